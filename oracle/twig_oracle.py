@@ -1,0 +1,239 @@
+"""fp64 CPU oracle for the TwigVLM / TwigVLM++ inference hot path.
+
+TEST INFRASTRUCTURE ONLY.  This is a plain, slow, exact-definition
+implementation used to check the CUDA library; nothing in the product path
+may import it, and it imports nothing from the product.  All floating-point
+inputs are float64 arrays (bf16 values widened exactly by the caller); all
+arithmetic is float64; softmax is the two-pass textbook form (max, then
+sum); there is no tiling, no online rescaling and no key splitting.
+``numpy.matmul`` is the only library primitive used.
+
+Parity pins (tests/test_oracle_*.py): every function below is pinned by
+closed forms, invariants the paper states, reductions to a library routine
+(causal scaled-dot-product attention in float64) or brute force on tiny
+inputs.  ``ttp_scores`` has no paper-printed numeric example to compare with
+(the paper prints no score values): its pins are closed forms and
+invariants only.
+
+Readings of the paper where it leaves a choice (each is also a test):
+  * scoring query = the last prompt token; heads are averaged (Eq. 7).
+  * norm_scope 0: softmax over the whole causal row of that query (it sees
+    every prompt key), then the visual columns are sliced (Eq. 2/3/5);
+    norm_scope 1: softmax over the visual keys only (Eq. 7).
+  * TopR ties go to the lower index; kept tokens stay in sequence order.
+  * a tree node attends to the whole KV prefix, its ancestors and itself.
+  * node 0 (root) is the last accepted token; it is always accepted.
+  * child c is accepted iff draft_tok[c] == base_argmax[parent[c]] and its
+    parent is accepted; the winner is the deepest accepted node (lowest index
+    among equals); the bonus token is base_argmax[winner] (Sec. 5.4,
+    Appendix A, Algorithm 2).
+"""
+from __future__ import annotations
+
+import numpy as np
+
+
+# --------------------------------------------------------------------------
+# Eq. 4 / Eq. 6: average number of retained visual tokens
+# --------------------------------------------------------------------------
+def avg_retained_tokens(M: int, K: int, R: int, L: int, K_f=None) -> float:
+    """Eq. 4 (K_f None): [M*K + R*(L-K)]/L.  Eq. 6: [M*K + R*(K_f-K)]/L."""
+    upper = L if K_f is None else K_f
+    return (M * K + R * (upper - K)) / L
+
+
+# --------------------------------------------------------------------------
+# O1: visual-token importance scores (Eq. 3/5 attention-map reading, Eq. 7)
+# --------------------------------------------------------------------------
+def ttp_scores(q, k, prefix_len, vis_start, n_vis, norm_scope=0, scale=None):
+    """q [B,Hq,d], k [B,Hkv,Lmax,d] float64 -> s [B,Mmax] float64 (0 beyond n_vis).
+
+    For request b and query head h (KV head h // G, G = Hq/Hkv):
+      z_j = (q[b,h] . k[b,h//G,j]) * scale over the scope,
+      p = softmax(z),  s[b,m] = mean_h p_h[vis_start + m].
+    Scope: norm_scope 0 -> j in [0, prefix_len); 1 -> j in the visual span.
+    """
+    q = np.asarray(q, dtype=np.float64)
+    k = np.asarray(k, dtype=np.float64)
+    B, Hq, d = q.shape
+    Hkv = k.shape[1]
+    G = Hq // Hkv
+    if scale is None:
+        scale = 1.0 / np.sqrt(d)
+    m_max = int(np.max(n_vis)) if B else 0
+    s = np.zeros((B, m_max), dtype=np.float64)
+    for b in range(B):
+        lp, vs, m = int(prefix_len[b]), int(vis_start[b]), int(n_vis[b])
+        if m == 0:
+            continue
+        lo, hi = (0, lp) if norm_scope == 0 else (vs, vs + m)
+        for h in range(Hq):
+            z = np.matmul(k[b, h // G, lo:hi, :], q[b, h, :]) * scale
+            e = np.exp(z - np.max(z))
+            p = e / np.sum(e)
+            s[b, :m] += p[vs - lo: vs - lo + m]
+        s[b, :m] /= Hq
+    return s
+
+
+# --------------------------------------------------------------------------
+# O2: TopR with the lowest-index tie rule (Eq. 3)
+# --------------------------------------------------------------------------
+def topk_lowest_index(s, R: int):
+    """Indices of the R largest entries of s; among equal values the lower
+    index wins; returned ascending."""
+    s = np.asarray(s)
+    order = sorted(range(len(s)), key=lambda m: (-s[m], m))
+    return np.array(sorted(order[:R]), dtype=np.int32)
+
+
+# --------------------------------------------------------------------------
+# O3: pruned sequence and the row gather (Eq. 3 / Eq. 5 applied to KV rows)
+# --------------------------------------------------------------------------
+def prune_index_list(prefix_len: int, vis_start: int, n_vis: int, kept):
+    """text before the image, kept visual tokens (ascending), text after."""
+    kept = [int(x) for x in kept]
+    return np.array(list(range(vis_start)) + [vis_start + m for m in kept]
+                    + list(range(vis_start + n_vis, prefix_len)), dtype=np.int64)
+
+
+def gather_compact(src_k, src_v, pos_in, prefix_len, vis_start, n_vis, kept_list, dst_k, dst_v, pos_out):
+    """dst[l,b,h,j,:] = src[l,b,h,idx_b[j],:], pos_out[b,j] = pos_in[b,idx_b[j]].
+
+    Arrays of any dtype (bit patterns are moved verbatim); dst/pos_out are
+    updated in place, rows >= new_len are left as they were.  Returns new_len.
+    """
+    B = src_k.shape[1]
+    new_len = np.zeros(B, dtype=np.int32)
+    for b in range(B):
+        idx = prune_index_list(int(prefix_len[b]), int(vis_start[b]), int(n_vis[b]), kept_list[b])
+        n = len(idx)
+        new_len[b] = n
+        for j in range(n):
+            dst_k[:, b, :, j, :] = src_k[:, b, :, idx[j], :]
+            dst_v[:, b, :, j, :] = src_v[:, b, :, idx[j], :]
+            pos_out[b, j] = pos_in[b, idx[j]]
+    return new_len
+
+
+# --------------------------------------------------------------------------
+# O4: tree-masked verification attention (Sec. 5.4, Appendix A, Eq. 2)
+# --------------------------------------------------------------------------
+def ancestors_or_self(parent, i: int):
+    out = []
+    x = int(i)
+    while x >= 0:
+        out.append(x)
+        x = int(parent[x])
+    return out[::-1]
+
+
+def tree_mask(parent, n_nodes: int, kv_len: int):
+    """Topology-aware causal mask of one request: visible[i, j] for node i over
+    the key sequence (cache rows 0..kv_len-1, then tree nodes 0..n_nodes-1)."""
+    vis = np.zeros((n_nodes, kv_len + n_nodes), dtype=bool)
+    vis[:, :kv_len] = True
+    for i in range(n_nodes):
+        for a in ancestors_or_self(parent, i):
+            vis[i, kv_len + a] = True
+    return vis
+
+
+def masked_attention(q_rows, keys, vals, visible, scale):
+    """Eq. 2 with mask: softmax over the visible keys of (q.k)*scale, times V.
+    q_rows [n,d], keys/vals [m,d], visible [n,m] bool.  Returns (out [n,d], lse [n])."""
+    z = np.matmul(q_rows, keys.T) * scale
+    z = np.where(visible, z, -np.inf)
+    zmax = np.max(z, axis=1, keepdims=True)
+    e = np.exp(z - zmax)
+    se = np.sum(e, axis=1, keepdims=True)
+    return np.matmul(e / se, vals), (zmax + np.log(se))[:, 0]
+
+
+def tree_attention(q, tree_k, tree_v, cache_k, cache_v, kv_len, n_nodes, parent, scale=None,
+                   samples=None):
+    """q [B,T,Hq,d]; tree_k/v [B,Hkv,T,d]; cache_k/v [B,Hkv,Lmax,d] (one layer).
+
+    Node i of request b, head h: keys/values are cache rows [0, kv_len[b]) of
+    KV head h//G followed by the tree rows, of which only i's ancestors and i
+    itself are visible; out = softmax(q.k * scale) @ v, lse = log-sum-exp of
+    the visible scaled logits.
+    Returns out [B,T,Hq,d] and lse [B,Hq,T]; rows of nodes >= n_nodes[b] are 0.
+    With ``samples`` (a list of (b, i, h)) only those rows are computed.
+    """
+    q = np.asarray(q, dtype=np.float64)
+    B, T, Hq, d = q.shape
+    Hkv = tree_k.shape[1]
+    G = Hq // Hkv
+    if scale is None:
+        scale = 1.0 / np.sqrt(d)
+    out = np.zeros((B, T, Hq, d), dtype=np.float64)
+    lse = np.zeros((B, Hq, T), dtype=np.float64)
+
+    def head_inputs(b, h):
+        L, n = int(kv_len[b]), int(n_nodes[b])
+        g = h // G
+        keys = np.concatenate([cache_k[b, g, :L, :], tree_k[b, g, :n, :]], axis=0).astype(np.float64)
+        vals = np.concatenate([cache_v[b, g, :L, :], tree_v[b, g, :n, :]], axis=0).astype(np.float64)
+        return keys, vals
+
+    if samples is not None:
+        for (b, i, h) in samples:
+            keys, vals = head_inputs(b, h)
+            vis = tree_mask(parent[b], int(n_nodes[b]), int(kv_len[b]))
+            o, l = masked_attention(q[b, i:i + 1, h, :], keys, vals, vis[i:i + 1], scale)
+            out[b, i, h, :] = o[0]
+            lse[b, h, i] = l[0]
+        return out, lse
+
+    for b in range(B):
+        n = int(n_nodes[b])
+        if n == 0:
+            continue
+        vis = tree_mask(parent[b], n, int(kv_len[b]))
+        for h in range(Hq):
+            keys, vals = head_inputs(b, h)
+            o, l = masked_attention(q[b, :n, h, :], keys, vals, vis, scale)
+            out[b, :n, h, :] = o
+            lse[b, h, :n] = l
+    return out, lse
+
+
+# --------------------------------------------------------------------------
+# O5: greedy tree acceptance (Sec. 5.4, Appendix A, Algorithm 2)
+# --------------------------------------------------------------------------
+def tree_accept(parent, draft_tok, base_argmax, n_nodes: int):
+    """One request.  Returns (accept_len, path, bonus).
+
+    A node is accepted when every edge (u -> c) on its root path has
+    draft_tok[c] == base_argmax[u].  The winner is the accepted node of
+    greatest depth, lowest index among equals; path = root..winner;
+    accept_len = depth(winner) (draft tokens accepted, root excluded);
+    bonus = base_argmax[winner].
+    """
+    best, best_depth = 0, 0
+    for i in range(int(n_nodes)):
+        chain = ancestors_or_self(parent, i)
+        ok = all(int(draft_tok[c]) == int(base_argmax[u]) for u, c in zip(chain[:-1], chain[1:]))
+        depth = len(chain) - 1
+        if ok and depth > best_depth:
+            best, best_depth = i, depth
+    path = ancestors_or_self(parent, best)
+    return best_depth, np.array(path, dtype=np.int32), int(base_argmax[best])
+
+
+# --------------------------------------------------------------------------
+# O6: append the accepted nodes' K/V rows to the cache
+# --------------------------------------------------------------------------
+def accept_compact(tree_k, tree_v, cache_k, cache_v, kv_len, paths):
+    """tree_k/v [Nl,B,Hkv,T,d]; cache_k/v [Nl,B,Hkv,Lmax,d] updated in place:
+    cache[l,b,h,kv_len[b]+j,:] = tree[l,b,h,path_b[j],:]; returns new kv_len."""
+    B = cache_k.shape[1]
+    new_len = np.array(kv_len, dtype=np.int32).copy()
+    for b in range(B):
+        base = int(kv_len[b])
+        for j, node in enumerate(paths[b]):
+            cache_k[:, b, :, base + j, :] = tree_k[:, b, :, int(node), :]
+            cache_v[:, b, :, base + j, :] = tree_v[:, b, :, int(node), :]
+        new_len[b] = base + len(paths[b])
+    return new_len
