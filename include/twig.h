@@ -1,0 +1,190 @@
+/*
+ * twig.h — C ABI of the B200 (sm_100a) kernels for the inference hot path of
+ * TwigVLM / TwigVLM++ ("Growing a Multi-head Twig via Distillation and
+ * Reinforcement Learning to Accelerate Large Vision-Language Models").
+ *
+ * Three calls make up the path:
+ *   ttp_score_topk_compact   twig-guided token pruning (Sec. 4.2 "TTP", Eq. 3, Eq. 5, Eq. 7/8)
+ *   tree_verify_attention    tree attention of the verification pass (Sec. 5.4, Appendix A, Algorithm 2)
+ *   tree_accept_compact      tree traversal / acceptance + bonus token + KV append (Sec. 5.4, Appendix A)
+ * The three stages of the first call are exported on their own as well.
+ *
+ * Conventions shared by every entry point
+ * ---------------------------------------
+ * Pointers: every data pointer is DEVICE memory unless marked "host".  The
+ *   twig_kv descriptor structs themselves are host memory, read during the
+ *   call.  The caller owns every buffer; the library allocates nothing.
+ * dtype: K, V, Q and attention outputs are bf16 (2 bytes); scores and lse are
+ *   fp32; all lengths, indices and token ids are int32.
+ * Layout: head_dim is contiguous and is 64 or 128.  Strides are in ELEMENTS.
+ *   Base pointers and row strides must make every row 16-byte aligned.
+ *   q-head h reads kv-head h / (n_q_heads / n_kv_heads).
+ * Stream: `stream` is a cudaStream_t passed as void* (NULL = default stream).
+ *   Calls enqueue work and return; they never synchronise, and they read
+ *   per-request metadata (lengths, parents, tokens) on the device.
+ * Errors: anything the host can check returns a twig_status != TWIG_OK and
+ *   launches nothing.  Data-dependent faults (a parent index out of range,
+ *   keep > n_vis, a cache that would overflow ...) set dev_status[b] to a
+ *   TWIG_DEV_* code and skip request b; kernels never trap or spin.
+ *   dev_status (int32 [batch], may be NULL) is only ever written with
+ *   non-zero codes: clear it before the call if you want to read it after.
+ * Positions: K is cached after the rotary embedding, so rows are moved
+ *   verbatim and kept tokens keep their ORIGINAL position ids (pos_ids are
+ *   carried through the gather, never recomputed).
+ */
+#ifndef TWIG_H_
+#define TWIG_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  TWIG_OK = 0,
+  TWIG_ERR_NULL = 1,        /* a required pointer is NULL                          */
+  TWIG_ERR_SHAPE = 2,       /* a size is non-positive or inconsistent               */
+  TWIG_ERR_UNSUPPORTED = 3, /* head_dim not 64/128, t_max > 64, n_vis bound > max  */
+  TWIG_ERR_WORKSPACE = 4,   /* ws_bytes < twig_workspace_bytes(...)                 */
+  TWIG_ERR_CUDA = 5,        /* a CUDA runtime call failed (launch error)            */
+  TWIG_ERR_ALIGN = 6        /* a pointer or stride breaks the 16-byte row rule      */
+} twig_status;
+
+/* per-request device status codes (written to dev_status[b]) */
+enum {
+  TWIG_DEV_OK = 0,
+  TWIG_DEV_BAD_LAYOUT = 1, /* vis_start/n_vis/prefix_len inconsistent or out of bounds */
+  TWIG_DEV_BAD_KEEP = 2,   /* keep < 0 or keep > n_vis                                 */
+  TWIG_DEV_BAD_INDEX = 3,  /* kept_idx not strictly ascending within [0, n_vis)        */
+  TWIG_DEV_BAD_TREE = 4,   /* n_nodes out of [0, t_max] or parent[i] not in [-1, i)    */
+  TWIG_DEV_OVERFLOW = 5    /* kv_len < 0 or kv_len + rows to append > max_len          */
+};
+
+#define TWIG_MAX_NODES 64      /* draft-tree nodes per request (root included)      */
+#define TWIG_MAX_VISUAL 16384  /* visual tokens per request                         */
+#define TWIG_MAX_BATCH 4096    /* requests per call                                 */
+
+/* One K/V tensor family: element (l, b, h, pos, c) of K is at
+ * k[l*stride_layer + b*stride_batch + h*stride_head + pos*stride_pos + c]. */
+typedef struct {
+  void *k, *v;             /* device, bf16 */
+  int64_t stride_layer, stride_batch, stride_head, stride_pos;
+  int32_t n_layers, batch, n_kv_heads, head_dim, max_len;
+} twig_kv;
+
+const char *twig_status_str(twig_status s);
+
+/* Bytes of device scratch the calls below need for these bounds (max_len is
+ * the longest prompt / cache length any of them will see). */
+size_t twig_workspace_bytes(int32_t batch, int32_t n_q_heads, int32_t head_dim, int32_t max_len,
+                            int32_t max_nodes);
+
+/* ---- TTP stage 1: importance score of every visual token -----------------
+ * Eq. 3 / Eq. 5 (attention map of the last twig layer, row of the last prompt
+ * token) and Eq. 7 (P-Head score).  For query head h:
+ *   p_h = softmax_j( twig_q[b,h] . twig_k[b, h/G, j] * softmax_scale ),
+ *   scores[b, m] = (1/n_q_heads) * sum_h p_h[vis_start[b] + m],  m < n_vis[b].
+ * norm_scope 0: the softmax runs over j in [0, prefix_len[b]) (the last
+ * query's full causal row); 1: over the visual span only (Eq. 7; scores sum
+ * to 1).  softmax_scale 0 means 1/sqrt(head_dim).
+ *   twig_q   [batch, n_q_heads, head_dim] contiguous (post-rotary, post-gate)
+ *   twig_k   rows at twig_k + b*k_stride_batch + h*k_stride_head + j*k_stride_pos
+ *   k_max_len  host bound on prefix_len (sizes the grid and the scratch)
+ *   scores   [batch, m_max] fp32 out; entries m >= n_vis[b] are set to 0
+ * Scratch: ws/ws_bytes from twig_workspace_bytes(batch, n_q_heads, head_dim, k_max_len, .).
+ */
+twig_status ttp_score(const void *twig_q, const void *twig_k, int64_t k_stride_batch,
+                      int64_t k_stride_head, int64_t k_stride_pos, int32_t k_max_len,
+                      const int32_t *prefix_len, const int32_t *vis_start, const int32_t *n_vis,
+                      int32_t batch, int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim,
+                      int32_t norm_scope, float softmax_scale, float *scores, int32_t m_max,
+                      int32_t *dev_status, void *ws, size_t ws_bytes, void *stream);
+
+/* ---- TTP stage 2: TopR of Eq. 3 --------------------------------------------
+ * kept_idx[b, 0..keep[b]) = indices of the keep[b] largest scores[b, 0..n_vis[b]),
+ * equal scores resolved to the LOWER index, written in ascending index order
+ * (sequence order is kept); entries past keep[b] are set to -1.  The choice is
+ * exact on the fp32 bit patterns.  Scores must not be NaN.
+ *   kept_idx [batch, r_max] int32 out;  m_max <= TWIG_MAX_VISUAL.
+ */
+twig_status ttp_topk(const float *scores, const int32_t *n_vis, const int32_t *keep, int32_t batch,
+                     int32_t m_max, int32_t r_max, int32_t *kept_idx, int32_t *dev_status,
+                     void *stream);
+
+/* ---- TTP stage 3: prune the KV cache (Eq. 5 applied to cached rows) --------
+ * New sequence of request b = [0, vis_start) ++ (vis_start + kept_idx[b, :keep])
+ * ++ [vis_start + n_vis, prefix_len).  For every layer and kv head,
+ * dst row j = src row idx[j] (bytes copied verbatim), pos_out[b, j] =
+ * pos_in[b, idx[j]], new_len[b] = prefix_len - n_vis + keep.  keep = 0 drops
+ * every visual token (the FinalWipe form); keep = n_vis is the identity.
+ * dst must not overlap src.  pos_in/pos_out ([batch, pos_stride], may both be
+ * NULL) and new_len (may be NULL) are int32.
+ */
+twig_status ttp_compact(const twig_kv *src, const twig_kv *dst, const int32_t *kept_idx,
+                        int32_t r_max, const int32_t *keep, const int32_t *prefix_len,
+                        const int32_t *vis_start, const int32_t *n_vis, const int32_t *pos_in,
+                        int32_t *pos_out, int32_t pos_stride, int32_t *new_len,
+                        int32_t *dev_status, void *stream);
+
+/* ---- TTP, all three stages (Sec. 4.2, Algorithm 1 "pruning", Algorithm 2) --
+ * Arguments as above; scores and kept_idx are outputs the caller may inspect. */
+twig_status ttp_score_topk_compact(
+    const void *twig_q, const void *twig_k, int64_t k_stride_batch, int64_t k_stride_head,
+    int64_t k_stride_pos, int32_t k_max_len, const int32_t *prefix_len, const int32_t *vis_start,
+    const int32_t *n_vis, const int32_t *keep, int32_t n_q_heads, int32_t norm_scope,
+    float softmax_scale, float *scores, int32_t m_max, int32_t *kept_idx, int32_t r_max,
+    const twig_kv *src, const twig_kv *dst, const int32_t *pos_in, int32_t *pos_out,
+    int32_t pos_stride, int32_t *new_len, int32_t *dev_status, void *ws, size_t ws_bytes,
+    void *stream);
+
+/* ---- Tree attention of the verification pass, one layer per call ------------
+ * Sec. 5.4 / Appendix A ("topology-aware causal mask so that each node attends
+ * only to its ancestors"), Eq. 2.  Node i < n_nodes[b] of request b, head h:
+ *   keys/values = cache rows [0, kv_len[b]) of layer `layer`, kv head h/G,
+ *                 followed by tree rows j with j an ancestor of i or i itself;
+ *   out[b,i,h,:] = softmax(q[b,i,h] . k * softmax_scale) @ v   (fp32 accumulate, bf16 out)
+ *   lse[b,h,i]   = log sum exp of the visible scaled logits    (optional)
+ *   q, out   [batch, t_max, n_q_heads, head_dim] bf16 contiguous
+ *   tree_k/v [batch, n_kv_heads, t_max, head_dim] bf16 contiguous (this layer's draft-tree K/V)
+ *   parent   [batch, t_max] int32; parent[b,0] = -1, parent[b,i] in [0, i)
+ *   lse      [batch, n_q_heads, t_max] fp32 or NULL
+ * t_max <= TWIG_MAX_NODES.  Rows of nodes >= n_nodes[b] are not written.
+ * softmax_scale 0 means 1/sqrt(head_dim).  ws may be NULL when ws_bytes is 0
+ * (the current kernels combine key splits on chip and use no scratch).
+ */
+twig_status tree_verify_attention(const void *q, const void *tree_k, const void *tree_v,
+                                  const twig_kv *cache, int32_t layer, const int32_t *kv_len,
+                                  const int32_t *n_nodes, const int32_t *parent, int32_t t_max,
+                                  int32_t n_q_heads, float softmax_scale, void *out, float *lse,
+                                  int32_t *dev_status, void *ws, size_t ws_bytes, void *stream);
+
+/* ---- Acceptance + bonus token + KV append, all layers in one call ------------
+ * Sec. 5.4 / Appendix A / Algorithm 2.  Node 0 is the last accepted token and is
+ * always accepted; child c is accepted iff its parent is and
+ * draft_tok[b,c] == base_argmax[b,parent[c]] (base_argmax[b,u] is the target's
+ * greedy token after consuming node u).  The winner is the accepted node of
+ * greatest depth (lowest index among equals);
+ *   path[b, 0..accept_len[b]] = root..winner, remaining entries -1,
+ *   accept_len[b] = depth(winner)   (accepted draft tokens, root excluded),
+ *   bonus_tok[b]  = base_argmax[b, winner].
+ * Then for every layer l and kv head: cache row kv_len[b] + j = tree row
+ * path[b, j] (j <= accept_len[b]) and kv_len[b] += accept_len[b] + 1.
+ *   tree_k_all/v_all [n_layers, batch, n_kv_heads, t_max, head_dim] bf16 contiguous
+ *   path [batch, d_max]; d_max must be >= the deepest level count (<= t_max)
+ * Requests with n_nodes[b] == 0 are idle: nothing is written for them.
+ * Two calls that are in flight at once on one device must not share a batch
+ * slot b (the completion ticket of slot b is library state).
+ */
+twig_status tree_accept_compact(const int32_t *parent, const int32_t *draft_tok,
+                                const int32_t *base_argmax, const int32_t *n_nodes, int32_t t_max,
+                                int32_t d_max, const void *tree_k_all, const void *tree_v_all,
+                                const twig_kv *cache, int32_t *kv_len, int32_t *accept_len,
+                                int32_t *path, int32_t *bonus_tok, int32_t *dev_status,
+                                void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TWIG_H_ */

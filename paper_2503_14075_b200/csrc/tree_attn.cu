@@ -1,0 +1,501 @@
+// Tree attention of the verification pass (Sec. 5.4, Appendix A, Algorithm 2;
+// Eq. 2 with the causal mask replaced by the tree's ancestor mask).
+//
+// Every draft-tree node attends to the whole cached prefix, to its ancestors
+// and to itself.  The T*G query rows that share one kv head (T nodes, G query
+// heads per kv head) form the M side of two dense contractions, S = Q K^T and
+// O = P V, run on bf16 tensor-core MMA with fp32 accumulation.  The key axis
+// (prefix rows followed by the tree's own rows) is cut into tiles; a thread
+// block cluster splits the tiles between its CTAs, every CTA keeps a
+// flash-style running (max, sum, O) per row, and the partial results are
+// merged through distributed shared memory, so nothing but Q, K, V and the
+// final output touches HBM.
+#include <cooperative_groups.h>
+
+#include "twig_common.cuh"
+
+namespace cg = cooperative_groups;
+
+namespace twig {
+
+struct AttnParams {
+  const __nv_bfloat16 *q, *tree_k, *tree_v, *cache_k, *cache_v;   // cache_* point at the layer
+  long long c_sb, c_sh, c_sp;
+  const int *kv_len, *n_nodes, *parent;
+  __nv_bfloat16 *out;
+  float *lse;
+  int *dev_status;
+  int t_max, n_q_heads, n_kv_heads, group, max_len, row_blocks;
+  float scale_log2;   // softmax_scale * log2(e)
+};
+
+// ---- small PTX wrappers ----------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void *p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void cp_async_16(uint32_t dst, const void *src, bool valid) {
+  const int n = valid ? 16 : 0;
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(n) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t *>(&v);
+}
+
+// Byte offset of 16-byte chunk `c` of row `r` in a [rows x D] bf16 tile.  The
+// tile is stored as D/64 panels of 128-byte rows; within a panel the chunk
+// index is XORed with (row & 7), which makes ldmatrix conflict-free.
+template <int ROWS>
+__device__ __forceinline__ uint32_t tile_off(int r, int c) {
+  return (uint32_t)((c >> 3) * ROWS * 128 + r * 128 + (((c & 7) ^ (r & 7)) << 4));
+}
+
+template <int D_, int WM_, int WN_, int KC_, int STAGES_>
+struct AttnCfg {
+  static constexpr int D = D_, WM = WM_, WN = WN_, KC = KC_, STAGES = STAGES_;
+  static constexpr int ROWS = 16 * WM;          // query rows per CTA
+  static constexpr int KT = KC * WN;            // keys per tile
+  static constexpr int THREADS = 32 * WM * WN;
+  static constexpr int CPR = D / 8;             // 16-byte chunks per row
+  static constexpr int Q_BYTES = ROWS * D * 2;
+  static constexpr int TILE_BYTES = KT * D * 2;
+  static constexpr int OD = D + 8;              // padded fp32 row of a partial O
+  static constexpr int PART_BYTES = WN * ROWS * OD * 4;
+  static constexpr int STAGE_BYTES = 2 * STAGES * TILE_BYTES;
+  static constexpr int BODY_BYTES = STAGE_BYTES > PART_BYTES ? STAGE_BYTES : PART_BYTES;
+  static constexpr int SMEM_BYTES = Q_BYTES + BODY_BYTES;
+};
+
+template <class C>
+__global__ void __launch_bounds__(C::THREADS)
+tree_attn_kernel(const AttnParams p) {
+  constexpr int D = C::D, ROWS = C::ROWS, KT = C::KT, KC = C::KC, WN = C::WN, STAGES = C::STAGES;
+  constexpr int NT = KC / 8;       // key n-tiles per warp per tile
+  constexpr int DT = D / 8;        // head-dim n-tiles of O
+  constexpr int KS = D / 16;       // k-steps of Q K^T
+  extern __shared__ __align__(1024) unsigned char smem[];
+  __shared__ unsigned long long s_mask[TWIG_MAX_NODES];
+  __shared__ float s_m[WN * ROWS], s_l[WN * ROWS];
+  __shared__ int s_bad;
+
+  cg::cluster_group cluster = cg::this_cluster();
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int wm = warp / WN, wn = warp % WN;
+  const int split = blockIdx.x, n_splits = gridDim.x;
+  const int hk = blockIdx.y / p.row_blocks, rb = blockIdx.y % p.row_blocks;
+  const int b = blockIdx.z;
+
+  // ---- per-request metadata; every exit below is uniform over the cluster ----
+  const int n = p.n_nodes[b], L = p.kv_len[b];
+  if (n == 0) return;
+  const bool first = split == 0 && blockIdx.y == 0 && tid == 0;
+  if (n < 0 || n > p.t_max) {
+    if (first) flag_status(p.dev_status, b, TWIG_DEV_BAD_TREE);
+    return;
+  }
+  if (L < 0 || L > p.max_len) {
+    if (first) flag_status(p.dev_status, b, TWIG_DEV_OVERFLOW);
+    return;
+  }
+  const int rows_total = n * p.group, row0 = rb * ROWS;
+  if (row0 >= rows_total) return;
+  if (tid == 0) s_bad = 0;
+  __syncthreads();
+  const int *par = p.parent + (long long)b * p.t_max;
+  if (tid < n) {
+    const int pr = par[tid];
+    if ((tid == 0) ? (pr != -1) : (pr < 0 || pr >= tid)) s_bad = 1;
+  }
+  __syncthreads();
+  if (s_bad) {
+    if (first) flag_status(p.dev_status, b, TWIG_DEV_BAD_TREE);
+    return;
+  }
+  if (tid < n) {          // ancestor-or-self bitmask; parent[x] < x bounds the walk
+    unsigned long long m = 0;
+    int x = tid;
+    while (x >= 0) {
+      m |= 1ull << x;
+      x = par[x];
+    }
+    s_mask[tid] = m;
+  }
+
+  const uint32_t q_s = smem_u32(smem);
+  const uint32_t k_s = q_s + C::Q_BYTES;
+  const uint32_t v_s = k_s + STAGES * C::TILE_BYTES;
+
+  // ---- key tiles of this CTA --------------------------------------------------
+  const int NK = L + n;
+  const int n_tiles = (NK + KT - 1) / KT;
+  const int per = (n_tiles + n_splits - 1) / n_splits;
+  const int t_begin = split * per;
+  const int t_end = min(n_tiles, t_begin + per);
+
+  const __nv_bfloat16 *ck = p.cache_k + b * p.c_sb + hk * p.c_sh;
+  const __nv_bfloat16 *cv = p.cache_v + b * p.c_sb + hk * p.c_sh;
+  const __nv_bfloat16 *tk = p.tree_k + ((long long)b * p.n_kv_heads + hk) * p.t_max * D;
+  const __nv_bfloat16 *tv = p.tree_v + ((long long)b * p.n_kv_heads + hk) * p.t_max * D;
+
+  auto load_tile = [&](int t, int stage) {
+    constexpr int CHUNKS = KT * C::CPR;
+#pragma unroll
+    for (int i = 0; i < (CHUNKS + C::THREADS - 1) / C::THREADS; ++i) {
+      const int cid = i * C::THREADS + tid;
+      if (CHUNKS % C::THREADS != 0 && cid >= CHUNKS) break;
+      const int r = cid / C::CPR, c = cid % C::CPR;
+      const int vj = t * KT + r;
+      const __nv_bfloat16 *sk = ck, *sv = cv;
+      bool valid = false;
+      if (vj < L) {
+        sk = ck + (long long)vj * p.c_sp + c * 8;
+        sv = cv + (long long)vj * p.c_sp + c * 8;
+        valid = true;
+      } else if (vj < NK) {
+        sk = tk + (vj - L) * D + c * 8;
+        sv = tv + (vj - L) * D + c * 8;
+        valid = true;
+      }
+      const uint32_t off = stage * C::TILE_BYTES + tile_off<KT>(r, c);
+      cp_async_16(k_s + off, sk, valid);
+      cp_async_16(v_s + off, sv, valid);
+    }
+  };
+
+  // ---- Q tile (zero rows past the request's last row) -------------------------
+  {
+    constexpr int CHUNKS = ROWS * C::CPR;
+#pragma unroll
+    for (int i = 0; i < (CHUNKS + C::THREADS - 1) / C::THREADS; ++i) {
+      const int cid = i * C::THREADS + tid;
+      if (CHUNKS % C::THREADS != 0 && cid >= CHUNKS) break;
+      const int r = cid / C::CPR, c = cid % C::CPR;
+      const int gr = row0 + r;
+      const bool valid = gr < rows_total;
+      const int node = valid ? gr / p.group : 0, g = valid ? gr % p.group : 0;
+      const __nv_bfloat16 *src =
+          p.q + (((long long)b * p.t_max + node) * p.n_q_heads + hk * p.group + g) * D + c * 8;
+      cp_async_16(q_s + tile_off<ROWS>(r, c), src, valid);
+    }
+  }
+#pragma unroll
+  for (int s = 0; s < STAGES - 1; ++s) {
+    if (t_begin + s < t_end) load_tile(t_begin + s, s);
+    cp_async_commit();        // the first group also carries Q
+  }
+
+  // ---- per-thread state --------------------------------------------------------
+  const int gq = lane >> 2, tq = lane & 3;
+  const int r_lo = wm * 16 + gq, r_hi = r_lo + 8;         // CTA-local rows of this thread
+  uint32_t qf[KS][4];
+  float o[DT][4];
+#pragma unroll
+  for (int i = 0; i < DT; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
+  float m_lo = -INFINITY, m_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;
+  unsigned long long mask_lo = 0, mask_hi = 0;
+  bool q_loaded = false;
+
+  for (int t = t_begin; t < t_end; ++t) {
+    const int it = t - t_begin;
+    cp_async_wait<STAGES - 2>();
+    __syncthreads();
+    {   // refill the stage that was consumed one iteration ago
+      const int tn = t + STAGES - 1;
+      if (tn < t_end) load_tile(tn, (it + STAGES - 1) % STAGES);
+      cp_async_commit();
+    }
+    if (!q_loaded) {
+      q_loaded = true;
+#pragma unroll
+      for (int ks = 0; ks < KS; ++ks) {
+        const int r = wm * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+        ldsm_x4(q_s + tile_off<ROWS>(r, ks * 2 + (lane >> 4)), qf[ks]);
+      }
+      const int g_lo = row0 + r_lo, g_hi = row0 + r_hi;
+      mask_lo = g_lo < rows_total ? s_mask[g_lo / p.group] : 0ull;
+      mask_hi = g_hi < rows_total ? s_mask[g_hi / p.group] : 0ull;
+    }
+    const int stage = it % STAGES;
+    const uint32_t kst = k_s + stage * C::TILE_BYTES, vst = v_s + stage * C::TILE_BYTES;
+    const int kbase = wn * KC;
+
+    // S = Q K^T for this warp's KC keys
+    float s[NT][4];
+#pragma unroll
+    for (int i = 0; i < NT; ++i) s[i][0] = s[i][1] = s[i][2] = s[i][3] = 0.f;
+#pragma unroll
+    for (int ks = 0; ks < KS; ++ks) {
+#pragma unroll
+      for (int np = 0; np < NT / 2; ++np) {
+        uint32_t kb[4];
+        const int key = kbase + np * 16 + (lane & 7) + (lane >> 4) * 8;
+        ldsm_x4(kst + tile_off<KT>(key, ks * 2 + ((lane >> 3) & 1)), kb);
+        mma_bf16(s[2 * np], qf[ks], kb[0], kb[1]);
+        mma_bf16(s[2 * np + 1], qf[ks], kb[2], kb[3]);
+      }
+    }
+
+    // scale into the exp2 domain; mask the tile that holds the prefix end / the tree
+    const int key0 = t * KT + kbase;
+    if (key0 + KC > L) {
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int vj = key0 + nt * 8 + tq * 2 + (e & 1);
+          const unsigned long long mk = (e & 2) ? mask_hi : mask_lo;
+          const bool vis = vj < L || (vj < NK && ((mk >> (vj - L)) & 1ull));
+          s[nt][e] = vis ? s[nt][e] * p.scale_log2 : -INFINITY;
+        }
+      }
+    } else {
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) s[nt][e] *= p.scale_log2;
+      }
+    }
+
+    // online softmax
+    float mx_lo = -INFINITY, mx_hi = -INFINITY;
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+      mx_lo = fmaxf(mx_lo, fmaxf(s[nt][0], s[nt][1]));
+      mx_hi = fmaxf(mx_hi, fmaxf(s[nt][2], s[nt][3]));
+    }
+    mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 1));
+    mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 2));
+    mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 1));
+    mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 2));
+    const float mn_lo = fmaxf(m_lo, mx_lo), mn_hi = fmaxf(m_hi, mx_hi);
+    const float use_lo = mn_lo == -INFINITY ? 0.f : mn_lo, use_hi = mn_hi == -INFINITY ? 0.f : mn_hi;
+    const float a_lo = exp2f(m_lo - use_lo), a_hi = exp2f(m_hi - use_hi);
+    m_lo = mn_lo;
+    m_hi = mn_hi;
+    float sum_lo = 0.f, sum_hi = 0.f;
+    uint32_t pf[NT / 2][4];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+      const float p0 = exp2f(s[nt][0] - use_lo), p1 = exp2f(s[nt][1] - use_lo);
+      const float p2 = exp2f(s[nt][2] - use_hi), p3 = exp2f(s[nt][3] - use_hi);
+      sum_lo += p0 + p1;
+      sum_hi += p2 + p3;
+      pf[nt / 2][(nt & 1) * 2 + 0] = pack_bf16(p0, p1);
+      pf[nt / 2][(nt & 1) * 2 + 1] = pack_bf16(p2, p3);
+    }
+    l_lo = l_lo * a_lo + sum_lo;
+    l_hi = l_hi * a_hi + sum_hi;
+#pragma unroll
+    for (int i = 0; i < DT; ++i) {
+      o[i][0] *= a_lo;
+      o[i][1] *= a_lo;
+      o[i][2] *= a_hi;
+      o[i][3] *= a_hi;
+    }
+
+    // O += P V
+#pragma unroll
+    for (int kk = 0; kk < NT / 2; ++kk) {
+#pragma unroll
+      for (int dp = 0; dp < DT / 2; ++dp) {
+        uint32_t vb[4];
+        const int key = kbase + kk * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+        ldsm_x4_t(vst + tile_off<KT>(key, dp * 2 + (lane >> 4)), vb);
+        mma_bf16(o[2 * dp], pf[kk], vb[0], vb[1]);
+        mma_bf16(o[2 * dp + 1], pf[kk], vb[2], vb[3]);
+      }
+    }
+  }
+  cp_async_wait<0>();
+  __syncthreads();            // all warps are done with the stage buffers
+
+  // ---- this warp's partial (m, l, O) -> shared memory ---------------------------
+  l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1);
+  l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
+  l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1);
+  l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
+  float *part = reinterpret_cast<float *>(smem + C::Q_BYTES);
+  {
+    float *po_lo = part + ((size_t)wn * ROWS + r_lo) * C::OD, *po_hi = part + ((size_t)wn * ROWS + r_hi) * C::OD;
+#pragma unroll
+    for (int i = 0; i < DT; ++i) {
+      *reinterpret_cast<float2 *>(po_lo + i * 8 + tq * 2) = make_float2(o[i][0], o[i][1]);
+      *reinterpret_cast<float2 *>(po_hi + i * 8 + tq * 2) = make_float2(o[i][2], o[i][3]);
+    }
+    if (tq == 0) {
+      s_m[wn * ROWS + r_lo] = m_lo;
+      s_l[wn * ROWS + r_lo] = l_lo;
+      s_m[wn * ROWS + r_hi] = m_hi;
+      s_l[wn * ROWS + r_hi] = l_hi;
+    }
+  }
+  cluster.sync();
+
+  // ---- merge the n_splits * WN partials; this CTA finishes a slice of the rows ---
+  {
+    constexpr int TPR = D / 4;                        // threads per row, 4 floats each
+    constexpr int RPP = C::THREADS / TPR;             // rows per pass
+    const int rows_per = (ROWS + n_splits - 1) / n_splits;
+    const int r_begin = split * rows_per, r_end = min(ROWS, r_begin + rows_per);
+    const int c4 = (tid % TPR) * 4;
+    for (int r = r_begin + tid / TPR; r < r_end; r += RPP) {
+      const int gr = row0 + r;
+      if (gr >= rows_total) continue;
+      float mstar = -INFINITY;
+      for (int cta = 0; cta < n_splits; ++cta) {
+        const float *rm = cluster.map_shared_rank(s_m, cta);
+#pragma unroll
+        for (int w = 0; w < WN; ++w) mstar = fmaxf(mstar, rm[w * ROWS + r]);
+      }
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+      float lsum = 0.f;
+      for (int cta = 0; cta < n_splits; ++cta) {
+        const float *rm = cluster.map_shared_rank(s_m, cta);
+        const float *rl = cluster.map_shared_rank(s_l, cta);
+        const float *ro = cluster.map_shared_rank(part, cta);
+#pragma unroll
+        for (int w = 0; w < WN; ++w) {
+          const float wgt = exp2f(rm[w * ROWS + r] - mstar);
+          if (wgt == 0.f) continue;
+          lsum = fmaf(wgt, rl[w * ROWS + r], lsum);
+          const float4 v = *reinterpret_cast<const float4 *>(ro + ((size_t)w * ROWS + r) * C::OD + c4);
+          acc.x = fmaf(wgt, v.x, acc.x);
+          acc.y = fmaf(wgt, v.y, acc.y);
+          acc.z = fmaf(wgt, v.z, acc.z);
+          acc.w = fmaf(wgt, v.w, acc.w);
+        }
+      }
+      const float inv = 1.f / lsum;
+      const int node = gr / p.group, g = gr % p.group;
+      const int h = hk * p.group + g;
+      uint2 packed;
+      packed.x = pack_bf16(acc.x * inv, acc.y * inv);
+      packed.y = pack_bf16(acc.z * inv, acc.w * inv);
+      *reinterpret_cast<uint2 *>(p.out + (((long long)b * p.t_max + node) * p.n_q_heads + h) * D + c4) = packed;
+      if (p.lse && c4 == 0)
+        p.lse[((long long)b * p.n_q_heads + h) * p.t_max + node] = (mstar + log2f(lsum)) * 0.6931471805599453f;
+    }
+  }
+  cluster.sync();             // keep this CTA's shared memory alive until every peer has read it
+}
+
+// ---------------------------------------------------------------------------
+// host side
+// ---------------------------------------------------------------------------
+template <class C>
+static twig_status launch_attn(const AttnParams &p, int batch, int n_splits, cudaStream_t st) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(tree_attn_kernel<C>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             C::SMEM_BYTES) != cudaSuccess)
+      return TWIG_ERR_CUDA;
+    attr_set = true;
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(n_splits, p.n_kv_heads * p.row_blocks, batch);
+  cfg.blockDim = dim3(C::THREADS);
+  cfg.dynamicSmemBytes = C::SMEM_BYTES;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = n_splits;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (cudaLaunchKernelEx(&cfg, tree_attn_kernel<C>, p) != cudaSuccess) return TWIG_ERR_CUDA;
+  return TWIG_OK;
+}
+
+static int pick_splits(int items, int max_tiles) {
+  int s = 1;
+  while (s < 8 && items * s < 2 * 148 && s * 2 <= max_tiles) s *= 2;
+  return s;
+}
+
+template <int D>
+static twig_status dispatch_attn(AttnParams &p, int batch, int rows, cudaStream_t st) {
+  using C16 = AttnCfg<D, 1, 4, 16, 3>;
+  using C32 = AttnCfg<D, 2, 4, 16, 3>;
+  using C64 = AttnCfg<D, 4, 2, 32, 3>;
+  using C128 = AttnCfg<D, 8, 1, 64, 3>;
+  const int rows_per_cta = rows <= 16 ? 16 : rows <= 32 ? 32 : rows <= 64 ? 64 : 128;
+  p.row_blocks = (rows + rows_per_cta - 1) / rows_per_cta;
+  if ((long long)p.n_kv_heads * p.row_blocks > 65535) return TWIG_ERR_UNSUPPORTED;
+  const int max_tiles = (p.max_len + p.t_max + 63) / 64;
+  const int n_splits = pick_splits(batch * p.n_kv_heads * p.row_blocks, max_tiles);
+  switch (rows_per_cta) {
+    case 16: return launch_attn<C16>(p, batch, n_splits, st);
+    case 32: return launch_attn<C32>(p, batch, n_splits, st);
+    case 64: return launch_attn<C64>(p, batch, n_splits, st);
+    default: return launch_attn<C128>(p, batch, n_splits, st);
+  }
+}
+
+}  // namespace twig
+
+using namespace twig;
+
+extern "C" twig_status tree_verify_attention(const void *q, const void *tree_k, const void *tree_v,
+                                             const twig_kv *cache, int32_t layer,
+                                             const int32_t *kv_len, const int32_t *n_nodes,
+                                             const int32_t *parent, int32_t t_max,
+                                             int32_t n_q_heads, float softmax_scale, void *out,
+                                             float *lse, int32_t *dev_status, void *ws,
+                                             size_t ws_bytes, void *stream) {
+  (void)ws;
+  (void)ws_bytes;
+  if (!q || !tree_k || !tree_v || !kv_len || !n_nodes || !parent || !out) return TWIG_ERR_NULL;
+  twig_status s = check_kv(cache);
+  if (s != TWIG_OK) return s;
+  if (t_max <= 0 || n_q_heads <= 0 || layer < 0 || layer >= cache->n_layers) return TWIG_ERR_SHAPE;
+  if (n_q_heads % cache->n_kv_heads) return TWIG_ERR_SHAPE;
+  if (t_max > TWIG_MAX_NODES) return TWIG_ERR_UNSUPPORTED;
+  if (!aligned16(q) || !aligned16(tree_k) || !aligned16(tree_v) || !aligned16(out)) return TWIG_ERR_ALIGN;
+
+  AttnParams p;
+  p.q = static_cast<const __nv_bfloat16 *>(q);
+  p.tree_k = static_cast<const __nv_bfloat16 *>(tree_k);
+  p.tree_v = static_cast<const __nv_bfloat16 *>(tree_v);
+  p.cache_k = static_cast<const __nv_bfloat16 *>(cache->k) + layer * cache->stride_layer;
+  p.cache_v = static_cast<const __nv_bfloat16 *>(cache->v) + layer * cache->stride_layer;
+  p.c_sb = cache->stride_batch;
+  p.c_sh = cache->stride_head;
+  p.c_sp = cache->stride_pos;
+  p.kv_len = kv_len;
+  p.n_nodes = n_nodes;
+  p.parent = parent;
+  p.out = static_cast<__nv_bfloat16 *>(out);
+  p.lse = lse;
+  p.dev_status = dev_status;
+  p.t_max = t_max;
+  p.n_q_heads = n_q_heads;
+  p.n_kv_heads = cache->n_kv_heads;
+  p.group = n_q_heads / cache->n_kv_heads;
+  p.max_len = cache->max_len;
+  p.row_blocks = 1;
+  const float scale = softmax_scale != 0.f ? softmax_scale : 1.f / sqrtf((float)cache->head_dim);
+  p.scale_log2 = scale * 1.4426950408889634f;
+  const int rows = t_max * p.group;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  return cache->head_dim == 128 ? dispatch_attn<128>(p, cache->batch, rows, st)
+                                : dispatch_attn<64>(p, cache->batch, rows, st);
+}

@@ -1,0 +1,516 @@
+// Twig-guided token pruning (TTP): importance scores, TopR selection and the
+// gather that compacts the kept rows of the KV cache.
+//
+// Scores follow Eq. 3 / Eq. 5 (row of the last prompt token in the attention
+// map of the last twig layer) and Eq. 7 (softmax over the visual tokens, mean
+// over heads).  TopR is Eq. 3's selection with the lower index winning ties
+// and sequence order kept.  The gather applies the pruned token list to the
+// cached K/V rows of every layer; position ids travel with their rows.
+#include "twig_common.cuh"
+
+namespace twig {
+
+constexpr int kScoreThreads = 256;
+constexpr int kScoreKeysPerCta = 128;
+constexpr int kMaxGroup = 16;   // query heads per kv head
+constexpr int kMaxQHeads = 128;
+constexpr int kTopkThreads = 1024;
+
+// per-request layout check shared by the three stages
+__device__ __forceinline__ bool layout_ok(int lp, int vs, int nv, int k_max_len, int m_max) {
+  return lp >= 0 && lp <= k_max_len && vs >= 0 && nv >= 0 && nv <= m_max && vs <= lp &&
+         nv <= lp - vs;
+}
+
+// ---------------------------------------------------------------------------
+// Stage 1a: scaled logits of the last prompt query against every key in scope.
+// One CTA = 128 keys of one kv head; the G query heads of the group share the
+// key read.  D/8 lanes cover one key row (16 bytes each).
+// ---------------------------------------------------------------------------
+template <int D>
+__global__ void __launch_bounds__(kScoreThreads)
+ttp_logits_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restrict__ k,
+                  long long ksb, long long ksh, long long ksp, int k_max_len,
+                  const int *__restrict__ prefix_len, const int *__restrict__ vis_start,
+                  const int *__restrict__ n_vis, int n_q_heads, int group, int norm_scope,
+                  float scale, float *__restrict__ logits, int lstride, int m_max,
+                  int *dev_status) {
+  constexpr int LPK = D / 8;               // lanes per key row
+  constexpr int KPP = kScoreThreads / LPK; // keys per pass of the CTA
+  constexpr int PASSES = kScoreKeysPerCta / KPP;
+  __shared__ float qs[kMaxGroup * D];
+
+  const int b = blockIdx.z, hk = blockIdx.y;
+  const int lp = prefix_len[b], vs = vis_start[b], nv = n_vis[b];
+  if (!layout_ok(lp, vs, nv, k_max_len, m_max)) {
+    if (threadIdx.x == 0 && blockIdx.x == 0 && hk == 0) flag_status(dev_status, b, TWIG_DEV_BAD_LAYOUT);
+    return;
+  }
+  const int lo = norm_scope ? vs : 0, hi = norm_scope ? vs + nv : lp;
+  const int j0 = blockIdx.x * kScoreKeysPerCta;
+  if (j0 >= hi || j0 + kScoreKeysPerCta <= lo) return;
+
+  for (int i = threadIdx.x; i < group * D; i += kScoreThreads)
+    qs[i] = __bfloat162float(q[((long long)b * n_q_heads + hk * group) * D + i]) * scale;
+  __syncthreads();
+
+  const int sub = threadIdx.x % LPK, slot = threadIdx.x / LPK;
+  const __nv_bfloat16 *kb = k + b * ksb + hk * ksh + sub * 8;
+  uint4 kr[PASSES];
+#pragma unroll
+  for (int p = 0; p < PASSES; ++p) {
+    const int j = j0 + p * KPP + slot;
+    kr[p] = (j >= lo && j < hi) ? ld_nc_16(kb + (long long)j * ksp) : make_uint4(0, 0, 0, 0);
+  }
+  for (int g = 0; g < group; ++g) {
+    const float4 qa = *reinterpret_cast<const float4 *>(qs + g * D + sub * 8);
+    const float4 qb = *reinterpret_cast<const float4 *>(qs + g * D + sub * 8 + 4);
+    float *lrow = logits + ((long long)b * n_q_heads + hk * group + g) * lstride;
+#pragma unroll
+    for (int p = 0; p < PASSES; ++p) {
+      float acc = bf16_lo(kr[p].x) * qa.x;
+      acc = fmaf(bf16_hi(kr[p].x), qa.y, acc);
+      acc = fmaf(bf16_lo(kr[p].y), qa.z, acc);
+      acc = fmaf(bf16_hi(kr[p].y), qa.w, acc);
+      acc = fmaf(bf16_lo(kr[p].z), qb.x, acc);
+      acc = fmaf(bf16_hi(kr[p].z), qb.y, acc);
+      acc = fmaf(bf16_lo(kr[p].w), qb.z, acc);
+      acc = fmaf(bf16_hi(kr[p].w), qb.w, acc);
+#pragma unroll
+      for (int o = LPK / 2; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+      const int j = j0 + p * KPP + slot;
+      if (sub == 0 && j >= lo && j < hi) lrow[j] = acc;
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------
+// Stage 1b + 2: softmax per head, mean over heads -> scores; then exact TopR.
+// One CTA of 1024 threads per request.  mode bit 0: compute scores from the
+// logits; bit 1: select.  Without bit 0 the scores are read from `scores`.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t order_key(float x) {
+  const uint32_t u = __float_as_uint(x);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+// exclusive block scan of `x` over 1024 threads; returns the block total in `total`
+__device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t x, uint32_t *warp_sums, uint32_t &total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  uint32_t inc = x;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const uint32_t y = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += y;
+  }
+  if (lane == 31) warp_sums[warp] = inc;
+  __syncthreads();
+  if (warp == 0) {
+    uint32_t w = warp_sums[lane], winc = w;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t y = __shfl_up_sync(0xffffffffu, winc, o);
+      if (lane >= o) winc += y;
+    }
+    warp_sums[lane] = winc - w;
+    if (lane == 31) warp_sums[32] = winc;
+  }
+  __syncthreads();
+  const uint32_t res = warp_sums[warp] + inc - x;
+  total = warp_sums[32];
+  __syncthreads();
+  return res;
+}
+
+__global__ void __launch_bounds__(kTopkThreads)
+ttp_finalize_topk_kernel(const float *__restrict__ logits, int lstride, int n_q_heads, int k_max_len,
+                         const int *__restrict__ prefix_len, const int *__restrict__ vis_start,
+                         const int *__restrict__ n_vis, const int *__restrict__ keep, int norm_scope,
+                         float *__restrict__ scores, int m_max, int *__restrict__ kept_idx, int r_max,
+                         int *dev_status, int mode) {
+  extern __shared__ uint32_t keys[];                 // [m_max] fp32 scores, then ordered keys
+  __shared__ float h_max[kMaxQHeads], h_inv[kMaxQHeads];
+  __shared__ uint32_t hist[256];
+  __shared__ uint32_t warp_sums[33];
+  __shared__ uint32_t sel_digit, sel_remaining;
+
+  const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int nv = n_vis[b];
+  float *sc = scores + (long long)b * m_max;
+
+  if (mode & 1) {
+    const int lp = prefix_len[b], vs = vis_start[b];
+    if (!layout_ok(lp, vs, nv, k_max_len, m_max)) {
+      if (tid == 0) flag_status(dev_status, b, TWIG_DEV_BAD_LAYOUT);
+      return;
+    }
+    const int lo = norm_scope ? vs : 0, hi = norm_scope ? vs + nv : lp;
+    for (int h = warp; h < n_q_heads; h += kTopkThreads / 32) {
+      const float *z = logits + ((long long)b * n_q_heads + h) * lstride;
+      float mx = -INFINITY;
+      for (int j = lo + lane; j < hi; j += 32) mx = fmaxf(mx, z[j]);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+      float sum = 0.f;
+      for (int j = lo + lane; j < hi; j += 32) sum += expf(z[j] - mx);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+      if (lane == 0) {
+        h_max[h] = mx;
+        h_inv[h] = 1.f / sum;
+      }
+    }
+    __syncthreads();
+    const float inv_h = 1.f / (float)n_q_heads;
+    for (int m = tid; m < m_max; m += kTopkThreads) {
+      float acc = 0.f;
+      if (m < nv) {
+        const float *z = logits + (long long)b * n_q_heads * lstride + vs + m;
+        for (int h = 0; h < n_q_heads; ++h) acc += expf(z[(long long)h * lstride] - h_max[h]) * h_inv[h];
+        acc *= inv_h;
+      }
+      sc[m] = acc;
+      keys[m] = order_key(acc);
+    }
+  } else {
+    if (nv < 0 || nv > m_max) {
+      if (tid == 0) flag_status(dev_status, b, TWIG_DEV_BAD_LAYOUT);
+      return;
+    }
+    for (int m = tid; m < nv; m += kTopkThreads) keys[m] = order_key(sc[m]);
+  }
+  if (!(mode & 2)) return;
+  const int R = keep[b];
+  if (R < 0 || R > nv || R > r_max) {
+    if (tid == 0) flag_status(dev_status, b, TWIG_DEV_BAD_KEEP);
+    return;
+  }
+  int *out = kept_idx + (long long)b * r_max;
+  for (int i = R + tid; i < r_max; i += kTopkThreads) out[i] = -1;
+  if (R == 0) return;
+  __syncthreads();
+
+  // radix select, 8 bits per pass from the top: the R-th largest key
+  uint32_t prefix = 0, mask = 0;
+  uint32_t remaining = (uint32_t)R;
+#pragma unroll 1
+  for (int shift = 24; shift >= 0; shift -= 8) {
+    if (tid < 256) hist[tid] = 0;
+    __syncthreads();
+    for (int m = tid; m < nv; m += kTopkThreads) {
+      const uint32_t key = keys[m];
+      if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+    }
+    __syncthreads();
+    if (warp == 0) {
+      uint32_t c[8], mine = 0;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        c[i] = hist[lane * 8 + i];
+        mine += c[i];
+      }
+      uint32_t suf = mine;   // inclusive suffix sum over lanes (lane 31 = top digits)
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t y = __shfl_down_sync(0xffffffffu, suf, o);
+        if (lane + o < 32) suf += y;
+      }
+      uint32_t above = suf - mine;
+      if (above < remaining && remaining <= suf) {
+#pragma unroll
+        for (int i = 7; i >= 0; --i) {
+          if (above < remaining && remaining <= above + c[i]) {
+            sel_digit = lane * 8 + i;
+            sel_remaining = remaining - above;
+          }
+          above += c[i];
+        }
+      }
+    }
+    __syncthreads();
+    prefix |= sel_digit << shift;
+    mask |= 255u << shift;
+    remaining = sel_remaining;
+    __syncthreads();
+  }
+  const uint32_t tau = prefix, need_eq = remaining;
+
+  // ordered compaction: keys above tau, plus the first need_eq keys equal to tau
+  uint32_t run_gt = 0, run_eq = 0;
+  for (int base = 0; base < nv; base += kTopkThreads) {
+    const int m = base + tid;
+    const uint32_t key = (m < nv) ? keys[m] : 0u;
+    const uint32_t gt = (m < nv && key > tau), eq = (m < nv && key == tau);
+    uint32_t total;
+    const uint32_t ex = block_exclusive_scan(gt | (eq << 16), warp_sums, total);
+    const uint32_t gt_before = run_gt + (ex & 0xffffu), eq_before = run_eq + (ex >> 16);
+    if (gt || (eq && eq_before < need_eq)) out[gt_before + min(eq_before, need_eq)] = m;
+    run_gt += total & 0xffffu;
+    run_eq += total >> 16;
+  }
+}
+
+// ---------------------------------------------------------------------------
+// Stage 3: gather the rows of the pruned sequence, all layers and kv heads.
+// One CTA = 64 destination rows of one (layer, kv head, request), K and V.
+// ---------------------------------------------------------------------------
+constexpr int kGatherThreads = 256;
+constexpr int kGatherRows = 64;
+
+template <int D>
+__global__ void __launch_bounds__(kGatherThreads)
+kv_gather_kernel(KvView src, KvViewMut dst, const int *__restrict__ kept_idx, int r_max,
+                 const int *__restrict__ keep, const int *__restrict__ prefix_len,
+                 const int *__restrict__ vis_start, const int *__restrict__ n_vis,
+                 const int *__restrict__ pos_in, int *__restrict__ pos_out, int pos_stride,
+                 int *__restrict__ new_len, int *dev_status) {
+  constexpr int LPR = D / 8;                   // lanes per row
+  constexpr int RPP = kGatherThreads / LPR;    // rows per pass
+  constexpr int PASSES = kGatherRows / RPP;
+  const int b = blockIdx.z;
+  const int layer = blockIdx.y / src.n_kv_heads, h = blockIdx.y % src.n_kv_heads;
+  const int lp = prefix_len[b], vs = vis_start[b], nv = n_vis[b], kp = keep[b];
+  const bool first = blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0;
+  if (!layout_ok(lp, vs, nv, src.max_len, TWIG_MAX_VISUAL)) {
+    if (first) flag_status(dev_status, b, TWIG_DEV_BAD_LAYOUT);
+    return;
+  }
+  if (kp < 0 || kp > nv || kp > r_max) {
+    if (first) flag_status(dev_status, b, TWIG_DEV_BAD_KEEP);
+    return;
+  }
+  const int nl = lp - nv + kp;
+  if (nl > dst.max_len) {
+    if (first) flag_status(dev_status, b, TWIG_DEV_OVERFLOW);
+    return;
+  }
+  if (first && new_len) new_len[b] = nl;
+  const int j0 = blockIdx.x * kGatherRows;
+  if (j0 >= nl) return;
+
+  const int sub = threadIdx.x % LPR, slot = threadIdx.x / LPR;
+  const long long sbase = layer * src.stride_layer + b * src.stride_batch + h * src.stride_head + sub * 8;
+  const long long dbase = layer * dst.stride_layer + b * dst.stride_batch + h * dst.stride_head + sub * 8;
+  const int *kidx = kept_idx + (long long)b * r_max;
+
+  int srow[PASSES];
+  uint4 kr[PASSES], vr[PASSES];
+#pragma unroll
+  for (int p = 0; p < PASSES; ++p) {
+    const int j = j0 + p * RPP + slot;
+    int s = -1;
+    if (j < nl) {
+      if (j < vs) {
+        s = j;
+      } else if (j < vs + kp) {
+        const int kk = kidx[j - vs];
+        const int prev = (j > vs) ? kidx[j - vs - 1] : -1;
+        if (kk < 0 || kk >= nv || kk <= prev) {
+          if (sub == 0 && blockIdx.y == 0) flag_status(dev_status, b, TWIG_DEV_BAD_INDEX);
+        } else {
+          s = vs + kk;
+        }
+      } else {
+        s = j - kp + nv;
+      }
+    }
+    srow[p] = s;
+    if (s >= 0) {
+      kr[p] = ld_nc_16(src.k + sbase + (long long)s * src.stride_pos);
+      vr[p] = ld_nc_16(src.v + sbase + (long long)s * src.stride_pos);
+    }
+  }
+#pragma unroll
+  for (int p = 0; p < PASSES; ++p) {
+    const int j = j0 + p * RPP + slot;
+    if (srow[p] >= 0) {
+      st_16(dst.k + dbase + (long long)j * dst.stride_pos, kr[p]);
+      st_16(dst.v + dbase + (long long)j * dst.stride_pos, vr[p]);
+      if (blockIdx.y == 0 && sub == 0 && pos_in && pos_out)
+        pos_out[(long long)b * pos_stride + j] = pos_in[(long long)b * pos_stride + srow[p]];
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------
+// host side
+// ---------------------------------------------------------------------------
+static inline int logits_stride(int k_max_len) { return (k_max_len + 3) & ~3; }
+
+size_t score_workspace_bytes(int batch, int n_q_heads, int max_len) {
+  return (size_t)batch * n_q_heads * logits_stride(max_len) * sizeof(float);
+}
+
+struct ScoreArgs {
+  const void *twig_q, *twig_k;
+  int64_t ksb, ksh, ksp;
+  int k_max_len;
+  const int *prefix_len, *vis_start, *n_vis;
+  int batch, n_q_heads, n_kv_heads, head_dim, norm_scope;
+  float softmax_scale;
+  float *scores;
+  int m_max;
+};
+
+static twig_status check_score_args(const ScoreArgs &a, const void *ws, size_t ws_bytes) {
+  if (!a.twig_q || !a.twig_k || !a.prefix_len || !a.vis_start || !a.n_vis || !a.scores || !ws)
+    return TWIG_ERR_NULL;
+  if (a.batch <= 0 || a.n_q_heads <= 0 || a.n_kv_heads <= 0 || a.k_max_len <= 0 || a.m_max <= 0)
+    return TWIG_ERR_SHAPE;
+  if (a.n_q_heads % a.n_kv_heads) return TWIG_ERR_SHAPE;
+  if (a.head_dim != 64 && a.head_dim != 128) return TWIG_ERR_UNSUPPORTED;
+  if (a.n_q_heads / a.n_kv_heads > kMaxGroup || a.n_q_heads > kMaxQHeads) return TWIG_ERR_UNSUPPORTED;
+  if (a.m_max > TWIG_MAX_VISUAL || a.batch > TWIG_MAX_BATCH) return TWIG_ERR_UNSUPPORTED;
+  if (a.norm_scope != 0 && a.norm_scope != 1) return TWIG_ERR_UNSUPPORTED;
+  if (a.ksp < a.head_dim) return TWIG_ERR_SHAPE;
+  if (!aligned16(a.twig_q) || !aligned16(a.twig_k) || !aligned16(ws) || ((a.ksb | a.ksh | a.ksp) & 7))
+    return TWIG_ERR_ALIGN;
+  if (ws_bytes < score_workspace_bytes(a.batch, a.n_q_heads, a.k_max_len)) return TWIG_ERR_WORKSPACE;
+  return TWIG_OK;
+}
+
+static twig_status launch_logits(const ScoreArgs &a, int *dev_status, void *ws, cudaStream_t st) {
+  const float scale = a.softmax_scale != 0.f ? a.softmax_scale : 1.f / sqrtf((float)a.head_dim);
+  dim3 grid((a.k_max_len + kScoreKeysPerCta - 1) / kScoreKeysPerCta, a.n_kv_heads, a.batch);
+  const int group = a.n_q_heads / a.n_kv_heads;
+  const int ls = logits_stride(a.k_max_len);
+  auto q = static_cast<const __nv_bfloat16 *>(a.twig_q);
+  auto k = static_cast<const __nv_bfloat16 *>(a.twig_k);
+  if (a.head_dim == 128)
+    ttp_logits_kernel<128><<<grid, kScoreThreads, 0, st>>>(q, k, a.ksb, a.ksh, a.ksp, a.k_max_len,
+        a.prefix_len, a.vis_start, a.n_vis, a.n_q_heads, group, a.norm_scope, scale,
+        static_cast<float *>(ws), ls, a.m_max, dev_status);
+  else
+    ttp_logits_kernel<64><<<grid, kScoreThreads, 0, st>>>(q, k, a.ksb, a.ksh, a.ksp, a.k_max_len,
+        a.prefix_len, a.vis_start, a.n_vis, a.n_q_heads, group, a.norm_scope, scale,
+        static_cast<float *>(ws), ls, a.m_max, dev_status);
+  return launch_status();
+}
+
+static twig_status launch_finalize(const float *logits, const ScoreArgs &a, const int *keep,
+                                   int *kept_idx, int r_max, int *dev_status, int mode,
+                                   cudaStream_t st) {
+  static bool attr_set = false;
+  const size_t smem = (size_t)a.m_max * sizeof(uint32_t);
+  if (smem > 48 * 1024 && !attr_set) {
+    if (cudaFuncSetAttribute(ttp_finalize_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             TWIG_MAX_VISUAL * (int)sizeof(uint32_t)) != cudaSuccess)
+      return TWIG_ERR_CUDA;
+    attr_set = true;
+  }
+  ttp_finalize_topk_kernel<<<a.batch, kTopkThreads, smem, st>>>(
+      logits, logits_stride(a.k_max_len), a.n_q_heads, a.k_max_len, a.prefix_len, a.vis_start,
+      a.n_vis, keep, a.norm_scope, a.scores, a.m_max, kept_idx, r_max, dev_status, mode);
+  return launch_status();
+}
+
+static twig_status check_compact_args(const twig_kv *src, const twig_kv *dst, const int *kept_idx,
+                                      int r_max, const int *keep, const int *prefix_len,
+                                      const int *vis_start, const int *n_vis, const int *pos_in,
+                                      int *pos_out, int pos_stride) {
+  twig_status s = check_kv(src);
+  if (s != TWIG_OK) return s;
+  s = check_kv(dst);
+  if (s != TWIG_OK) return s;
+  if (!kept_idx || !keep || !prefix_len || !vis_start || !n_vis) return TWIG_ERR_NULL;
+  if ((pos_in == nullptr) != (pos_out == nullptr)) return TWIG_ERR_NULL;
+  if (r_max <= 0 || (pos_in && pos_stride <= 0)) return TWIG_ERR_SHAPE;
+  if (src->head_dim != dst->head_dim || src->n_layers != dst->n_layers || src->batch != dst->batch ||
+      src->n_kv_heads != dst->n_kv_heads)
+    return TWIG_ERR_SHAPE;
+  if (src->k == dst->k || src->v == dst->v || src->k == dst->v || src->v == dst->k)
+    return TWIG_ERR_UNSUPPORTED;   // in-place compaction is not offered
+  if ((long long)src->n_layers * src->n_kv_heads > 65535) return TWIG_ERR_UNSUPPORTED;
+  return TWIG_OK;
+}
+
+static twig_status launch_gather(const twig_kv *src, const twig_kv *dst, const int *kept_idx, int r_max,
+                                 const int *keep, const int *prefix_len, const int *vis_start,
+                                 const int *n_vis, const int *pos_in, int *pos_out, int pos_stride,
+                                 int *new_len, int *dev_status, cudaStream_t st) {
+  const int rows_bound = src->max_len < dst->max_len ? src->max_len : dst->max_len;
+  dim3 grid((rows_bound + kGatherRows - 1) / kGatherRows, src->n_layers * src->n_kv_heads, src->batch);
+  if (src->head_dim == 128)
+    kv_gather_kernel<128><<<grid, kGatherThreads, 0, st>>>(view_of(src), view_of_mut(dst), kept_idx, r_max,
+        keep, prefix_len, vis_start, n_vis, pos_in, pos_out, pos_stride, new_len, dev_status);
+  else
+    kv_gather_kernel<64><<<grid, kGatherThreads, 0, st>>>(view_of(src), view_of_mut(dst), kept_idx, r_max,
+        keep, prefix_len, vis_start, n_vis, pos_in, pos_out, pos_stride, new_len, dev_status);
+  return launch_status();
+}
+
+}  // namespace twig
+
+using namespace twig;
+
+extern "C" twig_status ttp_score(const void *twig_q, const void *twig_k, int64_t k_stride_batch,
+                                 int64_t k_stride_head, int64_t k_stride_pos, int32_t k_max_len,
+                                 const int32_t *prefix_len, const int32_t *vis_start,
+                                 const int32_t *n_vis, int32_t batch, int32_t n_q_heads,
+                                 int32_t n_kv_heads, int32_t head_dim, int32_t norm_scope,
+                                 float softmax_scale, float *scores, int32_t m_max,
+                                 int32_t *dev_status, void *ws, size_t ws_bytes, void *stream) {
+  ScoreArgs a{twig_q, twig_k, k_stride_batch, k_stride_head, k_stride_pos, k_max_len, prefix_len,
+              vis_start, n_vis, batch, n_q_heads, n_kv_heads, head_dim, norm_scope, softmax_scale,
+              scores, m_max};
+  twig_status s = check_score_args(a, ws, ws_bytes);
+  if (s != TWIG_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  s = launch_logits(a, dev_status, ws, st);
+  if (s != TWIG_OK) return s;
+  return launch_finalize(static_cast<const float *>(ws), a, nullptr, nullptr, 0, dev_status, 1, st);
+}
+
+extern "C" twig_status ttp_topk(const float *scores, const int32_t *n_vis, const int32_t *keep,
+                                int32_t batch, int32_t m_max, int32_t r_max, int32_t *kept_idx,
+                                int32_t *dev_status, void *stream) {
+  if (!scores || !n_vis || !keep || !kept_idx) return TWIG_ERR_NULL;
+  if (batch <= 0 || m_max <= 0 || r_max <= 0) return TWIG_ERR_SHAPE;
+  if (m_max > TWIG_MAX_VISUAL || batch > TWIG_MAX_BATCH) return TWIG_ERR_UNSUPPORTED;
+  ScoreArgs a{};
+  a.n_vis = n_vis;
+  a.batch = batch;
+  a.scores = const_cast<float *>(scores);
+  a.m_max = m_max;
+  a.k_max_len = 1;
+  return launch_finalize(nullptr, a, keep, kept_idx, r_max, dev_status, 2,
+                         static_cast<cudaStream_t>(stream));
+}
+
+extern "C" twig_status ttp_compact(const twig_kv *src, const twig_kv *dst, const int32_t *kept_idx,
+                                   int32_t r_max, const int32_t *keep, const int32_t *prefix_len,
+                                   const int32_t *vis_start, const int32_t *n_vis,
+                                   const int32_t *pos_in, int32_t *pos_out, int32_t pos_stride,
+                                   int32_t *new_len, int32_t *dev_status, void *stream) {
+  twig_status s = check_compact_args(src, dst, kept_idx, r_max, keep, prefix_len, vis_start, n_vis,
+                                     pos_in, pos_out, pos_stride);
+  if (s != TWIG_OK) return s;
+  return launch_gather(src, dst, kept_idx, r_max, keep, prefix_len, vis_start, n_vis, pos_in, pos_out,
+                       pos_stride, new_len, dev_status, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" twig_status ttp_score_topk_compact(
+    const void *twig_q, const void *twig_k, int64_t k_stride_batch, int64_t k_stride_head,
+    int64_t k_stride_pos, int32_t k_max_len, const int32_t *prefix_len, const int32_t *vis_start,
+    const int32_t *n_vis, const int32_t *keep, int32_t n_q_heads, int32_t norm_scope,
+    float softmax_scale, float *scores, int32_t m_max, int32_t *kept_idx, int32_t r_max,
+    const twig_kv *src, const twig_kv *dst, const int32_t *pos_in, int32_t *pos_out,
+    int32_t pos_stride, int32_t *new_len, int32_t *dev_status, void *ws, size_t ws_bytes,
+    void *stream) {
+  twig_status s = check_compact_args(src, dst, kept_idx, r_max, keep, prefix_len, vis_start, n_vis,
+                                     pos_in, pos_out, pos_stride);
+  if (s != TWIG_OK) return s;
+  ScoreArgs a{twig_q, twig_k, k_stride_batch, k_stride_head, k_stride_pos, k_max_len, prefix_len,
+              vis_start, n_vis, src->batch, n_q_heads, src->n_kv_heads, src->head_dim, norm_scope,
+              softmax_scale, scores, m_max};
+  s = check_score_args(a, ws, ws_bytes);
+  if (s != TWIG_OK) return s;
+  if (k_max_len > src->max_len) return TWIG_ERR_SHAPE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  s = launch_logits(a, dev_status, ws, st);
+  if (s != TWIG_OK) return s;
+  s = launch_finalize(static_cast<const float *>(ws), a, keep, kept_idx, r_max, dev_status, 3, st);
+  if (s != TWIG_OK) return s;
+  return launch_gather(src, dst, kept_idx, r_max, keep, prefix_len, vis_start, n_vis, pos_in, pos_out,
+                       pos_stride, new_len, dev_status, st);
+}

@@ -1,0 +1,155 @@
+"""ctypes binding of libtwig.so: the same entry points as include/twig.h.
+
+Argument marshalling only.  Tensors are torch CUDA tensors (torch supplies the
+device memory and the stream); every step of the path runs in the library's
+kernels.  There is no fallback: if the library is missing this module raises
+at import, and a non-zero status raises ``TwigError``.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+from . import build as _build
+
+_LIB_PATH = _build.LIB
+if not os.path.exists(_LIB_PATH):
+    raise ImportError(
+        f"{_LIB_PATH} is missing: build it with `python -m paper_2503_14075_b200.build` "
+        "(nvcc, sm_100a); there is no CPU fallback")
+_lib = C.CDLL(_LIB_PATH)
+
+STATUS_NAMES = {0: "TWIG_OK", 1: "TWIG_ERR_NULL", 2: "TWIG_ERR_SHAPE", 3: "TWIG_ERR_UNSUPPORTED",
+                4: "TWIG_ERR_WORKSPACE", 5: "TWIG_ERR_CUDA", 6: "TWIG_ERR_ALIGN"}
+DEV_OK, DEV_BAD_LAYOUT, DEV_BAD_KEEP, DEV_BAD_INDEX, DEV_BAD_TREE, DEV_OVERFLOW = range(6)
+MAX_NODES, MAX_VISUAL, MAX_BATCH = 64, 16384, 4096
+
+EXPORTS = ["twig_status_str", "twig_workspace_bytes", "ttp_score", "ttp_topk", "ttp_compact",
+           "ttp_score_topk_compact", "tree_verify_attention", "tree_accept_compact"]
+
+
+class TwigError(RuntimeError):
+    def __init__(self, code: int):
+        self.code = code
+        super().__init__(f"{STATUS_NAMES.get(code, code)}: {_lib.twig_status_str(code).decode()}")
+
+
+class KV(C.Structure):
+    """Mirror of ``twig_kv`` (strides in elements)."""
+    _fields_ = [("k", C.c_void_p), ("v", C.c_void_p),
+                ("stride_layer", C.c_int64), ("stride_batch", C.c_int64),
+                ("stride_head", C.c_int64), ("stride_pos", C.c_int64),
+                ("n_layers", C.c_int32), ("batch", C.c_int32), ("n_kv_heads", C.c_int32),
+                ("head_dim", C.c_int32), ("max_len", C.c_int32)]
+
+    @classmethod
+    def of(cls, k: torch.Tensor, v: torch.Tensor) -> "KV":
+        """k, v: [n_layers, batch, n_kv_heads, max_len, head_dim] bf16 CUDA tensors."""
+        assert k.dim() == 5 and k.shape == v.shape and k.stride() == v.stride() and k.stride(4) == 1
+        kv = cls(k.data_ptr(), v.data_ptr(), k.stride(0), k.stride(1), k.stride(2), k.stride(3),
+                 k.shape[0], k.shape[1], k.shape[2], k.shape[4], k.shape[3])
+        kv._keep = (k, v)
+        return kv
+
+
+_vp, _i32, _i64, _f32, _sz = C.c_void_p, C.c_int32, C.c_int64, C.c_float, C.c_size_t
+_kvp = C.POINTER(KV)
+_lib.twig_status_str.restype = C.c_char_p
+_lib.twig_status_str.argtypes = [C.c_int]
+_lib.twig_workspace_bytes.restype = _sz
+_lib.twig_workspace_bytes.argtypes = [_i32] * 5
+_lib.ttp_score.restype = C.c_int
+_lib.ttp_score.argtypes = [_vp, _vp, _i64, _i64, _i64, _i32, _vp, _vp, _vp, _i32, _i32, _i32, _i32, _i32,
+                           _f32, _vp, _i32, _vp, _vp, _sz, _vp]
+_lib.ttp_topk.restype = C.c_int
+_lib.ttp_topk.argtypes = [_vp, _vp, _vp, _i32, _i32, _i32, _vp, _vp, _vp]
+_lib.ttp_compact.restype = C.c_int
+_lib.ttp_compact.argtypes = [_kvp, _kvp, _vp, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _vp]
+_lib.ttp_score_topk_compact.restype = C.c_int
+_lib.ttp_score_topk_compact.argtypes = [_vp, _vp, _i64, _i64, _i64, _i32, _vp, _vp, _vp, _vp, _i32, _i32,
+                                        _f32, _vp, _i32, _vp, _i32, _kvp, _kvp, _vp, _vp, _i32, _vp, _vp,
+                                        _vp, _sz, _vp]
+_lib.tree_verify_attention.restype = C.c_int
+_lib.tree_verify_attention.argtypes = [_vp, _vp, _vp, _kvp, _i32, _vp, _vp, _vp, _i32, _i32, _f32, _vp, _vp,
+                                       _vp, _vp, _sz, _vp]
+_lib.tree_accept_compact.restype = C.c_int
+_lib.tree_accept_compact.argtypes = [_vp, _vp, _vp, _vp, _i32, _i32, _vp, _vp, _kvp, _vp, _vp, _vp, _vp,
+                                     _vp, _vp]
+
+
+def _p(t):
+    return None if t is None else t.data_ptr()
+
+
+def _stream(stream=None):
+    return (stream or torch.cuda.current_stream()).cuda_stream
+
+
+def _check(code: int):
+    if code != 0:
+        raise TwigError(code)
+
+
+def lib_path() -> str:
+    return _LIB_PATH
+
+
+def twig_workspace_bytes(batch, n_q_heads, head_dim, max_len, max_nodes) -> int:
+    return int(_lib.twig_workspace_bytes(batch, n_q_heads, head_dim, max_len, max_nodes))
+
+
+def ttp_score(twig_q, twig_k, prefix_len, vis_start, n_vis, scores, ws, norm_scope=0,
+              softmax_scale=0.0, dev_status=None, stream=None):
+    """twig_q [B,Hq,d], twig_k [B,Hkv,Lmax,d] bf16; scores [B,m_max] fp32 (out)."""
+    B, Hq, d = twig_q.shape
+    _check(_lib.ttp_score(_p(twig_q), _p(twig_k), twig_k.stride(0), twig_k.stride(1), twig_k.stride(2),
+                          twig_k.shape[2], _p(prefix_len), _p(vis_start), _p(n_vis), B, Hq,
+                          twig_k.shape[1], d, norm_scope, softmax_scale, _p(scores), scores.shape[1],
+                          _p(dev_status), _p(ws), ws.numel() * ws.element_size(), _stream(stream)))
+
+
+def ttp_topk(scores, n_vis, keep, kept_idx, dev_status=None, stream=None):
+    """scores [B,m_max] fp32; kept_idx [B,r_max] int32 (out, ascending, -1 padded)."""
+    _check(_lib.ttp_topk(_p(scores), _p(n_vis), _p(keep), scores.shape[0], scores.shape[1],
+                         kept_idx.shape[1], _p(kept_idx), _p(dev_status), _stream(stream)))
+
+
+def ttp_compact(src: KV, dst: KV, kept_idx, keep, prefix_len, vis_start, n_vis, pos_in=None,
+                pos_out=None, new_len=None, dev_status=None, stream=None):
+    pos_stride = pos_in.shape[1] if pos_in is not None else 0
+    _check(_lib.ttp_compact(C.byref(src), C.byref(dst), _p(kept_idx), kept_idx.shape[1], _p(keep),
+                            _p(prefix_len), _p(vis_start), _p(n_vis), _p(pos_in), _p(pos_out),
+                            pos_stride, _p(new_len), _p(dev_status), _stream(stream)))
+
+
+def ttp_score_topk_compact(twig_q, twig_k, prefix_len, vis_start, n_vis, keep, scores, kept_idx,
+                           src: KV, dst: KV, ws, pos_in=None, pos_out=None, new_len=None,
+                           norm_scope=0, softmax_scale=0.0, dev_status=None, stream=None):
+    pos_stride = pos_in.shape[1] if pos_in is not None else 0
+    _check(_lib.ttp_score_topk_compact(
+        _p(twig_q), _p(twig_k), twig_k.stride(0), twig_k.stride(1), twig_k.stride(2), twig_k.shape[2],
+        _p(prefix_len), _p(vis_start), _p(n_vis), _p(keep), twig_q.shape[1], norm_scope, softmax_scale,
+        _p(scores), scores.shape[1], _p(kept_idx), kept_idx.shape[1], C.byref(src), C.byref(dst),
+        _p(pos_in), _p(pos_out), pos_stride, _p(new_len), _p(dev_status), _p(ws),
+        ws.numel() * ws.element_size(), _stream(stream)))
+
+
+def tree_verify_attention(q, tree_k, tree_v, cache: KV, layer, kv_len, n_nodes, parent, out, lse=None,
+                          softmax_scale=0.0, dev_status=None, ws=None, stream=None):
+    """q/out [B,T,Hq,d]; tree_k/v [B,Hkv,T,d]; parent [B,T] int32; lse [B,Hq,T] fp32 or None."""
+    B, T, Hq, d = q.shape
+    ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
+    _check(_lib.tree_verify_attention(_p(q), _p(tree_k), _p(tree_v), C.byref(cache), layer, _p(kv_len),
+                                      _p(n_nodes), _p(parent), T, Hq, softmax_scale, _p(out), _p(lse),
+                                      _p(dev_status), _p(ws), ws_bytes, _stream(stream)))
+
+
+def tree_accept_compact(parent, draft_tok, base_argmax, n_nodes, tree_k_all, tree_v_all, cache: KV,
+                        kv_len, accept_len, path, bonus_tok, dev_status=None, stream=None):
+    """tree_k_all/v_all [Nl,B,Hkv,T,d]; path [B,d_max] int32 (out)."""
+    _check(_lib.tree_accept_compact(_p(parent), _p(draft_tok), _p(base_argmax), _p(n_nodes),
+                                    parent.shape[1], path.shape[1], _p(tree_k_all), _p(tree_v_all),
+                                    C.byref(cache), _p(kv_len), _p(accept_len), _p(path), _p(bonus_tok),
+                                    _p(dev_status), _stream(stream)))

@@ -1,0 +1,177 @@
+"""GPU parity: tree-masked verification attention against the oracle."""
+import zlib
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import twig_oracle as O
+from paper_2503_14075_b200 import synth
+from gpu_common import (DEV, MAX_ABS_TOL, REL_L2_TOL, dev_bf16, dev_i32, f64, host_bits, max_abs,
+                        rel_l2_rows)
+
+pytestmark = pytest.mark.gpu
+CANARY = 0x7FC1          # a bf16 NaN pattern: untouched rows are recognisable, stray reads poison
+
+
+@pytest.fixture(scope="module")
+def tw():
+    from paper_2503_14075_b200 import twig
+    return twig
+
+
+def run_attention(tw, wl, ver, cache_k, cache_v, kv_len, layer=0, max_len=None, lse=True):
+    """cache_k/v: uint16 [Nl,B,Hkv,Lmax,d].  Returns (out bits [B,T,Hq,d], lse [B,Hq,T], status)."""
+    B, T, Hq, d = ver["q"].shape[1:]
+    ck, cv = dev_bf16(cache_k), dev_bf16(cache_v)
+    out = torch.zeros((B, T, Hq, d), dtype=torch.int16, device=DEV)
+    out.fill_(CANARY)
+    out = out.view(torch.bfloat16)
+    lse_t = torch.full((B, Hq, T), -123.0, dtype=torch.float32, device=DEV) if lse else None
+    status = torch.zeros(B, dtype=torch.int32, device=DEV)
+    tw.tree_verify_attention(dev_bf16(ver["q"][layer]), dev_bf16(ver["tree_k"][layer]), dev_bf16(ver["tree_v"][layer]),
+                             tw.KV.of(ck, cv), layer, dev_i32(kv_len), dev_i32(ver["n_nodes"]), dev_i32(ver["parent"]),
+                             out, lse=lse_t, dev_status=status)
+    torch.cuda.synchronize()
+    return host_bits(out), (lse_t.cpu().numpy() if lse else None), status.cpu().numpy()
+
+
+def oracle_attention(ver, cache_k, cache_v, kv_len, layer=0, samples=None):
+    return O.tree_attention(f64(ver["q"][layer]), f64(ver["tree_k"][layer]), f64(ver["tree_v"][layer]),
+                            f64(cache_k[layer]), f64(cache_v[layer]), kv_len, ver["n_nodes"], ver["parent"],
+                            samples=samples)
+
+
+def check(got_bits, got_lse, want, want_lse, n_nodes, tag=""):
+    got = f64(got_bits)
+    B = got.shape[0]
+    for b in range(B):
+        n = int(n_nodes[b])
+        assert np.all(got_bits[b, n:] == CANARY), tag            # padded nodes are not written
+        if n == 0:
+            continue
+        assert not np.isnan(got[b, :n]).any(), tag
+        assert max_abs(got[b, :n], want[b, :n]) <= MAX_ABS_TOL * max(1.0, np.abs(want[b, :n]).max()), tag
+        assert rel_l2_rows(got[b, :n], want[b, :n]) <= REL_L2_TOL, (tag, rel_l2_rows(got[b, :n], want[b, :n]))
+        if got_lse is not None:
+            assert max_abs(got_lse[b, :, :n], want_lse[b, :, :n]) <= 1e-3 * max(1.0, np.abs(want_lse[b]).max()), tag
+
+
+def _wl(B, Hq, Hkv, d, n_nodes, depth, index=9):
+    return synth.Workload(index, "test", 1, B, Hq, Hkv, d, [0] * B, [0] * B, [0] * B, [0] * B, list(n_nodes),
+                          list(depth), 0.6)
+
+
+SHAPES = [
+    # name, B, Hq, Hkv, d, n_nodes, depth, kv_len
+    ("c1", 1, 4, 4, 64, [8], [3], [64]),
+    ("t1-decode", 2, 4, 4, 128, [1, 1], [1, 1], [130, 1]),
+    ("rows32", 2, 8, 8, 128, [26, 17], [5, 4], [163, 291]),
+    ("rows64", 2, 4, 4, 128, [64, 33], [8, 6], [448, 700]),
+    ("gqa-rows128", 2, 8, 2, 128, [30, 32], [6, 5], [257, 64]),
+    ("gqa7-rows448", 1, 14, 2, 128, [64], [6], [384]),
+    ("d64-rows64", 3, 6, 3, 64, [32, 5, 20], [6, 2, 4], [0, 100, 513]),
+    ("empty-prefix", 1, 4, 4, 128, [9], [4], [0]),
+    ("idle-request", 3, 4, 4, 128, [12, 0, 7], [3, 2, 3], [77, 50, 200]),
+]
+
+
+@pytest.mark.parametrize("shape", SHAPES, ids=[s[0] for s in SHAPES])
+@pytest.mark.parametrize("gain_name", ["timing", "sharp", "sharp4"])
+def test_tree_attention_matches_oracle(tw, shape, gain_name):
+    name, B, Hq, Hkv, d, n_nodes, depth, kv_len = shape
+    gain = {"timing": 1.0, "sharp": d ** 0.5, "sharp4": 2.0 * d ** 0.5}[gain_name]   # logit std 1/d, 1, 4
+    wl = _wl(B, Hq, Hkv, d, n_nodes, depth)
+    rng = synth.rng_for(9, zlib.crc32(name.encode()) % 1000)
+    ver = synth.make_verify_inputs(wl, rng, n_layers=1, gain=gain)
+    max_len = max(kv_len) + 70
+    ck, cv = synth.make_cache(wl, rng, max_len, n_layers=1, gain=gain)
+    for b in range(B):                       # rows past kv_len must never be read
+        ck[0, b, :, kv_len[b]:] = CANARY
+        cv[0, b, :, kv_len[b]:] = CANARY
+    got, lse, status = run_attention(tw, wl, ver, ck, cv, kv_len)
+    assert not status.any()
+    want, want_lse = oracle_attention(ver, ck, cv, np.array(kv_len))
+    check(got, lse, want, want_lse, ver["n_nodes"], name)
+
+
+@pytest.mark.parametrize("kind", ["chain", "star"])
+def test_special_trees(tw, kind):
+    T = 20
+    wl = _wl(2, 4, 4, 128, [T, T], [T, 2])
+    rng = synth.rng_for(9, 77)
+    ver = synth.make_verify_inputs(wl, rng, n_layers=1, gain=128 ** 0.5)
+    ver["parent"][:] = synth.chain_tree(T) if kind == "chain" else synth.star_tree(T)
+    ck, cv = synth.make_cache(wl, rng, 300, n_layers=1, gain=128 ** 0.5)
+    kv_len = [190, 3]
+    got, lse, status = run_attention(tw, wl, ver, ck, cv, kv_len)
+    want, want_lse = oracle_attention(ver, ck, cv, np.array(kv_len))
+    check(got, lse, want, want_lse, ver["n_nodes"], kind)
+
+
+def test_bad_tree_and_overflow_set_status(tw):
+    wl = _wl(4, 4, 4, 128, [6, 6, 6, 6], [3, 3, 3, 3])
+    rng = synth.rng_for(9, 78)
+    ver = synth.make_verify_inputs(wl, rng, n_layers=1)
+    ver["parent"][1, 3] = 3            # parent must be an earlier node
+    ver["parent"][2, 0] = 0            # root must have parent -1
+    ck, cv = synth.make_cache(wl, rng, 64, n_layers=1)
+    got, lse, status = run_attention(tw, wl, ver, ck, cv, [10, 10, 10, 65])
+    assert status.tolist() == [0, tw.DEV_BAD_TREE, tw.DEV_BAD_TREE, tw.DEV_OVERFLOW]
+    assert np.all(got[1:] == CANARY)                                   # skipped requests untouched
+    want, want_lse = oracle_attention(ver, ck, cv, np.array([10, 0, 0, 0]))
+    check(got[:1], lse[:1], want[:1], want_lse[:1], ver["n_nodes"][:1])
+
+
+FULL = [
+    # workload, kv lengths to test (pruned prompt ... final length)
+    (2, [163, 291]),
+    (3, None),
+    (4, [448, 1472]),
+    (5, [384, 8128]),
+]
+
+
+@pytest.mark.parametrize("index,lens", FULL, ids=["c2", "c3", "c4", "c5"])
+def test_full_size_configs(tw, index, lens):
+    """Full-size shapes of the benchmark configurations, one layer, every output row
+    against the oracle (timing distribution), plus sampled rows of a sharp variant."""
+    wl = synth.workload(index)
+    rng = synth.rng_for(index, 11)
+    if lens is None:      # heterogeneous: pruned prompt + part of the generation target
+        lens_list = [[p + g // 2 for p, g in zip(wl.pruned_len, wl.gen_target)]]
+    else:
+        lens_list = [[l] * wl.batch for l in lens]
+    max_len = max(max(l) for l in lens_list) + 64
+    for gain, sampled in ((1.0, False), (wl.head_dim ** 0.5, True)):
+        ver = synth.make_verify_inputs(wl, rng, n_layers=1, gain=gain)
+        ck, cv = synth.make_cache(wl, rng, max_len, n_layers=1, gain=gain)
+        for kv_len in lens_list:
+            got, lse, status = run_attention(tw, wl, ver, ck, cv, kv_len)
+            assert not status.any()
+            if not sampled:
+                want, want_lse = oracle_attention(ver, ck, cv, np.array(kv_len))
+                check(got, lse, want, want_lse, ver["n_nodes"], f"c{index} L={kv_len[0]}")
+            else:
+                srng = np.random.default_rng(index)
+                smp = [(int(srng.integers(wl.batch)), 0, 0)]
+                for _ in range(24):
+                    b = int(srng.integers(wl.batch))
+                    smp.append((b, int(srng.integers(wl.n_nodes[b])), int(srng.integers(wl.n_q_heads))))
+                want, want_lse = O.tree_attention(f64(ver["q"][0]), f64(ver["tree_k"][0]), f64(ver["tree_v"][0]),
+                                                  _F64View(ck[0]), _F64View(cv[0]), np.array(kv_len), ver["n_nodes"],
+                                                  ver["parent"], samples=smp)
+                g = f64(got)
+                for (b, i, h) in smp:
+                    assert rel_l2_rows(g[b, i, h][None], want[b, i, h][None]) <= REL_L2_TOL
+                    assert abs(lse[b, h, i] - want_lse[b, h, i]) <= 1e-3 * max(1.0, abs(want_lse[b, h, i]))
+
+
+class _F64View:
+    """Lazily widens slices of a bf16 bit-pattern array (avoids a full fp64 copy of a big cache)."""
+
+    def __init__(self, bits):
+        self.bits = bits
+
+    def __getitem__(self, idx):
+        return synth.bf16_to_f64(self.bits[idx])
