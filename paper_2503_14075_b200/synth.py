@@ -103,8 +103,8 @@ def random_tree(rng: np.random.Generator, n_nodes: int, depth_levels: int) -> np
     """parent[i] ~ U{j < i : depth(j) < depth_levels-1}; redrawn until the
     tree has exactly ``depth_levels`` levels (root included)."""
     depth_levels = max(2, min(depth_levels, n_nodes))
-    if n_nodes == 1:
-        return np.array([-1], dtype=np.int32)
+    if n_nodes <= 1:
+        return np.full(n_nodes, -1, dtype=np.int32)
     while True:
         parent = np.full(n_nodes, -1, dtype=np.int32)
         dep = np.zeros(n_nodes, dtype=np.int32)
