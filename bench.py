@@ -1,0 +1,617 @@
+#!/usr/bin/env python
+"""Benchmark of the TwigVLM/TwigVLM++ inference hot path on B200.
+
+One bench "step" is one pass of the whole path over one batch of synthetic
+requests: twig-guided pruning of the prompt's KV cache (score, TopR, gather over
+all layers), then the tree-verification loop until every request has emitted its
+target number of tokens (tree attention in each of the layers + acceptance and
+KV append per verify step).  The metric is tree-verify steps per second.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2503_14075_b200 import synth  # noqa: E402
+
+METRIC = "tree_verify_steps_per_s"
+UNIT = "verify steps/s"
+N_ROT = 4          # request replicas visited round-robin so that no launch finds its KV in L2
+POOL = 8           # distinct per-step Q / tree-K/V sets per replica (cycled)
+MAX_STEPS = 110    # bound on verify steps per request
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained"), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.gpu)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, smax, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                smax = float(f[2])
+            except ValueError:
+                continue
+            for name, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": smax,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ----------------------------------------------------------------------------------
+# our arm
+# ----------------------------------------------------------------------------------
+class Replica:
+    """One request of the workload with all of its device buffers."""
+
+    def __init__(self, wl, stream_id, torch, tw, dev, max_len):
+        self.wl = wl
+        rng = synth.rng_for(wl.index, stream_id)
+        B, Hq, Hkv, d, T, nl = wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.t_max, wl.n_layers
+
+        def bf(x):
+            return torch.from_numpy(np.ascontiguousarray(x).view(np.int16)).to(dev).view(torch.bfloat16)
+
+        def i32(x):
+            return torch.from_numpy(np.ascontiguousarray(x, dtype=np.int32)).to(dev)
+
+        pre = synth.make_prefill(wl, rng)
+        self.host_twig = (pre["twig_q"], pre["twig_k"])
+        self.twig_q, self.twig_k = bf(pre["twig_q"]), bf(pre["twig_k"])
+        self.src_k, self.src_v = bf(pre["cache_k"]), bf(pre["cache_v"])
+        del pre["cache_k"], pre["cache_v"]
+        self.prefix_len, self.vis_start = i32(pre["prefix_len"]), i32(pre["vis_start"])
+        self.n_vis, self.keep = i32(pre["n_vis"]), i32(pre["keep"])
+        self.pos_in = i32(pre["pos_ids"])
+        self.pos_out = torch.zeros_like(self.pos_in)
+        self.dst_k = torch.zeros((nl, B, Hkv, max_len, d), dtype=torch.bfloat16, device=dev)
+        self.dst_v = torch.zeros_like(self.dst_k)
+        self.src = tw.KV.of(self.src_k, self.src_v)
+        self.cache = tw.KV.of(self.dst_k, self.dst_v)
+        self.scores = torch.zeros((B, max(wl.n_vis)), dtype=torch.float32, device=dev)
+        self.kept = torch.zeros((B, max(wl.keep)), dtype=torch.int32, device=dev)
+        self.kv_len = torch.zeros(B, dtype=torch.int32, device=dev)
+        self.status = torch.zeros(B, dtype=torch.int32, device=dev)
+        self.ws = torch.empty(tw.twig_workspace_bytes(B, Hq, d, self.twig_k.shape[2], T), dtype=torch.uint8,
+                              device=dev)
+        # verify-step inputs: a pool of Q / tree K,V sets, and token ids for every step
+        self.pool_host, self.q, self.tree_k, self.tree_v = [], [], [], []
+        for _ in range(POOL):
+            ver = synth.make_verify_inputs(wl, rng)
+            self.pool_host.append((ver["q"], ver["tree_k"], ver["tree_v"]))
+            self.q.append(bf(ver["q"]))
+            self.tree_k.append(bf(ver["tree_k"]))
+            self.tree_v.append(bf(ver["tree_v"]))
+        self.parent_host, self.n_nodes_host = ver["parent"], ver["n_nodes"]
+        self.parent, self.n_nodes = i32(ver["parent"]), i32(ver["n_nodes"])
+        draft = np.zeros((MAX_STEPS, B, T), dtype=np.int32)
+        tgt = np.zeros_like(draft)
+        for s in range(MAX_STEPS):
+            for b in range(B):
+                n = wl.n_nodes[b]
+                draft[s, b, :n], tgt[s, b, :n] = synth.draft_and_target_tokens(rng, ver["parent"][b, :n], wl.match_p)
+        self.draft_host, self.tgt_host = draft, tgt
+        self.draft, self.tgt = i32(draft), i32(tgt)
+        self.out = torch.zeros((B, T, Hq, d), dtype=torch.bfloat16, device=dev)
+        self.accept_len = torch.zeros(B, dtype=torch.int32, device=dev)
+        self.path = torch.zeros((B, T), dtype=torch.int32, device=dev)
+        self.bonus = torch.zeros(B, dtype=torch.int32, device=dev)
+        self.n_steps = MAX_STEPS
+
+    def prune(self, tw):
+        tw.ttp_score_topk_compact(self.twig_q, self.twig_k, self.prefix_len, self.vis_start, self.n_vis, self.keep,
+                                  self.scores, self.kept, self.src, self.cache, self.ws, pos_in=self.pos_in,
+                                  pos_out=self.pos_out, new_len=self.kv_len, dev_status=self.status)
+
+    def attention_layers(self, tw, s):
+        slot = s % POOL
+        q, tk, tv = self.q[slot], self.tree_k[slot], self.tree_v[slot]
+        for layer in range(self.wl.n_layers):
+            tw.tree_verify_attention(q[layer], tk[layer], tv[layer], self.cache, layer, self.kv_len, self.n_nodes,
+                                     self.parent, self.out, dev_status=self.status)
+
+    def accept(self, tw, s):
+        slot = s % POOL
+        tw.tree_accept_compact(self.parent, self.draft[s], self.tgt[s], self.n_nodes, self.tree_k[slot],
+                               self.tree_v[slot], self.cache, self.kv_len, self.accept_len, self.path, self.bonus,
+                               dev_status=self.status)
+
+
+def attn_bytes_per_launch(wl, kv_len):
+    """Algorithmic bytes of one tree-attention layer-call: K and V rows of the prefix and
+    of the tree, Q read, O written, parent ids."""
+    tot = 0
+    for b in range(wl.batch):
+        n = wl.n_nodes[b]
+        tot += wl.kv_row_bytes() * (kv_len[b] + n) + 2 * n * wl.n_q_heads * wl.head_dim * 2 + 8 * n
+    return tot
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2503_14075_b200 import build as _build
+    _build.build()
+    from paper_2503_14075_b200 import twig as tw
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+    wl = synth.workload(args.workload)
+    peaks = load_peaks()
+    max_len = ((max(wl.pruned_len) + max(wl.gen_target) + wl.t_max + 8 + 31) // 32) * 32
+
+    reps = [Replica(wl, 100 + rank * N_ROT + r, torch, tw, dev, max_len) for r in range(N_ROT)]
+    stream = torch.cuda.current_stream()
+
+    # ---- dry run: how many verify steps each request needs to emit its target ------------
+    for rp in reps:
+        rp.prune(tw)
+        emitted, s = np.zeros(wl.batch, dtype=np.int64), 0
+        lens = []
+        while s < MAX_STEPS and np.any(emitted < np.asarray(wl.gen_target)):
+            lens.append(rp.kv_len.cpu().numpy().copy())
+            rp.attention_layers(tw, s)
+            rp.accept(tw, s)
+            emitted += rp.accept_len.cpu().numpy() + 1
+            s += 1
+        rp.n_steps, rp.lens, rp.emitted = s, lens, int(emitted.sum())
+        assert not rp.status.cpu().numpy().any(), "device status set"
+    torch.cuda.synchronize()
+    total_verify = sum(rp.n_steps for rp in reps)
+    max_s = max(rp.n_steps for rp in reps)
+    attn_launches = total_verify * wl.n_layers
+    attn_bytes = sum(attn_bytes_per_launch(wl, l) for rp in reps for l in rp.lens) * wl.n_layers
+
+    # ---- CUDA graphs: one per (replica, verify step); each layer stays its own launch ----
+    graphs = None
+    if not args.no_graph:
+        side = torch.cuda.Stream()
+        graphs = [[None] * rp.n_steps for rp in reps]
+        with torch.cuda.stream(side):
+            for r, rp in enumerate(reps):
+                for s in range(rp.n_steps):
+                    g = torch.cuda.CUDAGraph()
+                    with torch.cuda.graph(g, stream=side):
+                        rp.attention_layers(tw, s)
+                        rp.accept(tw, s)
+                    graphs[r][s] = g
+        torch.cuda.synchronize()
+
+    ev_pairs = []
+
+    def one_step(record=False):
+        for rp in reps:
+            rp.prune(tw)
+        for s in range(max_s):
+            for r, rp in enumerate(reps):
+                if s >= rp.n_steps:
+                    continue
+                if record:
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record(stream)
+                if graphs is not None:
+                    graphs[r][s].replay()
+                else:
+                    rp.attention_layers(tw, s)
+                    rp.accept(tw, s)
+                if record:
+                    e1.record(stream)
+                    ev_pairs.append((e0, e1))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        one_step()
+    barrier()
+    sampler = ClockSampler(local)
+    sampler.start()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    t0.record(stream)
+    for _ in range(args.steps):
+        one_step(record=True)
+    t1.record(stream)
+    barrier()
+    clocks = sampler.stop()
+    ms = t0.elapsed_time(t1)
+    if world > 1:
+        tt = torch.tensor([ms], device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        ms = float(tt.item())
+    verify_ms = sum(a.elapsed_time(b) for a, b in ev_pairs)          # attention x layers + accept, per verify step
+    value = total_verify * args.steps * world / (ms * 1e-3)
+
+    # ---- dominant kernel alone: the 32 attention launches of every verify step, timed live ------
+    for rp in reps:
+        rp.prune(tw)
+    att_pairs = []
+    for s in range(max_s):
+        for rp in reps:
+            if s >= rp.n_steps:
+                continue
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            rp.attention_layers(tw, s)
+            e1.record(stream)
+            rp.accept(tw, s)
+            att_pairs.append((e0, e1))
+    torch.cuda.synchronize()
+    att_ms = sum(a.elapsed_time(b) for a, b in att_pairs)
+    att_us_per_launch = att_ms * 1e3 / attn_launches
+    # inside the graph the same launches run back to back; per-launch time there:
+    graph_us_per_launch = verify_ms * 1e3 / (args.steps * total_verify * (wl.n_layers + 1))
+    use_us = min(att_us_per_launch, graph_us_per_launch) if graphs is not None else att_us_per_launch
+    bytes_per_launch = attn_bytes / attn_launches
+    achieved = bytes_per_launch / (use_us * 1e-6) / 1e9
+    roofline = {"kernel": "tree_attn_kernel", "bound": "hbm", "achieved": round(achieved, 1),
+                "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": round(achieved / peaks["hbm_gbs"], 4),
+                "peak_source": peaks["source"], "traffic": None,
+                "bytes_per_launch": int(bytes_per_launch), "us_per_launch": round(use_us, 3),
+                "us_per_launch_direct": round(att_us_per_launch, 3),
+                "us_per_launch_in_graph": round(graph_us_per_launch, 3),
+                "note": "one launch = one layer of one verify step (3.5-5.6 MB): launch-latency sized"}
+
+    # ---- prune latency (the third quantity of the metric) --------------------------------------
+    pr = []
+    for _ in range(3):
+        for rp in reps:
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            rp.prune(tw)
+            e1.record(stream)
+            pr.append((e0, e1))
+    torch.cuda.synchronize()
+    prune_us = statistics.median(a.elapsed_time(b) for a, b in pr) * 1e3
+    prune_bytes = 2 * max(wl.pruned_len) * wl.kv_row_bytes() * wl.n_layers + \
+        wl.n_kv_heads * max(wl.prefix_len) * wl.head_dim * 2
+
+    # ---- end to end through the public API with host buffers -----------------------------------
+    e2e = run_e2e(torch, tw, wl, reps, stream, world, dev, dist if world > 1 else None)
+
+    out = {
+        "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": round(ms / args.steps, 4), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": wl.name, "requests_per_step": N_ROT, "layers": wl.n_layers, "heads": wl.n_q_heads,
+                   "head_dim": wl.head_dim, "tree_nodes": wl.t_max, "prefix": wl.prefix_len[0], "keep": wl.keep[0],
+                   "tokens_per_request": wl.gen_target[0], "verify_steps_per_bench_step": total_verify,
+                   "tokens_emitted_per_bench_step": sum(rp.emitted for rp in reps),
+                   "launch_mode": "direct" if graphs is None else "cuda-graph per verify step, one launch per layer",
+                   "l2": f"inputs larger than L2: {N_ROT} request replicas round-robin, >= {3 * 113} MB touched "
+                         "between two uses of a buffer"},
+        "clocks": clocks, "gpu_launches": args.steps * (3 * N_ROT + total_verify * (wl.n_layers + 1)),
+        "e2e": e2e, "roofline": roofline,
+        "verify_us_per_step": round(verify_ms * 1e3 / (args.steps * total_verify), 2),
+        "ttp_prune_latency_us": round(prune_us, 2),
+        "ttp_prune_gbs": round(prune_bytes / (prune_us * 1e-6) / 1e9, 1),
+        "tokens_per_s": round(sum(rp.emitted for rp in reps) * args.steps * world / (ms * 1e-3), 1),
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        out["cpu_baseline"] = cpu_baseline(wl, reps[0], budget_s=args.cpu_budget)
+    if rank == 0 and world == 1 and args.extra:
+        out["other_kernels"] = extra_rooflines(torch, tw, peaks, dev)
+    if rank == 0:
+        print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def run_e2e(torch, tw, wl, reps, stream, world, dev, dist):
+    """Same loop through the public API, every verify step's inputs (Q, tree K/V of all
+    layers, tree and token ids) copied from pinned host memory and its result (accept
+    length, path, bonus token) read back before the next step.  The prompt's KV cache is
+    device-resident state, like the model weights."""
+    rp = reps[0]
+    pin = []
+    for (q, tk, tv) in rp.pool_host:
+        pin.append(tuple(torch.from_numpy(np.ascontiguousarray(x).view(np.int16)).pin_memory() for x in (q, tk, tv)))
+    tq_pin = tuple(torch.from_numpy(np.ascontiguousarray(x).view(np.int16)).pin_memory() for x in rp.host_twig)
+    par_pin = torch.from_numpy(rp.parent_host).pin_memory()
+    draft_pin = torch.from_numpy(rp.draft_host).pin_memory()
+    tgt_pin = torch.from_numpy(rp.tgt_host).pin_memory()
+    res_pin = torch.zeros((wl.batch, 2 + wl.t_max), dtype=torch.int32).pin_memory()
+    res_dev = torch.zeros((wl.batch, 2 + wl.t_max), dtype=torch.int32, device=dev)
+    d_q, d_tk, d_tv = (torch.empty_like(rp.q[0]), torch.empty_like(rp.tree_k[0]), torch.empty_like(rp.tree_v[0]))
+    h2d = d2h = 0
+
+    def request():
+        nonlocal h2d, d2h
+        h2d = d2h = 0
+        rp.twig_q.view(torch.int16).copy_(tq_pin[0], non_blocking=True)
+        rp.twig_k.view(torch.int16).copy_(tq_pin[1], non_blocking=True)
+        h2d += tq_pin[0].numel() * 2 + tq_pin[1].numel() * 2
+        rp.prune(tw)
+        for s in range(rp.n_steps):
+            slot = s % POOL
+            d_q.view(torch.int16).copy_(pin[slot][0], non_blocking=True)
+            d_tk.view(torch.int16).copy_(pin[slot][1], non_blocking=True)
+            d_tv.view(torch.int16).copy_(pin[slot][2], non_blocking=True)
+            rp.parent.copy_(par_pin, non_blocking=True)
+            rp.draft[s].copy_(draft_pin[s], non_blocking=True)
+            rp.tgt[s].copy_(tgt_pin[s], non_blocking=True)
+            h2d += 2 * (d_q.numel() + d_tk.numel() + d_tv.numel()) + 4 * 3 * par_pin.numel()
+            for layer in range(wl.n_layers):
+                tw.tree_verify_attention(d_q[layer], d_tk[layer], d_tv[layer], rp.cache, layer, rp.kv_len,
+                                         rp.n_nodes, rp.parent, rp.out, dev_status=rp.status)
+            tw.tree_accept_compact(rp.parent, rp.draft[s], rp.tgt[s], rp.n_nodes, d_tk, d_tv, rp.cache, rp.kv_len,
+                                   rp.accept_len, rp.path, rp.bonus, dev_status=rp.status)
+            res_dev[:, 0] = rp.accept_len
+            res_dev[:, 1] = rp.bonus
+            res_dev[:, 2:] = rp.path
+            res_pin.copy_(res_dev, non_blocking=True)
+            stream.synchronize()               # the host needs the accepted tokens to draft the next tree
+            d2h += res_pin.numel() * 4
+
+    request()
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    n_req = 3
+    t0 = time.perf_counter()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(n_req):
+        request()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms = max(e0.elapsed_time(e1), (time.perf_counter() - t0) * 1e3 * 0.0)
+    if dist is not None:
+        tt = torch.tensor([ms], device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        ms = float(tt.item())
+    return {"value": round(rp.n_steps * n_req * world / (ms * 1e-3), 1), "unit": UNIT,
+            "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+            "note": "per bench step = one request; Q and tree K/V of all layers cross PCIe every verify step"}
+
+
+def extra_rooflines(torch, tw, peaks, dev):
+    """HBM-sized launches of the two bandwidth kernels (the high-resolution configuration):
+    tree attention at KV length 1472 with batch 4, and the pruning gather over 32 layers."""
+    res = {}
+    wl = synth.workload(4)
+    rng = synth.rng_for(4, 500)
+    nl = 8                                   # layers resident at once: 8 x 2 x 50 MB of cache > L2
+    L = wl.final_kv_len
+    B, Hq, Hkv, d, T = wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.t_max
+
+    def bf(x):
+        return torch.from_numpy(np.ascontiguousarray(x).view(np.int16)).to(dev).view(torch.bfloat16)
+
+    ck, cv = synth.make_cache(wl, rng, L + T, n_layers=nl)
+    ck, cv = bf(ck), bf(cv)
+    ver = synth.make_verify_inputs(wl, rng, n_layers=nl)
+    q, tk, tv = bf(ver["q"]), bf(ver["tree_k"]), bf(ver["tree_v"])
+    par = torch.from_numpy(ver["parent"]).to(dev)
+    nn = torch.from_numpy(ver["n_nodes"]).to(dev)
+    kvl = torch.full((B,), L, dtype=torch.int32, device=dev)
+    out = torch.zeros((B, T, Hq, d), dtype=torch.bfloat16, device=dev)
+    cache = tw.KV.of(ck, cv)
+    stream = torch.cuda.current_stream()
+
+    def loop():
+        for layer in range(nl):
+            tw.tree_verify_attention(q[layer], tk[layer], tv[layer], cache, layer, kvl, nn, par, out)
+    for _ in range(3):
+        loop()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    reps = 10
+    e0.record(stream)
+    for _ in range(reps):
+        loop()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    us = e0.elapsed_time(e1) * 1e3 / (reps * nl)
+    by = attn_bytes_per_launch(wl, [L] * B)
+    res["tree_attn_c4_L1472"] = {"bound": "hbm", "bytes_per_launch": by, "us_per_launch": round(us, 2),
+                                 "achieved": round(by / us / 1e3, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                 "frac": round(by / us / 1e3 / peaks["hbm_gbs"], 4)}
+    del ck, cv, cache
+    # pruning gather, 2 layers at a time of the B=4 x 3008-token prompt cache
+    nl = 2
+    pre = synth.make_prefill(wl, rng, n_layers=nl)
+    sk, sv = bf(pre["cache_k"]), bf(pre["cache_v"])
+    dk = torch.zeros((nl, B, Hkv, max(wl.pruned_len) + 8, d), dtype=torch.bfloat16, device=dev)
+    dv = torch.zeros_like(dk)
+    i32 = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(dev)  # noqa: E731
+    kept = np.stack([np.sort(rng.choice(wl.n_vis[b], wl.keep[b], replace=False)) for b in range(B)]).astype(np.int32)
+    args = (tw.KV.of(sk, sv), tw.KV.of(dk, dv), i32(kept), i32(pre["keep"]), i32(pre["prefix_len"]),
+            i32(pre["vis_start"]), i32(pre["n_vis"]))
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    ts = []
+    for it in range(8):
+        flush.fill_(it)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        tw.ttp_compact(*args)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        ts.append(e0.elapsed_time(e1) * 1e3)
+    us = statistics.median(ts[3:])
+    by = 2 * sum(wl.pruned_len) * wl.kv_row_bytes() * nl
+    res["kv_gather_c4_2layers"] = {"bound": "hbm", "bytes_per_launch": by, "us_per_launch": round(us, 2),
+                                   "achieved": round(by / us / 1e3, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                   "frac": round(by / us / 1e3 / peaks["hbm_gbs"], 4), "l2": "flushed between launches"}
+    return res
+
+
+# ----------------------------------------------------------------------------------
+# CPU oracle arm
+# ----------------------------------------------------------------------------------
+def oracle_verify_steps(wl, host, n_steps, n_layers):
+    """Runs the oracle: prune (all `n_layers`), then `n_steps` verify steps.  Returns seconds
+    spent in the verify steps and in the prune."""
+    from oracle import twig_oracle as O
+    f64 = synth.bf16_to_f64
+    pre, vers, draft, tgt = host["pre"], host["vers"], host["draft"], host["tgt"]
+    B, Hkv, d, T = wl.batch, wl.n_kv_heads, wl.head_dim, wl.t_max
+    max_len = max(wl.pruned_len) + n_steps * T + 8
+    t0 = time.perf_counter()
+    s = O.ttp_scores(f64(pre["twig_q"]), f64(pre["twig_k"]), pre["prefix_len"], pre["vis_start"], pre["n_vis"])
+    kept = [O.topk_lowest_index(s[b, :wl.n_vis[b]], wl.keep[b]).tolist() for b in range(B)]
+    ck = np.zeros((n_layers, B, Hkv, max_len, d), dtype=np.uint16)
+    cv = ck.copy()
+    pos = np.zeros_like(pre["pos_ids"])
+    kv_len = O.gather_compact(pre["cache_k"][:n_layers], pre["cache_v"][:n_layers], pre["pos_ids"], pre["prefix_len"],
+                              pre["vis_start"], pre["n_vis"], kept, ck, cv, pos)
+    t_prune = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    for st in range(n_steps):
+        ver = vers[st % len(vers)]
+        for layer in range(n_layers):
+            O.tree_attention(f64(ver["q"][layer]), f64(ver["tree_k"][layer]), f64(ver["tree_v"][layer]),
+                             f64(ck[layer]), f64(cv[layer]), kv_len, ver["n_nodes"], ver["parent"])
+        paths = []
+        for b in range(B):
+            _, p, _ = O.tree_accept(ver["parent"][b], draft[st][b], tgt[st][b], wl.n_nodes[b])
+            paths.append(p.tolist())
+        kv_len = O.accept_compact(ver["tree_k"][:n_layers], ver["tree_v"][:n_layers], ck, cv, kv_len, paths)
+    return time.perf_counter() - t0, t_prune
+
+
+def oracle_host_inputs(wl, n_pool=2, n_tok=16, stream_id=100):
+    rng = synth.rng_for(wl.index, stream_id)
+    pre = synth.make_prefill(wl, rng)
+    vers = [synth.make_verify_inputs(wl, rng) for _ in range(n_pool)]
+    draft, tgt = [], []
+    for _ in range(n_tok):
+        dd = np.zeros((wl.batch, wl.t_max), dtype=np.int32)
+        tt = np.zeros_like(dd)
+        for b in range(wl.batch):
+            n = wl.n_nodes[b]
+            dd[b, :n], tt[b, :n] = synth.draft_and_target_tokens(rng, vers[0]["parent"][b, :n], wl.match_p)
+        draft.append(dd)
+        tgt.append(tt)
+    return {"pre": pre, "vers": vers, "draft": draft, "tgt": tgt}
+
+
+def cpu_baseline(wl, rep0, budget_s=20.0):
+    """The oracle as it stands, single-threaded, on a bounded sample: the first verify steps of
+    one request (every layer each)."""
+    from threadpoolctl import threadpool_limits
+    host = oracle_host_inputs(wl)
+    with threadpool_limits(limits=1):
+        t1, _ = oracle_verify_steps(wl, host, 1, wl.n_layers)
+        n = int(max(1, min(16, budget_s / max(t1, 1e-3))))
+        tn, t_prune = oracle_verify_steps(wl, host, n, wl.n_layers)
+    return {"value": round(n / tn, 3), "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": f"first {n} verify steps of one request, all {wl.n_layers} layers each (numpy fp64, 1 thread); "
+                      f"oracle prune of the same request took {t_prune:.2f} s",
+            "host_cores_available": os.cpu_count()}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from threadpoolctl import threadpool_limits
+    wl = synth.workload(args.workload)
+    host = oracle_host_inputs(wl)
+    per = 2          # verify steps per timed step (bounded sample)
+    with threadpool_limits(limits=1):
+        for _ in range(min(args.warmup, 1)):
+            oracle_verify_steps(wl, host, 1, wl.n_layers)
+        tot = 0.0
+        k = max(1, min(args.steps, 5))
+        for _ in range(k):
+            t, _ = oracle_verify_steps(wl, host, per, wl.n_layers)
+            tot += t
+    value = per * k / tot
+    sample = f"{per} verify steps (all {wl.n_layers} layers) per step, {k} steps, numpy fp64, 1 thread"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": round(value, 3), "unit": UNIT,
+        "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": k, "warmup": min(args.warmup, 1),
+        "ms_per_step": round(tot / k * 1e3, 2), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic", "config": {"workload": wl.name},
+        "cpu_baseline": {"value": round(value, 3), "unit": UNIT, "kind": "oracle", "cores": 1, "sample": sample},
+        "e2e": {"value": round(value, 3), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", type=int, default=2)
+    ap.add_argument("--no-graph", action="store_true", help="launch every kernel directly instead of graph replay")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extra", dest="extra", action="store_false",
+                    help="skip the HBM-sized launches of the attention and gather kernels")
+    ap.add_argument("--cpu-budget", type=float, default=15.0)
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

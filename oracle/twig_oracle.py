@@ -120,11 +120,16 @@ def gather_compact(src_k, src_v, pos_in, prefix_len, vis_start, n_vis, kept_list
 # O4: tree-masked verification attention (Sec. 5.4, Appendix A, Eq. 2)
 # --------------------------------------------------------------------------
 def ancestors_or_self(parent, i: int):
+    """Root path of node i, root first.  A parent array must have parent[0] = -1
+    and parent[x] in [0, x) for x > 0; anything else is rejected."""
     out = []
     x = int(i)
     while x >= 0:
         out.append(x)
-        x = int(parent[x])
+        p = int(parent[x])
+        if not (-1 <= p < x) or (x == 0) != (p == -1):
+            raise ValueError(f"invalid parent array: parent[{x}] = {p}")
+        x = p
     return out[::-1]
 
 

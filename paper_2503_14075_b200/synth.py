@@ -100,21 +100,23 @@ def fixed_branching_tree(branching: Sequence[int], n_keep: Optional[int] = None)
 
 
 def random_tree(rng: np.random.Generator, n_nodes: int, depth_levels: int) -> np.ndarray:
-    """parent[i] ~ U{j < i : depth(j) < depth_levels-1}; redrawn until the
-    tree has exactly ``depth_levels`` levels (root included)."""
-    depth_levels = max(2, min(depth_levels, n_nodes))
+    """Random tree with exactly ``depth_levels`` levels (root included): nodes
+    0..depth_levels-1 form a spine (a chain), every later node i draws
+    parent[i] ~ U{j < i : depth(j) < depth_levels-1}."""
     if n_nodes <= 1:
         return np.full(n_nodes, -1, dtype=np.int32)
-    while True:
-        parent = np.full(n_nodes, -1, dtype=np.int32)
-        dep = np.zeros(n_nodes, dtype=np.int32)
-        for i in range(1, n_nodes):
+    depth_levels = max(2, min(depth_levels, n_nodes))
+    parent = np.full(n_nodes, -1, dtype=np.int32)
+    dep = np.zeros(n_nodes, dtype=np.int32)
+    for i in range(1, n_nodes):
+        if i < depth_levels:
+            j = i - 1
+        else:
             cand = np.nonzero(dep[:i] < depth_levels - 1)[0]
             j = int(cand[rng.integers(len(cand))])
-            parent[i] = j
-            dep[i] = dep[j] + 1
-        if dep.max() == depth_levels - 1:
-            return parent
+        parent[i] = j
+        dep[i] = dep[j] + 1
+    return parent
 
 
 def draft_and_target_tokens(rng: np.random.Generator, parent: np.ndarray, match_p: float,

@@ -119,8 +119,9 @@ def test_bad_tree_and_overflow_set_status(tw):
     got, lse, status = run_attention(tw, wl, ver, ck, cv, [10, 10, 10, 65])
     assert status.tolist() == [0, tw.DEV_BAD_TREE, tw.DEV_BAD_TREE, tw.DEV_OVERFLOW]
     assert np.all(got[1:] == CANARY)                                   # skipped requests untouched
-    want, want_lse = oracle_attention(ver, ck, cv, np.array([10, 0, 0, 0]))
-    check(got[:1], lse[:1], want[:1], want_lse[:1], ver["n_nodes"][:1])
+    good = {k: (v[:, :1] if k in ("q", "tree_k", "tree_v") else v[:1]) for k, v in ver.items()}
+    want, want_lse = oracle_attention(good, ck[:, :1], cv[:, :1], np.array([10]))      # the valid request only
+    check(got[:1], lse[:1], want, want_lse, good["n_nodes"])
 
 
 FULL = [

@@ -417,6 +417,12 @@ def test_accept_special_cases_and_statistics():
     assert abs(tot / n_trials - want) < 0.03
 
 
+def test_invalid_parent_arrays_are_rejected():
+    for bad in ([0, 0], [-1, 1], [-1, 0, 2], [-1, -1]):
+        with pytest.raises(ValueError):
+            O.ancestors_or_self(np.array(bad), len(bad) - 1)
+
+
 def test_speculative_decoding_is_lossless_with_toy_target():
     """With a deterministic toy target next = f(sequence), draft-tree verification
     must emit exactly the greedy sequence of f, whatever the drafts are."""
