@@ -182,8 +182,8 @@ def attn_bytes_per_launch(wl, kv_len):
     tot = 0
     for b in range(wl.batch):
         n = wl.n_nodes[b]
-        tot += wl.kv_row_bytes() * (kv_len[b] + n) + 2 * n * wl.n_q_heads * wl.head_dim * 2 + 8 * n
-    return tot
+        tot += wl.kv_row_bytes() * (int(kv_len[b]) + n) + 2 * n * wl.n_q_heads * wl.head_dim * 2 + 8 * n
+    return int(tot)
 
 
 def run_ours(args):

@@ -8,8 +8,9 @@
 // (prefix rows followed by the tree's own rows) is cut into tiles; a thread
 // block cluster splits the tiles between its CTAs, every CTA keeps a
 // flash-style running (max, sum, O) per row, and the partial results are
-// merged through distributed shared memory, so nothing but Q, K, V and the
-// final output touches HBM.
+// merged through distributed shared memory (each CTA pushes its per-row partial
+// to the CTA that owns the row), so nothing but Q, K, V and the final output
+// touches HBM.
 #include <cooperative_groups.h>
 
 #include "twig_common.cuh"
@@ -68,32 +69,36 @@ __device__ __forceinline__ uint32_t tile_off(int r, int c) {
   return (uint32_t)((c >> 3) * ROWS * 128 + r * 128 + (((c & 7) ^ (r & 7)) << 4));
 }
 
-template <int D_, int WM_, int WN_, int KC_, int STAGES_>
+template <int D_, int WM_, int WN_, int KC_, int STAGES_, int MIN_CTAS_>
 struct AttnCfg {
-  static constexpr int D = D_, WM = WM_, WN = WN_, KC = KC_, STAGES = STAGES_;
+  static constexpr int D = D_, WM = WM_, WN = WN_, KC = KC_, STAGES = STAGES_, MIN_CTAS = MIN_CTAS_;
   static constexpr int ROWS = 16 * WM;          // query rows per CTA
   static constexpr int KT = KC * WN;            // keys per tile
   static constexpr int THREADS = 32 * WM * WN;
   static constexpr int CPR = D / 8;             // 16-byte chunks per row
   static constexpr int Q_BYTES = ROWS * D * 2;
   static constexpr int TILE_BYTES = KT * D * 2;
-  static constexpr int OD = D + 8;              // padded fp32 row of a partial O
-  static constexpr int PART_BYTES = WN * ROWS * OD * 4;
   static constexpr int STAGE_BYTES = 2 * STAGES * TILE_BYTES;
-  static constexpr int BODY_BYTES = STAGE_BYTES > PART_BYTES ? STAGE_BYTES : PART_BYTES;
-  static constexpr int SMEM_BYTES = Q_BYTES + BODY_BYTES;
+  // after the key loop the stage ring is reused: XCH holds the partial O of the
+  // warps with wn > 0 (fragment order), RECV the per-split partials a CTA owns
+  static constexpr int XCH_BYTES = (WN - 1) * ROWS * D * 4;
+  static constexpr int RECV_BYTES = ROWS * D * 4;
+  static_assert(XCH_BYTES + RECV_BYTES <= STAGE_BYTES, "epilogue buffers must fit in the stage ring");
+  static constexpr int SMEM_BYTES = Q_BYTES + STAGE_BYTES;
 };
 
 template <class C>
-__global__ void __launch_bounds__(C::THREADS)
+__global__ void __launch_bounds__(C::THREADS, C::MIN_CTAS)
 tree_attn_kernel(const AttnParams p) {
-  constexpr int D = C::D, ROWS = C::ROWS, KT = C::KT, KC = C::KC, WN = C::WN, STAGES = C::STAGES;
+  constexpr int D = C::D, ROWS = C::ROWS, KT = C::KT, KC = C::KC, WM = C::WM, WN = C::WN, STAGES = C::STAGES;
   constexpr int NT = KC / 8;       // key n-tiles per warp per tile
   constexpr int DT = D / 8;        // head-dim n-tiles of O
   constexpr int KS = D / 16;       // k-steps of Q K^T
   extern __shared__ __align__(1024) unsigned char smem[];
   __shared__ unsigned long long s_mask[TWIG_MAX_NODES];
-  __shared__ float s_m[WN * ROWS], s_l[WN * ROWS];
+  __shared__ int s_par[TWIG_MAX_NODES];
+  __shared__ float4 s_xml[(WN > 1 ? WN - 1 : 1) * WM * 32];   // (m_lo, m_hi, l_lo, l_hi) of warps wn > 0
+  __shared__ float r_m[ROWS], r_l[ROWS];                       // received (m, l): [sender][owned row]
   __shared__ int s_bad;
 
   cg::cluster_group cluster = cg::this_cluster();
@@ -117,27 +122,6 @@ tree_attn_kernel(const AttnParams p) {
   }
   const int rows_total = n * p.group, row0 = rb * ROWS;
   if (row0 >= rows_total) return;
-  if (tid == 0) s_bad = 0;
-  __syncthreads();
-  const int *par = p.parent + (long long)b * p.t_max;
-  if (tid < n) {
-    const int pr = par[tid];
-    if ((tid == 0) ? (pr != -1) : (pr < 0 || pr >= tid)) s_bad = 1;
-  }
-  __syncthreads();
-  if (s_bad) {
-    if (first) flag_status(p.dev_status, b, TWIG_DEV_BAD_TREE);
-    return;
-  }
-  if (tid < n) {          // ancestor-or-self bitmask; parent[x] < x bounds the walk
-    unsigned long long m = 0;
-    int x = tid;
-    while (x >= 0) {
-      m |= 1ull << x;
-      x = par[x];
-    }
-    s_mask[tid] = m;
-  }
 
   const uint32_t q_s = smem_u32(smem);
   const uint32_t k_s = q_s + C::Q_BYTES;
@@ -180,7 +164,7 @@ tree_attn_kernel(const AttnParams p) {
     }
   };
 
-  // ---- Q tile (zero rows past the request's last row) -------------------------
+  // ---- start the copies first: Q tile (zero rows past the last row) and the first key tiles ----
   {
     constexpr int CHUNKS = ROWS * C::CPR;
 #pragma unroll
@@ -202,16 +186,39 @@ tree_attn_kernel(const AttnParams p) {
     cp_async_commit();        // the first group also carries Q
   }
 
+  // ---- while they fly: parent array -> shared memory, validation, ancestor masks ----
+  if (tid == 0) s_bad = 0;
+  __syncthreads();
+  if (tid < n) {
+    const int pr = p.parent[(long long)b * p.t_max + tid];
+    s_par[tid] = pr;
+    if ((tid == 0) ? (pr != -1) : (pr < 0 || pr >= tid)) s_bad = 1;
+  }
+  __syncthreads();
+  if (s_bad) {
+    if (first) flag_status(p.dev_status, b, TWIG_DEV_BAD_TREE);
+    cp_async_wait<0>();       // nothing may still be writing this CTA's shared memory
+    return;
+  }
+  if (tid < n) {          // ancestor-or-self bitmask; parent[x] < x bounds the walk
+    unsigned long long m = 0;
+    int x = tid;
+    while (x >= 0) {
+      m |= 1ull << x;
+      x = s_par[x];
+    }
+    s_mask[tid] = m;
+  }
+
   // ---- per-thread state --------------------------------------------------------
   const int gq = lane >> 2, tq = lane & 3;
   const int r_lo = wm * 16 + gq, r_hi = r_lo + 8;         // CTA-local rows of this thread
-  uint32_t qf[KS][4];
   float o[DT][4];
 #pragma unroll
   for (int i = 0; i < DT; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
   float m_lo = -INFINITY, m_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;
-  unsigned long long mask_lo = 0, mask_hi = 0;
-  bool q_loaded = false;
+  const uint32_t q_frag = q_s + (wm * 16 + (lane & 7) + ((lane >> 3) & 1) * 8) * 128;   // row base; chunk added per k-step
+  const int q_sw = (lane & 7);           // row & 7 of this lane's ldmatrix row
 
   for (int t = t_begin; t < t_end; ++t) {
     const int it = t - t_begin;
@@ -221,17 +228,6 @@ tree_attn_kernel(const AttnParams p) {
       const int tn = t + STAGES - 1;
       if (tn < t_end) load_tile(tn, (it + STAGES - 1) % STAGES);
       cp_async_commit();
-    }
-    if (!q_loaded) {
-      q_loaded = true;
-#pragma unroll
-      for (int ks = 0; ks < KS; ++ks) {
-        const int r = wm * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
-        ldsm_x4(q_s + tile_off<ROWS>(r, ks * 2 + (lane >> 4)), qf[ks]);
-      }
-      const int g_lo = row0 + r_lo, g_hi = row0 + r_hi;
-      mask_lo = g_lo < rows_total ? s_mask[g_lo / p.group] : 0ull;
-      mask_hi = g_hi < rows_total ? s_mask[g_hi / p.group] : 0ull;
     }
     const int stage = it % STAGES;
     const uint32_t kst = k_s + stage * C::TILE_BYTES, vst = v_s + stage * C::TILE_BYTES;
@@ -243,19 +239,27 @@ tree_attn_kernel(const AttnParams p) {
     for (int i = 0; i < NT; ++i) s[i][0] = s[i][1] = s[i][2] = s[i][3] = 0.f;
 #pragma unroll
     for (int ks = 0; ks < KS; ++ks) {
+      uint32_t qf[4];
+      {
+        const int c = ks * 2 + (lane >> 4);
+        ldsm_x4(q_frag + (c >> 3) * ROWS * 128 + (((c & 7) ^ q_sw) << 4), qf);
+      }
 #pragma unroll
       for (int np = 0; np < NT / 2; ++np) {
         uint32_t kb[4];
         const int key = kbase + np * 16 + (lane & 7) + (lane >> 4) * 8;
         ldsm_x4(kst + tile_off<KT>(key, ks * 2 + ((lane >> 3) & 1)), kb);
-        mma_bf16(s[2 * np], qf[ks], kb[0], kb[1]);
-        mma_bf16(s[2 * np + 1], qf[ks], kb[2], kb[3]);
+        mma_bf16(s[2 * np], qf, kb[0], kb[1]);
+        mma_bf16(s[2 * np + 1], qf, kb[2], kb[3]);
       }
     }
 
     // scale into the exp2 domain; mask the tile that holds the prefix end / the tree
     const int key0 = t * KT + kbase;
     if (key0 + KC > L) {
+      const int g_lo = row0 + r_lo, g_hi = row0 + r_hi;
+      const unsigned long long mask_lo = g_lo < rows_total ? s_mask[g_lo / p.group] : 0ull;
+      const unsigned long long mask_hi = g_hi < rows_total ? s_mask[g_hi / p.group] : 0ull;
 #pragma unroll
       for (int nt = 0; nt < NT; ++nt) {
 #pragma unroll
@@ -325,58 +329,102 @@ tree_attn_kernel(const AttnParams p) {
     }
   }
   cp_async_wait<0>();
-  __syncthreads();            // all warps are done with the stage buffers
+  __syncthreads();            // all warps are done with the stage ring; it is reused below
 
-  // ---- this warp's partial (m, l, O) -> shared memory ---------------------------
   l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1);
   l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
   l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1);
   l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
-  float *part = reinterpret_cast<float *>(smem + C::Q_BYTES);
-  {
-    float *po_lo = part + ((size_t)wn * ROWS + r_lo) * C::OD, *po_hi = part + ((size_t)wn * ROWS + r_hi) * C::OD;
+
+  // ---- merge the WN key-slices inside the CTA: warps wn > 0 hand their fragments to wn == 0 ----
+  float4 *xch = reinterpret_cast<float4 *>(smem + C::Q_BYTES);
+  if (WN > 1) {
+    if (wn > 0) {
+      float4 *dst = xch + ((size_t)((wn - 1) * WM + wm) * DT) * 32 + lane;
 #pragma unroll
-    for (int i = 0; i < DT; ++i) {
-      *reinterpret_cast<float2 *>(po_lo + i * 8 + tq * 2) = make_float2(o[i][0], o[i][1]);
-      *reinterpret_cast<float2 *>(po_hi + i * 8 + tq * 2) = make_float2(o[i][2], o[i][3]);
+      for (int i = 0; i < DT; ++i) dst[i * 32] = make_float4(o[i][0], o[i][1], o[i][2], o[i][3]);
+      s_xml[((wn - 1) * WM + wm) * 32 + lane] = make_float4(m_lo, m_hi, l_lo, l_hi);
     }
-    if (tq == 0) {
-      s_m[wn * ROWS + r_lo] = m_lo;
-      s_l[wn * ROWS + r_lo] = l_lo;
-      s_m[wn * ROWS + r_hi] = m_hi;
-      s_l[wn * ROWS + r_hi] = l_hi;
+    __syncthreads();
+    if (wn == 0) {
+#pragma unroll
+      for (int w = 1; w < WN; ++w) {
+        const float4 ml = s_xml[((w - 1) * WM + wm) * 32 + lane];
+        const float mn_lo = fmaxf(m_lo, ml.x), mn_hi = fmaxf(m_hi, ml.y);
+        const float use_lo = mn_lo == -INFINITY ? 0.f : mn_lo, use_hi = mn_hi == -INFINITY ? 0.f : mn_hi;
+        const float a_lo = exp2f(m_lo - use_lo), a_hi = exp2f(m_hi - use_hi);
+        const float b_lo = exp2f(ml.x - use_lo), b_hi = exp2f(ml.y - use_hi);
+        m_lo = mn_lo;
+        m_hi = mn_hi;
+        l_lo = l_lo * a_lo + ml.z * b_lo;
+        l_hi = l_hi * a_hi + ml.w * b_hi;
+        const float4 *src = xch + ((size_t)((w - 1) * WM + wm) * DT) * 32 + lane;
+#pragma unroll
+        for (int i = 0; i < DT; ++i) {
+          const float4 v = src[i * 32];
+          o[i][0] = o[i][0] * a_lo + v.x * b_lo;
+          o[i][1] = o[i][1] * a_lo + v.y * b_lo;
+          o[i][2] = o[i][2] * a_hi + v.z * b_hi;
+          o[i][3] = o[i][3] * a_hi + v.w * b_hi;
+        }
+      }
     }
   }
-  cluster.sync();
 
-  // ---- merge the n_splits * WN partials; this CTA finishes a slice of the rows ---
+  // ---- merge the key splits of the cluster ------------------------------------------
+  // Every CTA owns ROWS / n_splits rows.  Once all CTAs have left their key loops (first
+  // cluster barrier) each one writes its per-row partial (m, l, O) into the owner's shared
+  // memory; after the second barrier the owner combines its n_splits partials and stores.
+  const int rows_per = ROWS / n_splits;
+  float *recv = reinterpret_cast<float *>(smem + C::Q_BYTES + C::XCH_BYTES);
+  if (n_splits > 1) cluster.sync();
+  if (wn == 0) {
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+      const int r = half ? r_hi : r_lo;
+      const int owner = r / rows_per, lr = r % rows_per;
+      const int slot = split * rows_per + lr;
+      float *ro = recv + (size_t)slot * D, *rm = r_m + slot, *rl = r_l + slot;
+      if (n_splits > 1) {
+        ro = cluster.map_shared_rank(ro, owner);
+        rm = cluster.map_shared_rank(rm, owner);
+        rl = cluster.map_shared_rank(rl, owner);
+      }
+#pragma unroll
+      for (int i = 0; i < DT; ++i)     // 8-float groups are XOR-swizzled by the row to spread banks
+        *reinterpret_cast<float2 *>(ro + ((i ^ (lr & 7)) << 3) + tq * 2) =
+            half ? make_float2(o[i][2], o[i][3]) : make_float2(o[i][0], o[i][1]);
+      if (tq == 0) {
+        *rm = half ? m_hi : m_lo;
+        *rl = half ? l_hi : l_lo;
+      }
+    }
+  }
+  if (n_splits > 1) cluster.sync(); else __syncthreads();
+
   {
     constexpr int TPR = D / 4;                        // threads per row, 4 floats each
     constexpr int RPP = C::THREADS / TPR;             // rows per pass
-    const int rows_per = (ROWS + n_splits - 1) / n_splits;
-    const int r_begin = split * rows_per, r_end = min(ROWS, r_begin + rows_per);
     const int c4 = (tid % TPR) * 4;
-    for (int r = r_begin + tid / TPR; r < r_end; r += RPP) {
-      const int gr = row0 + r;
+    for (int lr = tid / TPR; lr < rows_per; lr += RPP) {
+      const int gr = row0 + split * rows_per + lr;
       if (gr >= rows_total) continue;
+      float mv[8];
       float mstar = -INFINITY;
-      for (int cta = 0; cta < n_splits; ++cta) {
-        const float *rm = cluster.map_shared_rank(s_m, cta);
 #pragma unroll
-        for (int w = 0; w < WN; ++w) mstar = fmaxf(mstar, rm[w * ROWS + r]);
+      for (int sd = 0; sd < 8; ++sd) {
+        mv[sd] = sd < n_splits ? r_m[sd * rows_per + lr] : -INFINITY;
+        mstar = fmaxf(mstar, mv[sd]);
       }
       float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
       float lsum = 0.f;
-      for (int cta = 0; cta < n_splits; ++cta) {
-        const float *rm = cluster.map_shared_rank(s_m, cta);
-        const float *rl = cluster.map_shared_rank(s_l, cta);
-        const float *ro = cluster.map_shared_rank(part, cta);
+      const int col = (((c4 >> 3) ^ (lr & 7)) << 3) + (c4 & 7);
 #pragma unroll
-        for (int w = 0; w < WN; ++w) {
-          const float wgt = exp2f(rm[w * ROWS + r] - mstar);
-          if (wgt == 0.f) continue;
-          lsum = fmaf(wgt, rl[w * ROWS + r], lsum);
-          const float4 v = *reinterpret_cast<const float4 *>(ro + ((size_t)w * ROWS + r) * C::OD + c4);
+      for (int sd = 0; sd < 8; ++sd) {
+        if (sd < n_splits) {
+          const float wgt = exp2f(mv[sd] - mstar);
+          lsum = fmaf(wgt, r_l[sd * rows_per + lr], lsum);
+          const float4 v = *reinterpret_cast<const float4 *>(recv + (size_t)(sd * rows_per + lr) * D + col);
           acc.x = fmaf(wgt, v.x, acc.x);
           acc.y = fmaf(wgt, v.y, acc.y);
           acc.z = fmaf(wgt, v.z, acc.z);
@@ -394,7 +442,6 @@ tree_attn_kernel(const AttnParams p) {
         p.lse[((long long)b * p.n_q_heads + h) * p.t_max + node] = (mstar + log2f(lsum)) * 0.6931471805599453f;
     }
   }
-  cluster.sync();             // keep this CTA's shared memory alive until every peer has read it
 }
 
 // ---------------------------------------------------------------------------
@@ -433,10 +480,10 @@ static int pick_splits(int items, int max_tiles) {
 
 template <int D>
 static twig_status dispatch_attn(AttnParams &p, int batch, int rows, cudaStream_t st) {
-  using C16 = AttnCfg<D, 1, 4, 16, 3>;
-  using C32 = AttnCfg<D, 2, 4, 16, 3>;
-  using C64 = AttnCfg<D, 4, 2, 32, 3>;
-  using C128 = AttnCfg<D, 8, 1, 64, 3>;
+  using C16 = AttnCfg<D, 1, 4, 16, 3, 2>;
+  using C32 = AttnCfg<D, 2, 4, 16, 3, 2>;
+  using C64 = AttnCfg<D, 4, 2, 32, 2, 2>;
+  using C128 = AttnCfg<D, 8, 1, 64, 2, 1>;
   const int rows_per_cta = rows <= 16 ? 16 : rows <= 32 ? 32 : rows <= 64 ? 64 : 128;
   p.row_blocks = (rows + rows_per_cta - 1) / rows_per_cta;
   if ((long long)p.n_kv_heads * p.row_blocks > 65535) return TWIG_ERR_UNSUPPORTED;

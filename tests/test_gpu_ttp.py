@@ -238,7 +238,8 @@ def test_fused_prune_matches_stage_chain(tw, name, scope):
         assert np.array_equal(kept.cpu().numpy()[b, :r], want_idx)
         kept_lists.append(want_idx.tolist())
         full = set(O.topk_lowest_index(want_s[b, :m], r).tolist())
-        overlap.append(len(full & set(want_idx.tolist())) / max(1, r))
+        if r > 0:
+            overlap.append(len(full & set(want_idx.tolist())) / r)
     ok = np.zeros((nl, B, Hkv, dst_len, d), dtype=np.uint16)
     ov = ok.copy()
     opos = np.full((B, lmax), -1, dtype=np.int32)
