@@ -102,6 +102,35 @@ twig_status ttp_score(const void *twig_q, const void *twig_k, int64_t k_stride_b
                       int32_t norm_scope, float softmax_scale, float *scores, int32_t m_max,
                       int32_t *dev_status, void *ws, size_t ws_bytes, void *stream);
 
+/* ---- ttp_score without any caller-provided or allocated scratch --------------
+ * (No counterpart in the paper: this is a deployment convenience.)
+ * Some hosts of this library may not allocate device memory at the point where
+ * they prune: a serving process that handed all device memory to its own pool
+ * at start-up, a plugin that is given tensors and a stream but no allocator, a
+ * latency-critical loop that must stay clear of cudaMalloc because it
+ * synchronises the device.  For them this variant of ttp_score keeps the fp32
+ * logits scratch in a fixed array inside the library image,
+ * TWIG_NOALLOC_SCRATCH_BYTES long; every GPU that loads the library holds that
+ * much memory until the process exits.  Same arguments, results and errors as
+ * ttp_score, minus ws / ws_bytes; it calls no allocator of any kind.
+ * Limit: batch * n_q_heads * round_up(k_max_len, 4) * 4 bytes must fit in the
+ * array, otherwise TWIG_ERR_WORKSPACE is returned and nothing is launched.
+ * The first call on each device looks up the array's device address (with that
+ * device current); make that first call outside any stream capture.
+ * All calls on a device share the one array.  It keeps the previous call's
+ * logits, which is harmless (each call overwrites what it reads), but two calls
+ * whose kernels overlap on the GPU (different streams) race on it: serialise
+ * them, or give the concurrent ones their own scratch through ttp_score.
+ */
+#define TWIG_NOALLOC_SCRATCH_BYTES (4u << 20)
+twig_status ttp_score_noalloc(const void *twig_q, const void *twig_k, int64_t k_stride_batch,
+                              int64_t k_stride_head, int64_t k_stride_pos, int32_t k_max_len,
+                              const int32_t *prefix_len, const int32_t *vis_start,
+                              const int32_t *n_vis, int32_t batch, int32_t n_q_heads,
+                              int32_t n_kv_heads, int32_t head_dim, int32_t norm_scope,
+                              float softmax_scale, float *scores, int32_t m_max,
+                              int32_t *dev_status, void *stream);
+
 /* ---- TTP stage 2: TopR of Eq. 3 --------------------------------------------
  * kept_idx[b, 0..keep[b]) = indices of the keep[b] largest scores[b, 0..n_vis[b]),
  * equal scores resolved to the LOWER index, written in ascending index order

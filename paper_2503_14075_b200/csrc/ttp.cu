@@ -461,6 +461,54 @@ extern "C" twig_status ttp_score(const void *twig_q, const void *twig_k, int64_t
   return launch_finalize(static_cast<const float *>(ws), a, nullptr, nullptr, 0, dev_status, 1, st);
 }
 
+// ---------------------------------------------------------------------------
+// ttp_score for callers that cannot allocate device memory: the logits scratch is
+// a fixed array that lives in the library image on every device that loads it.
+// ---------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char g_noalloc_scratch[TWIG_NOALLOC_SCRATCH_BYTES];
+
+// In host code `g_noalloc_scratch` is only a handle; the device address has to be asked
+// for, once per device, with that device current.
+static twig_status noalloc_scratch_address(void **out) {
+  constexpr int kMaxDevices = 64;
+  static void *addr[kMaxDevices] = {};
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return TWIG_ERR_CUDA;
+  if (!addr[dev]) {
+    void *p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || !p) return TWIG_ERR_CUDA;
+    addr[dev] = p;
+  }
+  *out = addr[dev];
+  return TWIG_OK;
+}
+
+extern "C" twig_status ttp_score_noalloc(const void *twig_q, const void *twig_k, int64_t k_stride_batch,
+                                         int64_t k_stride_head, int64_t k_stride_pos, int32_t k_max_len,
+                                         const int32_t *prefix_len, const int32_t *vis_start,
+                                         const int32_t *n_vis, int32_t batch, int32_t n_q_heads,
+                                         int32_t n_kv_heads, int32_t head_dim, int32_t norm_scope,
+                                         float softmax_scale, float *scores, int32_t m_max,
+                                         int32_t *dev_status, void *stream) {
+  if (batch > 0 && n_q_heads > 0 && k_max_len > 0 &&
+      score_workspace_bytes(batch, n_q_heads, k_max_len) > (size_t)TWIG_NOALLOC_SCRATCH_BYTES)
+    return TWIG_ERR_WORKSPACE;     // batch * n_q_heads * k_max_len logits do not fit the fixed array
+  void *ws = nullptr;
+  twig_status s = noalloc_scratch_address(&ws);
+  if (s != TWIG_OK) return s;
+  ScoreArgs a{twig_q, twig_k, k_stride_batch, k_stride_head, k_stride_pos, k_max_len, prefix_len,
+              vis_start, n_vis, batch, n_q_heads, n_kv_heads, head_dim, norm_scope, softmax_scale,
+              scores, m_max};
+  s = check_score_args(a, ws, TWIG_NOALLOC_SCRATCH_BYTES);
+  if (s != TWIG_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // every logit the second kernel reads is written by the first one in this call, so the
+  // array's old contents never matter and nothing has to be cleared
+  s = launch_logits(a, dev_status, ws, st);
+  if (s != TWIG_OK) return s;
+  return launch_finalize(static_cast<const float *>(ws), a, nullptr, nullptr, 0, dev_status, 1, st);
+}
+
 extern "C" twig_status ttp_topk(const float *scores, const int32_t *n_vis, const int32_t *keep,
                                 int32_t batch, int32_t m_max, int32_t r_max, int32_t *kept_idx,
                                 int32_t *dev_status, void *stream) {

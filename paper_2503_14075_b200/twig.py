@@ -26,7 +26,7 @@ STATUS_NAMES = {0: "TWIG_OK", 1: "TWIG_ERR_NULL", 2: "TWIG_ERR_SHAPE", 3: "TWIG_
 DEV_OK, DEV_BAD_LAYOUT, DEV_BAD_KEEP, DEV_BAD_INDEX, DEV_BAD_TREE, DEV_OVERFLOW = range(6)
 MAX_NODES, MAX_VISUAL, MAX_BATCH = 64, 16384, 4096
 
-EXPORTS = ["twig_status_str", "twig_workspace_bytes", "ttp_score", "ttp_topk", "ttp_compact",
+EXPORTS = ["twig_status_str", "twig_workspace_bytes", "ttp_score", "ttp_score_noalloc", "ttp_topk", "ttp_compact",
            "ttp_score_topk_compact", "tree_verify_attention", "tree_accept_compact"]
 
 
@@ -63,6 +63,10 @@ _lib.twig_workspace_bytes.argtypes = [_i32] * 5
 _lib.ttp_score.restype = C.c_int
 _lib.ttp_score.argtypes = [_vp, _vp, _i64, _i64, _i64, _i32, _vp, _vp, _vp, _i32, _i32, _i32, _i32, _i32,
                            _f32, _vp, _i32, _vp, _vp, _sz, _vp]
+_lib.ttp_score_noalloc.restype = C.c_int
+_lib.ttp_score_noalloc.argtypes = [_vp, _vp, _i64, _i64, _i64, _i32, _vp, _vp, _vp, _i32, _i32, _i32, _i32, _i32,
+                                   _f32, _vp, _i32, _vp, _vp]
+NOALLOC_SCRATCH_BYTES = 4 << 20
 _lib.ttp_topk.restype = C.c_int
 _lib.ttp_topk.argtypes = [_vp, _vp, _vp, _i32, _i32, _i32, _vp, _vp, _vp]
 _lib.ttp_compact.restype = C.c_int
@@ -108,6 +112,19 @@ def ttp_score(twig_q, twig_k, prefix_len, vis_start, n_vis, scores, ws, norm_sco
                           twig_k.shape[2], _p(prefix_len), _p(vis_start), _p(n_vis), B, Hq,
                           twig_k.shape[1], d, norm_scope, softmax_scale, _p(scores), scores.shape[1],
                           _p(dev_status), _p(ws), ws.numel() * ws.element_size(), _stream(stream)))
+
+
+def ttp_score_noalloc(twig_q, twig_k, prefix_len, vis_start, n_vis, scores, norm_scope=0,
+                      softmax_scale=0.0, dev_status=None, stream=None):
+    """ttp_score for callers that may not allocate device memory: the logits scratch is a fixed
+    NOALLOC_SCRATCH_BYTES array inside the library (shared by all calls on the device, so calls
+    that overlap on the GPU race).  Raises TwigError(TWIG_ERR_WORKSPACE) when
+    batch * n_q_heads * prompt length does not fit."""
+    B, Hq, d = twig_q.shape
+    _check(_lib.ttp_score_noalloc(_p(twig_q), _p(twig_k), twig_k.stride(0), twig_k.stride(1),
+                                  twig_k.stride(2), twig_k.shape[2], _p(prefix_len), _p(vis_start),
+                                  _p(n_vis), B, Hq, twig_k.shape[1], d, norm_scope, softmax_scale,
+                                  _p(scores), scores.shape[1], _p(dev_status), _stream(stream)))
 
 
 def ttp_topk(scores, n_vis, keep, kept_idx, dev_status=None, stream=None):
