@@ -59,7 +59,8 @@ enum {
   TWIG_DEV_BAD_KEEP = 2,   /* keep < 0 or keep > n_vis                                 */
   TWIG_DEV_BAD_INDEX = 3,  /* kept_idx not strictly ascending within [0, n_vis)        */
   TWIG_DEV_BAD_TREE = 4,   /* n_nodes out of [0, t_max] or parent[i] not in [-1, i)    */
-  TWIG_DEV_OVERFLOW = 5    /* kv_len < 0 or kv_len + rows to append > max_len          */
+  TWIG_DEV_OVERFLOW = 5,   /* kv_len < 0 or kv_len + rows to append > max_len          */
+  TWIG_DEV_INTERNAL = 6    /* a bounded on-chip wait ran out; the request's output is not written */
 };
 
 #define TWIG_MAX_NODES 64      /* draft-tree nodes per request (root included)      */
@@ -188,6 +189,11 @@ twig_status tree_verify_attention(const void *q, const void *tree_k, const void 
                                   const int32_t *n_nodes, const int32_t *parent, int32_t t_max,
                                   int32_t n_q_heads, float softmax_scale, void *out, float *lse,
                                   int32_t *dev_status, void *ws, size_t ws_bytes, void *stream);
+
+/* Selects the tree-attention kernel: 0 = automatic (default), 1 = mma.sync kernel,
+ * 2 = tcgen05 kernel (head_dim 128 only; other shapes fall back to 1).  Both compute
+ * the same function; this is a tuning and testing control.  Returns the previous value. */
+int32_t twig_set_attention_path(int32_t path);
 
 /* ---- Acceptance + bonus token + KV append, all layers in one call ------------
  * Sec. 5.4 / Appendix A / Algorithm 2.  Node 0 is the last accepted token and is

@@ -13,53 +13,11 @@
 // touches HBM.
 #include <cooperative_groups.h>
 
-#include "twig_common.cuh"
+#include "tree_attn.cuh"
 
 namespace cg = cooperative_groups;
 
 namespace twig {
-
-struct AttnParams {
-  const __nv_bfloat16 *q, *tree_k, *tree_v, *cache_k, *cache_v;   // cache_* point at the layer
-  long long c_sb, c_sh, c_sp;
-  const int *kv_len, *n_nodes, *parent;
-  __nv_bfloat16 *out;
-  float *lse;
-  int *dev_status;
-  int t_max, n_q_heads, n_kv_heads, group, max_len, row_blocks;
-  float scale_log2;   // softmax_scale * log2(e)
-};
-
-// ---- small PTX wrappers ----------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void *p) {
-  return (uint32_t)__cvta_generic_to_shared(p);
-}
-__device__ __forceinline__ void cp_async_16(uint32_t dst, const void *src, bool valid) {
-  const int n = valid ? 16 : 0;
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(n) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() {
-  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
-}
-__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t (&r)[4]) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
-}
-__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t (&r)[4]) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
-}
-__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-  return *reinterpret_cast<uint32_t *>(&v);
-}
 
 // Byte offset of 16-byte chunk `c` of row `r` in a [rows x D] bf16 tile.  The
 // tile is stored as D/64 panels of 128-byte rows; within a panel the chunk
@@ -291,15 +249,15 @@ tree_attn_kernel(const AttnParams p) {
     mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 2));
     const float mn_lo = fmaxf(m_lo, mx_lo), mn_hi = fmaxf(m_hi, mx_hi);
     const float use_lo = mn_lo == -INFINITY ? 0.f : mn_lo, use_hi = mn_hi == -INFINITY ? 0.f : mn_hi;
-    const float a_lo = exp2f(m_lo - use_lo), a_hi = exp2f(m_hi - use_hi);
+    const float a_lo = fast_exp2(m_lo - use_lo), a_hi = fast_exp2(m_hi - use_hi);
     m_lo = mn_lo;
     m_hi = mn_hi;
     float sum_lo = 0.f, sum_hi = 0.f;
     uint32_t pf[NT / 2][4];
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
-      const float p0 = exp2f(s[nt][0] - use_lo), p1 = exp2f(s[nt][1] - use_lo);
-      const float p2 = exp2f(s[nt][2] - use_hi), p3 = exp2f(s[nt][3] - use_hi);
+      const float p0 = fast_exp2(s[nt][0] - use_lo), p1 = fast_exp2(s[nt][1] - use_lo);
+      const float p2 = fast_exp2(s[nt][2] - use_hi), p3 = fast_exp2(s[nt][3] - use_hi);
       sum_lo += p0 + p1;
       sum_hi += p2 + p3;
       pf[nt / 2][(nt & 1) * 2 + 0] = pack_bf16(p0, p1);
@@ -352,8 +310,8 @@ tree_attn_kernel(const AttnParams p) {
         const float4 ml = s_xml[((w - 1) * WM + wm) * 32 + lane];
         const float mn_lo = fmaxf(m_lo, ml.x), mn_hi = fmaxf(m_hi, ml.y);
         const float use_lo = mn_lo == -INFINITY ? 0.f : mn_lo, use_hi = mn_hi == -INFINITY ? 0.f : mn_hi;
-        const float a_lo = exp2f(m_lo - use_lo), a_hi = exp2f(m_hi - use_hi);
-        const float b_lo = exp2f(ml.x - use_lo), b_hi = exp2f(ml.y - use_hi);
+        const float a_lo = fast_exp2(m_lo - use_lo), a_hi = fast_exp2(m_hi - use_hi);
+        const float b_lo = fast_exp2(ml.x - use_lo), b_hi = fast_exp2(ml.y - use_hi);
         m_lo = mn_lo;
         m_hi = mn_hi;
         l_lo = l_lo * a_lo + ml.z * b_lo;
@@ -422,7 +380,7 @@ tree_attn_kernel(const AttnParams p) {
 #pragma unroll
       for (int sd = 0; sd < 8; ++sd) {
         if (sd < n_splits) {
-          const float wgt = exp2f(mv[sd] - mstar);
+          const float wgt = fast_exp2(mv[sd] - mstar);
           lsum = fmaf(wgt, r_l[sd * rows_per + lr], lsum);
           const float4 v = *reinterpret_cast<const float4 *>(recv + (size_t)(sd * rows_per + lr) * D + col);
           acc.x = fmaf(wgt, v.x, acc.x);
@@ -472,7 +430,7 @@ static twig_status launch_attn(const AttnParams &p, int batch, int n_splits, cud
   return TWIG_OK;
 }
 
-static int pick_splits(int items, int max_tiles) {
+int pick_splits(int items, int max_tiles) {
   int s = 1;
   while (s < 8 && items * s < 2 * 148 && s * 2 <= max_tiles) s *= 2;
   return s;
@@ -500,6 +458,14 @@ static twig_status dispatch_attn(AttnParams &p, int batch, int rows, cudaStream_
 }  // namespace twig
 
 using namespace twig;
+
+static int g_attention_path = 0;
+
+extern "C" int32_t twig_set_attention_path(int32_t path) {
+  const int prev = g_attention_path;
+  if (path >= 0 && path <= 2) g_attention_path = path;
+  return prev;
+}
 
 extern "C" twig_status tree_verify_attention(const void *q, const void *tree_k, const void *tree_v,
                                              const twig_kv *cache, int32_t layer,
@@ -543,6 +509,8 @@ extern "C" twig_status tree_verify_attention(const void *q, const void *tree_k, 
   p.scale_log2 = scale * 1.4426950408889634f;
   const int rows = t_max * p.group;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (cache->head_dim == 128 && (g_attention_path == 2 || (g_attention_path == 0 && rows > 32)))
+    return launch_tree_attn_umma(p, cache->batch, rows, st);
   return cache->head_dim == 128 ? dispatch_attn<128>(p, cache->batch, rows, st)
                                 : dispatch_attn<64>(p, cache->batch, rows, st);
 }

@@ -23,10 +23,10 @@ _lib = C.CDLL(_LIB_PATH)
 
 STATUS_NAMES = {0: "TWIG_OK", 1: "TWIG_ERR_NULL", 2: "TWIG_ERR_SHAPE", 3: "TWIG_ERR_UNSUPPORTED",
                 4: "TWIG_ERR_WORKSPACE", 5: "TWIG_ERR_CUDA", 6: "TWIG_ERR_ALIGN"}
-DEV_OK, DEV_BAD_LAYOUT, DEV_BAD_KEEP, DEV_BAD_INDEX, DEV_BAD_TREE, DEV_OVERFLOW = range(6)
+DEV_OK, DEV_BAD_LAYOUT, DEV_BAD_KEEP, DEV_BAD_INDEX, DEV_BAD_TREE, DEV_OVERFLOW, DEV_INTERNAL = range(7)
 MAX_NODES, MAX_VISUAL, MAX_BATCH = 64, 16384, 4096
 
-EXPORTS = ["twig_status_str", "twig_workspace_bytes", "ttp_score", "ttp_score_noalloc", "ttp_topk", "ttp_compact",
+EXPORTS = ["twig_status_str", "twig_set_attention_path", "twig_workspace_bytes", "ttp_score", "ttp_score_noalloc", "ttp_topk", "ttp_compact",
            "ttp_score_topk_compact", "tree_verify_attention", "tree_accept_compact"]
 
 
@@ -58,6 +58,8 @@ _vp, _i32, _i64, _f32, _sz = C.c_void_p, C.c_int32, C.c_int64, C.c_float, C.c_si
 _kvp = C.POINTER(KV)
 _lib.twig_status_str.restype = C.c_char_p
 _lib.twig_status_str.argtypes = [C.c_int]
+_lib.twig_set_attention_path.restype = C.c_int32
+_lib.twig_set_attention_path.argtypes = [C.c_int32]
 _lib.twig_workspace_bytes.restype = _sz
 _lib.twig_workspace_bytes.argtypes = [_i32] * 5
 _lib.ttp_score.restype = C.c_int
@@ -98,6 +100,11 @@ def _check(code: int):
 
 def lib_path() -> str:
     return _LIB_PATH
+
+
+def twig_set_attention_path(path: int) -> int:
+    """0 automatic, 1 mma.sync kernel, 2 tcgen05 kernel; returns the previous setting."""
+    return int(_lib.twig_set_attention_path(int(path)))
 
 
 def twig_workspace_bytes(batch, n_q_heads, head_dim, max_len, max_nodes) -> int:

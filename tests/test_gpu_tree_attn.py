@@ -20,9 +20,11 @@ def tw():
     return twig
 
 
-def run_attention(tw, wl, ver, cache_k, cache_v, kv_len, layer=0, max_len=None, lse=True):
-    """cache_k/v: uint16 [Nl,B,Hkv,Lmax,d].  Returns (out bits [B,T,Hq,d], lse [B,Hq,T], status)."""
+def run_attention(tw, wl, ver, cache_k, cache_v, kv_len, layer=0, max_len=None, lse=True, path=0):
+    """cache_k/v: uint16 [Nl,B,Hkv,Lmax,d].  Returns (out bits [B,T,Hq,d], lse [B,Hq,T], status).
+    path: 0 automatic, 1 mma.sync kernel, 2 tcgen05 kernel."""
     B, T, Hq, d = ver["q"].shape[1:]
+    tw.twig_set_attention_path(path)
     ck, cv = dev_bf16(cache_k), dev_bf16(cache_v)
     out = torch.zeros((B, T, Hq, d), dtype=torch.int16, device=DEV)
     out.fill_(CANARY)
@@ -33,6 +35,7 @@ def run_attention(tw, wl, ver, cache_k, cache_v, kv_len, layer=0, max_len=None, 
                              tw.KV.of(ck, cv), layer, dev_i32(kv_len), dev_i32(ver["n_nodes"]), dev_i32(ver["parent"]),
                              out, lse=lse_t, dev_status=status)
     torch.cuda.synchronize()
+    tw.twig_set_attention_path(0)
     return host_bits(out), (lse_t.cpu().numpy() if lse else None), status.cpu().numpy()
 
 
@@ -78,8 +81,11 @@ SHAPES = [
 
 @pytest.mark.parametrize("shape", SHAPES, ids=[s[0] for s in SHAPES])
 @pytest.mark.parametrize("gain_name", ["timing", "sharp", "sharp4"])
-def test_tree_attention_matches_oracle(tw, shape, gain_name):
+@pytest.mark.parametrize("path", [1, 2], ids=["mma", "tcgen05"])
+def test_tree_attention_matches_oracle(tw, shape, gain_name, path):
     name, B, Hq, Hkv, d, n_nodes, depth, kv_len = shape
+    if path == 2 and d != 128:
+        pytest.skip("the tcgen05 kernel covers head_dim 128")
     gain = {"timing": 1.0, "sharp": d ** 0.5, "sharp4": 2.0 * d ** 0.5}[gain_name]   # logit std 1/d, 1, 4
     wl = _wl(B, Hq, Hkv, d, n_nodes, depth)
     rng = synth.rng_for(9, zlib.crc32(name.encode()) % 1000)
@@ -89,14 +95,15 @@ def test_tree_attention_matches_oracle(tw, shape, gain_name):
     for b in range(B):                       # rows past kv_len must never be read
         ck[0, b, :, kv_len[b]:] = CANARY
         cv[0, b, :, kv_len[b]:] = CANARY
-    got, lse, status = run_attention(tw, wl, ver, ck, cv, kv_len)
+    got, lse, status = run_attention(tw, wl, ver, ck, cv, kv_len, path=path)
     assert not status.any()
     want, want_lse = oracle_attention(ver, ck, cv, np.array(kv_len))
     check(got, lse, want, want_lse, ver["n_nodes"], name)
 
 
+@pytest.mark.parametrize("path", [1, 2], ids=["mma", "tcgen05"])
 @pytest.mark.parametrize("kind", ["chain", "star"])
-def test_special_trees(tw, kind):
+def test_special_trees(tw, kind, path):
     T = 20
     wl = _wl(2, 4, 4, 128, [T, T], [T, 2])
     rng = synth.rng_for(9, 77)
@@ -104,19 +111,20 @@ def test_special_trees(tw, kind):
     ver["parent"][:] = synth.chain_tree(T) if kind == "chain" else synth.star_tree(T)
     ck, cv = synth.make_cache(wl, rng, 300, n_layers=1, gain=128 ** 0.5)
     kv_len = [190, 3]
-    got, lse, status = run_attention(tw, wl, ver, ck, cv, kv_len)
+    got, lse, status = run_attention(tw, wl, ver, ck, cv, kv_len, path=path)
     want, want_lse = oracle_attention(ver, ck, cv, np.array(kv_len))
     check(got, lse, want, want_lse, ver["n_nodes"], kind)
 
 
-def test_bad_tree_and_overflow_set_status(tw):
+@pytest.mark.parametrize("path", [1, 2], ids=["mma", "tcgen05"])
+def test_bad_tree_and_overflow_set_status(tw, path):
     wl = _wl(4, 4, 4, 128, [6, 6, 6, 6], [3, 3, 3, 3])
     rng = synth.rng_for(9, 78)
     ver = synth.make_verify_inputs(wl, rng, n_layers=1)
     ver["parent"][1, 3] = 3            # parent must be an earlier node
     ver["parent"][2, 0] = 0            # root must have parent -1
     ck, cv = synth.make_cache(wl, rng, 64, n_layers=1)
-    got, lse, status = run_attention(tw, wl, ver, ck, cv, [10, 10, 10, 65])
+    got, lse, status = run_attention(tw, wl, ver, ck, cv, [10, 10, 10, 65], path=path)
     assert status.tolist() == [0, tw.DEV_BAD_TREE, tw.DEV_BAD_TREE, tw.DEV_OVERFLOW]
     assert np.all(got[1:] == CANARY)                                   # skipped requests untouched
     good = {k: (v[:, :1] if k in ("q", "tree_k", "tree_v") else v[:1]) for k, v in ver.items()}
@@ -133,8 +141,9 @@ FULL = [
 ]
 
 
+@pytest.mark.parametrize("path", [1, 2], ids=["mma", "tcgen05"])
 @pytest.mark.parametrize("index,lens", FULL, ids=["c2", "c3", "c4", "c5"])
-def test_full_size_configs(tw, index, lens):
+def test_full_size_configs(tw, index, lens, path):
     """Full-size shapes of the benchmark configurations, one layer, every output row
     against the oracle (timing distribution), plus sampled rows of a sharp variant."""
     wl = synth.workload(index)
@@ -148,7 +157,7 @@ def test_full_size_configs(tw, index, lens):
         ver = synth.make_verify_inputs(wl, rng, n_layers=1, gain=gain)
         ck, cv = synth.make_cache(wl, rng, max_len, n_layers=1, gain=gain)
         for kv_len in lens_list:
-            got, lse, status = run_attention(tw, wl, ver, ck, cv, kv_len)
+            got, lse, status = run_attention(tw, wl, ver, ck, cv, kv_len, path=path)
             assert not status.any()
             if not sampled:
                 want, want_lse = oracle_attention(ver, ck, cv, np.array(kv_len))
