@@ -54,13 +54,14 @@ def case_attn(a):
     kvl = torch.full((wl.batch,), L, dtype=torch.int32, device=DEV)
     out = torch.zeros((wl.batch, wl.t_max, wl.n_q_heads, wl.head_dim), dtype=torch.bfloat16, device=DEV)
     cache = tw.KV.of(ck, cv)
+    tw.twig_set_attention_path(a.path)
 
     def run():
         for layer in range(nl):
             tw.tree_verify_attention(q[layer], tk[layer], tv[layer], cache, layer, kvl, nn, par, out)
     us = _time(run, a.iters) / nl
     by = sum(wl.kv_row_bytes() * (L + n) + 2 * n * wl.n_q_heads * wl.head_dim * 2 + 8 * n for n in wl.n_nodes)
-    print(f"attn {wl.name} L={L}: {us:.2f} us/launch, {by / us / 1e3:.1f} GB/s algorithmic ({by} B/launch)")
+    print(f"attn path={a.path} {wl.name} L={L}: {us:.2f} us/launch, {by / us / 1e3:.1f} GB/s algorithmic ({by} B/launch)")
 
 
 def case_gather(a):
@@ -133,6 +134,7 @@ def main():
     ap.add_argument("--kv-len", type=int, default=0)
     ap.add_argument("--layers", type=int, default=2)
     ap.add_argument("--iters", type=int, default=3)
+    ap.add_argument("--path", type=int, default=0, help="attention kernel: 0 auto, 1 mma.sync, 2 tcgen05")
     a = ap.parse_args()
     {"attn": case_attn, "gather": case_gather, "score": case_score, "accept": case_accept}[a.case](a)
 
