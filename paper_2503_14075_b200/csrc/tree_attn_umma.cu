@@ -8,9 +8,12 @@
 //   softmax step  tcgen05.ld of the row, running max / sum, P (bf16) back to shared memory
 //   O_t = P V     tcgen05.mma, M = 128, N = 128, K = 4 x 16, V read MN-major (no transpose copy)
 //   O += O_t      tcgen05.ld, rescaled accumulation in registers
-// K/V tiles are staged by 16-byte cp.async in the 128-byte-swizzled layout that the
-// matrix descriptors name.  The instruction always multiplies 128 rows; rows past
-// ROWS read whatever follows in shared memory and land in lanes nobody reads.
+// K and V tiles travel separately through a ring of five 16 KB slots, filled by 16-byte
+// cp.async in the 128-byte-swizzled layout that the matrix descriptors name; a K slot is
+// refilled as soon as its S product has completed, a V slot after its P V product, so four
+// tiles (64 KB) per CTA are in flight while one is being consumed.  The instruction
+// always multiplies 128 rows; rows past ROWS read whatever follows in shared memory
+// and land in lanes nobody reads.
 // Key splits of a cluster are merged through distributed shared memory exactly as
 // in the mma.sync kernel (each CTA pushes its per-row partial to the row's owner).
 #include <cooperative_groups.h>
@@ -26,7 +29,7 @@ namespace {
 constexpr int kD = 128;          // head_dim
 constexpr int kKT = 64;          // keys per tile
 constexpr int kThreads = 128;
-constexpr int kStages = 2;
+constexpr int kSlots = 5;                         // ring of K / V tiles (K0 V0 K1 V1 K2 ...)
 constexpr int kTileBytes = kKT * kD * 2;          // one K (or V) tile: 16 KB
 constexpr int kPanelBytes = kKT * 128;            // 64-column panel of a K/V tile
 constexpr uint32_t kTmemCols = 256;               // S: columns [0,64), O tile: [128,256)
@@ -95,7 +98,7 @@ template <int ROWS>
 struct UmmaCfg {
   static constexpr int Q_BYTES = ROWS * kD * 2;          // two 64-column panels of ROWS x 128 B
   static constexpr int P_BYTES = ROWS * 128;             // ROWS x 64 keys bf16
-  static constexpr int RING_BYTES = 2 * kStages * kTileBytes;
+  static constexpr int RING_BYTES = kSlots * kTileBytes;
   static constexpr int RECV_BYTES = ROWS * kD * 4;
   static_assert(RECV_BYTES <= RING_BYTES, "split-merge buffer must fit in the stage ring");
   static_assert(Q_BYTES % 1024 == 0 && P_BYTES % 1024 == 0, "swizzled tiles start on 1024 bytes");
@@ -137,8 +140,7 @@ tree_attn_umma_kernel(const AttnParams p) {
 
   const uint32_t q_s = smem_u32(smem);
   const uint32_t p_s = q_s + C::Q_BYTES;
-  const uint32_t k_s = p_s + C::P_BYTES;
-  const uint32_t v_s = k_s + kStages * kTileBytes;
+  const uint32_t ring_s = p_s + C::P_BYTES;
 
   const int NK = L + n;
   const int n_tiles = (NK + kKT - 1) / kKT;
@@ -151,38 +153,36 @@ tree_attn_umma_kernel(const AttnParams p) {
   const __nv_bfloat16 *tk = p.tree_k + ((long long)b * p.n_kv_heads + hk) * p.t_max * kD;
   const __nv_bfloat16 *tv = p.tree_v + ((long long)b * p.n_kv_heads + hk) * p.t_max * kD;
 
-  // A thread copies chunk (tid & 15) of rows (tid >> 4) + 8 i, i = 0..7, of K and of V.
+  // A thread copies chunk (tid & 15) of rows (tid >> 4) + 8 i, i = 0..7, of a K or V tile.
+  // Unit u of this CTA is K (u even) or V (u odd) of its tile u / 2 and lives in slot u % kSlots.
   const int ld_c = tid & 15, ld_r0 = tid >> 4;
   const uint32_t ld_off0 = (uint32_t)((ld_c >> 3) * kPanelBytes + ld_r0 * 128 + (((ld_c & 7) ^ (ld_r0 & 7)) << 4));
-  auto load_tile = [&](int t, int stage) {
-    const uint32_t kd = k_s + stage * kTileBytes + ld_off0, vd = v_s + stage * kTileBytes + ld_off0;
+  auto load_unit = [&](int u) {
+    const int t = t_begin + (u >> 1);
+    if (t >= t_end) return;
+    const uint32_t dst = ring_s + (u % kSlots) * kTileBytes + ld_off0;
+    const __nv_bfloat16 *cbase = (u & 1) ? cv : ck, *tbase = (u & 1) ? tv : tk;
     const int j0 = t * kKT + ld_r0;
     if (t * kKT + kKT <= L) {               // whole tile inside the cached prefix
-      const __nv_bfloat16 *sk = ck + (long long)j0 * p.c_sp + ld_c * 8;
-      const __nv_bfloat16 *sv = cv + (long long)j0 * p.c_sp + ld_c * 8;
+      const __nv_bfloat16 *src = cbase + (long long)j0 * p.c_sp + ld_c * 8;
       const long long step = 8 * p.c_sp;
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {         // rows 8 apart keep (row & 7): same swizzle, +1024 bytes
-        cp_async_16(kd + i * 1024, sk + i * step, true);
-        cp_async_16(vd + i * 1024, sv + i * step, true);
-      }
+      for (int i = 0; i < 8; ++i)           // rows 8 apart keep (row & 7): same swizzle, +1024 bytes
+        cp_async_16(dst + i * 1024, src + i * step, true);
     } else {
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
         const int vj = j0 + 8 * i;
-        const __nv_bfloat16 *sk = ck, *sv = cv;
+        const __nv_bfloat16 *src = cbase;
         bool valid = false;
         if (vj < L) {
-          sk = ck + (long long)vj * p.c_sp + ld_c * 8;
-          sv = cv + (long long)vj * p.c_sp + ld_c * 8;
+          src = cbase + (long long)vj * p.c_sp + ld_c * 8;
           valid = true;
         } else if (vj < NK) {
-          sk = tk + (vj - L) * kD + ld_c * 8;
-          sv = tv + (vj - L) * kD + ld_c * 8;
+          src = tbase + (vj - L) * kD + ld_c * 8;
           valid = true;
         }
-        cp_async_16(kd + i * 1024, sk, valid);
-        cp_async_16(vd + i * 1024, sv, valid);
+        cp_async_16(dst + i * 1024, src, valid);
       }
     }
   };
@@ -198,10 +198,13 @@ tree_attn_umma_kernel(const AttnParams p) {
         p.q + (((long long)b * p.t_max + node) * p.n_q_heads + hk * p.group + g) * kD + ld_c * 8;
     cp_async_16(q_s + (ld_c >> 3) * ROWS * 128 + r * 128 + (((ld_c & 7) ^ (r & 7)) << 4), src, valid);
   }
-  if (t_begin < t_end) load_tile(t_begin, 0);
-  cp_async_commit();
-  if (t_begin + 1 < t_end) load_tile(t_begin + 1, 1);
-  cp_async_commit();
+  load_unit(0);
+  cp_async_commit();              // this group also carries Q
+#pragma unroll
+  for (int u = 1; u < kSlots; ++u) {
+    load_unit(u);
+    cp_async_commit();
+  }
 
   // ---- while they fly: parents, validation, ancestor masks ---------------------
   if (tid == 0) s_bad = 0;
@@ -258,13 +261,13 @@ tree_attn_umma_kernel(const AttnParams p) {
   bool ok = true;
 
   for (int t = t_begin; t < t_end; ++t) {
-    const int it = t - t_begin, stage = it & 1;
-    cp_async_wait<1>();            // this tile has landed (the next one may still be in flight)
+    const int it = t - t_begin;
+    cp_async_wait<kSlots - 1>();   // this tile's K has landed (four later units may still be in flight)
     fence_async_smem();            // make the copied bytes visible to the tensor core's reads
     __syncthreads();
     if (tid == 0) {
       tc_fence_after();
-      const uint32_t kb = k_s + stage * kTileBytes;
+      const uint32_t kb = ring_s + ((2 * it) % kSlots) * kTileBytes;
 #pragma unroll
       for (int ks = 0; ks < kD / 16; ++ks) {
         const uint32_t qa = q_s + (ks >> 2) * ROWS * 128 + (ks & 3) * 32;
@@ -277,6 +280,8 @@ tree_attn_umma_kernel(const AttnParams p) {
     if (ok) ok = mbar_wait(bar_s, ph_s);
     ph_s ^= 1;
     tc_fence_after();
+    if (ok) load_unit(2 * it + kSlots);      // the K slot is free: S has been computed
+    cp_async_commit();
     if (warp_rows && ok) {
       uint32_t sr[2][32];
       tmem_ld32(t_lane + 0, sr[0]);
@@ -327,12 +332,13 @@ tree_attn_umma_kernel(const AttnParams p) {
       }
       l_run = l_run * alpha + sum;
     }
-    fence_async_smem();            // P was written with ordinary stores
+    cp_async_wait<kSlots - 1>();   // this tile's V has landed
+    fence_async_smem();            // ... and P was written with ordinary stores
     tc_fence_before();
     ok = __syncthreads_and(ok);
     if (tid == 0 && ok) {
       tc_fence_after();
-      const uint32_t vb = v_s + stage * kTileBytes;
+      const uint32_t vb = ring_s + ((2 * it + 1) % kSlots) * kTileBytes;
 #pragma unroll
       for (int j = 0; j < kKT / 16; ++j)
         umma(tmem_o, smem_desc(p_s + j * 32, 16), smem_desc(vb + j * 2048, kPanelBytes), kIdescO, j > 0);
@@ -345,6 +351,8 @@ tree_attn_umma_kernel(const AttnParams p) {
     if (ok) ok = mbar_wait(bar_o, ph_o);
     ph_o ^= 1;
     tc_fence_after();
+    if (ok) load_unit(2 * it + kSlots + 1);  // the V slot is free: the O tile has been computed
+    cp_async_commit();
     if (warp_rows && ok) {
 #pragma unroll
       for (int ch = 0; ch < 4; ++ch) {
@@ -356,10 +364,8 @@ tree_attn_umma_kernel(const AttnParams p) {
       }
     }
     tc_fence_before();
-    ok = __syncthreads_and(ok);     // S, O tile, P and this stage are free again
+    ok = __syncthreads_and(ok);     // S, the O tile and P are free again
     if (!ok) break;
-    if (t + 2 < t_end) load_tile(t + 2, stage);
-    cp_async_commit();
   }
   cp_async_wait<0>();
   tc_fence_before();
