@@ -3,19 +3,22 @@
 //
 // One CTA of 128 threads owns up to ROWS query rows (tree node x query head of
 // one kv head) and a share of the key tiles; thread r owns row r, which is also
-// lane r of tensor memory.  Per 64-key tile:
-//   S = Q K^T     tcgen05.mma, M = 128, N = 64, K = 8 x 16, operands in shared memory
-//   softmax step  tcgen05.ld of the row, running max / sum, P (bf16) back to shared memory
-//   O_t = P V     tcgen05.mma, M = 128, N = 128, K = 4 x 16, V read MN-major (no transpose copy)
-//   O += O_t      tcgen05.ld, rescaled accumulation in registers
+// lane r of tensor memory.  Per 64-key tile t:
+//   S(t) = Q K^T   tcgen05.mma, M = 128, N = 64, K = 8 x 16, operands in shared memory;
+//                  it is issued one tile ahead, so it runs while tile t-1 is in its softmax
+//   softmax step   tcgen05.ld of the row, running max / sum, P (bf16) back to shared memory
+//   O += P V       tcgen05.mma, M = 128, N = 128, K = 4 x 16, V read MN-major (no transpose
+//                  copy), accumulating in tensor memory across tiles
+// The running maximum is only raised when a tile exceeds it by more than 2^8; then (rarely)
+// the O accumulator is rescaled in tensor memory (ld, multiply, st).  P stays below 2^8,
+// which bf16 and the fp32 sums hold without loss of accuracy.
 // K and V tiles travel separately through a ring of five 16 KB slots, filled by 16-byte
 // cp.async in the 128-byte-swizzled layout that the matrix descriptors name; a K slot is
-// refilled as soon as its S product has completed, a V slot after its P V product, so four
-// tiles (64 KB) per CTA are in flight while one is being consumed.  The instruction
-// always multiplies 128 rows; rows past ROWS read whatever follows in shared memory
-// and land in lanes nobody reads.
-// Key splits of a cluster are merged through distributed shared memory exactly as
-// in the mma.sync kernel (each CTA pushes its per-row partial to the row's owner).
+// refilled as soon as its S product has completed, a V slot after its P V product.
+// The instruction always multiplies 128 rows; rows past ROWS read whatever follows in
+// shared memory and land in lanes nobody reads.  Key splits of a cluster are merged
+// through distributed shared memory as in the mma.sync kernel (each CTA pushes its
+// per-row partial to the row's owner); without splits every thread stores its own row.
 #include <cooperative_groups.h>
 
 #include "tree_attn.cuh"
@@ -32,7 +35,8 @@ constexpr int kThreads = 128;
 constexpr int kSlots = 5;                         // ring of K / V tiles (K0 V0 K1 V1 K2 ...)
 constexpr int kTileBytes = kKT * kD * 2;          // one K (or V) tile: 16 KB
 constexpr int kPanelBytes = kKT * 128;            // 64-column panel of a K/V tile
-constexpr uint32_t kTmemCols = 256;               // S: columns [0,64), O tile: [128,256)
+constexpr uint32_t kTmemCols = 256;               // S: columns [0,64) and [64,128); O: [128,256)
+constexpr float kLazyMax = 8.f;                   // raise the running max only beyond this (log2 units)
 constexpr int kSpinLimit = 1 << 22;
 
 // ---- descriptors -------------------------------------------------------------
@@ -92,6 +96,16 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
       : "r"(taddr));
 }
 #undef TWIG_R8
+#define TWIG_S8(a, o) "r"(a[o]), "r"(a[o + 1]), "r"(a[o + 2]), "r"(a[o + 3]), "r"(a[o + 4]), "r"(a[o + 5]), "r"(a[o + 6]), "r"(a[o + 7])
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+      ::"r"(taddr), TWIG_S8(v, 0), TWIG_S8(v, 8), TWIG_S8(v, 16), TWIG_S8(v, 24)
+      : "memory");
+}
+#undef TWIG_S8
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 template <int ROWS>
@@ -154,13 +168,13 @@ tree_attn_umma_kernel(const AttnParams p) {
   const __nv_bfloat16 *tv = p.tree_v + ((long long)b * p.n_kv_heads + hk) * p.t_max * kD;
 
   // A thread copies chunk (tid & 15) of rows (tid >> 4) + 8 i, i = 0..7, of a K or V tile.
-  // Unit u of this CTA is K (u even) or V (u odd) of its tile u / 2 and lives in slot u % kSlots.
+  // Unit u of this CTA is K (u even) or V (u odd) of its tile u / 2.
   const int ld_c = tid & 15, ld_r0 = tid >> 4;
   const uint32_t ld_off0 = (uint32_t)((ld_c >> 3) * kPanelBytes + ld_r0 * 128 + (((ld_c & 7) ^ (ld_r0 & 7)) << 4));
-  auto load_unit = [&](int u) {
+  auto load_unit = [&](int u, int slot) {
     const int t = t_begin + (u >> 1);
     if (t >= t_end) return;
-    const uint32_t dst = ring_s + (u % kSlots) * kTileBytes + ld_off0;
+    const uint32_t dst = ring_s + slot * kTileBytes + ld_off0;
     const __nv_bfloat16 *cbase = (u & 1) ? cv : ck, *tbase = (u & 1) ? tv : tk;
     const int j0 = t * kKT + ld_r0;
     if (t * kKT + kKT <= L) {               // whole tile inside the cached prefix
@@ -198,12 +212,15 @@ tree_attn_umma_kernel(const AttnParams p) {
         p.q + (((long long)b * p.t_max + node) * p.n_q_heads + hk * p.group + g) * kD + ld_c * 8;
     cp_async_16(q_s + (ld_c >> 3) * ROWS * 128 + r * 128 + (((ld_c & 7) ^ (r & 7)) << 4), src, valid);
   }
-  load_unit(0);
-  cp_async_commit();              // this group also carries Q
+  // Ring slots: K(0) in 0, K(t) in 2 (t odd) or 4 (t even); V(t) in 1, 3, 0 for t mod 3 = 0, 1, 2.
+  // Units are issued in order, one commit group each: 0..4 here, V(2) when K(0) has been
+  // consumed, then K(t+2) when K(t) has been consumed and V(t+2) when V(t-1) has been.
+  auto slot_k = [](int t) { return t == 0 ? 0 : ((t & 1) ? 2 : 4); };
+  auto slot_v = [](int t) { return t % 3 == 0 ? 1 : (t % 3 == 1 ? 3 : 0); };
 #pragma unroll
-  for (int u = 1; u < kSlots; ++u) {
-    load_unit(u);
-    cp_async_commit();
+  for (int u = 0; u < kSlots; ++u) {
+    load_unit(u, u);
+    cp_async_commit();              // the first group also carries Q
   }
 
   // ---- while they fly: parents, validation, ancestor masks ---------------------
@@ -245,50 +262,79 @@ tree_attn_umma_kernel(const AttnParams p) {
   tc_fence_after();
   const uint32_t tmem = s_tmem;
   const uint32_t t_lane = tmem + ((uint32_t)(warp * 32) << 16);     // this warp's 32 lanes
-  const uint32_t tmem_s = tmem, tmem_o = tmem + 128;
+  const uint32_t tmem_o = tmem + 128;
 
   // ---- per-thread state: thread r owns row r ------------------------------------
   const bool warp_rows = warp * 32 < ROWS && row0 + warp * 32 < rows_total;   // warp-uniform
   const int gr = row0 + tid;
   const bool row_valid = tid < ROWS && gr < rows_total;
   const unsigned long long my_mask = row_valid ? s_mask[gr / p.group] : 0ull;
-  float o[kD];
-#pragma unroll
-  for (int i = 0; i < kD; ++i) o[i] = 0.f;
-  float m_run = -INFINITY, l_run = 0.f;
+  float m_run = -INFINITY, l_run = 0.f;     // m_run is in the exp2 domain (scaled logits)
   uint32_t ph_s = 0, ph_o = 0;
   constexpr uint32_t kIdescS = instr_desc(kKT, false), kIdescO = instr_desc(kD, true);
+  const int n_my = t_end - t_begin;
   bool ok = true;
+  // the thread that issues the MMAs sits in a warp without rows where there is one, so that
+  // the (blocking) issue does not hold back a warp's softmax
+  constexpr int kIssuer = ROWS <= 64 ? 96 : 0;
 
-  for (int t = t_begin; t < t_end; ++t) {
-    const int it = t - t_begin;
-    cp_async_wait<kSlots - 1>();   // this tile's K has landed (four later units may still be in flight)
+  auto issue_s = [&](int it) {              // S(it) = Q K(it)^T into S buffer it & 1
+    const uint32_t kb = ring_s + slot_k(it) * kTileBytes;
+#pragma unroll
+    for (int ks = 0; ks < kD / 16; ++ks) {
+      const uint32_t qa = q_s + (ks >> 2) * ROWS * 128 + (ks & 3) * 32;
+      const uint32_t ka = kb + (ks >> 2) * kPanelBytes + (ks & 3) * 32;
+      umma(tmem + (it & 1) * kKT, smem_desc(qa, 16), smem_desc(ka, 16), kIdescS, ks > 0);
+    }
+    umma_commit(bar_s);
+  };
+
+  if (n_my > 0) {
+    cp_async_wait<kSlots - 1>();   // Q and K(0) have landed
     fence_async_smem();            // make the copied bytes visible to the tensor core's reads
     __syncthreads();
-    if (tid == 0) {
+    if (tid == kIssuer) {
       tc_fence_after();
-      const uint32_t kb = ring_s + ((2 * it) % kSlots) * kTileBytes;
-#pragma unroll
-      for (int ks = 0; ks < kD / 16; ++ks) {
-        const uint32_t qa = q_s + (ks >> 2) * ROWS * 128 + (ks & 3) * 32;
-        const uint32_t ka = kb + (ks >> 2) * kPanelBytes + (ks & 3) * 32;
-        umma(tmem_s, smem_desc(qa, 16), smem_desc(ka, 16), kIdescS, ks > 0);
-      }
-      umma_commit(bar_s);
+      issue_s(0);
     }
-    float alpha = 1.f;
+  }
+
+  for (int it = 0; it < n_my; ++it) {
+    const int t = t_begin + it;
+    // S(it) is ready, so K(it)'s slot is free
     if (ok) ok = mbar_wait(bar_s, ph_s);
+    ok = __all_sync(0xffffffffu, ok);
     ph_s ^= 1;
     tc_fence_after();
-    if (ok) load_unit(2 * it + kSlots);      // the K slot is free: S has been computed
+    if (ok) {
+      if (it == 0) load_unit(5, slot_v(2)); else load_unit(2 * it + 4, slot_k(it + 2));
+    }
     cp_async_commit();
+    // K(it+1) and V(it) have landed: start S(it+1) so that it runs under this tile's softmax
+    cp_async_wait<2>();
+    fence_async_smem();
+    tc_fence_before();
+    ok = __syncthreads_and(ok);
+    if (tid == kIssuer && ok && it + 1 < n_my) {
+      tc_fence_after();
+      issue_s(it + 1);
+    }
+    // the previous P V product must be complete before P is overwritten or O is rescaled
+    if (it > 0) {
+      if (ok) ok = mbar_wait(bar_o, ph_o);
+      ok = __all_sync(0xffffffffu, ok);
+      ph_o ^= 1;
+      tc_fence_after();
+      if (ok) load_unit(2 * it + 5, slot_v(it + 2));
+      cp_async_commit();
+    }
     if (warp_rows && ok) {
       uint32_t sr[2][32];
-      tmem_ld32(t_lane + 0, sr[0]);
-      tmem_ld32(t_lane + 32, sr[1]);
+      const uint32_t ts = t_lane + (it & 1) * kKT;
+      tmem_ld32(ts, sr[0]);
+      tmem_ld32(ts + 32, sr[1]);
       tmem_ld_wait();
       const int key0 = t * kKT;
-      float mx = -INFINITY;
       if (key0 + kKT > L) {        // the tile that holds the prefix end and / or the tree
 #pragma unroll
         for (int h = 0; h < 2; ++h)
@@ -296,25 +342,34 @@ tree_attn_umma_kernel(const AttnParams p) {
           for (int j = 0; j < 32; ++j) {
             const int vj = key0 + h * 32 + j;
             const bool vis = vj < L || (vj < NK && ((my_mask >> (vj - L)) & 1ull));
-            const float x = vis ? __uint_as_float(sr[h][j]) * p.scale_log2 : -INFINITY;
-            sr[h][j] = __float_as_uint(x);
-            mx = fmaxf(mx, x);
-          }
-      } else {
-#pragma unroll
-        for (int h = 0; h < 2; ++h)
-#pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            const float x = __uint_as_float(sr[h][j]) * p.scale_log2;
-            sr[h][j] = __float_as_uint(x);
-            mx = fmaxf(mx, x);
+            if (!vis) sr[h][j] = 0xff800000u;     // -inf
           }
       }
-      const float m_new = fmaxf(m_run, mx);
+      float mx = -INFINITY;
+#pragma unroll
+      for (int j = 0; j < 32; j += 2)
+        mx = fmaxf(mx, fmaxf(fmaxf(__uint_as_float(sr[0][j]), __uint_as_float(sr[0][j + 1])),
+                             fmaxf(__uint_as_float(sr[1][j]), __uint_as_float(sr[1][j + 1]))));
+      mx *= p.scale_log2;                         // scale > 0, so the max commutes with it
+      const bool raise = mx > m_run + kLazyMax;   // also true for the first finite maximum
+      const float m_new = raise ? mx : m_run;
       const float m_use = m_new == -INFINITY ? 0.f : m_new;
-      alpha = fast_exp2(m_run - m_use);
+      if (__any_sync(0xffffffffu, raise && it > 0)) {
+        const float alpha = fast_exp2(m_run - m_use);     // 1 for rows that keep their maximum
+        l_run *= alpha;
+#pragma unroll
+        for (int ch = 0; ch < 4; ++ch) {
+          uint32_t v[32];
+          tmem_ld32(t_lane + 128 + ch * 32, v);
+          tmem_ld_wait();
+#pragma unroll
+          for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) * alpha);
+          tmem_st32(t_lane + 128 + ch * 32, v);
+        }
+        tmem_st_wait();
+      }
       m_run = m_new;
-      float sum = 0.f;
+      float sum0 = 0.f, sum1 = 0.f;
       const uint32_t prow = p_s + tid * 128;
 #pragma unroll
       for (int c = 0; c < 8; ++c) {          // chunk c = keys 8c .. 8c+7 of this row
@@ -322,77 +377,92 @@ tree_attn_umma_kernel(const AttnParams p) {
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
           const int j = c * 8 + e * 2;
-          const float p0 = fast_exp2(__uint_as_float(sr[j >> 5][j & 31]) - m_use);
-          const float p1 = fast_exp2(__uint_as_float(sr[(j + 1) >> 5][(j + 1) & 31]) - m_use);
-          sum += p0 + p1;
+          const float p0 = fast_exp2(fmaf(__uint_as_float(sr[j >> 5][j & 31]), p.scale_log2, -m_use));
+          const float p1 = fast_exp2(fmaf(__uint_as_float(sr[(j + 1) >> 5][(j + 1) & 31]), p.scale_log2, -m_use));
+          sum0 += p0;
+          sum1 += p1;
           w[e] = pack_bf16(p0, p1);
         }
         asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(prow + ((c ^ (tid & 7)) << 4)), "r"(w[0]), "r"(w[1]),
                      "r"(w[2]), "r"(w[3]) : "memory");
       }
-      l_run = l_run * alpha + sum;
+      l_run += sum0 + sum1;
     }
-    cp_async_wait<kSlots - 1>();   // this tile's V has landed
-    fence_async_smem();            // ... and P was written with ordinary stores
+    fence_async_smem();            // P was written with ordinary stores
     tc_fence_before();
     ok = __syncthreads_and(ok);
-    if (tid == 0 && ok) {
+    if (tid == kIssuer && ok) {
       tc_fence_after();
-      const uint32_t vb = ring_s + ((2 * it + 1) % kSlots) * kTileBytes;
+      const uint32_t vb = ring_s + slot_v(it) * kTileBytes;
 #pragma unroll
       for (int j = 0; j < kKT / 16; ++j)
-        umma(tmem_o, smem_desc(p_s + j * 32, 16), smem_desc(vb + j * 2048, kPanelBytes), kIdescO, j > 0);
+        umma(tmem_o, smem_desc(p_s + j * 32, 16), smem_desc(vb + j * 2048, kPanelBytes), kIdescO, (it > 0) || (j > 0));
       umma_commit(bar_o);
     }
-    if (warp_rows && alpha != 1.f) {          // overlaps with the P V product
+  }
+  // the accumulated O of this CTA's tiles
+  float o[kD];
+  if (n_my > 0 && ok) ok = mbar_wait(bar_o, ph_o);
+  ok = __all_sync(0xffffffffu, ok);
+  tc_fence_after();
+  if (n_my > 0 && warp_rows && ok) {
 #pragma unroll
-      for (int i = 0; i < kD; ++i) o[i] *= alpha;
+    for (int ch = 0; ch < 4; ++ch) {
+      uint32_t v[32];
+      tmem_ld32(t_lane + 128 + ch * 32, v);
+      tmem_ld_wait();
+#pragma unroll
+      for (int j = 0; j < 32; ++j) o[ch * 32 + j] = __uint_as_float(v[j]);
     }
-    if (ok) ok = mbar_wait(bar_o, ph_o);
-    ph_o ^= 1;
-    tc_fence_after();
-    if (ok) load_unit(2 * it + kSlots + 1);  // the V slot is free: the O tile has been computed
-    cp_async_commit();
-    if (warp_rows && ok) {
+  } else {
 #pragma unroll
-      for (int ch = 0; ch < 4; ++ch) {
-        uint32_t v[32];
-        tmem_ld32(t_lane + 128 + ch * 32, v);
-        tmem_ld_wait();
-#pragma unroll
-        for (int j = 0; j < 32; ++j) o[ch * 32 + j] += __uint_as_float(v[j]);
-      }
-    }
-    tc_fence_before();
-    ok = __syncthreads_and(ok);     // S, the O tile and P are free again
-    if (!ok) break;
+    for (int i = 0; i < kD; ++i) o[i] = 0.f;
   }
   cp_async_wait<0>();
   tc_fence_before();
-  __syncthreads();
+  ok = __syncthreads_and(ok);
   if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
   if (!ok && tid == 0) flag_status(p.dev_status, b, TWIG_DEV_INTERNAL);
+
+  // ---- no key splits: every thread finishes and stores its own row -------------------
+  if (n_splits == 1) {
+    if (row_valid && ok) {
+      const float inv = 1.f / l_run;
+      const int node = gr / p.group, g = gr % p.group;
+      const int h = hk * p.group + g;
+      __nv_bfloat16 *dst = p.out + (((long long)b * p.t_max + node) * p.n_q_heads + h) * kD;
+#pragma unroll
+      for (int c = 0; c < kD / 8; ++c) {
+        uint4 w;
+        w.x = pack_bf16(o[8 * c] * inv, o[8 * c + 1] * inv);
+        w.y = pack_bf16(o[8 * c + 2] * inv, o[8 * c + 3] * inv);
+        w.z = pack_bf16(o[8 * c + 4] * inv, o[8 * c + 5] * inv);
+        w.w = pack_bf16(o[8 * c + 6] * inv, o[8 * c + 7] * inv);
+        st_16(dst + 8 * c, w);
+      }
+      if (p.lse) p.lse[((long long)b * p.n_q_heads + h) * p.t_max + node] = (m_run + log2f(l_run)) * 0.6931471805599453f;
+    }
+    return;
+  }
 
   // ---- merge the key splits of the cluster (push to the row's owner, then reduce) ----
   const int rows_per = ROWS / n_splits;
   float *recv = reinterpret_cast<float *>(smem + C::Q_BYTES + C::P_BYTES);
-  if (n_splits > 1) cluster.sync();        // every CTA has left its key loop: the rings are free
+  cluster.sync();                          // every CTA has left its key loop: the rings are free
   if (tid < ROWS) {
     const int owner = tid / rows_per, lr = tid % rows_per;
     const int slot = split * rows_per + lr;
     float *ro = recv + (size_t)slot * kD, *rm = r_m + slot, *rl = r_l + slot;
-    if (n_splits > 1) {
-      ro = cluster.map_shared_rank(ro, owner);
-      rm = cluster.map_shared_rank(rm, owner);
-      rl = cluster.map_shared_rank(rl, owner);
-    }
+    ro = cluster.map_shared_rank(ro, owner);
+    rm = cluster.map_shared_rank(rm, owner);
+    rl = cluster.map_shared_rank(rl, owner);
 #pragma unroll
     for (int i = 0; i < kD / 4; ++i)        // float4 slots are XOR-swizzled by the row to spread banks
       *reinterpret_cast<float4 *>(ro + ((i ^ (lr & 31)) << 2)) = make_float4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
     *rm = m_run;
     *rl = l_run;
   }
-  if (n_splits > 1) cluster.sync(); else __syncthreads();
+  cluster.sync();
 
   {
     constexpr int TPR = kD / 4;                       // 32 threads per row, one float4 each
