@@ -432,7 +432,8 @@ static twig_status launch_attn(const AttnParams &p, int batch, int n_splits, cud
 
 int pick_splits(int items, int max_tiles) {
   int s = 1;
-  while (s < 8 && items * s < 2 * 148 && s * 2 <= max_tiles) s *= 2;
+  // double the key splits while all CTAs still fit in one wave of two CTAs per SM
+  while (s < 8 && items * s * 2 <= 2 * 148 && s * 2 <= max_tiles) s *= 2;
   return s;
 }
 
