@@ -1,24 +1,26 @@
 // Tree attention of the verification pass on the 5th-generation tensor cores
 // (Sec. 5.4, Appendix A, Algorithm 2; Eq. 2 with the tree's ancestor mask).
 //
-// One CTA of 128 threads owns up to ROWS query rows (tree node x query head of
-// one kv head) and a share of the key tiles; thread r owns row r, which is also
-// lane r of tensor memory.  Per 64-key tile t:
-//   S(t) = Q K^T   tcgen05.mma, M = 128, N = 64, K = 8 x 16, operands in shared memory;
-//                  it is issued one tile ahead, so it runs while tile t-1 is in its softmax
-//   softmax step   tcgen05.ld of the row, running max / sum, P (bf16) back to shared memory
-//   O += P V       tcgen05.mma, M = 128, N = 128, K = 4 x 16, V read MN-major (no transpose
-//                  copy), accumulating in tensor memory across tiles
+// One CTA owns up to ROWS query rows (tree node x query head of one kv head) and a
+// share of the 64-key tiles.  Its six warps have three roles that only meet at mbarriers:
+//   warp 4 (loader)   copies K and V tiles (16 KB units: K0 V0 K1 V1 ...) into a ring of five
+//                     slots with 16-byte cp.async, in the 128-byte-swizzled layout the matrix
+//                     descriptors name; it keeps three units in flight and refills a slot when
+//                     the MMA that read it has completed;
+//   warp 5 (issuer)   one thread issues S(t) = Q K(t)^T (tcgen05.mma, M = 128, N = 64, K = 8 x 16)
+//                     two tiles ahead into a double-buffered S in tensor memory, and
+//                     O += P(t) V(t) (M = 128, N = 128, K = 4 x 16, V read MN-major, accumulating
+//                     in tensor memory) as soon as the softmax warps have published P(t);
+//   warps 0-3 (softmax) thread r owns row r = tensor-memory lane r: tcgen05.ld of its S row,
+//                     running max / sum, P (bf16) back to shared memory.
 // The running maximum is only raised when a tile exceeds it by more than 2^8; then (rarely)
 // the O accumulator is rescaled in tensor memory (ld, multiply, st).  P stays below 2^8,
 // which bf16 and the fp32 sums hold without loss of accuracy.
-// K and V tiles travel separately through a ring of five 16 KB slots, filled by 16-byte
-// cp.async in the 128-byte-swizzled layout that the matrix descriptors name; a K slot is
-// refilled as soon as its S product has completed, a V slot after its P V product.
 // The instruction always multiplies 128 rows; rows past ROWS read whatever follows in
 // shared memory and land in lanes nobody reads.  Key splits of a cluster are merged
 // through distributed shared memory as in the mma.sync kernel (each CTA pushes its
 // per-row partial to the row's owner); without splits every thread stores its own row.
+// Every wait is bounded: if one runs out the request is flagged TWIG_DEV_INTERNAL.
 #include <cooperative_groups.h>
 
 #include "tree_attn.cuh"
@@ -31,7 +33,7 @@ namespace {
 
 constexpr int kD = 128;          // head_dim
 constexpr int kKT = 64;          // keys per tile
-constexpr int kThreads = 128;
+constexpr int kThreads = 192;          // warps 0-3 softmax, warp 4 loader, warp 5 MMA issuer
 constexpr int kSlots = 5;                         // ring of K / V tiles (K0 V0 K1 V1 K2 ...)
 constexpr int kTileBytes = kKT * kD * 2;          // one K (or V) tile: 16 KB
 constexpr int kPanelBytes = kKT * 128;            // 64-column panel of a K/V tile
@@ -72,9 +74,16 @@ __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.a
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-// Bounded wait on an mbarrier phase; false when the limit ran out.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+// Bounded wait on an mbarrier phase; false when the limit ran out or another role has failed.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *fail) {
   for (int i = 0; i < kSpinLimit; ++i) {
+    if ((i & 1023) == 1023 && *fail) return false;
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
@@ -127,18 +136,20 @@ tree_attn_umma_kernel(const AttnParams p) {
   __shared__ unsigned long long s_mask[TWIG_MAX_NODES];
   __shared__ int s_par[TWIG_MAX_NODES];
   __shared__ float r_m[ROWS], r_l[ROWS];
-  __shared__ __align__(8) unsigned long long s_bar[2];
+  // barriers: full[5], empty[5] (ring slots), s_ready[2], p_ready, o_done
+  __shared__ __align__(8) unsigned long long s_bar[2 * kSlots + 4];
   __shared__ uint32_t s_tmem;
-  __shared__ int s_bad;
+  __shared__ int s_bad, s_fail;
 
   cg::cluster_group cluster = cg::this_cluster();
-  const int tid = threadIdx.x, warp = tid >> 5;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int split = blockIdx.x, n_splits = gridDim.x;
   const int hk = blockIdx.y / p.row_blocks, rb = blockIdx.y % p.row_blocks;
   const int b = blockIdx.z;
 
   // ---- per-request metadata; every exit below is uniform over the cluster ----
   const int n = p.n_nodes[b], L = p.kv_len[b];
+  const int my_parent = tid < p.t_max ? p.parent[(long long)b * p.t_max + tid] : -1;
   if (n == 0) return;
   const bool first = split == 0 && blockIdx.y == 0 && tid == 0;
   if (n < 0 || n > p.t_max) {
@@ -155,86 +166,34 @@ tree_attn_umma_kernel(const AttnParams p) {
   const uint32_t q_s = smem_u32(smem);
   const uint32_t p_s = q_s + C::Q_BYTES;
   const uint32_t ring_s = p_s + C::P_BYTES;
+  const uint32_t bars = smem_u32(s_bar);
+  auto bar_full = [&](int slot) { return bars + 8 * slot; };
+  auto bar_empty = [&](int slot) { return bars + 8 * (kSlots + slot); };
+  auto bar_s = [&](int buf) { return bars + 8 * (2 * kSlots + buf); };
+  const uint32_t bar_p = bars + 8 * (2 * kSlots + 2), bar_o = bars + 8 * (2 * kSlots + 3);
 
   const int NK = L + n;
   const int n_tiles = (NK + kKT - 1) / kKT;
   const int per = (n_tiles + n_splits - 1) / n_splits;
   const int t_begin = split * per;
   const int t_end = min(n_tiles, t_begin + per);
+  const int n_my = max(0, t_end - t_begin);
+  // softmax warps that own rows of this request (a prefix of warps 0-3)
+  const int n_soft = min(ROWS / 32, (rows_total - row0 + 31) / 32);
 
-  const __nv_bfloat16 *ck = p.cache_k + b * p.c_sb + hk * p.c_sh;
-  const __nv_bfloat16 *cv = p.cache_v + b * p.c_sb + hk * p.c_sh;
-  const __nv_bfloat16 *tk = p.tree_k + ((long long)b * p.n_kv_heads + hk) * p.t_max * kD;
-  const __nv_bfloat16 *tv = p.tree_v + ((long long)b * p.n_kv_heads + hk) * p.t_max * kD;
-
-  // A thread copies chunk (tid & 15) of rows (tid >> 4) + 8 i, i = 0..7, of a K or V tile.
-  // Unit u of this CTA is K (u even) or V (u odd) of its tile u / 2.
-  const int ld_c = tid & 15, ld_r0 = tid >> 4;
-  const uint32_t ld_off0 = (uint32_t)((ld_c >> 3) * kPanelBytes + ld_r0 * 128 + (((ld_c & 7) ^ (ld_r0 & 7)) << 4));
-  auto load_unit = [&](int u, int slot) {
-    const int t = t_begin + (u >> 1);
-    if (t >= t_end) return;
-    const uint32_t dst = ring_s + slot * kTileBytes + ld_off0;
-    const __nv_bfloat16 *cbase = (u & 1) ? cv : ck, *tbase = (u & 1) ? tv : tk;
-    const int j0 = t * kKT + ld_r0;
-    if (t * kKT + kKT <= L) {               // whole tile inside the cached prefix
-      const __nv_bfloat16 *src = cbase + (long long)j0 * p.c_sp + ld_c * 8;
-      const long long step = 8 * p.c_sp;
-#pragma unroll
-      for (int i = 0; i < 8; ++i)           // rows 8 apart keep (row & 7): same swizzle, +1024 bytes
-        cp_async_16(dst + i * 1024, src + i * step, true);
-    } else {
-#pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        const int vj = j0 + 8 * i;
-        const __nv_bfloat16 *src = cbase;
-        bool valid = false;
-        if (vj < L) {
-          src = cbase + (long long)vj * p.c_sp + ld_c * 8;
-          valid = true;
-        } else if (vj < NK) {
-          src = tbase + (vj - L) * kD + ld_c * 8;
-          valid = true;
-        }
-        cp_async_16(dst + i * 1024, src, valid);
-      }
-    }
-  };
-
-  // ---- start the copies: Q (zero rows past the last row) and the first key tiles ----
-#pragma unroll
-  for (int i = 0; i < ROWS / 8; ++i) {
-    const int r = ld_r0 + 8 * i;
-    const int gr = row0 + r;
-    const bool valid = gr < rows_total;
-    const int node = valid ? gr / p.group : 0, g = valid ? gr % p.group : 0;
-    const __nv_bfloat16 *src =
-        p.q + (((long long)b * p.t_max + node) * p.n_q_heads + hk * p.group + g) * kD + ld_c * 8;
-    cp_async_16(q_s + (ld_c >> 3) * ROWS * 128 + r * 128 + (((ld_c & 7) ^ (r & 7)) << 4), src, valid);
+  // ---- parents, validation, ancestor masks; barriers; tensor memory ---------------
+  if (tid == 0) {
+    s_bad = 0;
+    s_fail = 0;
   }
-  // Ring slots: K(0) in 0, K(t) in 2 (t odd) or 4 (t even); V(t) in 1, 3, 0 for t mod 3 = 0, 1, 2.
-  // Units are issued in order, one commit group each: 0..4 here, V(2) when K(0) has been
-  // consumed, then K(t+2) when K(t) has been consumed and V(t+2) when V(t-1) has been.
-  auto slot_k = [](int t) { return t == 0 ? 0 : ((t & 1) ? 2 : 4); };
-  auto slot_v = [](int t) { return t % 3 == 0 ? 1 : (t % 3 == 1 ? 3 : 0); };
-#pragma unroll
-  for (int u = 0; u < kSlots; ++u) {
-    load_unit(u, u);
-    cp_async_commit();              // the first group also carries Q
-  }
-
-  // ---- while they fly: parents, validation, ancestor masks ---------------------
-  if (tid == 0) s_bad = 0;
   __syncthreads();
   if (tid < n) {
-    const int pr = p.parent[(long long)b * p.t_max + tid];
-    s_par[tid] = pr;
-    if ((tid == 0) ? (pr != -1) : (pr < 0 || pr >= tid)) s_bad = 1;
+    s_par[tid] = my_parent;
+    if ((tid == 0) ? (my_parent != -1) : (my_parent < 0 || my_parent >= tid)) s_bad = 1;
   }
   __syncthreads();
   if (s_bad) {
     if (first) flag_status(p.dev_status, b, TWIG_DEV_BAD_TREE);
-    cp_async_wait<0>();
     return;
   }
   if (tid < n) {
@@ -246,89 +205,148 @@ tree_attn_umma_kernel(const AttnParams p) {
     }
     s_mask[tid] = m;
   }
-  // tensor memory and the two completion barriers (S ready, O tile ready)
-  const uint32_t bar_s = smem_u32(&s_bar[0]), bar_o = smem_u32(&s_bar[1]);
-  if (warp == 0) {
+  if (tid == 0) {
+    for (int i = 0; i < kSlots; ++i) {
+      mbar_init(bar_full(i), 32);       // every loader lane arrives once per unit
+      mbar_init(bar_empty(i), 1);       // one tcgen05.commit
+    }
+    mbar_init(bar_s(0), 1);
+    mbar_init(bar_s(1), 1);
+    mbar_init(bar_p, n_soft);           // one arrival per softmax warp
+    mbar_init(bar_o, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 5) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem)), "r"(kTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-  }
-  if (tid == 0) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_s) : "memory");
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_o) : "memory");
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = s_tmem;
-  const uint32_t t_lane = tmem + ((uint32_t)(warp * 32) << 16);     // this warp's 32 lanes
   const uint32_t tmem_o = tmem + 128;
+  volatile int *fail = &s_fail;
 
-  // ---- per-thread state: thread r owns row r ------------------------------------
-  const bool warp_rows = warp * 32 < ROWS && row0 + warp * 32 < rows_total;   // warp-uniform
+  // per-row state of the softmax threads (also used by the epilogue)
   const int gr = row0 + tid;
   const bool row_valid = tid < ROWS && gr < rows_total;
-  const unsigned long long my_mask = row_valid ? s_mask[gr / p.group] : 0ull;
   float m_run = -INFINITY, l_run = 0.f;     // m_run is in the exp2 domain (scaled logits)
-  uint32_t ph_s = 0, ph_o = 0;
-  constexpr uint32_t kIdescS = instr_desc(kKT, false), kIdescO = instr_desc(kD, true);
-  const int n_my = t_end - t_begin;
-  bool ok = true;
-  // the thread that issues the MMAs sits in a warp without rows where there is one, so that
-  // the (blocking) issue does not hold back a warp's softmax
-  constexpr int kIssuer = ROWS <= 64 ? 96 : 0;
+  const uint32_t t_lane = tmem + ((uint32_t)((warp & 3) * 32) << 16);     // this warp's 32 lanes
 
-  auto issue_s = [&](int it) {              // S(it) = Q K(it)^T into S buffer it & 1
-    const uint32_t kb = ring_s + slot_k(it) * kTileBytes;
-#pragma unroll
-    for (int ks = 0; ks < kD / 16; ++ks) {
-      const uint32_t qa = q_s + (ks >> 2) * ROWS * 128 + (ks & 3) * 32;
-      const uint32_t ka = kb + (ks >> 2) * kPanelBytes + (ks & 3) * 32;
-      umma(tmem + (it & 1) * kKT, smem_desc(qa, 16), smem_desc(ka, 16), kIdescS, ks > 0);
+  if (warp == 4) {
+    // ================= loader =================
+    const __nv_bfloat16 *ck = p.cache_k + b * p.c_sb + hk * p.c_sh;
+    const __nv_bfloat16 *cv = p.cache_v + b * p.c_sb + hk * p.c_sh;
+    const __nv_bfloat16 *tk = p.tree_k + ((long long)b * p.n_kv_heads + hk) * p.t_max * kD;
+    const __nv_bfloat16 *tv = p.tree_v + ((long long)b * p.n_kv_heads + hk) * p.t_max * kD;
+    const int c = lane & 15, rbase = lane >> 4;      // chunk c of rows rbase, rbase + 2, ...
+    const uint32_t panel = (uint32_t)((c >> 3) * kPanelBytes);
+    // Q tile (zero rows past the request's last row): part of the first commit group
+    for (int r = rbase; r < ROWS && n_my > 0; r += 2) {
+      const int grow = row0 + r;
+      const bool valid = grow < rows_total;
+      const int node = valid ? grow / p.group : 0, g = valid ? grow % p.group : 0;
+      const __nv_bfloat16 *src =
+          p.q + (((long long)b * p.t_max + node) * p.n_q_heads + hk * p.group + g) * kD + c * 8;
+      cp_async_16(q_s + (c >> 3) * ROWS * 128 + r * 128 + (((c & 7) ^ (r & 7)) << 4), src, valid);
     }
-    umma_commit(bar_s);
-  };
-
-  if (n_my > 0) {
-    cp_async_wait<kSlots - 1>();   // Q and K(0) have landed
-    fence_async_smem();            // make the copied bytes visible to the tensor core's reads
-    __syncthreads();
-    if (tid == kIssuer) {
-      tc_fence_after();
-      issue_s(0);
-    }
-  }
-
-  for (int it = 0; it < n_my; ++it) {
-    const int t = t_begin + it;
-    // S(it) is ready, so K(it)'s slot is free
-    if (ok) ok = mbar_wait(bar_s, ph_s);
-    ok = __all_sync(0xffffffffu, ok);
-    ph_s ^= 1;
-    tc_fence_after();
-    if (ok) {
-      if (it == 0) load_unit(5, slot_v(2)); else load_unit(2 * it + 4, slot_k(it + 2));
-    }
-    cp_async_commit();
-    // K(it+1) and V(it) have landed: start S(it+1) so that it runs under this tile's softmax
-    cp_async_wait<2>();
-    fence_async_smem();
-    tc_fence_before();
-    ok = __syncthreads_and(ok);
-    if (tid == kIssuer && ok && it + 1 < n_my) {
-      tc_fence_after();
-      issue_s(it + 1);
-    }
-    // the previous P V product must be complete before P is overwritten or O is rescaled
-    if (it > 0) {
-      if (ok) ok = mbar_wait(bar_o, ph_o);
-      ok = __all_sync(0xffffffffu, ok);
-      ph_o ^= 1;
-      tc_fence_after();
-      if (ok) load_unit(2 * it + 5, slot_v(it + 2));
+    const int n_units = 2 * n_my;
+    bool ok = true;
+    for (int u = 0; u < n_units && ok; ++u) {
+      const int slot = u % kSlots, round = u / kSlots;
+      if (round > 0) ok = mbar_wait(bar_empty(slot), (round - 1) & 1, fail);
+      if (!ok) break;
+      const int t = t_begin + (u >> 1);
+      const uint32_t dst = ring_s + slot * kTileBytes + panel;
+      const __nv_bfloat16 *cbase = (u & 1) ? cv : ck, *tbase = (u & 1) ? tv : tk;
+      if (t * kKT + kKT <= L) {                 // whole tile inside the cached prefix
+        const __nv_bfloat16 *src = cbase + (long long)(t * kKT + rbase) * p.c_sp + c * 8;
+        const long long step = 2 * p.c_sp;
+#pragma unroll 8
+        for (int i = 0; i < kKT / 2; ++i) {
+          const int r = rbase + 2 * i;
+          cp_async_16(dst + r * 128 + (((c & 7) ^ (r & 7)) << 4), src + i * step, true);
+        }
+      } else {
+#pragma unroll 4
+        for (int i = 0; i < kKT / 2; ++i) {
+          const int r = rbase + 2 * i;
+          const int vj = t * kKT + r;
+          const __nv_bfloat16 *src = cbase;
+          bool valid = false;
+          if (vj < L) {
+            src = cbase + (long long)vj * p.c_sp + c * 8;
+            valid = true;
+          } else if (vj < NK) {
+            src = tbase + (vj - L) * kD + c * 8;
+            valid = true;
+          }
+          cp_async_16(dst + r * 128 + (((c & 7) ^ (r & 7)) << 4), src, valid);
+        }
+      }
       cp_async_commit();
+      if (u >= 3) {                             // unit u-3 has landed: publish it
+        cp_async_wait<3>();
+        fence_async_smem();
+        mbar_arrive(bar_full((u - 3) % kSlots));
+      }
     }
-    if (warp_rows && ok) {
+    cp_async_wait<0>();
+    fence_async_smem();
+    if (ok)
+      for (int u = max(0, n_units - 3); u < n_units; ++u) mbar_arrive(bar_full(u % kSlots));
+    if (!ok) s_fail = 1;
+  } else if (warp == 5) {
+    // ================= MMA issuer (one thread) =================
+    if (lane == 0) {
+      constexpr uint32_t kIdescS = instr_desc(kKT, false), kIdescO = instr_desc(kD, true);
+      bool ok = true;
+      auto wait_full = [&](int u) {
+        if (ok) ok = mbar_wait(bar_full(u % kSlots), (u / kSlots) & 1, fail);
+        fence_async_smem();
+        tc_fence_after();
+      };
+      auto issue_s = [&](int it) {            // S(it) = Q K(it)^T into S buffer it & 1
+        const int u = 2 * it;
+        wait_full(u);
+        if (!ok) return;
+        const uint32_t kb = ring_s + (u % kSlots) * kTileBytes;
+#pragma unroll
+        for (int ks = 0; ks < kD / 16; ++ks) {
+          const uint32_t qa = q_s + (ks >> 2) * ROWS * 128 + (ks & 3) * 32;
+          const uint32_t ka = kb + (ks >> 2) * kPanelBytes + (ks & 3) * 32;
+          umma(tmem + (it & 1) * kKT, smem_desc(qa, 16), smem_desc(ka, 16), kIdescS, ks > 0);
+        }
+        umma_commit(bar_s(it & 1));
+        umma_commit(bar_empty(u % kSlots));
+      };
+      if (n_my > 0) issue_s(0);
+      if (n_my > 1) issue_s(1);
+      for (int it = 0; it < n_my && ok; ++it) {
+        const int u = 2 * it + 1;
+        ok = mbar_wait(bar_p, it & 1, fail);          // P(it) is in shared memory, S(it) has been read
+        wait_full(u);
+        if (!ok) break;
+        const uint32_t vb = ring_s + (u % kSlots) * kTileBytes;
+#pragma unroll
+        for (int j = 0; j < kKT / 16; ++j)
+          umma(tmem_o, smem_desc(p_s + j * 32, 16), smem_desc(vb + j * 2048, kPanelBytes), kIdescO, (it > 0) || (j > 0));
+        umma_commit(bar_o);
+        umma_commit(bar_empty(u % kSlots));
+        if (it + 2 < n_my) issue_s(it + 2);
+      }
+      if (!ok) s_fail = 1;
+    }
+  } else if (warp < n_soft) {
+    // ================= softmax: thread r owns row r =================
+    const unsigned long long my_mask = row_valid ? s_mask[gr / p.group] : 0ull;
+    bool ok = true;
+    for (int it = 0; it < n_my; ++it) {
+      const int t = t_begin + it;
+      ok = mbar_wait(bar_s(it & 1), (it >> 1) & 1, fail);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
       uint32_t sr[2][32];
       const uint32_t ts = t_lane + (it & 1) * kKT;
       tmem_ld32(ts, sr[0]);
@@ -354,19 +372,25 @@ tree_attn_umma_kernel(const AttnParams p) {
       const bool raise = mx > m_run + kLazyMax;   // also true for the first finite maximum
       const float m_new = raise ? mx : m_run;
       const float m_use = m_new == -INFINITY ? 0.f : m_new;
-      if (__any_sync(0xffffffffu, raise && it > 0)) {
-        const float alpha = fast_exp2(m_run - m_use);     // 1 for rows that keep their maximum
-        l_run *= alpha;
+      if (it > 0) {                               // P is free and O is stable once P(it-1) V(it-1) is done
+        ok = mbar_wait(bar_o, (it - 1) & 1, fail);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after();
+        if (__any_sync(0xffffffffu, raise)) {
+          const float alpha = fast_exp2(m_run - m_use);   // 1 for rows that keep their maximum
+          l_run *= alpha;
 #pragma unroll
-        for (int ch = 0; ch < 4; ++ch) {
-          uint32_t v[32];
-          tmem_ld32(t_lane + 128 + ch * 32, v);
-          tmem_ld_wait();
+          for (int ch = 0; ch < 4; ++ch) {
+            uint32_t v[32];
+            tmem_ld32(t_lane + 128 + ch * 32, v);
+            tmem_ld_wait();
 #pragma unroll
-          for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) * alpha);
-          tmem_st32(t_lane + 128 + ch * 32, v);
+            for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) * alpha);
+            tmem_st32(t_lane + 128 + ch * 32, v);
+          }
+          tmem_st_wait();
         }
-        tmem_st_wait();
       }
       m_run = m_new;
       float sum0 = 0.f, sum1 = 0.f;
@@ -387,61 +411,52 @@ tree_attn_umma_kernel(const AttnParams p) {
                      "r"(w[2]), "r"(w[3]) : "memory");
       }
       l_run += sum0 + sum1;
+      fence_async_smem();            // P was written with ordinary stores
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_p);
     }
-    fence_async_smem();            // P was written with ordinary stores
-    tc_fence_before();
-    ok = __syncthreads_and(ok);
-    if (tid == kIssuer && ok) {
+    if (ok && n_my > 0) {
+      ok = mbar_wait(bar_o, (n_my - 1) & 1, fail);   // the last P V product has completed
       tc_fence_after();
-      const uint32_t vb = ring_s + slot_v(it) * kTileBytes;
-#pragma unroll
-      for (int j = 0; j < kKT / 16; ++j)
-        umma(tmem_o, smem_desc(p_s + j * 32, 16), smem_desc(vb + j * 2048, kPanelBytes), kIdescO, (it > 0) || (j > 0));
-      umma_commit(bar_o);
     }
+    if (!ok) s_fail = 1;
   }
-  // the accumulated O of this CTA's tiles
-  float o[kD];
-  if (n_my > 0 && ok) ok = mbar_wait(bar_o, ph_o);
-  ok = __all_sync(0xffffffffu, ok);
-  tc_fence_after();
-  if (n_my > 0 && warp_rows && ok) {
-#pragma unroll
-    for (int ch = 0; ch < 4; ++ch) {
-      uint32_t v[32];
-      tmem_ld32(t_lane + 128 + ch * 32, v);
-      tmem_ld_wait();
-#pragma unroll
-      for (int j = 0; j < 32; ++j) o[ch * 32 + j] = __uint_as_float(v[j]);
-    }
-  } else {
-#pragma unroll
-    for (int i = 0; i < kD; ++i) o[i] = 0.f;
-  }
-  cp_async_wait<0>();
-  tc_fence_before();
-  ok = __syncthreads_and(ok);
-  if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+  __syncthreads();
+  const bool ok = s_fail == 0;
   if (!ok && tid == 0) flag_status(p.dev_status, b, TWIG_DEV_INTERNAL);
+  const bool have_o = n_my > 0 && warp < n_soft && ok;      // this thread's O row is in tensor memory
 
-  // ---- no key splits: every thread finishes and stores its own row -------------------
   if (n_splits == 1) {
-    if (row_valid && ok) {
+    // ---- no key splits: every thread finishes and stores its own row ---------------
+    if (have_o) {                           // warp-uniform: the tensor-memory loads need the whole warp
       const float inv = 1.f / l_run;
-      const int node = gr / p.group, g = gr % p.group;
+      const int node = row_valid ? gr / p.group : 0, g = row_valid ? gr % p.group : 0;
       const int h = hk * p.group + g;
       __nv_bfloat16 *dst = p.out + (((long long)b * p.t_max + node) * p.n_q_heads + h) * kD;
 #pragma unroll
-      for (int c = 0; c < kD / 8; ++c) {
-        uint4 w;
-        w.x = pack_bf16(o[8 * c] * inv, o[8 * c + 1] * inv);
-        w.y = pack_bf16(o[8 * c + 2] * inv, o[8 * c + 3] * inv);
-        w.z = pack_bf16(o[8 * c + 4] * inv, o[8 * c + 5] * inv);
-        w.w = pack_bf16(o[8 * c + 6] * inv, o[8 * c + 7] * inv);
-        st_16(dst + 8 * c, w);
+      for (int ch = 0; ch < 4; ++ch) {
+        uint32_t v[32];
+        tmem_ld32(t_lane + 128 + ch * 32, v);
+        tmem_ld_wait();
+        if (row_valid) {
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            uint4 w;
+            w.x = pack_bf16(__uint_as_float(v[8 * c]) * inv, __uint_as_float(v[8 * c + 1]) * inv);
+            w.y = pack_bf16(__uint_as_float(v[8 * c + 2]) * inv, __uint_as_float(v[8 * c + 3]) * inv);
+            w.z = pack_bf16(__uint_as_float(v[8 * c + 4]) * inv, __uint_as_float(v[8 * c + 5]) * inv);
+            w.w = pack_bf16(__uint_as_float(v[8 * c + 6]) * inv, __uint_as_float(v[8 * c + 7]) * inv);
+            st_16(dst + ch * 32 + 8 * c, w);
+          }
+        }
       }
-      if (p.lse) p.lse[((long long)b * p.n_q_heads + h) * p.t_max + node] = (m_run + log2f(l_run)) * 0.6931471805599453f;
+      if (p.lse && row_valid)
+        p.lse[((long long)b * p.n_q_heads + h) * p.t_max + node] = (m_run + log2f(l_run)) * 0.6931471805599453f;
     }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 5) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
     return;
   }
 
@@ -452,17 +467,29 @@ tree_attn_umma_kernel(const AttnParams p) {
   if (tid < ROWS) {
     const int owner = tid / rows_per, lr = tid % rows_per;
     const int slot = split * rows_per + lr;
-    float *ro = recv + (size_t)slot * kD, *rm = r_m + slot, *rl = r_l + slot;
-    ro = cluster.map_shared_rank(ro, owner);
-    rm = cluster.map_shared_rank(rm, owner);
-    rl = cluster.map_shared_rank(rl, owner);
+    float *ro = cluster.map_shared_rank(recv + (size_t)slot * kD, owner);
 #pragma unroll
-    for (int i = 0; i < kD / 4; ++i)        // float4 slots are XOR-swizzled by the row to spread banks
-      *reinterpret_cast<float4 *>(ro + ((i ^ (lr & 31)) << 2)) = make_float4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
-    *rm = m_run;
-    *rl = l_run;
+    for (int ch = 0; ch < 4; ++ch) {
+      uint32_t v[32];
+      if (have_o) {                         // warp-uniform
+        tmem_ld32(t_lane + 128 + ch * 32, v);
+        tmem_ld_wait();
+      } else {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) v[j] = 0u;
+      }
+#pragma unroll
+      for (int i = 0; i < 8; ++i)           // float4 slots are XOR-swizzled by the row to spread banks
+        *reinterpret_cast<float4 *>(ro + (((ch * 8 + i) ^ (lr & 31)) << 2)) =
+            make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]), __uint_as_float(v[4 * i + 2]),
+                        __uint_as_float(v[4 * i + 3]));
+    }
+    *cluster.map_shared_rank(r_m + slot, owner) = m_run;
+    *cluster.map_shared_rank(r_l + slot, owner) = l_run;
   }
+  tc_fence_before();
   cluster.sync();
+  if (warp == 5) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
 
   {
     constexpr int TPR = kD / 4;                       // 32 threads per row, one float4 each
