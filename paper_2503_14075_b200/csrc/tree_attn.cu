@@ -491,6 +491,12 @@ extern "C" twig_status tree_verify_attention(const void *q, const void *tree_k, 
   p.tree_v = static_cast<const __nv_bfloat16 *>(tree_v);
   p.cache_k = static_cast<const __nv_bfloat16 *>(cache->k) + layer * cache->stride_layer;
   p.cache_v = static_cast<const __nv_bfloat16 *>(cache->v) + layer * cache->stride_layer;
+  p.cache_k0 = static_cast<const __nv_bfloat16 *>(cache->k);
+  p.cache_v0 = static_cast<const __nv_bfloat16 *>(cache->v);
+  p.c_sl = cache->stride_layer;
+  p.layer = layer;
+  p.n_layers = cache->n_layers;
+  p.batch = cache->batch;
   p.c_sb = cache->stride_batch;
   p.c_sh = cache->stride_head;
   p.c_sp = cache->stride_pos;
@@ -510,8 +516,11 @@ extern "C" twig_status tree_verify_attention(const void *q, const void *tree_k, 
   p.scale_log2 = scale * 1.4426950408889634f;
   const int rows = t_max * p.group;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (cache->head_dim == 128 && (g_attention_path == 2 || (g_attention_path == 0 && rows > 32)))
-    return launch_tree_attn_umma(p, cache->batch, rows, st);
+  if (cache->head_dim == 128 && softmax_scale >= 0.f &&
+      (g_attention_path == 2 || (g_attention_path == 0 && rows > 32))) {
+    const twig_status us = launch_tree_attn_umma(p, cache->batch, rows, st);
+    if (us != TWIG_ERR_UNSUPPORTED) return us;     // no tensor map for this layout: use the mma.sync kernel
+  }
   return cache->head_dim == 128 ? dispatch_attn<128>(p, cache->batch, rows, st)
                                 : dispatch_attn<64>(p, cache->batch, rows, st);
 }

@@ -14,6 +14,10 @@ struct AttnParams {
   float *lse;
   int *dev_status;
   int t_max, n_q_heads, n_kv_heads, group, max_len, row_blocks;
+  // whole cache (all layers), for the tensor maps of the tcgen05 path
+  const __nv_bfloat16 *cache_k0, *cache_v0;
+  long long c_sl;
+  int layer, n_layers, batch;
   float scale_log2;   // softmax_scale * log2(e)
 };
 

@@ -3,10 +3,13 @@
 //
 // One CTA owns up to ROWS query rows (tree node x query head of one kv head) and a
 // share of the 64-key tiles.  Its six warps have three roles that only meet at mbarriers:
-//   warp 4 (loader)   copies K and V tiles (16 KB units: K0 V0 K1 V1 ...) into a ring of five
-//                     slots with 16-byte cp.async, in the 128-byte-swizzled layout the matrix
-//                     descriptors name; it keeps three units in flight and refills a slot when
-//                     the MMA that read it has completed;
+//   warp 4 (loader)   brings K and V tiles (16 KB units: K0 V0 K1 V1 ...) into a ring of five
+//                     slots in the 128-byte-swizzled layout the matrix descriptors name: tiles
+//                     that lie wholly in the cached prefix by TMA (two 64 x 64 boxes of a 5-D
+//                     tensor map over the cache, completion counted on the slot's mbarrier),
+//                     the tile that holds the prefix end and the tree's own rows by 16-byte
+//                     cp.async with zero fill; a slot is refilled when the MMA that read it
+//                     has completed;
 //   warp 5 (issuer)   one thread issues S(t) = Q K(t)^T (tcgen05.mma, M = 128, N = 64, K = 8 x 16)
 //                     two tiles ahead into a double-buffered S in tensor memory, and
 //                     O += P(t) V(t) (M = 128, N = 128, K = 4 x 16, V read MN-major, accumulating
@@ -22,6 +25,9 @@
 // per-row partial to the row's owner); without splits every thread stores its own row.
 // Every wait is bounded: if one runs out the request is flagged TWIG_DEV_INTERNAL.
 #include <cooperative_groups.h>
+#include <cuda.h>
+
+#include <mutex>
 
 #include "tree_attn.cuh"
 
@@ -80,6 +86,17 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// One box of the 5-D cache tensor map -> shared memory; completion is counted on `bar`.
+__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int pos,
+                                            int head, int batch, int layer) {
+  asm volatile(
+      "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(x), "r"(pos), "r"(head), "r"(batch), "r"(layer)
+      : "memory");
+}
 // Bounded wait on an mbarrier phase; false when the limit ran out or another role has failed.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *fail) {
   for (int i = 0; i < kSpinLimit; ++i) {
@@ -130,14 +147,15 @@ struct UmmaCfg {
 
 template <int ROWS>
 __global__ void __launch_bounds__(kThreads, 2)
-tree_attn_umma_kernel(const AttnParams p) {
+tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap,
+                      const __grid_constant__ CUtensorMap vmap) {
   using C = UmmaCfg<ROWS>;
   extern __shared__ __align__(1024) unsigned char smem[];
   __shared__ unsigned long long s_mask[TWIG_MAX_NODES];
   __shared__ int s_par[TWIG_MAX_NODES];
   __shared__ float r_m[ROWS], r_l[ROWS];
-  // barriers: full[5], empty[5] (ring slots), s_ready[2], p_ready, o_done
-  __shared__ __align__(8) unsigned long long s_bar[2 * kSlots + 4];
+  // barriers: full[5], empty[5] (ring slots), s_ready[2], p_ready, o_done, q_ready
+  __shared__ __align__(8) unsigned long long s_bar[2 * kSlots + 5];
   __shared__ uint32_t s_tmem;
   __shared__ int s_bad, s_fail;
 
@@ -171,6 +189,7 @@ tree_attn_umma_kernel(const AttnParams p) {
   auto bar_empty = [&](int slot) { return bars + 8 * (kSlots + slot); };
   auto bar_s = [&](int buf) { return bars + 8 * (2 * kSlots + buf); };
   const uint32_t bar_p = bars + 8 * (2 * kSlots + 2), bar_o = bars + 8 * (2 * kSlots + 3);
+  const uint32_t bar_q = bars + 8 * (2 * kSlots + 4);
 
   const int NK = L + n;
   const int n_tiles = (NK + kKT - 1) / kKT;
@@ -214,6 +233,7 @@ tree_attn_umma_kernel(const AttnParams p) {
     mbar_init(bar_s(1), 1);
     mbar_init(bar_p, n_soft);           // one arrival per softmax warp
     mbar_init(bar_o, 1);
+    mbar_init(bar_q, 32);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 5) {
@@ -250,24 +270,38 @@ tree_attn_umma_kernel(const AttnParams p) {
           p.q + (((long long)b * p.t_max + node) * p.n_q_heads + hk * p.group + g) * kD + c * 8;
       cp_async_16(q_s + (c >> 3) * ROWS * 128 + r * 128 + (((c & 7) ^ (r & 7)) << 4), src, valid);
     }
+    cp_async_commit();
+    bool q_published = false;
+    auto publish_q = [&]() {                    // Q has landed: publish it once
+      if (!q_published) {
+        cp_async_wait<0>();
+        fence_async_smem();
+        mbar_arrive(bar_q);
+        q_published = true;
+      }
+    };
     const int n_units = 2 * n_my;
     bool ok = true;
     for (int u = 0; u < n_units && ok; ++u) {
       const int slot = u % kSlots, round = u / kSlots;
-      if (round > 0) ok = mbar_wait(bar_empty(slot), (round - 1) & 1, fail);
+      if (round > 0) {
+        publish_q();                            // (all ring slots are in flight by now)
+        ok = mbar_wait(bar_empty(slot), (round - 1) & 1, fail);
+      }
       if (!ok) break;
       const int t = t_begin + (u >> 1);
-      const uint32_t dst = ring_s + slot * kTileBytes + panel;
-      const __nv_bfloat16 *cbase = (u & 1) ? cv : ck, *tbase = (u & 1) ? tv : tk;
-      if (t * kKT + kKT <= L) {                 // whole tile inside the cached prefix
-        const __nv_bfloat16 *src = cbase + (long long)(t * kKT + rbase) * p.c_sp + c * 8;
-        const long long step = 2 * p.c_sp;
-#pragma unroll 8
-        for (int i = 0; i < kKT / 2; ++i) {
-          const int r = rbase + 2 * i;
-          cp_async_16(dst + r * 128 + (((c & 7) ^ (r & 7)) << 4), src + i * step, true);
+      const uint32_t dst = ring_s + slot * kTileBytes;
+      if (t * kKT + kKT <= L) {                 // whole tile inside the cached prefix: two TMA boxes
+        if (lane == 0) {
+          mbar_arrive_expect_tx(bar_full(slot), kTileBytes);
+          const CUtensorMap *map = (u & 1) ? &vmap : &kmap;
+          tma_load_5d(dst, map, bar_full(slot), 0, t * kKT, hk, b, p.layer);
+          tma_load_5d(dst + kPanelBytes, map, bar_full(slot), 64, t * kKT, hk, b, p.layer);
+        } else {
+          mbar_arrive(bar_full(slot));
         }
-      } else {
+      } else {                                  // prefix end and / or tree rows: cp.async with zero fill
+        const __nv_bfloat16 *cbase = (u & 1) ? cv : ck, *tbase = (u & 1) ? tv : tk;
 #pragma unroll 4
         for (int i = 0; i < kKT / 2; ++i) {
           const int r = rbase + 2 * i;
@@ -281,20 +315,19 @@ tree_attn_umma_kernel(const AttnParams p) {
             src = tbase + (vj - L) * kD + c * 8;
             valid = true;
           }
-          cp_async_16(dst + r * 128 + (((c & 7) ^ (r & 7)) << 4), src, valid);
+          cp_async_16(dst + panel + r * 128 + (((c & 7) ^ (r & 7)) << 4), src, valid);
         }
-      }
-      cp_async_commit();
-      if (u >= 3) {                             // unit u-3 has landed: publish it
-        cp_async_wait<3>();
+        cp_async_commit();
+        cp_async_wait<0>();                     // (this also completes the Q copies)
         fence_async_smem();
-        mbar_arrive(bar_full((u - 3) % kSlots));
+        if (!q_published) {
+          mbar_arrive(bar_q);
+          q_published = true;
+        }
+        mbar_arrive(bar_full(slot));
       }
     }
-    cp_async_wait<0>();
-    fence_async_smem();
-    if (ok)
-      for (int u = max(0, n_units - 3); u < n_units; ++u) mbar_arrive(bar_full(u % kSlots));
+    publish_q();
     if (!ok) s_fail = 1;
   } else if (warp == 5) {
     // ================= MMA issuer (one thread) =================
@@ -320,7 +353,10 @@ tree_attn_umma_kernel(const AttnParams p) {
         umma_commit(bar_s(it & 1));
         umma_commit(bar_empty(u % kSlots));
       };
-      if (n_my > 0) issue_s(0);
+      if (n_my > 0) {
+        ok = mbar_wait(bar_q, 0, fail);         // Q is in shared memory
+        issue_s(0);
+      }
       if (n_my > 1) issue_s(1);
       for (int it = 0; it < n_my && ok; ++it) {
         const int u = 2 * it + 1;
@@ -533,8 +569,74 @@ tree_attn_umma_kernel(const AttnParams p) {
   }
 }
 
+// ---- tensor maps over the whole K and V cache: dims (d, pos, head, batch, layer) ----
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct MapKey {
+  const void *k, *v;
+  long long sl, sb, sh, sp;
+  int n_layers, batch, heads, max_len;
+  bool operator==(const MapKey &o) const {
+    return k == o.k && v == o.v && sl == o.sl && sb == o.sb && sh == o.sh && sp == o.sp && n_layers == o.n_layers &&
+           batch == o.batch && heads == o.heads && max_len == o.max_len;
+  }
+};
+struct MapEntry {
+  MapKey key;
+  alignas(64) CUtensorMap kmap;
+  alignas(64) CUtensorMap vmap;
+  bool valid = false;
+};
+
+static bool encode_cache_map(EncodeTiledFn fn, CUtensorMap *out, const void *base, const MapKey &key) {
+  const cuuint64_t dims[5] = {(cuuint64_t)kD, (cuuint64_t)key.max_len, (cuuint64_t)key.heads, (cuuint64_t)key.batch,
+                              (cuuint64_t)key.n_layers};
+  const cuuint64_t strides[4] = {(cuuint64_t)key.sp * 2, (cuuint64_t)key.sh * 2, (cuuint64_t)key.sb * 2,
+                                 (cuuint64_t)key.sl * 2};
+  const cuuint32_t box[5] = {64, (cuuint32_t)kKT, 1, 1, 1};      // 128 bytes x 64 rows: one swizzled panel
+  const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+  return fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void *>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Returns the (cached) pair of maps for this cache layout, or nullptr when none can be made.
+static const MapEntry *cache_maps(const AttnParams &p) {
+  static std::mutex mu;
+  static EncodeTiledFn fn = nullptr;
+  static bool fn_tried = false;
+  static MapEntry table[16];
+  static int next = 0;
+  std::lock_guard<std::mutex> lock(mu);
+  if (!fn_tried) {
+    fn_tried = true;
+    void *ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  }
+  if (!fn) return nullptr;
+  // strides must be multiples of 16 bytes, and every dimension but the last needs stride * extent in range
+  if (p.c_sp <= 0 || p.c_sh <= 0 || p.c_sb < 0 || p.c_sl < 0) return nullptr;
+  MapKey key{p.cache_k0, p.cache_v0, p.n_layers > 1 ? p.c_sl : p.c_sp, p.batch > 1 ? p.c_sb : p.c_sp, p.c_sh, p.c_sp,
+             p.n_layers, p.batch, p.n_kv_heads, p.max_len};
+  if (p.n_kv_heads == 1) key.sh = key.sp;      // a stride of an extent-1 dimension is never used
+  for (auto &e : table)
+    if (e.valid && e.key == key) return &e;
+  MapEntry &e = table[next];
+  next = (next + 1) % 16;
+  e.valid = false;
+  if (!encode_cache_map(fn, &e.kmap, p.cache_k0, key) || !encode_cache_map(fn, &e.vmap, p.cache_v0, key)) return nullptr;
+  e.key = key;
+  e.valid = true;
+  return &e;
+}
+
 template <int ROWS>
-twig_status launch_umma(const AttnParams &p, int batch, int n_splits, cudaStream_t st) {
+twig_status launch_umma(const AttnParams &p, const MapEntry *maps, int batch, int n_splits, cudaStream_t st) {
   using C = UmmaCfg<ROWS>;
   static bool attr_set = false;
   if (!attr_set) {
@@ -555,7 +657,8 @@ twig_status launch_umma(const AttnParams &p, int batch, int n_splits, cudaStream
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  if (cudaLaunchKernelEx(&cfg, tree_attn_umma_kernel<ROWS>, p) != cudaSuccess) return TWIG_ERR_CUDA;
+  if (cudaLaunchKernelEx(&cfg, tree_attn_umma_kernel<ROWS>, p, maps->kmap, maps->vmap) != cudaSuccess)
+    return TWIG_ERR_CUDA;
   return TWIG_OK;
 }
 
@@ -565,12 +668,14 @@ twig_status launch_tree_attn_umma(AttnParams &p, int batch, int rows, cudaStream
   const int rows_per_cta = rows <= 32 ? 32 : rows <= 64 ? 64 : 128;
   p.row_blocks = (rows + rows_per_cta - 1) / rows_per_cta;
   if ((long long)p.n_kv_heads * p.row_blocks > 65535) return TWIG_ERR_UNSUPPORTED;
+  const MapEntry *maps = cache_maps(p);
+  if (!maps) return TWIG_ERR_UNSUPPORTED;
   const int max_tiles = (p.max_len + p.t_max + kKT - 1) / kKT;
   const int n_splits = pick_splits(batch * p.n_kv_heads * p.row_blocks, max_tiles);
   switch (rows_per_cta) {
-    case 32: return launch_umma<32>(p, batch, n_splits, st);
-    case 64: return launch_umma<64>(p, batch, n_splits, st);
-    default: return launch_umma<128>(p, batch, n_splits, st);
+    case 32: return launch_umma<32>(p, maps, batch, n_splits, st);
+    case 64: return launch_umma<64>(p, maps, batch, n_splits, st);
+    default: return launch_umma<128>(p, maps, batch, n_splits, st);
   }
 }
 
