@@ -14,12 +14,15 @@
 //                     two tiles ahead into a double-buffered S in tensor memory, and
 //                     O += P(t) V(t) (M = 128, N = 128, K = 4 x 16, V read MN-major, accumulating
 //                     in tensor memory) as soon as the softmax warps have published P(t);
-//   warps 0-3 (softmax) thread r owns row r = tensor-memory lane r: tcgen05.ld of its S row,
-//                     running max / sum, P (bf16) back to shared memory.
+//   warps 0-3 (softmax) one thread per row: tcgen05.ld of its S row, running max / sum,
+//                     P (bf16) back to shared memory.  With up to 64 rows the products use
+//                     M = 64, whose accumulator rows sit in lanes 0-15 of each of the four
+//                     32-lane quadrants of tensor memory (row r in lane 32 (r / 16) + r % 16),
+//                     so every warp works on 16 rows; with 128 rows M = 128 and row r is lane r.
 // The running maximum is only raised when a tile exceeds it by more than 2^8; then (rarely)
 // the O accumulator is rescaled in tensor memory (ld, multiply, st).  P stays below 2^8,
 // which bf16 and the fp32 sums hold without loss of accuracy.
-// The instruction always multiplies 128 rows; rows past ROWS read whatever follows in
+// The instruction multiplies 64 or 128 rows; rows past ROWS read whatever follows in
 // shared memory and land in lanes nobody reads.  Key splits of a cluster are merged
 // through distributed shared memory as in the mma.sync kernel (each CTA pushes its
 // per-row partial to the row's owner); without splits every thread stores its own row.
@@ -60,10 +63,10 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes)
   d |= (uint64_t)2 << 61;      // 128-byte swizzle
   return d;
 }
-// Instruction descriptor: bf16 x bf16 -> fp32, M = 128, A K-major.
-__host__ __device__ constexpr uint32_t instr_desc(int n, bool b_mn_major) {
+// Instruction descriptor: bf16 x bf16 -> fp32, M = m (64 or 128), A K-major.
+__host__ __device__ constexpr uint32_t instr_desc(int m, int n, bool b_mn_major) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((uint32_t)(n >> 3) << 17) |
-         ((uint32_t)(128 >> 4) << 24);
+         ((uint32_t)(m >> 4) << 24);
 }
 
 __device__ __forceinline__ void umma(uint32_t tmem_d, uint64_t a, uint64_t b, uint32_t idesc, uint32_t accumulate) {
@@ -143,6 +146,8 @@ struct UmmaCfg {
   static_assert(RECV_BYTES <= RING_BYTES, "split-merge buffer must fit in the stage ring");
   static_assert(Q_BYTES % 1024 == 0 && P_BYTES % 1024 == 0, "swizzled tiles start on 1024 bytes");
   static constexpr int SMEM_BYTES = Q_BYTES + P_BYTES + RING_BYTES;
+  static constexpr int MMA_M = ROWS <= 64 ? 64 : 128;
+  static constexpr int ROWS_PER_WARP = MMA_M == 64 ? 16 : 32;    // rows a softmax warp owns
 };
 
 template <int ROWS>
@@ -198,7 +203,8 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
   const int t_end = min(n_tiles, t_begin + per);
   const int n_my = max(0, t_end - t_begin);
   // softmax warps that own rows of this request (a prefix of warps 0-3)
-  const int n_soft = min(ROWS / 32, (rows_total - row0 + 31) / 32);
+  constexpr int RPW = C::ROWS_PER_WARP;
+  const int n_soft = min((ROWS + RPW - 1) / RPW, (rows_total - row0 + RPW - 1) / RPW);
 
   // ---- parents, validation, ancestor masks; barriers; tensor memory ---------------
   if (tid == 0) {
@@ -248,8 +254,10 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
   volatile int *fail = &s_fail;
 
   // per-row state of the softmax threads (also used by the epilogue)
-  const int gr = row0 + tid;
-  const bool row_valid = tid < ROWS && gr < rows_total;
+  const int row_local = C::MMA_M == 64 ? 16 * warp + lane : tid;
+  const bool row_active = warp < 4 && lane < RPW && row_local < ROWS;
+  const int gr = row0 + row_local;
+  const bool row_valid = row_active && gr < rows_total;
   float m_run = -INFINITY, l_run = 0.f;     // m_run is in the exp2 domain (scaled logits)
   const uint32_t t_lane = tmem + ((uint32_t)((warp & 3) * 32) << 16);     // this warp's 32 lanes
 
@@ -332,7 +340,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
   } else if (warp == 5) {
     // ================= MMA issuer (one thread) =================
     if (lane == 0) {
-      constexpr uint32_t kIdescS = instr_desc(kKT, false), kIdescO = instr_desc(kD, true);
+      constexpr uint32_t kIdescS = instr_desc(C::MMA_M, kKT, false), kIdescO = instr_desc(C::MMA_M, kD, true);
       bool ok = true;
       auto wait_full = [&](int u) {
         if (ok) ok = mbar_wait(bar_full(u % kSlots), (u / kSlots) & 1, fail);
@@ -405,7 +413,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
         mx = fmaxf(mx, fmaxf(fmaxf(__uint_as_float(sr[0][j]), __uint_as_float(sr[0][j + 1])),
                              fmaxf(__uint_as_float(sr[1][j]), __uint_as_float(sr[1][j + 1]))));
       mx *= p.scale_log2;                         // scale > 0, so the max commutes with it
-      const bool raise = mx > m_run + kLazyMax;   // also true for the first finite maximum
+      const bool raise = row_active && mx > m_run + kLazyMax;   // also true for the first finite maximum
       const float m_new = raise ? mx : m_run;
       const float m_use = m_new == -INFINITY ? 0.f : m_new;
       if (it > 0) {                               // P is free and O is stable once P(it-1) V(it-1) is done
@@ -430,7 +438,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
       }
       m_run = m_new;
       float sum0 = 0.f, sum1 = 0.f;
-      const uint32_t prow = p_s + tid * 128;
+      const uint32_t prow = p_s + row_local * 128;
 #pragma unroll
       for (int c = 0; c < 8; ++c) {          // chunk c = keys 8c .. 8c+7 of this row
         uint32_t w[4];
@@ -443,8 +451,9 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
           sum1 += p1;
           w[e] = pack_bf16(p0, p1);
         }
-        asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(prow + ((c ^ (tid & 7)) << 4)), "r"(w[0]), "r"(w[1]),
-                     "r"(w[2]), "r"(w[3]) : "memory");
+        if (row_active)
+          asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(prow + ((c ^ (row_local & 7)) << 4)), "r"(w[0]),
+                       "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
       }
       l_run += sum0 + sum1;
       fence_async_smem();            // P was written with ordinary stores
@@ -500,8 +509,9 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
   const int rows_per = ROWS / n_splits;
   float *recv = reinterpret_cast<float *>(smem + C::Q_BYTES + C::P_BYTES);
   cluster.sync();                          // every CTA has left its key loop: the rings are free
-  if (tid < ROWS) {
-    const int owner = tid / rows_per, lr = tid % rows_per;
+  if (warp < 4) {
+    const int rl_ = row_active ? row_local : 0;
+    const int owner = rl_ / rows_per, lr = rl_ % rows_per;
     const int slot = split * rows_per + lr;
     float *ro = cluster.map_shared_rank(recv + (size_t)slot * kD, owner);
 #pragma unroll
@@ -514,14 +524,18 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
 #pragma unroll
         for (int j = 0; j < 32; ++j) v[j] = 0u;
       }
+      if (row_active) {
 #pragma unroll
-      for (int i = 0; i < 8; ++i)           // float4 slots are XOR-swizzled by the row to spread banks
-        *reinterpret_cast<float4 *>(ro + (((ch * 8 + i) ^ (lr & 31)) << 2)) =
-            make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]), __uint_as_float(v[4 * i + 2]),
-                        __uint_as_float(v[4 * i + 3]));
+        for (int i = 0; i < 8; ++i)         // float4 slots are XOR-swizzled by the row to spread banks
+          *reinterpret_cast<float4 *>(ro + (((ch * 8 + i) ^ (lr & 31)) << 2)) =
+              make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]), __uint_as_float(v[4 * i + 2]),
+                          __uint_as_float(v[4 * i + 3]));
+      }
     }
-    *cluster.map_shared_rank(r_m + slot, owner) = m_run;
-    *cluster.map_shared_rank(r_l + slot, owner) = l_run;
+    if (row_active) {
+      *cluster.map_shared_rank(r_m + slot, owner) = m_run;
+      *cluster.map_shared_rank(r_l + slot, owner) = l_run;
+    }
   }
   tc_fence_before();
   cluster.sync();
