@@ -202,6 +202,7 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device(dev))
     wl = synth.workload(args.workload)
     peaks = load_peaks()
+    tw.twig_set_attention_path(args.attn_path)
     max_len = ((max(wl.pruned_len) + max(wl.gen_target) + wl.t_max + 8 + 31) // 32) * 32
 
     reps = [Replica(wl, 100 + rank * N_ROT + r, torch, tw, dev, max_len) for r in range(N_ROT)]
@@ -605,6 +606,7 @@ def main():
     ap.add_argument("--no-extra", dest="extra", action="store_false",
                     help="skip the HBM-sized launches of the attention and gather kernels")
     ap.add_argument("--cpu-budget", type=float, default=15.0)
+    ap.add_argument("--attn-path", type=int, default=0, help="tree-attention kernel: 0 auto, 1 mma.sync, 2 tcgen05")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
