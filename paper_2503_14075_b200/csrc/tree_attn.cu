@@ -516,8 +516,11 @@ extern "C" twig_status tree_verify_attention(const void *q, const void *tree_k, 
   p.scale_log2 = scale * 1.4426950408889634f;
   const int rows = t_max * p.group;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // automatic choice: the tcgen05 kernel once there are more than 32 query rows per kv head or
+  // enough (request, kv head) pairs to fill the GPU; the mma.sync kernel for small, latency-bound calls
+  const bool big = rows > 32 || (long long)cache->batch * cache->n_kv_heads >= 148;
   if (cache->head_dim == 128 && softmax_scale >= 0.f &&
-      (g_attention_path == 2 || (g_attention_path == 0 && rows > 32))) {
+      (g_attention_path == 2 || (g_attention_path == 0 && big))) {
     const twig_status us = launch_tree_attn_umma(p, cache->batch, rows, st);
     if (us != TWIG_ERR_UNSUPPORTED) return us;     // no tensor map for this layout: use the mma.sync kernel
   }
