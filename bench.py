@@ -203,6 +203,7 @@ def run_ours(args):
     wl = synth.workload(args.workload)
     peaks = load_peaks()
     tw.twig_set_attention_path(args.attn_path)
+    tw.twig_set_attention_splits(args.attn_splits)
     max_len = ((max(wl.pruned_len) + max(wl.gen_target) + wl.t_max + 8 + 31) // 32) * 32
 
     reps = [Replica(wl, 100 + rank * N_ROT + r, torch, tw, dev, max_len) for r in range(N_ROT)]
@@ -597,7 +598,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", type=int, default=2)
@@ -606,6 +607,7 @@ def main():
     ap.add_argument("--no-extra", dest="extra", action="store_false",
                     help="skip the HBM-sized launches of the attention and gather kernels")
     ap.add_argument("--cpu-budget", type=float, default=15.0)
+    ap.add_argument("--attn-splits", type=int, default=0, help="force key splits per cluster (0 auto)")
     ap.add_argument("--attn-path", type=int, default=0, help="tree-attention kernel: 0 auto, 1 mma.sync, 2 tcgen05")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup

@@ -195,6 +195,10 @@ twig_status tree_verify_attention(const void *q, const void *tree_k, const void 
  * the same function; this is a tuning and testing control.  Returns the previous value. */
 int32_t twig_set_attention_path(int32_t path);
 
+/* Forces the number of key splits (CTAs per cluster) of the tree-attention kernels:
+ * 1, 2, 4 or 8; 0 = automatic (default).  A tuning control.  Returns the previous value. */
+int32_t twig_set_attention_splits(int32_t splits);
+
 /* ---- Acceptance + bonus token + KV append, all layers in one call ------------
  * Sec. 5.4 / Appendix A / Algorithm 2.  Node 0 is the last accepted token and is
  * always accepted; child c is accepted iff its parent is and

@@ -430,7 +430,10 @@ static twig_status launch_attn(const AttnParams &p, int batch, int n_splits, cud
   return TWIG_OK;
 }
 
+static int g_forced_splits = 0;
+
 int pick_splits(int items, int max_tiles) {
+  if (g_forced_splits > 0) return g_forced_splits;
   int s = 1;
   // double the key splits while all CTAs still fit in one wave of two CTAs per SM
   while (s < 8 && items * s * 2 <= 2 * 148 && s * 2 <= max_tiles) s *= 2;
@@ -465,6 +468,12 @@ static int g_attention_path = 0;
 extern "C" int32_t twig_set_attention_path(int32_t path) {
   const int prev = g_attention_path;
   if (path >= 0 && path <= 2) g_attention_path = path;
+  return prev;
+}
+
+extern "C" int32_t twig_set_attention_splits(int32_t splits) {
+  const int prev = g_forced_splits;
+  if (splits == 0 || splits == 1 || splits == 2 || splits == 4 || splits == 8) g_forced_splits = splits;
   return prev;
 }
 

@@ -55,6 +55,7 @@ def case_attn(a):
     out = torch.zeros((wl.batch, wl.t_max, wl.n_q_heads, wl.head_dim), dtype=torch.bfloat16, device=DEV)
     cache = tw.KV.of(ck, cv)
     tw.twig_set_attention_path(a.path)
+    tw.twig_set_attention_splits(a.splits)
 
     def run():
         for layer in range(nl):
@@ -134,6 +135,7 @@ def main():
     ap.add_argument("--kv-len", type=int, default=0)
     ap.add_argument("--layers", type=int, default=2)
     ap.add_argument("--iters", type=int, default=3)
+    ap.add_argument("--splits", type=int, default=0, help="force key splits (0 auto)")
     ap.add_argument("--path", type=int, default=0, help="attention kernel: 0 auto, 1 mma.sync, 2 tcgen05")
     a = ap.parse_args()
     {"attn": case_attn, "gather": case_gather, "score": case_score, "accept": case_accept}[a.case](a)

@@ -26,7 +26,7 @@ STATUS_NAMES = {0: "TWIG_OK", 1: "TWIG_ERR_NULL", 2: "TWIG_ERR_SHAPE", 3: "TWIG_
 DEV_OK, DEV_BAD_LAYOUT, DEV_BAD_KEEP, DEV_BAD_INDEX, DEV_BAD_TREE, DEV_OVERFLOW, DEV_INTERNAL = range(7)
 MAX_NODES, MAX_VISUAL, MAX_BATCH = 64, 16384, 4096
 
-EXPORTS = ["twig_status_str", "twig_set_attention_path", "twig_workspace_bytes", "ttp_score", "ttp_score_noalloc", "ttp_topk", "ttp_compact",
+EXPORTS = ["twig_status_str", "twig_set_attention_path", "twig_set_attention_splits", "twig_workspace_bytes", "ttp_score", "ttp_score_noalloc", "ttp_topk", "ttp_compact",
            "ttp_score_topk_compact", "tree_verify_attention", "tree_accept_compact"]
 
 
@@ -60,6 +60,8 @@ _lib.twig_status_str.restype = C.c_char_p
 _lib.twig_status_str.argtypes = [C.c_int]
 _lib.twig_set_attention_path.restype = C.c_int32
 _lib.twig_set_attention_path.argtypes = [C.c_int32]
+_lib.twig_set_attention_splits.restype = C.c_int32
+_lib.twig_set_attention_splits.argtypes = [C.c_int32]
 _lib.twig_workspace_bytes.restype = _sz
 _lib.twig_workspace_bytes.argtypes = [_i32] * 5
 _lib.ttp_score.restype = C.c_int
@@ -105,6 +107,11 @@ def lib_path() -> str:
 def twig_set_attention_path(path: int) -> int:
     """0 automatic, 1 mma.sync kernel, 2 tcgen05 kernel; returns the previous setting."""
     return int(_lib.twig_set_attention_path(int(path)))
+
+
+def twig_set_attention_splits(splits: int) -> int:
+    """Force 1, 2, 4 or 8 key splits per (request, kv head, row block); 0 = automatic."""
+    return int(_lib.twig_set_attention_splits(int(splits)))
 
 
 def twig_workspace_bytes(batch, n_q_heads, head_dim, max_len, max_nodes) -> int:
