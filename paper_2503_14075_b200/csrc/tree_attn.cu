@@ -432,11 +432,11 @@ static twig_status launch_attn(const AttnParams &p, int batch, int n_splits, cud
 
 static int g_forced_splits = 0;
 
-int pick_splits(int items, int max_tiles) {
+int pick_splits(int items, int max_tiles, int ctas_per_sm) {
   if (g_forced_splits > 0) return g_forced_splits;
   int s = 1;
-  // double the key splits while all CTAs still fit in one wave of two CTAs per SM
-  while (s < 8 && items * s * 2 <= 2 * 148 && s * 2 <= max_tiles) s *= 2;
+  // double the key splits while all CTAs still fit in one wave
+  while (s < 8 && items * s * 2 <= ctas_per_sm * 148 && s * 2 <= max_tiles) s *= 2;
   return s;
 }
 
@@ -450,7 +450,7 @@ static twig_status dispatch_attn(AttnParams &p, int batch, int rows, cudaStream_
   p.row_blocks = (rows + rows_per_cta - 1) / rows_per_cta;
   if ((long long)p.n_kv_heads * p.row_blocks > 65535) return TWIG_ERR_UNSUPPORTED;
   const int max_tiles = (p.max_len + p.t_max + 63) / 64;
-  const int n_splits = pick_splits(batch * p.n_kv_heads * p.row_blocks, max_tiles);
+  const int n_splits = pick_splits(batch * p.n_kv_heads * p.row_blocks, max_tiles, 2);
   switch (rows_per_cta) {
     case 16: return launch_attn<C16>(p, batch, n_splits, st);
     case 32: return launch_attn<C32>(p, batch, n_splits, st);

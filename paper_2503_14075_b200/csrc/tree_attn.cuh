@@ -61,6 +61,6 @@ __device__ __forceinline__ float fast_exp2(float x) {
 
 // tcgen05 path (tree_attn_umma.cu): head_dim 128, rows = t_max * group.
 twig_status launch_tree_attn_umma(AttnParams &p, int batch, int rows, cudaStream_t st);
-int pick_splits(int items, int max_tiles);
+int pick_splits(int items, int max_tiles, int ctas_per_sm);
 
 }  // namespace twig

@@ -41,12 +41,8 @@ namespace twig {
 namespace {
 
 constexpr int kD = 128;          // head_dim
-constexpr int kKT = 64;          // keys per tile
 constexpr int kThreads = 192;          // warps 0-3 softmax, warp 4 loader, warp 5 MMA issuer
 constexpr int kSlots = 5;                         // ring of K / V tiles (K0 V0 K1 V1 K2 ...)
-constexpr int kTileBytes = kKT * kD * 2;          // one K (or V) tile: 16 KB
-constexpr int kPanelBytes = kKT * 128;            // 64-column panel of a K/V tile
-constexpr uint32_t kTmemCols = 256;               // S: columns [0,64) and [64,128); O: [128,256)
 constexpr float kLazyMax = 8.f;                   // raise the running max only beyond this (log2 units)
 constexpr int kSpinLimit = 1 << 22;
 
@@ -137,11 +133,18 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
-template <int ROWS>
+// KT = keys per tile: 64 (two CTAs per SM, 256 tensor-memory columns each) or 128 (one CTA per SM
+// with all 512 columns: half as many, twice as large MMA instructions per key).
+template <int ROWS, int KT>
 struct UmmaCfg {
+  static constexpr int TILE_BYTES = KT * kD * 2;         // one K (or V) tile: 16 or 32 KB
+  static constexpr int PANEL_BYTES = KT * 128;           // 64-column panel of a K/V tile
   static constexpr int Q_BYTES = ROWS * kD * 2;          // two 64-column panels of ROWS x 128 B
-  static constexpr int P_BYTES = ROWS * 128;             // ROWS x 64 keys bf16
-  static constexpr int RING_BYTES = kSlots * kTileBytes;
+  static constexpr int P_BYTES = ROWS * KT * 2;          // ROWS x KT keys bf16, KT/64 panels of ROWS x 128 B
+  static constexpr int RING_BYTES = kSlots * TILE_BYTES;
+  static constexpr uint32_t TMEM_COLS = KT == 64 ? 256 : 512;   // S: [0,KT) and [KT,2KT); O: [2KT, 2KT+128)
+  static constexpr uint32_t O_COL = 2 * KT;
+  static constexpr int MIN_CTAS = KT == 64 ? 2 : 1;
   static constexpr int RECV_BYTES = ROWS * kD * 4;
   static_assert(RECV_BYTES <= RING_BYTES, "split-merge buffer must fit in the stage ring");
   static_assert(Q_BYTES % 1024 == 0 && P_BYTES % 1024 == 0, "swizzled tiles start on 1024 bytes");
@@ -150,11 +153,12 @@ struct UmmaCfg {
   static constexpr int ROWS_PER_WARP = MMA_M == 64 ? 16 : 32;    // rows a softmax warp owns
 };
 
-template <int ROWS>
-__global__ void __launch_bounds__(kThreads, 2)
+template <int ROWS, int KT>
+__global__ void __launch_bounds__(kThreads, UmmaCfg<ROWS, KT>::MIN_CTAS)
 tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap,
                       const __grid_constant__ CUtensorMap vmap) {
-  using C = UmmaCfg<ROWS>;
+  using C = UmmaCfg<ROWS, KT>;
+  constexpr int kTileBytes = C::TILE_BYTES, kPanelBytes = C::PANEL_BYTES;
   extern __shared__ __align__(1024) unsigned char smem[];
   __shared__ unsigned long long s_mask[TWIG_MAX_NODES];
   __shared__ int s_par[TWIG_MAX_NODES];
@@ -197,7 +201,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
   const uint32_t bar_q = bars + 8 * (2 * kSlots + 4);
 
   const int NK = L + n;
-  const int n_tiles = (NK + kKT - 1) / kKT;
+  const int n_tiles = (NK + KT - 1) / KT;
   const int per = (n_tiles + n_splits - 1) / n_splits;
   const int t_begin = split * per;
   const int t_end = min(n_tiles, t_begin + per);
@@ -243,14 +247,14 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 5) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem)), "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem)), "r"(C::TMEM_COLS) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = s_tmem;
-  const uint32_t tmem_o = tmem + 128;
+  const uint32_t tmem_o = tmem + C::O_COL;
   volatile int *fail = &s_fail;
 
   // per-row state of the softmax threads (also used by the epilogue)
@@ -299,21 +303,21 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
       if (!ok) break;
       const int t = t_begin + (u >> 1);
       const uint32_t dst = ring_s + slot * kTileBytes;
-      if (t * kKT + kKT <= L) {                 // whole tile inside the cached prefix: two TMA boxes
+      if (t * KT + KT <= L) {                   // whole tile inside the cached prefix: two TMA boxes
         if (lane == 0) {
           mbar_arrive_expect_tx(bar_full(slot), kTileBytes);
           const CUtensorMap *map = (u & 1) ? &vmap : &kmap;
-          tma_load_5d(dst, map, bar_full(slot), 0, t * kKT, hk, b, p.layer);
-          tma_load_5d(dst + kPanelBytes, map, bar_full(slot), 64, t * kKT, hk, b, p.layer);
+          tma_load_5d(dst, map, bar_full(slot), 0, t * KT, hk, b, p.layer);
+          tma_load_5d(dst + kPanelBytes, map, bar_full(slot), 64, t * KT, hk, b, p.layer);
         } else {
           mbar_arrive(bar_full(slot));
         }
       } else {                                  // prefix end and / or tree rows: cp.async with zero fill
         const __nv_bfloat16 *cbase = (u & 1) ? cv : ck, *tbase = (u & 1) ? tv : tk;
 #pragma unroll 4
-        for (int i = 0; i < kKT / 2; ++i) {
+        for (int i = 0; i < KT / 2; ++i) {
           const int r = rbase + 2 * i;
-          const int vj = t * kKT + r;
+          const int vj = t * KT + r;
           const __nv_bfloat16 *src = cbase;
           bool valid = false;
           if (vj < L) {
@@ -340,7 +344,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
   } else if (warp == 5) {
     // ================= MMA issuer (one thread) =================
     if (lane == 0) {
-      constexpr uint32_t kIdescS = instr_desc(C::MMA_M, kKT, false), kIdescO = instr_desc(C::MMA_M, kD, true);
+      constexpr uint32_t kIdescS = instr_desc(C::MMA_M, KT, false), kIdescO = instr_desc(C::MMA_M, kD, true);
       bool ok = true;
       auto wait_full = [&](int u) {
         if (ok) ok = mbar_wait(bar_full(u % kSlots), (u / kSlots) & 1, fail);
@@ -356,7 +360,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
         for (int ks = 0; ks < kD / 16; ++ks) {
           const uint32_t qa = q_s + (ks >> 2) * ROWS * 128 + (ks & 3) * 32;
           const uint32_t ka = kb + (ks >> 2) * kPanelBytes + (ks & 3) * 32;
-          umma(tmem + (it & 1) * kKT, smem_desc(qa, 16), smem_desc(ka, 16), kIdescS, ks > 0);
+          umma(tmem + (it & 1) * KT, smem_desc(qa, 16), smem_desc(ka, 16), kIdescS, ks > 0);
         }
         umma_commit(bar_s(it & 1));
         umma_commit(bar_empty(u % kSlots));
@@ -373,8 +377,9 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
         if (!ok) break;
         const uint32_t vb = ring_s + (u % kSlots) * kTileBytes;
 #pragma unroll
-        for (int j = 0; j < kKT / 16; ++j)
-          umma(tmem_o, smem_desc(p_s + j * 32, 16), smem_desc(vb + j * 2048, kPanelBytes), kIdescO, (it > 0) || (j > 0));
+        for (int j = 0; j < KT / 16; ++j)          // 16 keys per step: P panel j / 4, V rows 16 j ..
+          umma(tmem_o, smem_desc(p_s + (j >> 2) * ROWS * 128 + (j & 3) * 32, 16),
+               smem_desc(vb + j * 2048, kPanelBytes), kIdescO, (it > 0) || (j > 0));
         umma_commit(bar_o);
         umma_commit(bar_empty(u % kSlots));
         if (it + 2 < n_my) issue_s(it + 2);
@@ -391,27 +396,35 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      uint32_t sr[2][32];
-      const uint32_t ts = t_lane + (it & 1) * kKT;
-      tmem_ld32(ts, sr[0]);
-      tmem_ld32(ts + 32, sr[1]);
-      tmem_ld_wait();
-      const int key0 = t * kKT;
-      if (key0 + kKT > L) {        // the tile that holds the prefix end and / or the tree
+      const uint32_t ts = t_lane + (it & 1) * KT;
+      // 64 keys of this row's S; the keys that hold the prefix end and / or the tree are masked
+      auto load_s = [&](int half, uint32_t (&sr)[2][32]) {
+        tmem_ld32(ts + half * 64, sr[0]);
+        tmem_ld32(ts + half * 64 + 32, sr[1]);
+        tmem_ld_wait();
+        const int key0 = t * KT + half * 64;
+        if (key0 + 64 > L) {
 #pragma unroll
-        for (int h = 0; h < 2; ++h)
+          for (int h = 0; h < 2; ++h)
 #pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            const int vj = key0 + h * 32 + j;
-            const bool vis = vj < L || (vj < NK && ((my_mask >> (vj - L)) & 1ull));
-            if (!vis) sr[h][j] = 0xff800000u;     // -inf
-          }
-      }
+            for (int j = 0; j < 32; ++j) {
+              const int vj = key0 + h * 32 + j;
+              const bool vis = vj < L || (vj < NK && ((my_mask >> (vj - L)) & 1ull));
+              if (!vis) sr[h][j] = 0xff800000u;     // -inf
+            }
+        }
+      };
+      // pass 1: the tile's row maximum
       float mx = -INFINITY;
+#pragma unroll 1
+      for (int half = 0; half < KT / 64; ++half) {
+        uint32_t sr[2][32];
+        load_s(half, sr);
 #pragma unroll
-      for (int j = 0; j < 32; j += 2)
-        mx = fmaxf(mx, fmaxf(fmaxf(__uint_as_float(sr[0][j]), __uint_as_float(sr[0][j + 1])),
-                             fmaxf(__uint_as_float(sr[1][j]), __uint_as_float(sr[1][j + 1]))));
+        for (int j = 0; j < 32; j += 2)
+          mx = fmaxf(mx, fmaxf(fmaxf(__uint_as_float(sr[0][j]), __uint_as_float(sr[0][j + 1])),
+                               fmaxf(__uint_as_float(sr[1][j]), __uint_as_float(sr[1][j + 1]))));
+      }
       mx *= p.scale_log2;                         // scale > 0, so the max commutes with it
       const bool raise = row_active && mx > m_run + kLazyMax;   // also true for the first finite maximum
       const float m_new = raise ? mx : m_run;
@@ -427,33 +440,39 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
 #pragma unroll
           for (int ch = 0; ch < 4; ++ch) {
             uint32_t v[32];
-            tmem_ld32(t_lane + 128 + ch * 32, v);
+            tmem_ld32(t_lane + C::O_COL + ch * 32, v);
             tmem_ld_wait();
 #pragma unroll
             for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) * alpha);
-            tmem_st32(t_lane + 128 + ch * 32, v);
+            tmem_st32(t_lane + C::O_COL + ch * 32, v);
           }
           tmem_st_wait();
         }
       }
       m_run = m_new;
+      // pass 2: P = exp2(S * scale - m), row sums, P (bf16) to shared memory
       float sum0 = 0.f, sum1 = 0.f;
-      const uint32_t prow = p_s + row_local * 128;
+#pragma unroll 1
+      for (int half = 0; half < KT / 64; ++half) {
+        uint32_t sr[2][32];
+        load_s(half, sr);
+        const uint32_t prow = p_s + half * ROWS * 128 + row_local * 128;
 #pragma unroll
-      for (int c = 0; c < 8; ++c) {          // chunk c = keys 8c .. 8c+7 of this row
-        uint32_t w[4];
+        for (int c = 0; c < 8; ++c) {          // chunk c = keys 8c .. 8c+7 of this row
+          uint32_t w[4];
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const int j = c * 8 + e * 2;
-          const float p0 = fast_exp2(fmaf(__uint_as_float(sr[j >> 5][j & 31]), p.scale_log2, -m_use));
-          const float p1 = fast_exp2(fmaf(__uint_as_float(sr[(j + 1) >> 5][(j + 1) & 31]), p.scale_log2, -m_use));
-          sum0 += p0;
-          sum1 += p1;
-          w[e] = pack_bf16(p0, p1);
+          for (int e = 0; e < 4; ++e) {
+            const int j = c * 8 + e * 2;
+            const float p0 = fast_exp2(fmaf(__uint_as_float(sr[j >> 5][j & 31]), p.scale_log2, -m_use));
+            const float p1 = fast_exp2(fmaf(__uint_as_float(sr[(j + 1) >> 5][(j + 1) & 31]), p.scale_log2, -m_use));
+            sum0 += p0;
+            sum1 += p1;
+            w[e] = pack_bf16(p0, p1);
+          }
+          if (row_active)
+            asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(prow + ((c ^ (row_local & 7)) << 4)), "r"(w[0]),
+                         "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
         }
-        if (row_active)
-          asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(prow + ((c ^ (row_local & 7)) << 4)), "r"(w[0]),
-                       "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
       }
       l_run += sum0 + sum1;
       fence_async_smem();            // P was written with ordinary stores
@@ -482,7 +501,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
 #pragma unroll
       for (int ch = 0; ch < 4; ++ch) {
         uint32_t v[32];
-        tmem_ld32(t_lane + 128 + ch * 32, v);
+        tmem_ld32(t_lane + C::O_COL + ch * 32, v);
         tmem_ld_wait();
         if (row_valid) {
 #pragma unroll
@@ -501,7 +520,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 5) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+    if (warp == 5) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(C::TMEM_COLS) : "memory");
     return;
   }
 
@@ -518,7 +537,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
     for (int ch = 0; ch < 4; ++ch) {
       uint32_t v[32];
       if (have_o) {                         // warp-uniform
-        tmem_ld32(t_lane + 128 + ch * 32, v);
+        tmem_ld32(t_lane + C::O_COL + ch * 32, v);
         tmem_ld_wait();
       } else {
 #pragma unroll
@@ -539,7 +558,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
   }
   tc_fence_before();
   cluster.sync();
-  if (warp == 5) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+  if (warp == 5) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(C::TMEM_COLS) : "memory");
 
   {
     constexpr int TPR = kD / 4;                       // 32 threads per row, one float4 each
@@ -591,10 +610,10 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
 struct MapKey {
   const void *k, *v;
   long long sl, sb, sh, sp;
-  int n_layers, batch, heads, max_len;
+  int n_layers, batch, heads, max_len, box_rows;
   bool operator==(const MapKey &o) const {
     return k == o.k && v == o.v && sl == o.sl && sb == o.sb && sh == o.sh && sp == o.sp && n_layers == o.n_layers &&
-           batch == o.batch && heads == o.heads && max_len == o.max_len;
+           batch == o.batch && heads == o.heads && max_len == o.max_len && box_rows == o.box_rows;
   }
 };
 struct MapEntry {
@@ -609,7 +628,7 @@ static bool encode_cache_map(EncodeTiledFn fn, CUtensorMap *out, const void *bas
                               (cuuint64_t)key.n_layers};
   const cuuint64_t strides[4] = {(cuuint64_t)key.sp * 2, (cuuint64_t)key.sh * 2, (cuuint64_t)key.sb * 2,
                                  (cuuint64_t)key.sl * 2};
-  const cuuint32_t box[5] = {64, (cuuint32_t)kKT, 1, 1, 1};      // 128 bytes x 64 rows: one swizzled panel
+  const cuuint32_t box[5] = {64, (cuuint32_t)key.box_rows, 1, 1, 1};   // 128 bytes x KT rows: one swizzled panel
   const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
   return fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void *>(base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -617,7 +636,7 @@ static bool encode_cache_map(EncodeTiledFn fn, CUtensorMap *out, const void *bas
 }
 
 // Returns the (cached) pair of maps for this cache layout, or nullptr when none can be made.
-static const MapEntry *cache_maps(const AttnParams &p) {
+static const MapEntry *cache_maps(const AttnParams &p, int box_rows) {
   static std::mutex mu;
   static EncodeTiledFn fn = nullptr;
   static bool fn_tried = false;
@@ -636,7 +655,7 @@ static const MapEntry *cache_maps(const AttnParams &p) {
   // strides must be multiples of 16 bytes, and every dimension but the last needs stride * extent in range
   if (p.c_sp <= 0 || p.c_sh <= 0 || p.c_sb < 0 || p.c_sl < 0) return nullptr;
   MapKey key{p.cache_k0, p.cache_v0, p.n_layers > 1 ? p.c_sl : p.c_sp, p.batch > 1 ? p.c_sb : p.c_sp, p.c_sh, p.c_sp,
-             p.n_layers, p.batch, p.n_kv_heads, p.max_len};
+             p.n_layers, p.batch, p.n_kv_heads, p.max_len, box_rows};
   if (p.n_kv_heads == 1) key.sh = key.sp;      // a stride of an extent-1 dimension is never used
   for (auto &e : table)
     if (e.valid && e.key == key) return &e;
@@ -649,12 +668,12 @@ static const MapEntry *cache_maps(const AttnParams &p) {
   return &e;
 }
 
-template <int ROWS>
+template <int ROWS, int KT>
 twig_status launch_umma(const AttnParams &p, const MapEntry *maps, int batch, int n_splits, cudaStream_t st) {
-  using C = UmmaCfg<ROWS>;
+  using C = UmmaCfg<ROWS, KT>;
   static bool attr_set = false;
   if (!attr_set) {
-    if (cudaFuncSetAttribute(tree_attn_umma_kernel<ROWS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    if (cudaFuncSetAttribute(tree_attn_umma_kernel<ROWS, KT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              C::SMEM_BYTES) != cudaSuccess)
       return TWIG_ERR_CUDA;
     attr_set = true;
@@ -671,7 +690,7 @@ twig_status launch_umma(const AttnParams &p, const MapEntry *maps, int batch, in
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  if (cudaLaunchKernelEx(&cfg, tree_attn_umma_kernel<ROWS>, p, maps->kmap, maps->vmap) != cudaSuccess)
+  if (cudaLaunchKernelEx(&cfg, tree_attn_umma_kernel<ROWS, KT>, p, maps->kmap, maps->vmap) != cudaSuccess)
     return TWIG_ERR_CUDA;
   return TWIG_OK;
 }
@@ -682,14 +701,23 @@ twig_status launch_tree_attn_umma(AttnParams &p, int batch, int rows, cudaStream
   const int rows_per_cta = rows <= 32 ? 32 : rows <= 64 ? 64 : 128;
   p.row_blocks = (rows + rows_per_cta - 1) / rows_per_cta;
   if ((long long)p.n_kv_heads * p.row_blocks > 65535) return TWIG_ERR_UNSUPPORTED;
-  const MapEntry *maps = cache_maps(p);
+  const int items = batch * p.n_kv_heads * p.row_blocks;
+  // Few, long work items: 128-key tiles, one CTA per SM (larger MMA instructions, all of tensor
+  // memory).  Many items, or short caches: 64-key tiles, two CTAs per SM.
+  const bool wide = rows_per_cta >= 64 && items <= 148 && p.max_len >= 1024;
+  const int kt = wide ? 128 : 64;
+  const MapEntry *maps = cache_maps(p, kt);
   if (!maps) return TWIG_ERR_UNSUPPORTED;
-  const int max_tiles = (p.max_len + p.t_max + kKT - 1) / kKT;
-  const int n_splits = pick_splits(batch * p.n_kv_heads * p.row_blocks, max_tiles);
+  const int max_tiles = (p.max_len + p.t_max + kt - 1) / kt;
+  const int n_splits = pick_splits(items, max_tiles, wide ? 1 : 2);
+  if (wide) {
+    if (rows_per_cta == 64) return launch_umma<64, 128>(p, maps, batch, n_splits, st);
+    return launch_umma<128, 128>(p, maps, batch, n_splits, st);
+  }
   switch (rows_per_cta) {
-    case 32: return launch_umma<32>(p, maps, batch, n_splits, st);
-    case 64: return launch_umma<64>(p, maps, batch, n_splits, st);
-    default: return launch_umma<128>(p, maps, batch, n_splits, st);
+    case 32: return launch_umma<32, 64>(p, maps, batch, n_splits, st);
+    case 64: return launch_umma<64, 64>(p, maps, batch, n_splits, st);
+    default: return launch_umma<128, 64>(p, maps, batch, n_splits, st);
   }
 }
 
