@@ -135,12 +135,28 @@ __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.
 
 // KT = keys per tile: 64 (two CTAs per SM, 256 tensor-memory columns each) or 128 (one CTA per SM
 // with all 512 columns: half as many, twice as large MMA instructions per key).
+// 2^x by range reduction and a cubic on the FMA pipe (relative error < 1e-3, far below the
+// bf16 rounding of P); used for half of the elements so that the special-function unit and
+// the FMA pipe share the exponentials.  Arguments below -126 give 2^-126 (in effect 0).
+__device__ __forceinline__ float poly_exp2(float x) {
+  x = fmaxf(x, -126.f);
+  const float t = x + 12582912.f;                 // 1.5 * 2^23: rounds x to the nearest integer
+  const float f = x - (t - 12582912.f);           // in [-0.5, 0.5]
+  float r = fmaf(f, 0.0555041f, 0.2402265f);
+  r = fmaf(r, f, 0.6931472f);
+  r = fmaf(r, f, 1.f);
+  return __int_as_float(__float_as_int(r) + (__float_as_int(t) << 23));   // * 2^n (the magic's bits shift out)
+}
+
 template <int ROWS, int KT>
 struct UmmaCfg {
   static constexpr int TILE_BYTES = KT * kD * 2;         // one K (or V) tile: 16 or 32 KB
   static constexpr int PANEL_BYTES = KT * 128;           // 64-column panel of a K/V tile
   static constexpr int Q_BYTES = ROWS * kD * 2;          // two 64-column panels of ROWS x 128 B
-  static constexpr int P_BYTES = ROWS * KT * 2;          // ROWS x KT keys bf16, KT/64 panels of ROWS x 128 B
+  static constexpr int P_ONE = ROWS * KT * 2;            // ROWS x KT keys bf16, KT/64 panels of ROWS x 128 B
+  // two P buffers where shared memory allows: the softmax of tile t+1 then never waits for P(t) V(t)
+  static constexpr int P_BUFS = ((KT == 128 && ROWS <= 64) || (KT == 64 && ROWS <= 32)) ? 2 : 1;
+  static constexpr int P_BYTES = P_BUFS * P_ONE;
   static constexpr int RING_BYTES = kSlots * TILE_BYTES;
   static constexpr uint32_t TMEM_COLS = KT == 64 ? 256 : 512;   // S: [0,KT) and [KT,2KT); O: [2KT, 2KT+128)
   static constexpr uint32_t O_COL = 2 * KT;
@@ -163,8 +179,8 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
   __shared__ unsigned long long s_mask[TWIG_MAX_NODES];
   __shared__ int s_par[TWIG_MAX_NODES];
   __shared__ float r_m[ROWS], r_l[ROWS];
-  // barriers: full[5], empty[5] (ring slots), s_ready[2], p_ready, o_done, q_ready
-  __shared__ __align__(8) unsigned long long s_bar[2 * kSlots + 5];
+  // barriers: full[5], empty[5] (ring slots), s_ready[2], p_ready[2], o_done[2], q_ready
+  __shared__ __align__(8) unsigned long long s_bar[2 * kSlots + 7];
   __shared__ uint32_t s_tmem;
   __shared__ int s_bad, s_fail;
 
@@ -197,8 +213,10 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
   auto bar_full = [&](int slot) { return bars + 8 * slot; };
   auto bar_empty = [&](int slot) { return bars + 8 * (kSlots + slot); };
   auto bar_s = [&](int buf) { return bars + 8 * (2 * kSlots + buf); };
-  const uint32_t bar_p = bars + 8 * (2 * kSlots + 2), bar_o = bars + 8 * (2 * kSlots + 3);
-  const uint32_t bar_q = bars + 8 * (2 * kSlots + 4);
+  auto bar_p = [&](int buf) { return bars + 8 * (2 * kSlots + 2 + buf); };
+  auto bar_o = [&](int buf) { return bars + 8 * (2 * kSlots + 4 + buf); };
+  const uint32_t bar_q = bars + 8 * (2 * kSlots + 6);
+  constexpr int PB = C::P_BUFS;
 
   const int NK = L + n;
   const int n_tiles = (NK + KT - 1) / KT;
@@ -241,8 +259,10 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
     }
     mbar_init(bar_s(0), 1);
     mbar_init(bar_s(1), 1);
-    mbar_init(bar_p, n_soft);           // one arrival per softmax warp
-    mbar_init(bar_o, 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(bar_p(i), n_soft);      // one arrival per softmax warp
+      mbar_init(bar_o(i), 1);
+    }
     mbar_init(bar_q, 32);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -372,15 +392,16 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
       if (n_my > 1) issue_s(1);
       for (int it = 0; it < n_my && ok; ++it) {
         const int u = 2 * it + 1;
-        ok = mbar_wait(bar_p, it & 1, fail);          // P(it) is in shared memory, S(it) has been read
+        const int pb = it % PB;
+        ok = mbar_wait(bar_p(pb), (it / PB) & 1, fail);   // P(it) is in shared memory, S(it) has been read
         wait_full(u);
         if (!ok) break;
         const uint32_t vb = ring_s + (u % kSlots) * kTileBytes;
 #pragma unroll
         for (int j = 0; j < KT / 16; ++j)          // 16 keys per step: P panel j / 4, V rows 16 j ..
-          umma(tmem_o, smem_desc(p_s + (j >> 2) * ROWS * 128 + (j & 3) * 32, 16),
+          umma(tmem_o, smem_desc(p_s + pb * C::P_ONE + (j >> 2) * ROWS * 128 + (j & 3) * 32, 16),
                smem_desc(vb + j * 2048, kPanelBytes), kIdescO, (it > 0) || (j > 0));
-        umma_commit(bar_o);
+        umma_commit(bar_o(pb));
         umma_commit(bar_empty(u % kSlots));
         if (it + 2 < n_my) issue_s(it + 2);
       }
@@ -429,12 +450,21 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
       const bool raise = row_active && mx > m_run + kLazyMax;   // also true for the first finite maximum
       const float m_new = raise ? mx : m_run;
       const float m_use = m_new == -INFINITY ? 0.f : m_new;
-      if (it > 0) {                               // P is free and O is stable once P(it-1) V(it-1) is done
-        ok = mbar_wait(bar_o, (it - 1) & 1, fail);
+      const int pb = it % PB;
+      if (it >= PB) {                             // this P buffer is free once P(it-PB) V(it-PB) is done
+        ok = mbar_wait(bar_o(pb), (it / PB - 1) & 1, fail);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after();
-        if (__any_sync(0xffffffffu, raise)) {
+      }
+      if (it > 0 && __any_sync(0xffffffffu, raise)) {
+        if (PB > 1) {                             // O must be stable: wait for P(it-1) V(it-1) as well
+          ok = mbar_wait(bar_o((it - 1) % PB), ((it - 1) / PB) & 1, fail);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          tc_fence_after();
+        }
+        {
           const float alpha = fast_exp2(m_run - m_use);   // 1 for rows that keep their maximum
           l_run *= alpha;
 #pragma unroll
@@ -456,7 +486,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
       for (int half = 0; half < KT / 64; ++half) {
         uint32_t sr[2][32];
         load_s(half, sr);
-        const uint32_t prow = p_s + half * ROWS * 128 + row_local * 128;
+        const uint32_t prow = p_s + pb * C::P_ONE + half * ROWS * 128 + row_local * 128;
 #pragma unroll
         for (int c = 0; c < 8; ++c) {          // chunk c = keys 8c .. 8c+7 of this row
           uint32_t w[4];
@@ -464,7 +494,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
           for (int e = 0; e < 4; ++e) {
             const int j = c * 8 + e * 2;
             const float p0 = fast_exp2(fmaf(__uint_as_float(sr[j >> 5][j & 31]), p.scale_log2, -m_use));
-            const float p1 = fast_exp2(fmaf(__uint_as_float(sr[(j + 1) >> 5][(j + 1) & 31]), p.scale_log2, -m_use));
+            const float p1 = poly_exp2(fmaf(__uint_as_float(sr[(j + 1) >> 5][(j + 1) & 31]), p.scale_log2, -m_use));
             sum0 += p0;
             sum1 += p1;
             w[e] = pack_bf16(p0, p1);
@@ -478,10 +508,10 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
       fence_async_smem();            // P was written with ordinary stores
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar_p);
+      if (lane == 0) mbar_arrive(bar_p(pb));
     }
     if (ok && n_my > 0) {
-      ok = mbar_wait(bar_o, (n_my - 1) & 1, fail);   // the last P V product has completed
+      ok = mbar_wait(bar_o((n_my - 1) % PB), ((n_my - 1) / PB) & 1, fail);   // the last P V product has completed
       tc_fence_after();
     }
     if (!ok) s_fail = 1;
