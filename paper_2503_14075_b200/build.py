@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
-LIB = os.path.join(HERE, "libtwig.so")
+LIB = os.environ.get("TWIG_LIB") or os.path.join(HERE, "libtwig.so")   # TWIG_LIB: load another build
 SOURCES = ["api.cu", "ttp.cu", "tree_attn.cu", "tree_attn_umma.cu", "tree_accept.cu"]
 
 

@@ -435,11 +435,11 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
             }
         }
       };
-      // pass 1: the tile's row maximum
+      // pass 1: the tile's row maximum (with 64-key tiles the row then stays in registers)
       float mx = -INFINITY;
+      uint32_t sr[2][32];
 #pragma unroll 1
       for (int half = 0; half < KT / 64; ++half) {
-        uint32_t sr[2][32];
         load_s(half, sr);
 #pragma unroll
         for (int j = 0; j < 32; j += 2)
@@ -484,8 +484,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
       float sum0 = 0.f, sum1 = 0.f;
 #pragma unroll 1
       for (int half = 0; half < KT / 64; ++half) {
-        uint32_t sr[2][32];
-        load_s(half, sr);
+        if (KT > 64) load_s(half, sr);
         const uint32_t prow = p_s + pb * C::P_ONE + half * ROWS * 128 + row_local * 128;
 #pragma unroll
         for (int c = 0; c < 8; ++c) {          // chunk c = keys 8c .. 8c+7 of this row
@@ -734,7 +733,7 @@ twig_status launch_tree_attn_umma(AttnParams &p, int batch, int rows, cudaStream
   const int items = batch * p.n_kv_heads * p.row_blocks;
   // Few, long work items: 128-key tiles, one CTA per SM (larger MMA instructions, all of tensor
   // memory).  Many items, or short caches: 64-key tiles, two CTAs per SM.
-  const bool wide = rows_per_cta >= 64 && items <= 148 && p.max_len >= 1024;
+  const bool wide = items <= 148 && ((rows_per_cta == 128 && p.max_len >= 1024) || (rows_per_cta == 64 && p.max_len >= 4096));
   const int kt = wide ? 128 : 64;
   const MapEntry *maps = cache_maps(p, kt);
   if (!maps) return TWIG_ERR_UNSUPPORTED;

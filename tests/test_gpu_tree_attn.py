@@ -76,7 +76,7 @@ SHAPES = [
     ("d64-rows64", 3, 6, 3, 64, [32, 5, 20], [6, 2, 4], [0, 100, 513]),
     ("empty-prefix", 1, 4, 4, 128, [9], [4], [0]),
     ("idle-request", 3, 4, 4, 128, [12, 0, 7], [3, 2, 3], [77, 50, 200]),
-    ("long-rows64", 2, 4, 4, 128, [64, 40], [8, 6], [1100, 130]),
+    ("long-rows64", 2, 4, 4, 128, [64, 40], [8, 6], [4100, 130]),
     ("long-gqa-rows128", 1, 8, 2, 128, [31], [5], [1500]),
 ]
 
