@@ -203,6 +203,7 @@ def run_ours(args):
     wl = synth.workload(args.workload)
     peaks = load_peaks()
     tw.twig_set_attention_path(args.attn_path)
+    tw.twig_set_launch_overlap(0 if args.no_overlap else 1)
     tw.twig_set_attention_splits(args.attn_splits)
     max_len = ((max(wl.pruned_len) + max(wl.gen_target) + wl.t_max + 8 + 31) // 32) * 32
 
@@ -607,6 +608,7 @@ def main():
     ap.add_argument("--no-extra", dest="extra", action="store_false",
                     help="skip the HBM-sized launches of the attention and gather kernels")
     ap.add_argument("--cpu-budget", type=float, default=15.0)
+    ap.add_argument("--no-overlap", action="store_true", help="plain launches (no programmatic stream serialization)")
     ap.add_argument("--attn-splits", type=int, default=0, help="force key splits per cluster (0 auto)")
     ap.add_argument("--attn-path", type=int, default=0, help="tree-attention kernel: 0 auto, 1 mma.sync, 2 tcgen05")
     args = ap.parse_args()

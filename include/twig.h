@@ -195,6 +195,12 @@ twig_status tree_verify_attention(const void *q, const void *tree_k, const void 
  * the same function; this is a tuning and testing control.  Returns the previous value. */
 int32_t twig_set_attention_path(int32_t path);
 
+/* Launch overlap (default on): tree_verify_attention and tree_accept_compact launch their kernels
+ * with programmatic stream serialization, so the next kernel of the stream is scheduled while the
+ * current one drains; each kernel waits on the device for its predecessor before it reads anything,
+ * so results do not change.  0 switches it off.  Returns the previous value. */
+int32_t twig_set_launch_overlap(int32_t on);
+
 /* Forces the number of key splits (CTAs per cluster) of the tree-attention kernels:
  * 1, 2, 4 or 8; 0 = automatic (default).  A tuning control.  Returns the previous value. */
 int32_t twig_set_attention_splits(int32_t splits);

@@ -5,6 +5,15 @@ namespace twig {
 size_t score_workspace_bytes(int batch, int n_q_heads, int max_len);
 }
 
+static bool g_launch_overlap = true;
+bool twig::launch_overlap_enabled() { return g_launch_overlap; }
+
+extern "C" int32_t twig_set_launch_overlap(int32_t on) {
+  const int prev = g_launch_overlap ? 1 : 0;
+  g_launch_overlap = on != 0;
+  return prev;
+}
+
 extern "C" const char *twig_status_str(twig_status s) {
   switch (s) {
     case TWIG_OK: return "ok";

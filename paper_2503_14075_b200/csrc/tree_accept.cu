@@ -27,6 +27,7 @@ tree_accept_compact_kernel(const int *__restrict__ parent, const int *__restrict
   __shared__ int s_path[TWIG_MAX_NODES];
   __shared__ int s_bad, s_best, s_len;
 
+  grid_dependency_sync();
   const int b = blockIdx.y, tid = threadIdx.x;
   const int n = n_nodes[b];
   if (n == 0) return;                                   // idle request
@@ -146,13 +147,22 @@ extern "C" twig_status tree_accept_compact(const int32_t *parent, const int32_t 
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   auto tk = static_cast<const __nv_bfloat16 *>(tree_k_all);
   auto tv = static_cast<const __nv_bfloat16 *>(tree_v_all);
-  if (cache->head_dim == 128)
-    tree_accept_compact_kernel<128><<<grid, kAcceptThreads, 0, st>>>(
-        parent, draft_tok, base_argmax, n_nodes, t_max, d_max, tk, tv, view_of_mut(cache), kv_len,
-        accept_len, path, bonus_tok, dev_status);
-  else
-    tree_accept_compact_kernel<64><<<grid, kAcceptThreads, 0, st>>>(
-        parent, draft_tok, base_argmax, n_nodes, t_max, d_max, tk, tv, view_of_mut(cache), kv_len,
-        accept_len, path, bonus_tok, dev_status);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(kAcceptThreads);
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = launch_overlap_enabled() ? 1 : 0;
+  const KvViewMut cv = view_of_mut(cache);
+  const cudaError_t err =
+      cache->head_dim == 128
+          ? cudaLaunchKernelEx(&cfg, tree_accept_compact_kernel<128>, parent, draft_tok, base_argmax, n_nodes, t_max,
+                               d_max, tk, tv, cv, kv_len, accept_len, path, bonus_tok, dev_status)
+          : cudaLaunchKernelEx(&cfg, tree_accept_compact_kernel<64>, parent, draft_tok, base_argmax, n_nodes, t_max,
+                               d_max, tk, tv, cv, kv_len, accept_len, path, bonus_tok, dev_status);
+  if (err != cudaSuccess) return TWIG_ERR_CUDA;
   return launch_status();
 }

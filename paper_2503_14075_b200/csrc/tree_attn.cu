@@ -66,6 +66,7 @@ tree_attn_kernel(const AttnParams p) {
   const int hk = blockIdx.y / p.row_blocks, rb = blockIdx.y % p.row_blocks;
   const int b = blockIdx.z;
 
+  grid_dependency_sync();
   // ---- per-request metadata; every exit below is uniform over the cluster ----
   const int n = p.n_nodes[b], L = p.kv_len[b];
   if (n == 0) return;
@@ -419,13 +420,15 @@ static twig_status launch_attn(const AttnParams &p, int batch, int n_splits, cud
   cfg.blockDim = dim3(C::THREADS);
   cfg.dynamicSmemBytes = C::SMEM_BYTES;
   cfg.stream = st;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = n_splits;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = launch_overlap_enabled() ? 2 : 1;
   if (cudaLaunchKernelEx(&cfg, tree_attn_kernel<C>, p) != cudaSuccess) return TWIG_ERR_CUDA;
   return TWIG_OK;
 }

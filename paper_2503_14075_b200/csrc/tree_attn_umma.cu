@@ -190,6 +190,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
   const int hk = blockIdx.y / p.row_blocks, rb = blockIdx.y % p.row_blocks;
   const int b = blockIdx.z;
 
+  grid_dependency_sync();
   // ---- per-request metadata; every exit below is uniform over the cluster ----
   const int n = p.n_nodes[b], L = p.kv_len[b];
   const int my_parent = tid < p.t_max ? p.parent[(long long)b * p.t_max + tid] : -1;
@@ -712,13 +713,15 @@ twig_status launch_umma(const AttnParams &p, const MapEntry *maps, int batch, in
   cfg.blockDim = dim3(kThreads);
   cfg.dynamicSmemBytes = C::SMEM_BYTES;
   cfg.stream = st;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = n_splits;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = launch_overlap_enabled() ? 2 : 1;
   if (cudaLaunchKernelEx(&cfg, tree_attn_umma_kernel<ROWS, KT>, p, maps->kmap, maps->vmap) != cudaSuccess)
     return TWIG_ERR_CUDA;
   return TWIG_OK;

@@ -70,11 +70,23 @@ inline KvViewMut view_of_mut(const twig_kv *kv) {
   return w;
 }
 
+// Whether kernels are launched with programmatic stream serialization (the next kernel of the
+// stream may be scheduled while this one drains; it waits on the device before reading anything).
+bool launch_overlap_enabled();
+
 inline twig_status launch_status() {
   return cudaGetLastError() == cudaSuccess ? TWIG_OK : TWIG_ERR_CUDA;
 }
 
 #ifdef __CUDACC__
+// First statement of every kernel that may be launched with programmatic stream serialization:
+// wait until the preceding kernel of the stream has completed and its writes are visible, then
+// allow the following kernel to be scheduled.  A no-op for ordinary launches.
+__device__ __forceinline__ void grid_dependency_sync() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
 __device__ __forceinline__ void flag_status(int *dev_status, int b, int code) {
   if (dev_status) atomicMax(dev_status + b, code);
 }

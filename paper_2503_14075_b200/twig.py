@@ -26,7 +26,7 @@ STATUS_NAMES = {0: "TWIG_OK", 1: "TWIG_ERR_NULL", 2: "TWIG_ERR_SHAPE", 3: "TWIG_
 DEV_OK, DEV_BAD_LAYOUT, DEV_BAD_KEEP, DEV_BAD_INDEX, DEV_BAD_TREE, DEV_OVERFLOW, DEV_INTERNAL = range(7)
 MAX_NODES, MAX_VISUAL, MAX_BATCH = 64, 16384, 4096
 
-EXPORTS = ["twig_status_str", "twig_set_attention_path", "twig_set_attention_splits", "twig_workspace_bytes", "ttp_score", "ttp_score_noalloc", "ttp_topk", "ttp_compact",
+EXPORTS = ["twig_status_str", "twig_set_launch_overlap", "twig_set_attention_path", "twig_set_attention_splits", "twig_workspace_bytes", "ttp_score", "ttp_score_noalloc", "ttp_topk", "ttp_compact",
            "ttp_score_topk_compact", "tree_verify_attention", "tree_accept_compact"]
 
 
@@ -60,6 +60,8 @@ _lib.twig_status_str.restype = C.c_char_p
 _lib.twig_status_str.argtypes = [C.c_int]
 _lib.twig_set_attention_path.restype = C.c_int32
 _lib.twig_set_attention_path.argtypes = [C.c_int32]
+_lib.twig_set_launch_overlap.restype = C.c_int32
+_lib.twig_set_launch_overlap.argtypes = [C.c_int32]
 _lib.twig_set_attention_splits.restype = C.c_int32
 _lib.twig_set_attention_splits.argtypes = [C.c_int32]
 _lib.twig_workspace_bytes.restype = _sz
@@ -107,6 +109,11 @@ def lib_path() -> str:
 def twig_set_attention_path(path: int) -> int:
     """0 automatic, 1 mma.sync kernel, 2 tcgen05 kernel; returns the previous setting."""
     return int(_lib.twig_set_attention_path(int(path)))
+
+
+def twig_set_launch_overlap(on: int) -> int:
+    """Programmatic stream serialization for the attention and accept kernels (default on)."""
+    return int(_lib.twig_set_launch_overlap(int(on)))
 
 
 def twig_set_attention_splits(splits: int) -> int:
