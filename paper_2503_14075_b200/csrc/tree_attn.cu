@@ -41,8 +41,13 @@ struct AttnCfg {
   // warps with wn > 0 (fragment order), RECV the per-split partials a CTA owns
   static constexpr int XCH_BYTES = (WN - 1) * ROWS * D * 4;
   static constexpr int RECV_BYTES = ROWS * D * 4;
-  static_assert(XCH_BYTES + RECV_BYTES <= STAGE_BYTES, "epilogue buffers must fit in the stage ring");
-  static constexpr int SMEM_BYTES = Q_BYTES + STAGE_BYTES;
+  // The small, latency-bound variants (one CTA per SM is enough for them) keep the split-merge
+  // buffer outside the stage ring: peers may then push as soon as they are done, and one
+  // cluster barrier of the epilogue goes away.
+  static constexpr bool RECV_OWN = ROWS <= 32;
+  static_assert(XCH_BYTES + (RECV_OWN ? 0 : RECV_BYTES) <= STAGE_BYTES, "epilogue buffers must fit in the stage ring");
+  static constexpr int RECV_OFFSET = RECV_OWN ? Q_BYTES + STAGE_BYTES : Q_BYTES + XCH_BYTES;
+  static constexpr int SMEM_BYTES = Q_BYTES + STAGE_BYTES + (RECV_OWN ? RECV_BYTES : 0);
 };
 
 template <class C>
@@ -69,6 +74,7 @@ tree_attn_kernel(const AttnParams p) {
   grid_dependency_sync();
   // ---- per-request metadata; every exit below is uniform over the cluster ----
   const int n = p.n_nodes[b], L = p.kv_len[b];
+  const int my_parent = tid < p.t_max ? p.parent[(long long)b * p.t_max + tid] : -1;   // (in flight with n, L)
   if (n == 0) return;
   const bool first = split == 0 && blockIdx.y == 0 && tid == 0;
   if (n < 0 || n > p.t_max) {
@@ -81,6 +87,8 @@ tree_attn_kernel(const AttnParams p) {
   }
   const int rows_total = n * p.group, row0 = rb * ROWS;
   if (row0 >= rows_total) return;
+  // with its own receive buffer a CTA only has to be running before peers may write to it
+  if (C::RECV_OWN && n_splits > 1) asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
 
   const uint32_t q_s = smem_u32(smem);
   const uint32_t k_s = q_s + C::Q_BYTES;
@@ -149,7 +157,7 @@ tree_attn_kernel(const AttnParams p) {
   if (tid == 0) s_bad = 0;
   __syncthreads();
   if (tid < n) {
-    const int pr = p.parent[(long long)b * p.t_max + tid];
+    const int pr = my_parent;
     s_par[tid] = pr;
     if ((tid == 0) ? (pr != -1) : (pr < 0 || pr >= tid)) s_bad = 1;
   }
@@ -335,8 +343,11 @@ tree_attn_kernel(const AttnParams p) {
   // cluster barrier) each one writes its per-row partial (m, l, O) into the owner's shared
   // memory; after the second barrier the owner combines its n_splits partials and stores.
   const int rows_per = ROWS / n_splits;
-  float *recv = reinterpret_cast<float *>(smem + C::Q_BYTES + C::XCH_BYTES);
-  if (n_splits > 1) cluster.sync();
+  float *recv = reinterpret_cast<float *>(smem + C::RECV_OFFSET);
+  if (n_splits > 1) {
+    if (C::RECV_OWN) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");   // every peer is running
+    else cluster.sync();                        // every peer has left its key loop: the rings are free
+  }
   if (wn == 0) {
 #pragma unroll
     for (int half = 0; half < 2; ++half) {
