@@ -434,26 +434,22 @@ def run_e2e(torch, tw, wl, reps, stream, world, dev, dist):
             "note": "per bench step = one request; Q and tree K/V of all layers cross PCIe every verify step"}
 
 
-def extra_rooflines(torch, tw, peaks, dev):
-    """HBM-sized launches of the two bandwidth kernels (the high-resolution configuration):
-    tree attention at KV length 1472 with batch 4, and the pruning gather over 32 layers."""
-    res = {}
-    wl = synth.workload(4)
-    rng = synth.rng_for(4, 500)
-    nl = 8                                   # layers resident at once: 8 x 2 x 50 MB of cache > L2
-    L = wl.final_kv_len
+def _time_attention(torch, tw, wl, kv_lens, nl, stream_id, dev, reps=10):
+    """Mean launch time (us) of tree_verify_attention over `nl` resident layers (their KV does
+    not fit L2 together), plus the algorithmic bytes and flops of one launch."""
+    rng = synth.rng_for(wl.index, stream_id)
     B, Hq, Hkv, d, T = wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.t_max
 
     def bf(x):
         return torch.from_numpy(np.ascontiguousarray(x).view(np.int16)).to(dev).view(torch.bfloat16)
 
-    ck, cv = synth.make_cache(wl, rng, L + T, n_layers=nl)
+    ck, cv = synth.make_cache(wl, rng, max(kv_lens) + T, n_layers=nl)
     ck, cv = bf(ck), bf(cv)
     ver = synth.make_verify_inputs(wl, rng, n_layers=nl)
     q, tk, tv = bf(ver["q"]), bf(ver["tree_k"]), bf(ver["tree_v"])
     par = torch.from_numpy(ver["parent"]).to(dev)
     nn = torch.from_numpy(ver["n_nodes"]).to(dev)
-    kvl = torch.full((B,), L, dtype=torch.int32, device=dev)
+    kvl = torch.from_numpy(np.asarray(kv_lens, dtype=np.int32)).to(dev)
     out = torch.zeros((B, T, Hq, d), dtype=torch.bfloat16, device=dev)
     cache = tw.KV.of(ck, cv)
     stream = torch.cuda.current_stream()
@@ -464,18 +460,47 @@ def extra_rooflines(torch, tw, peaks, dev):
     for _ in range(3):
         loop()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    reps = 10
     e0.record(stream)
     for _ in range(reps):
         loop()
     e1.record(stream)
     torch.cuda.synchronize()
     us = e0.elapsed_time(e1) * 1e3 / (reps * nl)
-    by = attn_bytes_per_launch(wl, [L] * B)
-    res["tree_attn_c4_L1472"] = {"bound": "hbm", "bytes_per_launch": by, "us_per_launch": round(us, 2),
-                                 "achieved": round(by / us / 1e3, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                                 "frac": round(by / us / 1e3 / peaks["hbm_gbs"], 4)}
-    del ck, cv, cache
+    by = attn_bytes_per_launch(wl, kv_lens)
+    flops = sum(4 * Hq * n * d * (int(l) + n) for n, l in zip(wl.n_nodes, kv_lens))
+    return us, by, flops
+
+
+def extra_rooflines(torch, tw, peaks, dev):
+    """HBM-sized launches of the bandwidth kernels on the larger configurations: tree attention
+    for the heterogeneous batch (c3), the high-resolution shape (c4) and the GQA long-context
+    shape (c5, tensor bound), and the pruning gather of c4."""
+    res = {}
+
+    def bf(x):
+        return torch.from_numpy(np.ascontiguousarray(x).view(np.int16)).to(dev).view(torch.bfloat16)
+
+    def hbm_entry(us, by):
+        return {"bound": "hbm", "bytes_per_launch": by, "us_per_launch": round(us, 2),
+                "achieved": round(by / us / 1e3, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": round(by / us / 1e3 / peaks["hbm_gbs"], 4)}
+
+    wl3 = synth.workload(3)
+    lens3 = [p + g // 2 for p, g in zip(wl3.pruned_len, wl3.gen_target)]      # half-way through generation
+    us, by, _ = _time_attention(torch, tw, wl3, lens3, 2, 501, dev)
+    res["tree_attn_c3_midway"] = hbm_entry(us, by)
+    wl = synth.workload(4)
+    B, Hq, Hkv, d, T = wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.t_max
+    us, by, _ = _time_attention(torch, tw, wl, [wl.final_kv_len] * B, 8, 500, dev)
+    res["tree_attn_c4_L1472"] = hbm_entry(us, by)
+    wl5 = synth.workload(5)
+    us, by, fl = _time_attention(torch, tw, wl5, [wl5.final_kv_len] * wl5.batch, 2, 502, dev, reps=5)
+    res["tree_attn_c5_L8128"] = {"bound": "tensor", "flops_per_launch": fl, "bytes_per_launch": by,
+                                 "us_per_launch": round(us, 2), "achieved": round(fl / us / 1e6, 1),
+                                 "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                                 "frac": round(fl / us / 1e6 / peaks["bf16_tflops"], 4),
+                                 "hbm_gbs": round(by / us / 1e3, 1)}
+    rng = synth.rng_for(4, 503)
     # pruning gather, 2 layers at a time of the B=4 x 3008-token prompt cache
     nl = 2
     pre = synth.make_prefill(wl, rng, n_layers=nl)
