@@ -501,6 +501,7 @@ def extra_rooflines(torch, tw, peaks, dev):
                                  "frac": round(fl / us / 1e6 / peaks["bf16_tflops"], 4),
                                  "hbm_gbs": round(by / us / 1e3, 1)}
     rng = synth.rng_for(4, 503)
+    stream = torch.cuda.current_stream()
     # pruning gather, 2 layers at a time of the B=4 x 3008-token prompt cache
     nl = 2
     pre = synth.make_prefill(wl, rng, n_layers=nl)
