@@ -158,6 +158,23 @@ twig_status ttp_compact(const twig_kv *src, const twig_kv *dst, const int32_t *k
                         int32_t *pos_out, int32_t pos_stride, int32_t *new_len,
                         int32_t *dev_status, void *stream);
 
+/* ---- TTP stage 3 on hidden states: Eq. 5 in the paper's literal form -------------
+ * The paper prunes the token sequence X^(K) that leaves layer K (and, with FinalWipe,
+ * drops every visual token after layer K_f: keep = 0).  Same index list as ttp_compact,
+ * applied to rows of any width: dst row j of request b = src row idx_b[j], bytes verbatim.
+ *   src, dst   device; row (b, i) at base + b*stride_batch + i*stride_row (strides in BYTES)
+ *   row_bytes  bytes per row, a multiple of 16 (e.g. d_model * 2); rows must be 16-byte aligned
+ *   src_rows / dst_rows   rows available per request in src / dst (bounds for the checks)
+ * new_len (may be NULL) receives prefix_len - n_vis + keep.  dst must not overlap src.
+ */
+twig_status ttp_compact_rows(const void *src, void *dst, int64_t row_bytes, int64_t src_stride_row,
+                             int64_t src_stride_batch, int32_t src_rows, int64_t dst_stride_row,
+                             int64_t dst_stride_batch, int32_t dst_rows, int32_t batch,
+                             const int32_t *kept_idx, int32_t r_max, const int32_t *keep,
+                             const int32_t *prefix_len, const int32_t *vis_start,
+                             const int32_t *n_vis, int32_t *new_len, int32_t *dev_status,
+                             void *stream);
+
 /* ---- TTP, all three stages (Sec. 4.2, Algorithm 1 "pruning", Algorithm 2) --
  * Arguments as above; scores and kept_idx are outputs the caller may inspect. */
 twig_status ttp_score_topk_compact(

@@ -116,6 +116,20 @@ def gather_compact(src_k, src_v, pos_in, prefix_len, vis_start, n_vis, kept_list
     return new_len
 
 
+def gather_rows(src, prefix_len, vis_start, n_vis, kept_list, dst):
+    """Eq. 5 in its literal form: prune a [B, L, ...] token sequence (the layer-K hidden
+    states X^(K)).  dst[b, j] = src[b, idx_b[j]]; rows >= new_len stay as they were.
+    kept_list[b] = [] removes every visual token (FinalWipe after layer K_f)."""
+    B = src.shape[0]
+    new_len = np.zeros(B, dtype=np.int32)
+    for b in range(B):
+        idx = prune_index_list(int(prefix_len[b]), int(vis_start[b]), int(n_vis[b]), kept_list[b])
+        new_len[b] = len(idx)
+        for j, i in enumerate(idx):
+            dst[b, j] = src[b, i]
+    return new_len
+
+
 # --------------------------------------------------------------------------
 # O4: tree-masked verification attention (Sec. 5.4, Appendix A, Eq. 2)
 # --------------------------------------------------------------------------

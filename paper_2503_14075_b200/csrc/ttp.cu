@@ -333,6 +333,83 @@ kv_gather_kernel(KvView src, KvViewMut dst, const int *__restrict__ kept_idx, in
 }
 
 // ---------------------------------------------------------------------------
+// Stage 3 on rows of any width (hidden states of layer K; FinalWipe with keep = 0).
+// One CTA = 4 destination rows of one request; 16-byte chunks, 8 loads in flight per thread.
+// ---------------------------------------------------------------------------
+constexpr int kRowGatherRows = 4;
+
+__global__ void __launch_bounds__(kGatherThreads)
+row_gather_kernel(const unsigned char *__restrict__ src, unsigned char *__restrict__ dst, long long row_bytes,
+                  long long s_row, long long s_batch, int src_rows, long long d_row, long long d_batch,
+                  int dst_rows, const int *__restrict__ kept_idx, int r_max, const int *__restrict__ keep,
+                  const int *__restrict__ prefix_len, const int *__restrict__ vis_start,
+                  const int *__restrict__ n_vis, int *__restrict__ new_len, int *dev_status) {
+  const int b = blockIdx.y;
+  const int lp = prefix_len[b], vs = vis_start[b], nv = n_vis[b], kp = keep[b];
+  const bool first = blockIdx.x == 0 && threadIdx.x == 0;
+  if (!layout_ok(lp, vs, nv, src_rows, TWIG_MAX_VISUAL)) {
+    if (first) flag_status(dev_status, b, TWIG_DEV_BAD_LAYOUT);
+    return;
+  }
+  if (kp < 0 || kp > nv || kp > r_max) {
+    if (first) flag_status(dev_status, b, TWIG_DEV_BAD_KEEP);
+    return;
+  }
+  const int nl = lp - nv + kp;
+  if (nl > dst_rows) {
+    if (first) flag_status(dev_status, b, TWIG_DEV_OVERFLOW);
+    return;
+  }
+  if (first && new_len) new_len[b] = nl;
+  const int j0 = blockIdx.x * kRowGatherRows;
+  if (j0 >= nl) return;
+  const int *kidx = kept_idx + (long long)b * r_max;
+  const unsigned char *sp[kRowGatherRows];
+  unsigned char *dp[kRowGatherRows];
+#pragma unroll
+  for (int r = 0; r < kRowGatherRows; ++r) {
+    const int j = j0 + r;
+    int s = -1;
+    if (j < nl) {
+      if (j < vs) {
+        s = j;
+      } else if (j < vs + kp) {
+        const int kk = kidx[j - vs];
+        const int prev = (j > vs) ? kidx[j - vs - 1] : -1;
+        if (kk < 0 || kk >= nv || kk <= prev) {
+          if (threadIdx.x == 0) flag_status(dev_status, b, TWIG_DEV_BAD_INDEX);
+        } else {
+          s = vs + kk;
+        }
+      } else {
+        s = j - kp + nv;
+      }
+    }
+    sp[r] = s >= 0 ? src + b * s_batch + (long long)s * s_row : nullptr;
+    dp[r] = dst + b * d_batch + (long long)j * d_row;
+  }
+  const long long chunks = row_bytes >> 4;
+  for (long long c0 = threadIdx.x; c0 < chunks; c0 += 2 * kGatherThreads) {
+    const long long c1 = c0 + kGatherThreads;
+    uint4 v0[kRowGatherRows], v1[kRowGatherRows];
+#pragma unroll
+    for (int r = 0; r < kRowGatherRows; ++r) {
+      if (sp[r]) {
+        v0[r] = ld_nc_16(sp[r] + (c0 << 4));
+        if (c1 < chunks) v1[r] = ld_nc_16(sp[r] + (c1 << 4));
+      }
+    }
+#pragma unroll
+    for (int r = 0; r < kRowGatherRows; ++r) {
+      if (sp[r]) {
+        st_16(dp[r] + (c0 << 4), v0[r]);
+        if (c1 < chunks) st_16(dp[r] + (c1 << 4), v1[r]);
+      }
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------
 static inline int logits_stride(int k_max_len) { return (k_max_len + 3) & ~3; }
@@ -561,4 +638,26 @@ extern "C" twig_status ttp_score_topk_compact(
   if (s != TWIG_OK) return s;
   return launch_gather(src, dst, kept_idx, r_max, keep, prefix_len, vis_start, n_vis, pos_in, pos_out,
                        pos_stride, new_len, dev_status, st);
+}
+
+extern "C" twig_status ttp_compact_rows(const void *src, void *dst, int64_t row_bytes, int64_t src_stride_row,
+                                        int64_t src_stride_batch, int32_t src_rows, int64_t dst_stride_row,
+                                        int64_t dst_stride_batch, int32_t dst_rows, int32_t batch,
+                                        const int32_t *kept_idx, int32_t r_max, const int32_t *keep,
+                                        const int32_t *prefix_len, const int32_t *vis_start,
+                                        const int32_t *n_vis, int32_t *new_len, int32_t *dev_status,
+                                        void *stream) {
+  if (!src || !dst || !kept_idx || !keep || !prefix_len || !vis_start || !n_vis) return TWIG_ERR_NULL;
+  if (row_bytes <= 0 || batch <= 0 || src_rows <= 0 || dst_rows <= 0 || r_max <= 0) return TWIG_ERR_SHAPE;
+  if (src_stride_row < row_bytes || dst_stride_row < row_bytes) return TWIG_ERR_SHAPE;
+  if (batch > TWIG_MAX_BATCH) return TWIG_ERR_UNSUPPORTED;
+  if (src == dst) return TWIG_ERR_UNSUPPORTED;
+  if ((row_bytes | src_stride_row | src_stride_batch | dst_stride_row | dst_stride_batch) & 15) return TWIG_ERR_ALIGN;
+  if (!aligned16(src) || !aligned16(dst)) return TWIG_ERR_ALIGN;
+  dim3 grid((dst_rows + kRowGatherRows - 1) / kRowGatherRows, batch);
+  row_gather_kernel<<<grid, kGatherThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+      static_cast<const unsigned char *>(src), static_cast<unsigned char *>(dst), row_bytes, src_stride_row,
+      src_stride_batch, src_rows, dst_stride_row, dst_stride_batch, dst_rows, kept_idx, r_max, keep, prefix_len,
+      vis_start, n_vis, new_len, dev_status);
+  return launch_status();
 }

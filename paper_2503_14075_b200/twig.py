@@ -26,7 +26,7 @@ STATUS_NAMES = {0: "TWIG_OK", 1: "TWIG_ERR_NULL", 2: "TWIG_ERR_SHAPE", 3: "TWIG_
 DEV_OK, DEV_BAD_LAYOUT, DEV_BAD_KEEP, DEV_BAD_INDEX, DEV_BAD_TREE, DEV_OVERFLOW, DEV_INTERNAL = range(7)
 MAX_NODES, MAX_VISUAL, MAX_BATCH = 64, 16384, 4096
 
-EXPORTS = ["twig_status_str", "twig_set_launch_overlap", "twig_set_attention_path", "twig_set_attention_splits", "twig_workspace_bytes", "ttp_score", "ttp_score_noalloc", "ttp_topk", "ttp_compact",
+EXPORTS = ["twig_status_str", "twig_set_launch_overlap", "twig_set_attention_path", "twig_set_attention_splits", "twig_workspace_bytes", "ttp_score", "ttp_score_noalloc", "ttp_topk", "ttp_compact", "ttp_compact_rows",
            "ttp_score_topk_compact", "tree_verify_attention", "tree_accept_compact"]
 
 
@@ -77,6 +77,9 @@ _lib.ttp_topk.restype = C.c_int
 _lib.ttp_topk.argtypes = [_vp, _vp, _vp, _i32, _i32, _i32, _vp, _vp, _vp]
 _lib.ttp_compact.restype = C.c_int
 _lib.ttp_compact.argtypes = [_kvp, _kvp, _vp, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _vp]
+_lib.ttp_compact_rows.restype = C.c_int
+_lib.ttp_compact_rows.argtypes = [_vp, _vp, _i64, _i64, _i64, _i32, _i64, _i64, _i32, _i32, _vp, _i32, _vp, _vp, _vp,
+                                  _vp, _vp, _vp, _vp]
 _lib.ttp_score_topk_compact.restype = C.c_int
 _lib.ttp_score_topk_compact.argtypes = [_vp, _vp, _i64, _i64, _i64, _i32, _vp, _vp, _vp, _vp, _i32, _i32,
                                         _f32, _vp, _i32, _vp, _i32, _kvp, _kvp, _vp, _vp, _i32, _vp, _vp,
@@ -160,6 +163,18 @@ def ttp_compact(src: KV, dst: KV, kept_idx, keep, prefix_len, vis_start, n_vis, 
     _check(_lib.ttp_compact(C.byref(src), C.byref(dst), _p(kept_idx), kept_idx.shape[1], _p(keep),
                             _p(prefix_len), _p(vis_start), _p(n_vis), _p(pos_in), _p(pos_out),
                             pos_stride, _p(new_len), _p(dev_status), _stream(stream)))
+
+
+def ttp_compact_rows(src, dst, kept_idx, keep, prefix_len, vis_start, n_vis, new_len=None, dev_status=None,
+                     stream=None):
+    """Prune a [B, L, width] token sequence (e.g. layer-K hidden states): dst[b, j] = src[b, idx_b[j]].
+    src/dst: CUDA tensors whose last dimension is contiguous and a multiple of 16 bytes."""
+    es = src.element_size()
+    assert src.dim() == 3 and dst.dim() == 3 and src.stride(2) == 1 and dst.stride(2) == 1
+    _check(_lib.ttp_compact_rows(_p(src), _p(dst), src.shape[2] * es, src.stride(1) * es, src.stride(0) * es,
+                                 src.shape[1], dst.stride(1) * es, dst.stride(0) * es, dst.shape[1], src.shape[0],
+                                 _p(kept_idx), kept_idx.shape[1], _p(keep), _p(prefix_len), _p(vis_start),
+                                 _p(n_vis), _p(new_len), _p(dev_status), _stream(stream)))
 
 
 def ttp_score_topk_compact(twig_q, twig_k, prefix_len, vis_start, n_vis, keep, scores, kept_idx,

@@ -249,3 +249,35 @@ def test_fused_prune_matches_stage_chain(tw, name, scope):
     assert np.array_equal(host_bits(dk), ok) and np.array_equal(host_bits(dv), ov)
     assert np.array_equal(pos_out.cpu().numpy(), opos)
     assert min(overlap) > 0.8        # informational: near-ties may flip between fp32 and fp64 scores
+
+
+@pytest.mark.parametrize("width", [4096, 1000 * 8, 8])
+def test_compact_rows_hidden_states_and_finalwipe(tw, width):
+    """Eq. 5 on rows of any width (layer-K hidden states), and keep = 0 (FinalWipe)."""
+    rng = np.random.default_rng(21)
+    lens = [(35, 576, 64), (3, 100, 0), (0, 7, 9)]
+    B = len(lens)
+    lp = [a + m + c for a, m, c in lens]
+    x = rng.integers(0, 1 << 16, size=(B, max(lp), width), dtype=np.uint16)
+    for kept_lists in ([sorted(rng.choice(m, size=min(m, 64), replace=False).tolist()) for _, m, _ in lens],
+                       [[] for _ in lens]):
+        r_max = max(1, max(len(k) for k in kept_lists))
+        kept = np.full((B, r_max), -1, dtype=np.int32)
+        for b, kl in enumerate(kept_lists):
+            kept[b, :len(kl)] = kl
+        keep = [len(k) for k in kept_lists]
+        src = dev_bf16(x)
+        dst_rows = max(l - m + k for l, (_, m, _), k in zip(lp, lens, keep)) + 2
+        dst = torch.zeros((B, dst_rows, width), dtype=torch.int16, device=DEV)
+        dst.fill_(0x7FC1)
+        dst = dst.view(torch.bfloat16)
+        new_len = torch.full((B,), -1, dtype=torch.int32, device=DEV)
+        status = torch.zeros(B, dtype=torch.int32, device=DEV)
+        tw.ttp_compact_rows(src, dst, dev_i32(kept), dev_i32(keep), dev_i32(lp), dev_i32([a for a, _, _ in lens]),
+                            dev_i32([m for _, m, _ in lens]), new_len=new_len, dev_status=status)
+        torch.cuda.synchronize()
+        want = np.full((B, dst_rows, width), 0x7FC1, dtype=np.uint16)
+        wlen = O.gather_rows(x, lp, [a for a, _, _ in lens], [m for _, m, _ in lens], kept_lists, want)
+        assert not status.cpu().numpy().any()
+        assert np.array_equal(new_len.cpu().numpy(), wlen)
+        assert np.array_equal(host_bits(dst), want)

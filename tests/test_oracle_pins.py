@@ -191,6 +191,23 @@ def test_gather_keep_all_is_identity_and_keep_none_is_text_only():
     assert n[0] == 4 and list(dk[0, 0, 0, :4, 0] % 1000) == [0, 1, 7, 8]
 
 
+def test_gather_rows_hidden_states_and_finalwipe():
+    B, L, D = 2, 11, 5
+    x = np.arange(B * L * D, dtype=np.int64).reshape(B, L, D)
+    lp, vs, nv = [11, 9], [3, 0], [6, 4]
+    dst = np.full_like(x, -1)
+    n = O.gather_rows(x, lp, vs, nv, [[0, 5], [1, 2, 3]], dst)
+    assert list(n) == [7, 8]
+    assert np.array_equal(dst[0, :7], x[0, [0, 1, 2, 3, 8, 9, 10]]) and np.all(dst[0, 7:] == -1)
+    assert np.array_equal(dst[1, :8], x[1, [1, 2, 3, 4, 5, 6, 7, 8]])
+    # FinalWipe: no visual token survives; keep-all: identity
+    dst[:] = -1
+    n = O.gather_rows(x, lp, vs, nv, [[], []], dst)
+    assert list(n) == [5, 5] and np.array_equal(dst[0, :5], x[0, [0, 1, 2, 9, 10]])
+    n = O.gather_rows(x, lp, vs, nv, [list(range(6)), list(range(4))], dst)
+    assert list(n) == lp and np.array_equal(dst[0], x[0]) and np.array_equal(dst[1, :9], x[1, :9])
+
+
 # ---------------------------------------------------------------- O4 tree attention
 def _attn_case(seed, B=2, T=6, Hq=4, Hkv=2, d=8, Lmax=11, kv_len=(7, 11), gain=1.0):
     rng = np.random.default_rng(seed)
