@@ -35,6 +35,9 @@ UNIT = "verify steps/s"
 N_ROT = 4          # request replicas visited round-robin so that no launch finds its KV in L2
 POOL = 8           # distinct per-step Q / tree-K/V sets per replica (cycled)
 MAX_STEPS = 110    # bound on verify steps per request
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel (tree_attn_kernel,
+# c2 shape, kv_len 227); set to None whenever that kernel changes after the capture
+ATTN_TRAFFIC_NCU = 4405248
 
 
 def load_peaks():
@@ -315,7 +318,9 @@ def run_ours(args):
     achieved = bytes_per_launch / (use_us * 1e-6) / 1e9
     roofline = {"kernel": "tree_attn_kernel", "bound": "hbm", "achieved": round(achieved, 1),
                 "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": round(achieved / peaks["hbm_gbs"], 4),
-                "peak_source": peaks["source"], "traffic": None,
+                "peak_source": peaks["source"], "traffic": ATTN_TRAFFIC_NCU,
+                "traffic_note": "dram read+write bytes of one launch at kv_len 227 (algorithmic 4571344 B there), "
+                                "from the ncu capture summarised in profiles/kernels_ncu_full.md",
                 "bytes_per_launch": int(bytes_per_launch), "us_per_launch": round(use_us, 3),
                 "us_per_launch_direct": round(att_us_per_launch, 3),
                 "us_per_launch_in_graph": round(graph_us_per_launch, 3),
