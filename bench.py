@@ -498,6 +498,9 @@ def extra_rooflines(torch, tw, peaks, dev):
     B, Hq, Hkv, d, T = wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.t_max
     us, by, _ = _time_attention(torch, tw, wl, [wl.final_kv_len] * B, 8, 500, dev)
     res["tree_attn_c4_L1472"] = hbm_entry(us, by)
+    # the same shape with a long cache (beyond the configuration's 1.5k): the kernel's steady state
+    us, by, _ = _time_attention(torch, tw, wl, [8128] * B, 2, 504, dev, reps=5)
+    res["tree_attn_c4shape_L8128"] = hbm_entry(us, by)
     wl5 = synth.workload(5)
     us, by, fl = _time_attention(torch, tw, wl5, [wl5.final_kv_len] * wl5.batch, 2, 502, dev, reps=5)
     res["tree_attn_c5_L8128"] = {"bound": "tensor", "flops_per_launch": fl, "bytes_per_launch": by,

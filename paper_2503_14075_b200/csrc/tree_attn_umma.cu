@@ -42,7 +42,7 @@ namespace {
 
 constexpr int kD = 128;          // head_dim
 constexpr int kThreads = 192;          // warps 0-3 softmax, warp 4 loader, warp 5 MMA issuer
-constexpr int kSlots = 5;                         // ring of K / V tiles (K0 V0 K1 V1 K2 ...)
+constexpr int kMaxSlots = 5;                      // ring of K / V tiles (K0 V0 K1 V1 K2 ...)
 constexpr float kLazyMax = 8.f;                   // raise the running max only beyond this (log2 units)
 constexpr int kSpinLimit = 1 << 22;
 
@@ -155,9 +155,11 @@ struct UmmaCfg {
   static constexpr int Q_BYTES = ROWS * kD * 2;          // two 64-column panels of ROWS x 128 B
   static constexpr int P_ONE = ROWS * KT * 2;            // ROWS x KT keys bf16, KT/64 panels of ROWS x 128 B
   // two P buffers where shared memory allows: the softmax of tile t+1 then never waits for P(t) V(t)
-  static constexpr int P_BUFS = ((KT == 128 && ROWS <= 64) || (KT == 64 && ROWS <= 32)) ? 2 : 1;
+  static constexpr int P_BUFS = (KT == 128 || (KT == 64 && ROWS <= 32)) ? 2 : 1;
   static constexpr int P_BYTES = P_BUFS * P_ONE;
-  static constexpr int RING_BYTES = kSlots * TILE_BYTES;
+  // 128 rows with 128-key tiles: four slots, so that two P buffers still fit in shared memory
+  static constexpr int SLOTS = (ROWS == 128 && KT == 128) ? 4 : kMaxSlots;
+  static constexpr int RING_BYTES = SLOTS * TILE_BYTES;
   static constexpr uint32_t TMEM_COLS = KT == 64 ? 256 : 512;   // S: [0,KT) and [KT,2KT); O: [2KT, 2KT+128)
   static constexpr uint32_t O_COL = 2 * KT;
   static constexpr int MIN_CTAS = KT == 64 ? 2 : 1;
@@ -174,13 +176,13 @@ __global__ void __launch_bounds__(kThreads, UmmaCfg<ROWS, KT>::MIN_CTAS)
 tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap,
                       const __grid_constant__ CUtensorMap vmap) {
   using C = UmmaCfg<ROWS, KT>;
-  constexpr int kTileBytes = C::TILE_BYTES, kPanelBytes = C::PANEL_BYTES;
+  constexpr int kTileBytes = C::TILE_BYTES, kPanelBytes = C::PANEL_BYTES, kSlots = C::SLOTS;
   extern __shared__ __align__(1024) unsigned char smem[];
   __shared__ unsigned long long s_mask[TWIG_MAX_NODES];
   __shared__ int s_par[TWIG_MAX_NODES];
   __shared__ float r_m[ROWS], r_l[ROWS];
   // barriers: full[5], empty[5] (ring slots), s_ready[2], p_ready[2], o_done[2], q_ready
-  __shared__ __align__(8) unsigned long long s_bar[2 * kSlots + 7];
+  __shared__ __align__(8) unsigned long long s_bar[2 * kMaxSlots + 7];
   __shared__ uint32_t s_tmem;
   __shared__ int s_bad, s_fail;
 
@@ -212,11 +214,11 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
   const uint32_t ring_s = p_s + C::P_BYTES;
   const uint32_t bars = smem_u32(s_bar);
   auto bar_full = [&](int slot) { return bars + 8 * slot; };
-  auto bar_empty = [&](int slot) { return bars + 8 * (kSlots + slot); };
-  auto bar_s = [&](int buf) { return bars + 8 * (2 * kSlots + buf); };
-  auto bar_p = [&](int buf) { return bars + 8 * (2 * kSlots + 2 + buf); };
-  auto bar_o = [&](int buf) { return bars + 8 * (2 * kSlots + 4 + buf); };
-  const uint32_t bar_q = bars + 8 * (2 * kSlots + 6);
+  auto bar_empty = [&](int slot) { return bars + 8 * (kMaxSlots + slot); };
+  auto bar_s = [&](int buf) { return bars + 8 * (2 * kMaxSlots + buf); };
+  auto bar_p = [&](int buf) { return bars + 8 * (2 * kMaxSlots + 2 + buf); };
+  auto bar_o = [&](int buf) { return bars + 8 * (2 * kMaxSlots + 4 + buf); };
+  const uint32_t bar_q = bars + 8 * (2 * kMaxSlots + 6);
   constexpr int PB = C::P_BUFS;
 
   const int NK = L + n;
