@@ -28,7 +28,7 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-from paper_2503_14075_b200 import synth  # noqa: E402
+from paper_2503_14075_b200 import replicas, synth  # noqa: E402
 
 METRIC = "tree_verify_steps_per_s"
 UNIT = "verify steps/s"
@@ -210,7 +210,7 @@ def run_ours(args):
     tw.twig_set_attention_splits(args.attn_splits)
     max_len = ((max(wl.pruned_len) + max(wl.gen_target) + wl.t_max + 8 + 31) // 32) * 32
 
-    reps = [Replica(wl, 100 + rank * N_ROT + r, torch, tw, dev, max_len) for r in range(N_ROT)]
+    reps = [Replica(wl, sid, torch, tw, dev, max_len) for sid in replicas.replica_streams(rank, N_ROT)]
     stream = torch.cuda.current_stream()
 
     # ---- dry run: how many verify steps each request needs to emit its target ------------
@@ -286,13 +286,10 @@ def run_ours(args):
     t1.record(stream)
     barrier()
     clocks = sampler.stop()
-    ms = t0.elapsed_time(t1)
-    if world > 1:
-        tt = torch.tensor([ms], device=dev)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        ms = float(tt.item())
+    # whole-job value: work summed over the ranks, time of the slowest rank
+    job_steps, ms = replicas.combine(total_verify * args.steps, t0.elapsed_time(t1), dev)
     verify_ms = sum(a.elapsed_time(b) for a, b in ev_pairs)          # attention x layers + accept, per verify step
-    value = total_verify * args.steps * world / (ms * 1e-3)
+    value = job_steps / (ms * 1e-3)
 
     # ---- dominant kernel alone: the 32 attention launches of every verify step, timed live ------
     for rp in reps:

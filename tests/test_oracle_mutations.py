@@ -1,0 +1,57 @@
+"""The pins must catch plausible mistakes.  Each case plants one mistake in a copy of the
+oracle's source (on the CPU, in memory), runs the pin tests against that copy and expects at
+least one of them to fail."""
+import os
+import types
+
+import pytest
+
+import test_oracle_pins as pins
+
+ORACLE_SRC = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "oracle", "twig_oracle.py")
+
+MUTATIONS = [
+    ("scores: scale dropped", "z = np.matmul(k[b, h // G, lo:hi, :], q[b, h, :]) * scale",
+     "z = np.matmul(k[b, h // G, lo:hi, :], q[b, h, :])"),
+    ("scores: heads summed, not averaged", "        s[b, :m] /= Hq\n", ""),
+    ("scores: wrong kv head for a query head", "z = np.matmul(k[b, h // G, lo:hi, :]", "z = np.matmul(k[b, h % Hkv, lo:hi, :]"),
+    ("scores: visual slice off by one", "p[vs - lo: vs - lo + m]", "p[vs - lo + 1: vs - lo + m + 1]"),
+    ("scores: eq. 7 scope ignored", "lo, hi = (0, lp) if norm_scope == 0 else (vs, vs + m)", "lo, hi = (0, lp)"),
+    ("top-k: ties to the higher index", "key=lambda m: (-s[m], m)", "key=lambda m: (-s[m], -m)"),
+    ("top-k: smallest instead of largest", "key=lambda m: (-s[m], m)", "key=lambda m: (s[m], m)"),
+    ("prune: text after the image dropped", "+ list(range(vis_start + n_vis, prefix_len))", ""),
+    ("prune: kept indices not offset", "[vis_start + m for m in kept]", "[m for m in kept]"),
+    ("attention: node does not see itself", "    while x >= 0:\n        out.append(x)", "    while x >= 0:\n        out.append(x) if x != i or x == 0 else None"),
+    ("attention: mask shifted by one key", "vis[i, kv_len + a] = True", "vis[i, min(kv_len + a + 1, kv_len + n_nodes - 1)] = True"),
+    ("attention: prefix end off by one", "vis[:, :kv_len] = True", "vis[:, :max(kv_len - 1, 0)] = True"),
+    ("attention: scale dropped", "z = np.matmul(q_rows, keys.T) * scale", "z = np.matmul(q_rows, keys.T)"),
+    ("attention: lse without the max", "(zmax + np.log(se))[:, 0]", "(np.log(se))[:, 0]"),
+    ("attention: wrong kv head", "        g = h // G\n", "        g = h % Hkv\n"),
+    ("accept: any matching node counts", "ok = all(", "ok = any([True] if len(chain) == 1 else []) or any("),
+    ("accept: compares with the node's own target", "int(base_argmax[u]) for u, c in zip(chain[:-1], chain[1:])",
+     "int(base_argmax[c]) for u, c in zip(chain[:-1], chain[1:])"),
+    ("accept: ties to the later node", "if ok and depth > best_depth:", "if ok and depth >= best_depth:"),
+    ("accept: bonus from the root", "return best_depth, np.array(path, dtype=np.int32), int(base_argmax[best])",
+     "return best_depth, np.array(path, dtype=np.int32), int(base_argmax[0])"),
+    ("append: rows written one position late", "cache_k[:, b, :, base + j, :]", "cache_k[:, b, :, base + j + 1, :]"),
+    ("append: length not advanced by the root", "new_len[b] = base + len(paths[b])", "new_len[b] = base + len(paths[b]) - 1"),
+    ("eq. 6: K_f ignored", "upper = L if K_f is None else K_f", "upper = L"),
+]
+
+PIN_TESTS = [getattr(pins, n) for n in dir(pins) if n.startswith("test_") and "generator" not in n and "bf16" not in n]
+
+
+@pytest.mark.parametrize("name,old,new", MUTATIONS, ids=[m[0] for m in MUTATIONS])
+def test_pins_catch_planted_mistake(monkeypatch, name, old, new):
+    src = open(ORACLE_SRC).read()
+    assert src.count(old) >= 1, "mutation target not found: " + name
+    mutant = types.ModuleType("twig_oracle_mutant")
+    exec(compile(src.replace(old, new, 1), "twig_oracle_mutant.py", "exec"), mutant.__dict__)
+    monkeypatch.setattr(pins, "O", mutant)
+    caught = []
+    for t in PIN_TESTS:
+        try:
+            t()
+        except Exception as e:          # an assertion, or a crash caused by the mistake
+            caught.append((t.__name__, type(e).__name__))
+    assert caught, f"no pin noticed: {name}"
