@@ -159,6 +159,7 @@ class Replica:
         self.path = torch.zeros((B, T), dtype=torch.int32, device=dev)
         self.bonus = torch.zeros(B, dtype=torch.int32, device=dev)
         self.n_steps = MAX_STEPS
+        self.early_prefix = True
 
     def prune(self, tw):
         tw.ttp_score_topk_compact(self.twig_q, self.twig_k, self.prefix_len, self.vis_start, self.n_vis, self.keep,
@@ -169,8 +170,12 @@ class Replica:
         slot = s % POOL
         q, tk, tv = self.q[slot], self.tree_k[slot], self.tree_v[slot]
         for layer in range(self.wl.n_layers):
+            # layer 0 follows the accept (or prune) kernel, which writes kv_len; the other layers follow
+            # the previous layer's attention, which leaves lengths and cache alone
+            tw.twig_set_early_prefix(1 if (layer > 0 and self.early_prefix) else 0)
             tw.tree_verify_attention(q[layer], tk[layer], tv[layer], self.cache, layer, self.kv_len, self.n_nodes,
                                      self.parent, self.out, dev_status=self.status)
+        tw.twig_set_early_prefix(0)
 
     def accept(self, tw, s):
         slot = s % POOL
@@ -211,6 +216,8 @@ def run_ours(args):
     max_len = ((max(wl.pruned_len) + max(wl.gen_target) + wl.t_max + 8 + 31) // 32) * 32
 
     reps = [Replica(wl, sid, torch, tw, dev, max_len) for sid in replicas.replica_streams(rank, N_ROT)]
+    for rp in reps:
+        rp.early_prefix = not args.no_early_prefix
     stream = torch.cuda.current_stream()
 
     # ---- dry run: how many verify steps each request needs to emit its target ------------
@@ -645,6 +652,7 @@ def main():
     ap.add_argument("--no-extra", dest="extra", action="store_false",
                     help="skip the HBM-sized launches of the attention and gather kernels")
     ap.add_argument("--cpu-budget", type=float, default=15.0)
+    ap.add_argument("--no-early-prefix", action="store_true", help="do not prefetch the KV prefix under the previous layer")
     ap.add_argument("--no-overlap", action="store_true", help="plain launches (no programmatic stream serialization)")
     ap.add_argument("--attn-splits", type=int, default=0, help="force key splits per cluster (0 auto)")
     ap.add_argument("--attn-path", type=int, default=0, help="tree-attention kernel: 0 auto, 1 mma.sync, 2 tcgen05")

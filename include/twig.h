@@ -218,6 +218,15 @@ int32_t twig_set_attention_path(int32_t path);
  * so results do not change.  0 switches it off.  Returns the previous value. */
 int32_t twig_set_launch_overlap(int32_t on);
 
+/* Early prefix (default off; needs launch overlap).  While it is on, the caller promises for every
+ * following tree_verify_attention call that the kernel preceding it in its stream writes neither
+ * kv_len, n_nodes, parent nor cache rows below kv_len (true between the layers of one verification
+ * step, where the preceding kernels are the previous layer's; false right after tree_accept_compact or
+ * ttp_compact, which write kv_len).  The small-call kernel then reads the lengths and prefetches the
+ * cached prefix while the preceding kernel is still draining; Q, tree_k and tree_v are still read only
+ * after it has completed.  Results do not change when the promise holds.  Returns the previous value. */
+int32_t twig_set_early_prefix(int32_t on);
+
 /* Forces the number of key splits (CTAs per cluster) of the tree-attention kernels:
  * 1, 2, 4 or 8; 0 = automatic (default).  A tuning control.  Returns the previous value. */
 int32_t twig_set_attention_splits(int32_t splits);

@@ -71,7 +71,11 @@ tree_attn_kernel(const AttnParams p) {
   const int hk = blockIdx.y / p.row_blocks, rb = blockIdx.y % p.row_blocks;
   const int b = blockIdx.z;
 
-  grid_dependency_sync();
+  // Normally nothing is read before the preceding kernel of the stream has completed.  With
+  // `early_prefix` the caller has promised that the preceding kernel writes neither the lengths,
+  // the parent array nor cache rows below kv_len: those are then read (and the prefix tiles
+  // prefetched) while that kernel is still draining, and only Q and the tree's rows wait.
+  if (!p.early_prefix) grid_dependency_sync();
   // ---- per-request metadata; every exit below is uniform over the cluster ----
   const int n = p.n_nodes[b], L = p.kv_len[b];
   const int my_parent = tid < p.t_max ? p.parent[(long long)b * p.t_max + tid] : -1;   // (in flight with n, L)
@@ -132,7 +136,17 @@ tree_attn_kernel(const AttnParams p) {
   };
 
   // ---- start the copies first: Q tile (zero rows past the last row) and the first key tiles ----
-  {
+  bool prefetched[STAGES > 1 ? STAGES - 1 : 1];
+  if (p.early_prefix) {
+#pragma unroll
+    for (int s = 0; s < STAGES - 1; ++s) {
+      const int t = t_begin + s;
+      prefetched[s] = t < t_end && t * KT + KT <= L;      // wholly inside the cached prefix
+      if (prefetched[s]) load_tile(t, s);
+      cp_async_commit();
+    }
+  }
+  auto load_q = [&]() {
     constexpr int CHUNKS = ROWS * C::CPR;
 #pragma unroll
     for (int i = 0; i < (CHUNKS + C::THREADS - 1) / C::THREADS; ++i) {
@@ -146,11 +160,14 @@ tree_attn_kernel(const AttnParams p) {
           p.q + (((long long)b * p.t_max + node) * p.n_q_heads + hk * p.group + g) * D + c * 8;
       cp_async_16(q_s + tile_off<ROWS>(r, c), src, valid);
     }
-  }
+  };
+  if (!p.early_prefix) {
+    load_q();
 #pragma unroll
-  for (int s = 0; s < STAGES - 1; ++s) {
-    if (t_begin + s < t_end) load_tile(t_begin + s, s);
-    cp_async_commit();        // the first group also carries Q
+    for (int s = 0; s < STAGES - 1; ++s) {
+      if (t_begin + s < t_end) load_tile(t_begin + s, s);
+      cp_async_commit();        // the first group also carries Q
+    }
   }
 
   // ---- while they fly: parent array -> shared memory, validation, ancestor masks ----
@@ -175,6 +192,16 @@ tree_attn_kernel(const AttnParams p) {
       x = s_par[x];
     }
     s_mask[tid] = m;
+  }
+
+  if (p.early_prefix) {     // now wait for the preceding kernel; then Q and the tiles that hold tree rows
+    grid_dependency_sync();
+    load_q();
+#pragma unroll
+    for (int s = 0; s < STAGES - 1; ++s)
+      if (t_begin + s < t_end && !prefetched[s]) load_tile(t_begin + s, s);
+    cp_async_commit();
+    cp_async_wait<0>();
   }
 
   // ---- per-thread state --------------------------------------------------------
@@ -456,8 +483,8 @@ int pick_splits(int items, int max_tiles, int ctas_per_sm) {
 
 template <int D>
 static twig_status dispatch_attn(AttnParams &p, int batch, int rows, cudaStream_t st) {
-  using C16 = AttnCfg<D, 1, 4, 16, 3, 2>;
-  using C32 = AttnCfg<D, 2, 4, 16, 3, 2>;
+  using C16 = AttnCfg<D, 1, 4, 16, 2, 2>;
+  using C32 = AttnCfg<D, 2, 4, 16, 2, 2>;
   using C64 = AttnCfg<D, 4, 2, 32, 2, 2>;
   using C128 = AttnCfg<D, 8, 1, 64, 2, 1>;
   const int rows_per_cta = rows <= 16 ? 16 : rows <= 32 ? 32 : rows <= 64 ? 64 : 128;
@@ -478,6 +505,14 @@ static twig_status dispatch_attn(AttnParams &p, int batch, int rows, cudaStream_
 using namespace twig;
 
 static int g_attention_path = 0;
+static int g_early_prefix = 0;
+
+extern "C" int32_t twig_set_early_prefix(int32_t on) {
+  const int prev = g_early_prefix;
+  g_early_prefix = on != 0;
+  return prev;
+}
+
 
 extern "C" int32_t twig_set_attention_path(int32_t path) {
   const int prev = g_attention_path;
@@ -535,6 +570,7 @@ extern "C" twig_status tree_verify_attention(const void *q, const void *tree_k, 
   p.group = n_q_heads / cache->n_kv_heads;
   p.max_len = cache->max_len;
   p.row_blocks = 1;
+  p.early_prefix = (g_early_prefix && launch_overlap_enabled()) ? 1 : 0;
   const float scale = softmax_scale != 0.f ? softmax_scale : 1.f / sqrtf((float)cache->head_dim);
   p.scale_log2 = scale * 1.4426950408889634f;
   const int rows = t_max * p.group;

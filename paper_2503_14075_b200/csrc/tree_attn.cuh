@@ -18,6 +18,7 @@ struct AttnParams {
   const __nv_bfloat16 *cache_k0, *cache_v0;
   long long c_sl;
   int layer, n_layers, batch;
+  int early_prefix;   // see twig_set_early_prefix
   float scale_log2;   // softmax_scale * log2(e)
 };
 

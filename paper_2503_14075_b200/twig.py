@@ -26,7 +26,7 @@ STATUS_NAMES = {0: "TWIG_OK", 1: "TWIG_ERR_NULL", 2: "TWIG_ERR_SHAPE", 3: "TWIG_
 DEV_OK, DEV_BAD_LAYOUT, DEV_BAD_KEEP, DEV_BAD_INDEX, DEV_BAD_TREE, DEV_OVERFLOW, DEV_INTERNAL = range(7)
 MAX_NODES, MAX_VISUAL, MAX_BATCH = 64, 16384, 4096
 
-EXPORTS = ["twig_status_str", "twig_set_launch_overlap", "twig_set_attention_path", "twig_set_attention_splits", "twig_workspace_bytes", "ttp_score", "ttp_score_noalloc", "ttp_topk", "ttp_compact", "ttp_compact_rows",
+EXPORTS = ["twig_status_str", "twig_set_launch_overlap", "twig_set_early_prefix", "twig_set_attention_path", "twig_set_attention_splits", "twig_workspace_bytes", "ttp_score", "ttp_score_noalloc", "ttp_topk", "ttp_compact", "ttp_compact_rows",
            "ttp_score_topk_compact", "tree_verify_attention", "tree_accept_compact"]
 
 
@@ -62,6 +62,8 @@ _lib.twig_set_attention_path.restype = C.c_int32
 _lib.twig_set_attention_path.argtypes = [C.c_int32]
 _lib.twig_set_launch_overlap.restype = C.c_int32
 _lib.twig_set_launch_overlap.argtypes = [C.c_int32]
+_lib.twig_set_early_prefix.restype = C.c_int32
+_lib.twig_set_early_prefix.argtypes = [C.c_int32]
 _lib.twig_set_attention_splits.restype = C.c_int32
 _lib.twig_set_attention_splits.argtypes = [C.c_int32]
 _lib.twig_workspace_bytes.restype = _sz
@@ -117,6 +119,12 @@ def twig_set_attention_path(path: int) -> int:
 def twig_set_launch_overlap(on: int) -> int:
     """Programmatic stream serialization for the attention and accept kernels (default on)."""
     return int(_lib.twig_set_launch_overlap(int(on)))
+
+
+def twig_set_early_prefix(on: int) -> int:
+    """Promise that the kernel before each following tree_verify_attention call leaves kv_len, n_nodes,
+    parent and the cache rows below kv_len alone (e.g. between the layers of one verify step)."""
+    return int(_lib.twig_set_early_prefix(int(on)))
 
 
 def twig_set_attention_splits(splits: int) -> int:

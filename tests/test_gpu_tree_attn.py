@@ -187,3 +187,38 @@ class _F64View:
 
     def __getitem__(self, idx):
         return synth.bf16_to_f64(self.bits[idx])
+
+
+@pytest.mark.parametrize("shape", [SHAPES[0], SHAPES[2], SHAPES[6]], ids=["c1", "rows32", "d64-rows64"])
+def test_early_prefix_gives_the_same_bits(tw, shape):
+    """With the early-prefix promise kept (nothing before the call writes lengths or cache), the
+    small-call kernel prefetches the prefix under its predecessor and must return identical bits."""
+    name, B, Hq, Hkv, d, n_nodes, depth, kv_len = shape
+    wl = _wl(B, Hq, Hkv, d, n_nodes, depth)
+    rng = synth.rng_for(9, 321)
+    ver = synth.make_verify_inputs(wl, rng, n_layers=1, gain=d ** 0.5)
+    ck, cv = synth.make_cache(wl, rng, max(kv_len) + 70, n_layers=1, gain=d ** 0.5)
+    ref, ref_lse, st0 = run_attention(tw, wl, ver, ck, cv, kv_len, path=1)
+    tw.twig_set_early_prefix(1)
+    try:
+        got, got_lse, st1 = run_attention(tw, wl, ver, ck, cv, kv_len, path=1)
+        # twice back to back on one stream: the second call prefetches under the first
+        B_, T, Hq_, d_ = ver["q"].shape[1:]
+        dck, dcv = dev_bf16(ck), dev_bf16(cv)
+        cache = tw.KV.of(dck, dcv)
+        q, tk, tv = dev_bf16(ver["q"][0]), dev_bf16(ver["tree_k"][0]), dev_bf16(ver["tree_v"][0])
+        kvl, nn, par = dev_i32(kv_len), dev_i32(ver["n_nodes"]), dev_i32(ver["parent"])
+        outs = [torch.zeros((B_, T, Hq_, d_), dtype=torch.bfloat16, device=DEV) for _ in range(3)]
+        tw.twig_set_attention_path(1)
+        for o in outs:
+            tw.tree_verify_attention(q, tk, tv, cache, 0, kvl, nn, par, o)
+        torch.cuda.synchronize()
+    finally:
+        tw.twig_set_early_prefix(0)
+        tw.twig_set_attention_path(0)
+    assert not st0.any() and not st1.any()
+    assert np.array_equal(got, ref) and np.array_equal(got_lse, ref_lse)
+    for b in range(B):
+        n = n_nodes[b]
+        for o in outs:
+            assert np.array_equal(host_bits(o)[b, :n], ref[b, :n])
