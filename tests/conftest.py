@@ -24,3 +24,13 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+def pytest_sessionstart(session):
+    """Build the C-ABI library if it is missing or older than its sources (nvcc cross-compiles
+    without a GPU), so that the tests never run against a stale binary."""
+    try:
+        from paper_2503_14075_b200 import build
+        build.build()
+    except Exception as e:  # pragma: no cover - the ABI test reports the failure properly
+        print("could not build libtwig.so:", e)
