@@ -545,6 +545,22 @@ def extra_rooflines(torch, tw, peaks, dev):
                                    "achieved": round(by / us / 1e3, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
                                    "frac": round(by / us / 1e3 / peaks["hbm_gbs"], 4),
                                    "l2": f"chain of {n_chain} launches over {n_sets} rotating 394 MB source sets"}
+    del sets
+    # greedy target token per tree node over the heterogeneous batch's trees (32000-entry bf16 rows);
+    # six logits buffers in turn, 190 MB together, so that every read is cold
+    V = 32000
+    nn3 = i32(wl3.n_nodes)
+    bufs = [torch.randn((wl3.batch, wl3.t_max, V), dtype=torch.bfloat16, device=dev) for _ in range(6)]
+    arg = torch.zeros((wl3.batch, wl3.t_max), dtype=torch.int32, device=dev)
+    for bfr in bufs:
+        tw.tree_base_argmax(bfr, nn3, arg)
+    e0.record(stream)
+    for i in range(n_chain):
+        tw.tree_base_argmax(bufs[i % 6], nn3, arg)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    us = e0.elapsed_time(e1) * 1e3 / n_chain
+    res["base_argmax_c3_V32000"] = hbm_entry(us, int(sum(wl3.n_nodes)) * V * 2)
     return res
 
 

@@ -231,6 +231,18 @@ int32_t twig_set_early_prefix(int32_t on);
  * 1, 2, 4 or 8; 0 = automatic (default).  A tuning control.  Returns the previous value. */
 int32_t twig_set_attention_splits(int32_t splits);
 
+/* ---- Greedy target token of every tree node (input of tree_accept_compact) -----
+ * Algorithm 2 ("argmax(tgt_probs[...])"), Sec. 5.4: base_argmax[b, i] = the index of the largest of
+ * logits[b, i, 0..vocab), the LOWEST index among equal values, for i < n_nodes[b]; other entries
+ * are left untouched.  Logits must not be NaN.
+ *   logits      [batch, t_max, vocab] at logits + (b*t_max + i)*row_stride (ELEMENTS), bf16
+ *               (logits_fp32 = 0) or fp32 (logits_fp32 = 1); rows 16-byte aligned
+ *   base_argmax [batch, t_max] int32 out
+ */
+twig_status tree_base_argmax(const void *logits, int32_t logits_fp32, int64_t row_stride, int32_t vocab,
+                             const int32_t *n_nodes, int32_t batch, int32_t t_max,
+                             int32_t *base_argmax, int32_t *dev_status, void *stream);
+
 /* ---- Acceptance + bonus token + KV append, all layers in one call ------------
  * Sec. 5.4 / Appendix A / Algorithm 2.  Node 0 is the last accepted token and is
  * always accepted; child c is accepted iff its parent is and

@@ -241,6 +241,23 @@ def tree_accept(parent, draft_tok, base_argmax, n_nodes: int):
     return best_depth, np.array(path, dtype=np.int32), int(base_argmax[best])
 
 
+def base_argmax(logits, n_nodes):
+    """Algorithm 2, "argmax(tgt_probs[...])": the target's greedy token after every tree node.
+    logits [B, T, V]; returns int32 [B, T] with the LOWEST index among equal maxima and 0 for
+    nodes >= n_nodes[b] (softmax is monotonic, so probabilities and logits agree)."""
+    logits = np.asarray(logits, dtype=np.float64)
+    B, T, V = logits.shape
+    out = np.zeros((B, T), dtype=np.int32)
+    for b in range(B):
+        for i in range(int(n_nodes[b])):
+            best, best_v = 0, logits[b, i, 0]
+            for v in range(1, V):
+                if logits[b, i, v] > best_v:
+                    best, best_v = v, logits[b, i, v]
+            out[b, i] = best
+    return out
+
+
 # --------------------------------------------------------------------------
 # O6: append the accepted nodes' K/V rows to the cache
 # --------------------------------------------------------------------------

@@ -124,9 +124,117 @@ tree_accept_compact_kernel(const int *__restrict__ parent, const int *__restrict
   }
 }
 
+// ---------------------------------------------------------------------------
+// Greedy target token per tree node: argmax over the vocabulary, lowest index on ties.
+// One CTA per (request, node) row; 16-byte loads, 4 in flight per thread.
+// ---------------------------------------------------------------------------
+constexpr int kArgmaxThreads = 256;
+
+__device__ __forceinline__ void argmax_take(float v, int i, float &best, int &bi) {
+  if (v > best || (v == best && i < bi)) {
+    best = v;
+    bi = i;
+  }
+}
+
+template <bool FP32>
+__global__ void __launch_bounds__(kArgmaxThreads)
+base_argmax_kernel(const void *__restrict__ logits, long long row_stride, int vocab,
+                   const int *__restrict__ n_nodes, int t_max, int *__restrict__ out, int *dev_status) {
+  constexpr int EPC = FP32 ? 4 : 8;                 // elements per 16-byte chunk
+  __shared__ float s_v[kArgmaxThreads / 32];
+  __shared__ int s_i[kArgmaxThreads / 32];
+  grid_dependency_sync();
+  const int b = blockIdx.y, node = blockIdx.x, tid = threadIdx.x;
+  const int n = n_nodes[b];
+  if (n < 0 || n > t_max) {
+    if (node == 0 && tid == 0) flag_status(dev_status, b, TWIG_DEV_BAD_TREE);
+    return;
+  }
+  if (node >= n) return;
+  const unsigned char *row = static_cast<const unsigned char *>(logits) +
+                             ((long long)b * t_max + node) * row_stride * (FP32 ? 4 : 2);
+  float best = -INFINITY;
+  int bi = 0x7fffffff;
+  const int chunks = vocab / EPC;
+  auto take_chunk = [&](const uint4 &w, int c) {
+    const int base = c * EPC;
+    if (FP32) {
+      argmax_take(__uint_as_float(w.x), base, best, bi);
+      argmax_take(__uint_as_float(w.y), base + 1, best, bi);
+      argmax_take(__uint_as_float(w.z), base + 2, best, bi);
+      argmax_take(__uint_as_float(w.w), base + 3, best, bi);
+    } else {
+      argmax_take(bf16_lo(w.x), base, best, bi);
+      argmax_take(bf16_hi(w.x), base + 1, best, bi);
+      argmax_take(bf16_lo(w.y), base + 2, best, bi);
+      argmax_take(bf16_hi(w.y), base + 3, best, bi);
+      argmax_take(bf16_lo(w.z), base + 4, best, bi);
+      argmax_take(bf16_hi(w.z), base + 5, best, bi);
+      argmax_take(bf16_lo(w.w), base + 6, best, bi);
+      argmax_take(bf16_hi(w.w), base + 7, best, bi);
+    }
+  };
+  int c = tid;
+  for (; c + 3 * kArgmaxThreads < chunks; c += 4 * kArgmaxThreads) {
+    uint4 w[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) w[u] = ld_nc_16(row + (long long)(c + u * kArgmaxThreads) * 16);
+#pragma unroll
+    for (int u = 0; u < 4; ++u) take_chunk(w[u], c + u * kArgmaxThreads);
+  }
+  for (; c < chunks; c += kArgmaxThreads) take_chunk(ld_nc_16(row + (long long)c * 16), c);
+  for (int i = chunks * EPC + tid; i < vocab; i += kArgmaxThreads) {     // tail that is no whole chunk
+    const float v = FP32 ? reinterpret_cast<const float *>(row)[i]
+                         : __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(row)[i]);
+    argmax_take(v, i, best, bi);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float ov = __shfl_xor_sync(0xffffffffu, best, o);
+    const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+    argmax_take(ov, oi, best, bi);
+  }
+  if ((tid & 31) == 0) {
+    s_v[tid >> 5] = best;
+    s_i[tid >> 5] = bi;
+  }
+  __syncthreads();
+  if (tid == 0) {
+    for (int w = 1; w < kArgmaxThreads / 32; ++w) argmax_take(s_v[w], s_i[w], best, bi);
+    out[(long long)b * t_max + node] = bi;
+  }
+}
+
 }  // namespace twig
 
 using namespace twig;
+
+extern "C" twig_status tree_base_argmax(const void *logits, int32_t logits_fp32, int64_t row_stride,
+                                        int32_t vocab, const int32_t *n_nodes, int32_t batch,
+                                        int32_t t_max, int32_t *base_argmax, int32_t *dev_status,
+                                        void *stream) {
+  if (!logits || !n_nodes || !base_argmax) return TWIG_ERR_NULL;
+  if (vocab <= 0 || batch <= 0 || t_max <= 0 || row_stride < vocab) return TWIG_ERR_SHAPE;
+  if (t_max > TWIG_MAX_NODES || batch > TWIG_MAX_BATCH) return TWIG_ERR_UNSUPPORTED;
+  const int esz = logits_fp32 ? 4 : 2;
+  if (!aligned16(logits) || (row_stride * esz) % 16) return TWIG_ERR_ALIGN;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(t_max, batch);
+  cfg.blockDim = dim3(kArgmaxThreads);
+  cfg.stream = static_cast<cudaStream_t>(stream);
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = launch_overlap_enabled() ? 1 : 0;
+  const long long rs = row_stride;
+  const cudaError_t err =
+      logits_fp32 ? cudaLaunchKernelEx(&cfg, base_argmax_kernel<true>, logits, rs, vocab, n_nodes, t_max, base_argmax, dev_status)
+                  : cudaLaunchKernelEx(&cfg, base_argmax_kernel<false>, logits, rs, vocab, n_nodes, t_max, base_argmax, dev_status);
+  return err == cudaSuccess ? TWIG_OK : TWIG_ERR_CUDA;
+}
+
 
 extern "C" twig_status tree_accept_compact(const int32_t *parent, const int32_t *draft_tok,
                                            const int32_t *base_argmax, const int32_t *n_nodes,

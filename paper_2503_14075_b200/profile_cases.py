@@ -4,6 +4,7 @@
   python -m paper_2503_14075_b200.profile_cases gather --workload 4 --layers 2 --iters 3
   python -m paper_2503_14075_b200.profile_cases score  --workload 4 --iters 3
   python -m paper_2503_14075_b200.profile_cases accept --workload 2 --layers 32 --iters 3
+  python -m paper_2503_14075_b200.profile_cases argmax --workload 4 --iters 3
 
 Every case holds well under a few GB on the device and launches a handful of kernels, so
 that a profiler capture ends by itself.  Prints the mean launch time from CUDA events.
@@ -128,17 +129,30 @@ def case_accept(a):
     print(f"accept {wl.name} {nl} layers: {us:.2f} us per (fill, accept) pair")
 
 
+def case_argmax(a):
+    wl = synth.workload(a.workload)
+    rng = synth.rng_for(a.workload, 904)
+    B, T, V = wl.batch, wl.t_max, a.vocab
+    logits = torch.from_numpy(rng.standard_normal((B, T, V), dtype=np.float32)).to(DEV).to(torch.bfloat16)
+    nn = _i32(wl.n_nodes)
+    out = torch.zeros((B, T), dtype=torch.int32, device=DEV)
+    us = _time(lambda: tw.tree_base_argmax(logits, nn, out), a.iters)
+    by = sum(wl.n_nodes) * V * 2
+    print(f"argmax {wl.name} V={V}: {us:.2f} us/launch, {by / us / 1e3:.1f} GB/s algorithmic ({by} B/launch)")
+
+
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("case", choices=["attn", "gather", "score", "accept"])
+    ap.add_argument("case", choices=["attn", "gather", "score", "accept", "argmax"])
     ap.add_argument("--workload", type=int, default=4)
     ap.add_argument("--kv-len", type=int, default=0)
     ap.add_argument("--layers", type=int, default=2)
     ap.add_argument("--iters", type=int, default=3)
+    ap.add_argument("--vocab", type=int, default=32000)
     ap.add_argument("--splits", type=int, default=0, help="force key splits (0 auto)")
     ap.add_argument("--path", type=int, default=0, help="attention kernel: 0 auto, 1 mma.sync, 2 tcgen05")
     a = ap.parse_args()
-    {"attn": case_attn, "gather": case_gather, "score": case_score, "accept": case_accept}[a.case](a)
+    {"attn": case_attn, "gather": case_gather, "score": case_score, "accept": case_accept, "argmax": case_argmax}[a.case](a)
 
 
 if __name__ == "__main__":

@@ -27,7 +27,7 @@ DEV_OK, DEV_BAD_LAYOUT, DEV_BAD_KEEP, DEV_BAD_INDEX, DEV_BAD_TREE, DEV_OVERFLOW,
 MAX_NODES, MAX_VISUAL, MAX_BATCH = 64, 16384, 4096
 
 EXPORTS = ["twig_status_str", "twig_set_launch_overlap", "twig_set_early_prefix", "twig_set_attention_path", "twig_set_attention_splits", "twig_workspace_bytes", "ttp_score", "ttp_score_noalloc", "ttp_topk", "ttp_compact", "ttp_compact_rows",
-           "ttp_score_topk_compact", "tree_verify_attention", "tree_accept_compact"]
+           "ttp_score_topk_compact", "tree_verify_attention", "tree_base_argmax", "tree_accept_compact"]
 
 
 class TwigError(RuntimeError):
@@ -89,6 +89,8 @@ _lib.ttp_score_topk_compact.argtypes = [_vp, _vp, _i64, _i64, _i64, _i32, _vp, _
 _lib.tree_verify_attention.restype = C.c_int
 _lib.tree_verify_attention.argtypes = [_vp, _vp, _vp, _kvp, _i32, _vp, _vp, _vp, _i32, _i32, _f32, _vp, _vp,
                                        _vp, _vp, _sz, _vp]
+_lib.tree_base_argmax.restype = C.c_int
+_lib.tree_base_argmax.argtypes = [_vp, _i32, _i64, _i32, _vp, _i32, _i32, _vp, _vp, _vp]
 _lib.tree_accept_compact.restype = C.c_int
 _lib.tree_accept_compact.argtypes = [_vp, _vp, _vp, _vp, _i32, _i32, _vp, _vp, _kvp, _vp, _vp, _vp, _vp,
                                      _vp, _vp]
@@ -205,6 +207,15 @@ def tree_verify_attention(q, tree_k, tree_v, cache: KV, layer, kv_len, n_nodes, 
     _check(_lib.tree_verify_attention(_p(q), _p(tree_k), _p(tree_v), C.byref(cache), layer, _p(kv_len),
                                       _p(n_nodes), _p(parent), T, Hq, softmax_scale, _p(out), _p(lse),
                                       _p(dev_status), _p(ws), ws_bytes, _stream(stream)))
+
+
+def tree_base_argmax(logits, n_nodes, base_argmax, dev_status=None, stream=None):
+    """logits [B, T, V] bf16 or fp32 (last dim contiguous); base_argmax [B, T] int32 (out):
+    the target's greedy token after every tree node, lowest index on ties."""
+    B, T, V = logits.shape
+    assert logits.stride(2) == 1 and logits.stride(0) == T * logits.stride(1)
+    _check(_lib.tree_base_argmax(_p(logits), 1 if logits.dtype == torch.float32 else 0, logits.stride(1), V,
+                                 _p(n_nodes), B, T, _p(base_argmax), _p(dev_status), _stream(stream)))
 
 
 def tree_accept_compact(parent, draft_tok, base_argmax, n_nodes, tree_k_all, tree_v_all, cache: KV,

@@ -175,3 +175,39 @@ def test_prune_then_verify_loop_matches_oracle(tw):
         torch.cuda.synchronize()
         assert not status.cpu().numpy().any()
         assert np.array_equal(host_bits(dk), ok) and np.array_equal(host_bits(dv), ov)
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "fp32"])
+@pytest.mark.parametrize("vocab", [32000, 32003, 7])
+def test_base_argmax_bit_exact(tw, dtype, vocab):
+    """Greedy target token per tree node: lowest index on ties (bf16 rounding makes ties common)."""
+    rng = np.random.default_rng(41)
+    B, T = 3, 9
+    n_nodes = [9, 4, 0]
+    x = rng.standard_normal((B, T, vocab)).astype(np.float32)
+    x[0, 1, :] = 0.25                                   # all equal -> index 0
+    if vocab > 10:
+        x[0, 2, [5, vocab - 1]] = 9.0                   # tie between far-apart indices
+        x[1, 0, vocab - 1] = 11.0                       # winner in the ragged tail
+    stride = (vocab + 7) // 8 * 8                       # rows start on 16 bytes
+    if dtype == "bf16":
+        bits = synth.f32_to_bf16(x)
+        padded = np.full((B, T, stride), 0x7F7F, dtype=bits.dtype)   # padding holds a huge value
+        padded[..., :vocab] = bits
+        dev = dev_bf16(padded)[..., :vocab]
+        ref_in = synth.bf16_to_f64(bits)
+    else:
+        padded = np.full((B, T, stride), 3e38, dtype=np.float32)
+        padded[..., :vocab] = x
+        dev = torch.from_numpy(padded).to(DEV)[..., :vocab]
+        ref_in = x.astype(np.float64)
+    out = torch.full((B, T), -5, dtype=torch.int32, device=DEV)
+    status = torch.zeros(B, dtype=torch.int32, device=DEV)
+    tw.tree_base_argmax(dev, dev_i32(n_nodes), out, dev_status=status)
+    torch.cuda.synchronize()
+    want = O.base_argmax(ref_in, n_nodes)
+    got = out.cpu().numpy()
+    assert not status.cpu().numpy().any()
+    for b in range(B):
+        assert np.array_equal(got[b, :n_nodes[b]], want[b, :n_nodes[b]])
+        assert np.all(got[b, n_nodes[b]:] == -5)

@@ -35,6 +35,7 @@ MUTATIONS = [
      "return best_depth, np.array(path, dtype=np.int32), int(base_argmax[0])"),
     ("append: rows written one position late", "cache_k[:, b, :, base + j, :]", "cache_k[:, b, :, base + j + 1, :]"),
     ("append: length not advanced by the root", "new_len[b] = base + len(paths[b])", "new_len[b] = base + len(paths[b]) - 1"),
+    ("argmax: ties to the higher index", "if logits[b, i, v] > best_v:", "if logits[b, i, v] >= best_v:"),
     ("eq. 6: K_f ignored", "upper = L if K_f is None else K_f", "upper = L"),
 ]
 

@@ -471,6 +471,22 @@ def test_speculative_decoding_is_lossless_with_toy_target():
     assert seq[:len(greedy)] == greedy
 
 
+def test_base_argmax_library_and_ties():
+    rng = np.random.default_rng(31)
+    x = rng.integers(-3, 4, size=(2, 5, 40)).astype(np.float64)          # many exact ties
+    got = O.base_argmax(x, [5, 3])
+    assert np.array_equal(got[0], np.argmax(x[0], axis=-1))               # numpy: first occurrence
+    assert np.array_equal(got[1, :3], np.argmax(x[1, :3], axis=-1)) and np.all(got[1, 3:] == 0)
+    y = np.zeros((1, 2, 9))
+    y[0, 0, [4, 7]] = 2.5
+    y[0, 1, 8] = 1e-300
+    assert O.base_argmax(y, [2]).tolist() == [[4, 8]]
+    # the argmax of the logits is the argmax of the probabilities the paper's pseudocode uses
+    import scipy.special as sp
+    z = rng.standard_normal((1, 4, 50))
+    assert np.array_equal(O.base_argmax(z, [4]), O.base_argmax(sp.softmax(z, axis=-1), [4]))
+
+
 # ---------------------------------------------------------------- O6 accept-compact
 def test_accept_compact_tail_rows_and_canaries():
     nl, B, H, T, L, d = 2, 2, 2, 5, 12, 3
