@@ -45,6 +45,11 @@ struct AttnCfg {
   // buffer outside the stage ring: peers may then push as soon as they are done, and one
   // cluster barrier of the epilogue goes away.
   static constexpr bool RECV_OWN = ROWS <= 32;
+  // The same variants spend far less time computing a tile than waiting for it, so they keep the
+  // whole ring in flight (a stage is refilled after its tile has been used) instead of one stage
+  // less (refilled before): STAGES rather than STAGES - 1 tiles are requested up front.
+  static constexpr bool FULL_RING = ROWS <= 32;
+  static constexpr int PRE = FULL_RING ? STAGES : STAGES - 1;
   static_assert(XCH_BYTES + (RECV_OWN ? 0 : RECV_BYTES) <= STAGE_BYTES, "epilogue buffers must fit in the stage ring");
   static constexpr int RECV_OFFSET = RECV_OWN ? Q_BYTES + STAGE_BYTES : Q_BYTES + XCH_BYTES;
   static constexpr int SMEM_BYTES = Q_BYTES + STAGE_BYTES + (RECV_OWN ? RECV_BYTES : 0);
@@ -136,10 +141,11 @@ tree_attn_kernel(const AttnParams p) {
   };
 
   // ---- start the copies first: Q tile (zero rows past the last row) and the first key tiles ----
-  bool prefetched[STAGES > 1 ? STAGES - 1 : 1];
+  constexpr int PRE = C::PRE;
+  bool prefetched[PRE > 0 ? PRE : 1];
   if (p.early_prefix) {
 #pragma unroll
-    for (int s = 0; s < STAGES - 1; ++s) {
+    for (int s = 0; s < PRE; ++s) {
       const int t = t_begin + s;
       prefetched[s] = t < t_end && t * KT + KT <= L;      // wholly inside the cached prefix
       if (prefetched[s]) load_tile(t, s);
@@ -164,7 +170,7 @@ tree_attn_kernel(const AttnParams p) {
   if (!p.early_prefix) {
     load_q();
 #pragma unroll
-    for (int s = 0; s < STAGES - 1; ++s) {
+    for (int s = 0; s < PRE; ++s) {
       if (t_begin + s < t_end) load_tile(t_begin + s, s);
       cp_async_commit();        // the first group also carries Q
     }
@@ -198,7 +204,7 @@ tree_attn_kernel(const AttnParams p) {
     grid_dependency_sync();
     load_q();
 #pragma unroll
-    for (int s = 0; s < STAGES - 1; ++s)
+    for (int s = 0; s < PRE; ++s)
       if (t_begin + s < t_end && !prefetched[s]) load_tile(t_begin + s, s);
     cp_async_commit();
     cp_async_wait<0>();
@@ -216,9 +222,9 @@ tree_attn_kernel(const AttnParams p) {
 
   for (int t = t_begin; t < t_end; ++t) {
     const int it = t - t_begin;
-    cp_async_wait<STAGES - 2>();
+    cp_async_wait<PRE - 1>();
     __syncthreads();
-    {   // refill the stage that was consumed one iteration ago
+    if (!C::FULL_RING) {   // refill the stage that was consumed one iteration ago
       const int tn = t + STAGES - 1;
       if (tn < t_end) load_tile(tn, (it + STAGES - 1) % STAGES);
       cp_async_commit();
@@ -320,6 +326,14 @@ tree_attn_kernel(const AttnParams p) {
         mma_bf16(o[2 * dp], pf[kk], vb[0], vb[1]);
         mma_bf16(o[2 * dp + 1], pf[kk], vb[2], vb[3]);
       }
+    }
+    if (C::FULL_RING) {    // refill this tile's own stage once every warp has finished with it
+      const int tn = t + STAGES;
+      if (tn < t_end) {
+        __syncthreads();
+        load_tile(tn, stage);
+      }
+      cp_async_commit();
     }
   }
   cp_async_wait<0>();
@@ -481,10 +495,15 @@ int pick_splits(int items, int max_tiles, int ctas_per_sm) {
   return s;
 }
 
+// warps that share the 64 keys of a tile in the 16- and 32-row variants
+#ifndef TWIG_SMALL_WN
+#define TWIG_SMALL_WN 4
+#endif
+
 template <int D>
 static twig_status dispatch_attn(AttnParams &p, int batch, int rows, cudaStream_t st) {
-  using C16 = AttnCfg<D, 1, 4, 16, 2, 2>;
-  using C32 = AttnCfg<D, 2, 4, 16, 2, 2>;
+  using C16 = AttnCfg<D, 1, TWIG_SMALL_WN, 64 / TWIG_SMALL_WN, 2, 2>;
+  using C32 = AttnCfg<D, 2, TWIG_SMALL_WN, 64 / TWIG_SMALL_WN, 2, 2>;
   using C64 = AttnCfg<D, 4, 2, 32, 2, 2>;
   using C128 = AttnCfg<D, 8, 1, 64, 2, 1>;
   const int rows_per_cta = rows <= 16 ? 16 : rows <= 32 ? 32 : rows <= 64 ? 64 : 128;
