@@ -32,41 +32,50 @@ struct AttnCfg {
   static constexpr int D = D_, WM = WM_, WN = WN_, KC = KC_, STAGES = STAGES_, MIN_CTAS = MIN_CTAS_;
   static constexpr int ROWS = 16 * WM;          // query rows per CTA
   static constexpr int KT = KC * WN;            // keys per tile
+  static constexpr int DW = D / WN;             // output columns per warp
   static constexpr int THREADS = 32 * WM * WN;
   static constexpr int CPR = D / 8;             // 16-byte chunks per row
   static constexpr int Q_BYTES = ROWS * D * 2;
+  static constexpr int P_BYTES = WN > 1 ? ROWS * KT * 2 : 0;   // bf16 probabilities of one tile
   static constexpr int TILE_BYTES = KT * D * 2;
   static constexpr int STAGE_BYTES = 2 * STAGES * TILE_BYTES;
-  // after the key loop the stage ring is reused: XCH holds the partial O of the
-  // warps with wn > 0 (fragment order), RECV the per-split partials a CTA owns
-  static constexpr int XCH_BYTES = (WN - 1) * ROWS * D * 4;
-  static constexpr int RECV_BYTES = ROWS * D * 4;
+  static constexpr int RECV_BYTES = ROWS * D * 4;              // the per-split partials a CTA owns
+  static_assert(KT == 64, "a row of P is one 128-byte swizzled line");
+  static_assert(DW % 16 == 0 && KC % 16 == 0, "warp slices are whole ldmatrix.x4 steps");
   // The small, latency-bound variants (one CTA per SM is enough for them) keep the split-merge
   // buffer outside the stage ring: peers may then push as soon as they are done, and one
-  // cluster barrier of the epilogue goes away.
+  // cluster barrier of the epilogue goes away.  The others reuse the ring after the key loop.
   static constexpr bool RECV_OWN = ROWS <= 32;
   // The same variants spend far less time computing a tile than waiting for it, so they keep the
   // whole ring in flight (a stage is refilled after its tile has been used) instead of one stage
   // less (refilled before): STAGES rather than STAGES - 1 tiles are requested up front.
   static constexpr bool FULL_RING = ROWS <= 32;
   static constexpr int PRE = FULL_RING ? STAGES : STAGES - 1;
-  static_assert(XCH_BYTES + (RECV_OWN ? 0 : RECV_BYTES) <= STAGE_BYTES, "epilogue buffers must fit in the stage ring");
-  static constexpr int RECV_OFFSET = RECV_OWN ? Q_BYTES + STAGE_BYTES : Q_BYTES + XCH_BYTES;
-  static constexpr int SMEM_BYTES = Q_BYTES + STAGE_BYTES + (RECV_OWN ? RECV_BYTES : 0);
+  static_assert(RECV_OWN || RECV_BYTES <= STAGE_BYTES, "the receive buffer must fit in the stage ring");
+  static constexpr int P_OFFSET = Q_BYTES;
+  static constexpr int K_OFFSET = Q_BYTES + P_BYTES;
+  static constexpr int RECV_OFFSET = RECV_OWN ? K_OFFSET + STAGE_BYTES : K_OFFSET;
+  static constexpr int SMEM_BYTES = K_OFFSET + STAGE_BYTES + (RECV_OWN ? RECV_BYTES : 0);
 };
 
+// The WM x WN warps of a CTA: warp (wm, wn) owns query rows [16 wm, 16 wm + 16).  For S = Q K^T it
+// takes the KC keys [wn KC, wn KC + KC) of the tile; the WN warps of a row group agree on the row
+// maxima through shared memory and leave their bf16 probabilities there; for O += P V every warp
+// reads all KT probabilities of its rows and accumulates the DW output columns [wn DW, wn DW + DW).
+// No warp ever holds another's partial O, so nothing but maxima, probabilities and row sums is
+// exchanged inside the CTA.
 template <class C>
 __global__ void __launch_bounds__(C::THREADS, C::MIN_CTAS)
 tree_attn_kernel(const AttnParams p) {
   constexpr int D = C::D, ROWS = C::ROWS, KT = C::KT, KC = C::KC, WM = C::WM, WN = C::WN, STAGES = C::STAGES;
-  constexpr int NT = KC / 8;       // key n-tiles per warp per tile
-  constexpr int DT = D / 8;        // head-dim n-tiles of O
+  constexpr int NT = KC / 8;       // key n-tiles of S per warp per tile
+  constexpr int OT = C::DW / 8;    // head-dim n-tiles of O per warp
   constexpr int KS = D / 16;       // k-steps of Q K^T
   extern __shared__ __align__(1024) unsigned char smem[];
   __shared__ unsigned long long s_mask[TWIG_MAX_NODES];
   __shared__ int s_par[TWIG_MAX_NODES];
-  __shared__ float4 s_xml[(WN > 1 ? WN - 1 : 1) * WM * 32];   // (m_lo, m_hi, l_lo, l_hi) of warps wn > 0
-  __shared__ float r_m[ROWS], r_l[ROWS];                       // received (m, l): [sender][owned row]
+  __shared__ float s_stat[WN][ROWS];                            // row maxima of a tile, later row sums
+  __shared__ float r_m[ROWS], r_l[ROWS];                        // received (m, l): [sender][owned row]
   __shared__ int s_bad;
 
   cg::cluster_group cluster = cg::this_cluster();
@@ -75,6 +84,10 @@ tree_attn_kernel(const AttnParams p) {
   const int split = blockIdx.x, n_splits = gridDim.x;
   const int hk = blockIdx.y / p.row_blocks, rb = blockIdx.y % p.row_blocks;
   const int b = blockIdx.z;
+  // barrier of the WN warps that share a row group (ids 1..WM; 0 is __syncthreads)
+  auto group_sync = [&]() {
+    if (WN > 1) asm volatile("bar.sync %0, %1;" ::"r"(1 + wm), "n"(32 * WN) : "memory");
+  };
 
   // Normally nothing is read before the preceding kernel of the stream has completed.  With
   // `early_prefix` the caller has promised that the preceding kernel writes neither the lengths,
@@ -100,7 +113,8 @@ tree_attn_kernel(const AttnParams p) {
   if (C::RECV_OWN && n_splits > 1) asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
 
   const uint32_t q_s = smem_u32(smem);
-  const uint32_t k_s = q_s + C::Q_BYTES;
+  const uint32_t p_s = q_s + C::P_OFFSET;
+  const uint32_t k_s = q_s + C::K_OFFSET;
   const uint32_t v_s = k_s + STAGES * C::TILE_BYTES;
 
   // ---- key tiles of this CTA --------------------------------------------------
@@ -199,6 +213,18 @@ tree_attn_kernel(const AttnParams p) {
     }
     s_mask[tid] = m;
   }
+  __syncthreads();
+
+  // ---- per-thread state --------------------------------------------------------
+  const int gq = lane >> 2, tq = lane & 3;
+  const int r_lo = wm * 16 + gq, r_hi = r_lo + 8;         // CTA-local rows of this thread
+  // ancestor masks of this thread's two rows (0 for rows past the last one)
+  unsigned long long mask_lo = 0ull, mask_hi = 0ull;
+  {
+    const int g_lo = row0 + r_lo, g_hi = row0 + r_hi;
+    if (g_lo < rows_total) mask_lo = s_mask[p.group == 1 ? g_lo : g_lo / p.group];
+    if (g_hi < rows_total) mask_hi = s_mask[p.group == 1 ? g_hi : g_hi / p.group];
+  }
 
   if (p.early_prefix) {     // now wait for the preceding kernel; then Q and the tiles that hold tree rows
     grid_dependency_sync();
@@ -210,15 +236,13 @@ tree_attn_kernel(const AttnParams p) {
     cp_async_wait<0>();
   }
 
-  // ---- per-thread state --------------------------------------------------------
-  const int gq = lane >> 2, tq = lane & 3;
-  const int r_lo = wm * 16 + gq, r_hi = r_lo + 8;         // CTA-local rows of this thread
-  float o[DT][4];
+  float o[OT][4];
 #pragma unroll
-  for (int i = 0; i < DT; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
-  float m_lo = -INFINITY, m_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;
-  const uint32_t q_frag = q_s + (wm * 16 + (lane & 7) + ((lane >> 3) & 1) * 8) * 128;   // row base; chunk added per k-step
-  const int q_sw = (lane & 7);           // row & 7 of this lane's ldmatrix row
+  for (int i = 0; i < OT; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
+  float m_lo = -INFINITY, m_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;     // l: this warp's keys only
+  const int sw = lane & 7;                                               // (row & 7) of this lane's ldmatrix row
+  const uint32_t a_row = (wm * 16 + (lane & 7) + ((lane >> 3) & 1) * 8) * 128;   // A-operand row of this lane
+  const uint32_t q_frag = q_s + a_row, p_frag = p_s + a_row;             // chunk added per k-step
 
   for (int t = t_begin; t < t_end; ++t) {
     const int it = t - t_begin;
@@ -242,7 +266,7 @@ tree_attn_kernel(const AttnParams p) {
       uint32_t qf[4];
       {
         const int c = ks * 2 + (lane >> 4);
-        ldsm_x4(q_frag + (c >> 3) * ROWS * 128 + (((c & 7) ^ q_sw) << 4), qf);
+        ldsm_x4(q_frag + (c >> 3) * ROWS * 128 + (((c & 7) ^ sw) << 4), qf);
       }
 #pragma unroll
       for (int np = 0; np < NT / 2; ++np) {
@@ -257,17 +281,26 @@ tree_attn_kernel(const AttnParams p) {
     // scale into the exp2 domain; mask the tile that holds the prefix end / the tree
     const int key0 = t * KT + kbase;
     if (key0 + KC > L) {
-      const int g_lo = row0 + r_lo, g_hi = row0 + r_hi;
-      const unsigned long long mask_lo = g_lo < rows_total ? s_mask[g_lo / p.group] : 0ull;
-      const unsigned long long mask_hi = g_hi < rows_total ? s_mask[g_hi / p.group] : 0ull;
+      // bit j of vis_*: key key0 + j is visible to the row (every prefix key; tree keys by the
+      // ancestor mask, whose bits at and above n are clear, so keys past the last one are hidden)
+      const int rel0 = key0 - L;                       // > -KC
+      unsigned long long vis_lo, vis_hi;
+      if (rel0 >= 0) {
+        vis_lo = rel0 < 64 ? mask_lo >> rel0 : 0ull;
+        vis_hi = rel0 < 64 ? mask_hi >> rel0 : 0ull;
+      } else {
+        const unsigned long long pre = (1ull << -rel0) - 1ull;
+        vis_lo = (mask_lo << -rel0) | pre;
+        vis_hi = (mask_hi << -rel0) | pre;
+      }
+      vis_lo >>= tq * 2;
+      vis_hi >>= tq * 2;
 #pragma unroll
       for (int nt = 0; nt < NT; ++nt) {
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-          const int vj = key0 + nt * 8 + tq * 2 + (e & 1);
-          const unsigned long long mk = (e & 2) ? mask_hi : mask_lo;
-          const bool vis = vj < L || (vj < NK && ((mk >> (vj - L)) & 1ull));
-          s[nt][e] = vis ? s[nt][e] * p.scale_log2 : -INFINITY;
+          const unsigned long long v = (e & 2) ? vis_hi : vis_lo;
+          s[nt][e] = ((v >> (nt * 8 + (e & 1))) & 1ull) ? s[nt][e] * p.scale_log2 : -INFINITY;
         }
       }
     } else {
@@ -278,7 +311,7 @@ tree_attn_kernel(const AttnParams p) {
       }
     }
 
-    // online softmax
+    // online softmax: row maxima over this warp's keys, then over the WN warps of the row group
     float mx_lo = -INFINITY, mx_hi = -INFINITY;
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
@@ -289,6 +322,18 @@ tree_attn_kernel(const AttnParams p) {
     mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 2));
     mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 1));
     mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 2));
+    if (WN > 1) {
+      if (tq == 0) {
+        s_stat[wn][r_lo] = mx_lo;
+        s_stat[wn][r_hi] = mx_hi;
+      }
+      group_sync();
+#pragma unroll
+      for (int w = 0; w < WN; ++w) {
+        mx_lo = fmaxf(mx_lo, s_stat[w][r_lo]);
+        mx_hi = fmaxf(mx_hi, s_stat[w][r_hi]);
+      }
+    }
     const float mn_lo = fmaxf(m_lo, mx_lo), mn_hi = fmaxf(m_hi, mx_hi);
     const float use_lo = mn_lo == -INFINITY ? 0.f : mn_lo, use_hi = mn_hi == -INFINITY ? 0.f : mn_hi;
     const float a_lo = fast_exp2(m_lo - use_lo), a_hi = fast_exp2(m_hi - use_hi);
@@ -308,23 +353,50 @@ tree_attn_kernel(const AttnParams p) {
     l_lo = l_lo * a_lo + sum_lo;
     l_hi = l_hi * a_hi + sum_hi;
 #pragma unroll
-    for (int i = 0; i < DT; ++i) {
+    for (int i = 0; i < OT; ++i) {
       o[i][0] *= a_lo;
       o[i][1] *= a_lo;
       o[i][2] *= a_hi;
       o[i][3] *= a_hi;
     }
 
-    // O += P V
+    if (WN > 1) {
+      // probabilities -> shared memory (rows of 128 bytes, 16-byte chunks XORed with the row)
 #pragma unroll
-    for (int kk = 0; kk < NT / 2; ++kk) {
+      for (int nt = 0; nt < NT; ++nt) {
+        const int c = wn * NT + nt;
+        asm volatile("st.shared.b32 [%0], %1;" ::"r"(p_s + r_lo * 128 + ((c ^ (r_lo & 7)) << 4) + tq * 4),
+                     "r"(pf[nt / 2][(nt & 1) * 2 + 0]) : "memory");
+        asm volatile("st.shared.b32 [%0], %1;" ::"r"(p_s + r_hi * 128 + ((c ^ (r_hi & 7)) << 4) + tq * 4),
+                     "r"(pf[nt / 2][(nt & 1) * 2 + 1]) : "memory");
+      }
+      group_sync();
+      // O[:, this warp's columns] += P[all keys of the tile] V
 #pragma unroll
-      for (int dp = 0; dp < DT / 2; ++dp) {
-        uint32_t vb[4];
-        const int key = kbase + kk * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
-        ldsm_x4_t(vst + tile_off<KT>(key, dp * 2 + (lane >> 4)), vb);
-        mma_bf16(o[2 * dp], pf[kk], vb[0], vb[1]);
-        mma_bf16(o[2 * dp + 1], pf[kk], vb[2], vb[3]);
+      for (int kk = 0; kk < KT / 16; ++kk) {
+        uint32_t pa[4];
+        ldsm_x4(p_frag + (((kk * 2 + (lane >> 4)) ^ sw) << 4), pa);
+#pragma unroll
+        for (int dp = 0; dp < OT / 2; ++dp) {
+          uint32_t vb[4];
+          const int key = kk * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+          ldsm_x4_t(vst + tile_off<KT>(key, wn * OT + dp * 2 + (lane >> 4)), vb);
+          mma_bf16(o[2 * dp], pa, vb[0], vb[1]);
+          mma_bf16(o[2 * dp + 1], pa, vb[2], vb[3]);
+        }
+      }
+    } else {
+      // one warp per row group: the probabilities stay in registers
+#pragma unroll
+      for (int kk = 0; kk < NT / 2; ++kk) {
+#pragma unroll
+        for (int dp = 0; dp < OT / 2; ++dp) {
+          uint32_t vb[4];
+          const int key = kk * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+          ldsm_x4_t(vst + tile_off<KT>(key, dp * 2 + (lane >> 4)), vb);
+          mma_bf16(o[2 * dp], pf[kk], vb[0], vb[1]);
+          mma_bf16(o[2 * dp + 1], pf[kk], vb[2], vb[3]);
+        }
       }
     }
     if (C::FULL_RING) {    // refill this tile's own stage once every warp has finished with it
@@ -337,78 +409,58 @@ tree_attn_kernel(const AttnParams p) {
     }
   }
   cp_async_wait<0>();
-  __syncthreads();            // all warps are done with the stage ring; it is reused below
 
+  // ---- row sums: add up the WN warps' shares ---------------------------------------------
   l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1);
   l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
   l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1);
   l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
-
-  // ---- merge the WN key-slices inside the CTA: warps wn > 0 hand their fragments to wn == 0 ----
-  float4 *xch = reinterpret_cast<float4 *>(smem + C::Q_BYTES);
   if (WN > 1) {
-    if (wn > 0) {
-      float4 *dst = xch + ((size_t)((wn - 1) * WM + wm) * DT) * 32 + lane;
-#pragma unroll
-      for (int i = 0; i < DT; ++i) dst[i * 32] = make_float4(o[i][0], o[i][1], o[i][2], o[i][3]);
-      s_xml[((wn - 1) * WM + wm) * 32 + lane] = make_float4(m_lo, m_hi, l_lo, l_hi);
+    // (every warp of the group has read the last tile's maxima: that was before the tile's second barrier)
+    if (tq == 0) {
+      s_stat[wn][r_lo] = l_lo;
+      s_stat[wn][r_hi] = l_hi;
     }
-    __syncthreads();
-    if (wn == 0) {
+    group_sync();
+    l_lo = l_hi = 0.f;
 #pragma unroll
-      for (int w = 1; w < WN; ++w) {
-        const float4 ml = s_xml[((w - 1) * WM + wm) * 32 + lane];
-        const float mn_lo = fmaxf(m_lo, ml.x), mn_hi = fmaxf(m_hi, ml.y);
-        const float use_lo = mn_lo == -INFINITY ? 0.f : mn_lo, use_hi = mn_hi == -INFINITY ? 0.f : mn_hi;
-        const float a_lo = fast_exp2(m_lo - use_lo), a_hi = fast_exp2(m_hi - use_hi);
-        const float b_lo = fast_exp2(ml.x - use_lo), b_hi = fast_exp2(ml.y - use_hi);
-        m_lo = mn_lo;
-        m_hi = mn_hi;
-        l_lo = l_lo * a_lo + ml.z * b_lo;
-        l_hi = l_hi * a_hi + ml.w * b_hi;
-        const float4 *src = xch + ((size_t)((w - 1) * WM + wm) * DT) * 32 + lane;
-#pragma unroll
-        for (int i = 0; i < DT; ++i) {
-          const float4 v = src[i * 32];
-          o[i][0] = o[i][0] * a_lo + v.x * b_lo;
-          o[i][1] = o[i][1] * a_lo + v.y * b_lo;
-          o[i][2] = o[i][2] * a_hi + v.z * b_hi;
-          o[i][3] = o[i][3] * a_hi + v.w * b_hi;
-        }
-      }
+    for (int w = 0; w < WN; ++w) {
+      l_lo += s_stat[w][r_lo];
+      l_hi += s_stat[w][r_hi];
     }
   }
 
   // ---- merge the key splits of the cluster ------------------------------------------
-  // Every CTA owns ROWS / n_splits rows.  Once all CTAs have left their key loops (first
-  // cluster barrier) each one writes its per-row partial (m, l, O) into the owner's shared
-  // memory; after the second barrier the owner combines its n_splits partials and stores.
+  // Every CTA owns ROWS / n_splits rows.  Each CTA writes its per-row partial (m, l, O) into the
+  // owner's shared memory (once the owner's buffer is free: at once if it is a buffer of its own,
+  // else after every CTA of the cluster has left its key loop); after the next cluster barrier
+  // the owner combines its n_splits partials and stores.
   const int rows_per = ROWS / n_splits;
   float *recv = reinterpret_cast<float *>(smem + C::RECV_OFFSET);
   if (n_splits > 1) {
     if (C::RECV_OWN) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");   // every peer is running
     else cluster.sync();                        // every peer has left its key loop: the rings are free
+  } else if (!C::RECV_OWN) {
+    __syncthreads();                            // all warps are done with the stage ring
   }
-  if (wn == 0) {
 #pragma unroll
-    for (int half = 0; half < 2; ++half) {
-      const int r = half ? r_hi : r_lo;
-      const int owner = r / rows_per, lr = r % rows_per;
-      const int slot = split * rows_per + lr;
-      float *ro = recv + (size_t)slot * D, *rm = r_m + slot, *rl = r_l + slot;
-      if (n_splits > 1) {
-        ro = cluster.map_shared_rank(ro, owner);
-        rm = cluster.map_shared_rank(rm, owner);
-        rl = cluster.map_shared_rank(rl, owner);
-      }
+  for (int half = 0; half < 2; ++half) {
+    const int r = half ? r_hi : r_lo;
+    const int owner = r / rows_per, lr = r % rows_per;
+    const int slot = split * rows_per + lr;
+    float *ro = recv + (size_t)slot * D, *rm = r_m + slot, *rl = r_l + slot;
+    if (n_splits > 1) {
+      ro = cluster.map_shared_rank(ro, owner);
+      rm = cluster.map_shared_rank(rm, owner);
+      rl = cluster.map_shared_rank(rl, owner);
+    }
 #pragma unroll
-      for (int i = 0; i < DT; ++i)     // 8-float groups are XOR-swizzled by the row to spread banks
-        *reinterpret_cast<float2 *>(ro + ((i ^ (lr & 7)) << 3) + tq * 2) =
-            half ? make_float2(o[i][2], o[i][3]) : make_float2(o[i][0], o[i][1]);
-      if (tq == 0) {
-        *rm = half ? m_hi : m_lo;
-        *rl = half ? l_hi : l_lo;
-      }
+    for (int i = 0; i < OT; ++i)     // 8-float groups are XOR-swizzled by the row to spread banks
+      *reinterpret_cast<float2 *>(ro + (((wn * OT + i) ^ (lr & 7)) << 3) + tq * 2) =
+          half ? make_float2(o[i][2], o[i][3]) : make_float2(o[i][0], o[i][1]);
+    if (wn == 0 && tq == 0) {
+      *rm = half ? m_hi : m_lo;
+      *rl = half ? l_hi : l_lo;
     }
   }
   if (n_splits > 1) cluster.sync(); else __syncthreads();
