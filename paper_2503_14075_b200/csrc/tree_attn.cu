@@ -67,7 +67,7 @@ struct AttnCfg {
 template <class C>
 __global__ void __launch_bounds__(C::THREADS, C::MIN_CTAS)
 tree_attn_kernel(const AttnParams p) {
-  constexpr int D = C::D, ROWS = C::ROWS, KT = C::KT, KC = C::KC, WM = C::WM, WN = C::WN, STAGES = C::STAGES;
+  constexpr int D = C::D, ROWS = C::ROWS, KT = C::KT, KC = C::KC, WN = C::WN, STAGES = C::STAGES;
   constexpr int NT = KC / 8;       // key n-tiles of S per warp per tile
   constexpr int OT = C::DW / 8;    // head-dim n-tiles of O per warp
   constexpr int KS = D / 16;       // k-steps of Q K^T
@@ -75,8 +75,9 @@ tree_attn_kernel(const AttnParams p) {
   __shared__ unsigned long long s_mask[TWIG_MAX_NODES];
   __shared__ int s_par[TWIG_MAX_NODES];
   __shared__ float s_stat[WN][ROWS];                            // row maxima of a tile, later row sums
-  __shared__ float r_m[ROWS], r_l[ROWS];                        // received (m, l): [sender][owned row]
+  __shared__ float2 r_ml[ROWS];                                 // received (m, l): [sender][owned row]
   __shared__ int s_bad;
+  __shared__ __align__(8) unsigned long long s_recv_bar;       // counts the bytes peers have pushed to this CTA
 
   cg::cluster_group cluster = cg::this_cluster();
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -109,8 +110,20 @@ tree_attn_kernel(const AttnParams p) {
   }
   const int rows_total = n * p.group, row0 = rb * ROWS;
   if (row0 >= rows_total) return;
-  // with its own receive buffer a CTA only has to be running before peers may write to it
-  if (C::RECV_OWN && n_splits > 1) asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  // Split merge: every CTA owns ROWS / n_splits rows and receives n_splits partials (m, l, O row)
+  // for each of them; its barrier completes when all of those bytes have landed.
+  const int rows_per = ROWS / n_splits;
+  const uint32_t recv_bar = smem_u32(&s_recv_bar);
+  if (n_splits > 1) {
+    if (tid == 0) {
+      mbar_init(recv_bar, 1);
+      mbar_arrive_expect_tx(recv_bar, (uint32_t)(n_splits * rows_per * (D * 4 + 8)));
+      mbar_init_fence_cluster();
+    }
+    __syncthreads();
+    // with its own receive buffer a CTA only has to be running before peers may write to it
+    if (C::RECV_OWN) asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  }
 
   const uint32_t q_s = smem_u32(smem);
   const uint32_t p_s = q_s + C::P_OFFSET;
@@ -431,11 +444,10 @@ tree_attn_kernel(const AttnParams p) {
   }
 
   // ---- merge the key splits of the cluster ------------------------------------------
-  // Every CTA owns ROWS / n_splits rows.  Each CTA writes its per-row partial (m, l, O) into the
-  // owner's shared memory (once the owner's buffer is free: at once if it is a buffer of its own,
-  // else after every CTA of the cluster has left its key loop); after the next cluster barrier
-  // the owner combines its n_splits partials and stores.
-  const int rows_per = ROWS / n_splits;
+  // Each CTA writes its per-row partial (m, l, O) into the owner's shared memory (once the owner's
+  // buffer is free: at once if it is a buffer of its own, else after every CTA of the cluster has
+  // left its key loop) with asynchronous stores that report to the owner's barrier; the owner
+  // waits for its bytes, combines its n_splits partials and stores.
   float *recv = reinterpret_cast<float *>(smem + C::RECV_OFFSET);
   if (n_splits > 1) {
     if (C::RECV_OWN) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");   // every peer is running
@@ -443,27 +455,50 @@ tree_attn_kernel(const AttnParams p) {
   } else if (!C::RECV_OWN) {
     __syncthreads();                            // all warps are done with the stage ring
   }
-#pragma unroll
-  for (int half = 0; half < 2; ++half) {
-    const int r = half ? r_hi : r_lo;
+  {
+    // The two lanes of a quad pair swap halves so that each holds four consecutive floats of one
+    // row: even lanes of the pair keep the low row, odd lanes the high row; 16-byte stores.
+    const bool odd = tq & 1;
+    const int r = odd ? r_hi : r_lo;
     const int owner = r / rows_per, lr = r % rows_per;
     const int slot = split * rows_per + lr;
-    float *ro = recv + (size_t)slot * D, *rm = r_m + slot, *rl = r_l + slot;
-    if (n_splits > 1) {
-      ro = cluster.map_shared_rank(ro, owner);
-      rm = cluster.map_shared_rank(rm, owner);
-      rl = cluster.map_shared_rank(rl, owner);
-    }
+    float *ro = recv + (size_t)slot * D;
+    const uint32_t ro_c = n_splits > 1 ? map_to_cta(smem_u32(ro), owner) : 0u;
+    const uint32_t bar_c = n_splits > 1 ? map_to_cta(recv_bar, owner) : 0u;
 #pragma unroll
-    for (int i = 0; i < OT; ++i)     // 8-float groups are XOR-swizzled by the row to spread banks
-      *reinterpret_cast<float2 *>(ro + (((wn * OT + i) ^ (lr & 7)) << 3) + tq * 2) =
-          half ? make_float2(o[i][2], o[i][3]) : make_float2(o[i][0], o[i][1]);
-    if (wn == 0 && tq == 0) {
-      *rm = half ? m_hi : m_lo;
-      *rl = half ? l_hi : l_lo;
+    for (int i = 0; i < OT; ++i) {
+      const float s0 = odd ? o[i][0] : o[i][2], s1 = odd ? o[i][1] : o[i][3];
+      const float g0 = __shfl_xor_sync(0xffffffffu, s0, 1), g1 = __shfl_xor_sync(0xffffffffu, s1, 1);
+      const float4 v = odd ? make_float4(g0, g1, o[i][2], o[i][3]) : make_float4(o[i][0], o[i][1], g0, g1);
+      // 8-float groups of a row are XOR-swizzled by the row to spread banks
+      const int off = (((wn * OT + i) ^ (lr & 7)) << 3) + (tq >> 1) * 4;
+      if (n_splits > 1) st_async_f32x4(ro_c + off * 4, v, bar_c);
+      else *reinterpret_cast<float4 *>(ro + off) = v;
+    }
+    if (wn == 0 && tq < 2) {
+      const float mm = odd ? m_hi : m_lo, ll = odd ? l_hi : l_lo;
+      if (n_splits > 1) st_async_f32x2(map_to_cta(smem_u32(r_ml + slot), owner), mm, ll, bar_c);
+      else r_ml[slot] = make_float2(mm, ll);
     }
   }
-  if (n_splits > 1) cluster.sync(); else __syncthreads();
+  if (n_splits > 1) {
+    // bounded: a peer that never delivers is reported, not waited for
+    bool landed = mbar_try_wait(recv_bar, 0);
+    if (!landed) {
+      unsigned long long t0, t1;
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
+      do {                                                    // at most 0.2 s
+        landed = mbar_try_wait(recv_bar, 0);
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t1));
+      } while (!landed && t1 - t0 < 200000000ull);
+    }
+    if (!landed) {
+      if (tid == 0) flag_status(p.dev_status, b, TWIG_DEV_INTERNAL);
+      return;
+    }
+  } else {
+    __syncthreads();
+  }
 
   {
     constexpr int TPR = D / 4;                        // threads per row, 4 floats each
@@ -476,7 +511,7 @@ tree_attn_kernel(const AttnParams p) {
       float mstar = -INFINITY;
 #pragma unroll
       for (int sd = 0; sd < 8; ++sd) {
-        mv[sd] = sd < n_splits ? r_m[sd * rows_per + lr] : -INFINITY;
+        mv[sd] = sd < n_splits ? r_ml[sd * rows_per + lr].x : -INFINITY;
         mstar = fmaxf(mstar, mv[sd]);
       }
       float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -486,7 +521,7 @@ tree_attn_kernel(const AttnParams p) {
       for (int sd = 0; sd < 8; ++sd) {
         if (sd < n_splits) {
           const float wgt = fast_exp2(mv[sd] - mstar);
-          lsum = fmaf(wgt, r_l[sd * rows_per + lr], lsum);
+          lsum = fmaf(wgt, r_ml[sd * rows_per + lr].y, lsum);
           const float4 v = *reinterpret_cast<const float4 *>(recv + (size_t)(sd * rows_per + lr) * D + col);
           acc.x = fmaf(wgt, v.x, acc.x);
           acc.y = fmaf(wgt, v.y, acc.y);
