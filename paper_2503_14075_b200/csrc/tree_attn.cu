@@ -116,8 +116,9 @@ tree_attn_kernel(const AttnParams p) {
   const uint32_t recv_bar = smem_u32(&s_recv_bar);
   if (n_splits > 1) {
     if (tid == 0) {
-      mbar_init(recv_bar, 1);
-      mbar_arrive_expect_tx(recv_bar, (uint32_t)(n_splits * rows_per * (D * 4 + 8)));
+      // one arrival that announces the peers' bytes, one per warp for this CTA's own share
+      mbar_init(recv_bar, 1 + C::THREADS / 32);
+      mbar_arrive_expect_tx(recv_bar, (uint32_t)((n_splits - 1) * rows_per * (D * 4 + 8)));
       mbar_init_fence_cluster();
     }
     __syncthreads();
@@ -463,8 +464,9 @@ tree_attn_kernel(const AttnParams p) {
     const int owner = r / rows_per, lr = r % rows_per;
     const int slot = split * rows_per + lr;
     float *ro = recv + (size_t)slot * D;
-    const uint32_t ro_c = n_splits > 1 ? map_to_cta(smem_u32(ro), owner) : 0u;
-    const uint32_t bar_c = n_splits > 1 ? map_to_cta(recv_bar, owner) : 0u;
+    const bool remote = owner != split;           // (n_splits == 1: never)
+    const uint32_t ro_c = remote ? map_to_cta(smem_u32(ro), owner) : 0u;
+    const uint32_t bar_c = remote ? map_to_cta(recv_bar, owner) : 0u;
 #pragma unroll
     for (int i = 0; i < OT; ++i) {
       const float s0 = odd ? o[i][0] : o[i][2], s1 = odd ? o[i][1] : o[i][3];
@@ -472,16 +474,18 @@ tree_attn_kernel(const AttnParams p) {
       const float4 v = odd ? make_float4(g0, g1, o[i][2], o[i][3]) : make_float4(o[i][0], o[i][1], g0, g1);
       // 8-float groups of a row are XOR-swizzled by the row to spread banks
       const int off = (((wn * OT + i) ^ (lr & 7)) << 3) + (tq >> 1) * 4;
-      if (n_splits > 1) st_async_f32x4(ro_c + off * 4, v, bar_c);
+      if (remote) st_async_f32x4(ro_c + off * 4, v, bar_c);
       else *reinterpret_cast<float4 *>(ro + off) = v;
     }
     if (wn == 0 && tq < 2) {
       const float mm = odd ? m_hi : m_lo, ll = odd ? l_hi : l_lo;
-      if (n_splits > 1) st_async_f32x2(map_to_cta(smem_u32(r_ml + slot), owner), mm, ll, bar_c);
+      if (remote) st_async_f32x2(map_to_cta(smem_u32(r_ml + slot), owner), mm, ll, bar_c);
       else r_ml[slot] = make_float2(mm, ll);
     }
   }
   if (n_splits > 1) {
+    __syncwarp();                     // the lanes' own-share stores come before lane 0's arrival
+    if (lane == 0) mbar_arrive(recv_bar);
     // bounded: a peer that never delivers is reported, not waited for
     bool landed = mbar_try_wait(recv_bar, 0);
     if (!landed) {
