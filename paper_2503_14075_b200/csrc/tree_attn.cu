@@ -39,7 +39,7 @@ struct AttnCfg {
   static constexpr int P_BYTES = WN > 1 ? ROWS * KT * 2 : 0;   // bf16 probabilities of one tile
   static constexpr int TILE_BYTES = KT * D * 2;
   static constexpr int STAGE_BYTES = 2 * STAGES * TILE_BYTES;
-  static constexpr int RECV_BYTES = ROWS * D * 4;              // the per-split partials a CTA owns
+  static constexpr int RECV_BYTES = ROWS * D * 2;              // the per-split partials a CTA owns (fp16)
   static_assert(KT == 64, "a row of P is one 128-byte swizzled line");
   static_assert(DW % 16 == 0 && KC % 16 == 0, "warp slices are whole ldmatrix.x4 steps");
   // The small, latency-bound variants (one CTA per SM is enough for them) keep the split-merge
@@ -118,7 +118,7 @@ tree_attn_kernel(const AttnParams p) {
     if (tid == 0) {
       // one arrival that announces the peers' bytes, one per warp for this CTA's own share
       mbar_init(recv_bar, 1 + C::THREADS / 32);
-      mbar_arrive_expect_tx(recv_bar, (uint32_t)((n_splits - 1) * rows_per * (D * 4 + 8)));
+      mbar_arrive_expect_tx(recv_bar, (uint32_t)((n_splits - 1) * rows_per * (D * 2 + 8)));
       mbar_init_fence_cluster();
     }
     __syncthreads();
@@ -445,11 +445,12 @@ tree_attn_kernel(const AttnParams p) {
   }
 
   // ---- merge the key splits of the cluster ------------------------------------------
-  // Each CTA writes its per-row partial (m, l, O) into the owner's shared memory (once the owner's
+  // Each CTA writes its per-row partial (m, l, O / l as fp16: |O / l| is bounded by the largest
+  // |V| entry, and fp16 rounds eight times finer than the bf16 output) into the owner's shared memory (once the owner's
   // buffer is free: at once if it is a buffer of its own, else after every CTA of the cluster has
   // left its key loop) with asynchronous stores that report to the owner's barrier; the owner
   // waits for its bytes, combines its n_splits partials and stores.
-  float *recv = reinterpret_cast<float *>(smem + C::RECV_OFFSET);
+  unsigned char *recv = smem + C::RECV_OFFSET;                 // [slot][D] fp16
   if (n_splits > 1) {
     if (C::RECV_OWN) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");   // every peer is running
     else cluster.sync();                        // every peer has left its key loop: the rings are free
@@ -463,7 +464,9 @@ tree_attn_kernel(const AttnParams p) {
     const int r = odd ? r_hi : r_lo;
     const int owner = r / rows_per, lr = r % rows_per;
     const int slot = split * rows_per + lr;
-    float *ro = recv + (size_t)slot * D;
+    unsigned char *ro = recv + (size_t)slot * D * 2;
+    const float my_l = odd ? l_hi : l_lo;
+    const float inv_l = my_l > 0.f ? 1.f / my_l : 0.f;
     const bool remote = owner != split;           // (n_splits == 1: never)
     const uint32_t ro_c = remote ? map_to_cta(smem_u32(ro), owner) : 0u;
     const uint32_t bar_c = remote ? map_to_cta(recv_bar, owner) : 0u;
@@ -472,10 +475,11 @@ tree_attn_kernel(const AttnParams p) {
       const float s0 = odd ? o[i][0] : o[i][2], s1 = odd ? o[i][1] : o[i][3];
       const float g0 = __shfl_xor_sync(0xffffffffu, s0, 1), g1 = __shfl_xor_sync(0xffffffffu, s1, 1);
       const float4 v = odd ? make_float4(g0, g1, o[i][2], o[i][3]) : make_float4(o[i][0], o[i][1], g0, g1);
-      // 8-float groups of a row are XOR-swizzled by the row to spread banks
-      const int off = (((wn * OT + i) ^ (lr & 7)) << 3) + (tq >> 1) * 4;
-      if (remote) st_async_f32x4(ro_c + off * 4, v, bar_c);
-      else *reinterpret_cast<float4 *>(ro + off) = v;
+      const uint32_t h0 = pack_f16(v.x * inv_l, v.y * inv_l), h1 = pack_f16(v.z * inv_l, v.w * inv_l);
+      // 8-column groups of a row are XOR-swizzled by the row to spread banks
+      const int off = ((((wn * OT + i) ^ (lr & 7)) << 3) + (tq >> 1) * 4) * 2;
+      if (remote) st_async_b32x2(ro_c + off, h0, h1, bar_c);
+      else *reinterpret_cast<uint2 *>(ro + off) = make_uint2(h0, h1);
     }
     if (wn == 0 && tq < 2) {
       const float mm = odd ? m_hi : m_lo, ll = odd ? l_hi : l_lo;
@@ -524,13 +528,14 @@ tree_attn_kernel(const AttnParams p) {
 #pragma unroll
       for (int sd = 0; sd < 8; ++sd) {
         if (sd < n_splits) {
-          const float wgt = fast_exp2(mv[sd] - mstar);
-          lsum = fmaf(wgt, r_ml[sd * rows_per + lr].y, lsum);
-          const float4 v = *reinterpret_cast<const float4 *>(recv + (size_t)(sd * rows_per + lr) * D + col);
-          acc.x = fmaf(wgt, v.x, acc.x);
-          acc.y = fmaf(wgt, v.y, acc.y);
-          acc.z = fmaf(wgt, v.z, acc.z);
-          acc.w = fmaf(wgt, v.w, acc.w);
+          const float wgt = fast_exp2(mv[sd] - mstar) * r_ml[sd * rows_per + lr].y;
+          lsum += wgt;
+          const uint2 raw = *reinterpret_cast<const uint2 *>(recv + ((size_t)(sd * rows_per + lr) * D + col) * 2);
+          const float2 v01 = unpack_f16(raw.x), v23 = unpack_f16(raw.y);
+          acc.x = fmaf(wgt, v01.x, acc.x);
+          acc.y = fmaf(wgt, v01.y, acc.y);
+          acc.z = fmaf(wgt, v23.x, acc.z);
+          acc.w = fmaf(wgt, v23.y, acc.w);
         }
       }
       const float inv = 1.f / lsum;
