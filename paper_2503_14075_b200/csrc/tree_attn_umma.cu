@@ -155,10 +155,11 @@ struct UmmaCfg {
   static constexpr int Q_BYTES = ROWS * kD * 2;          // two 64-column panels of ROWS x 128 B
   static constexpr int P_ONE = ROWS * KT * 2;            // ROWS x KT keys bf16, KT/64 panels of ROWS x 128 B
   // two P buffers where shared memory allows: the softmax of tile t+1 then never waits for P(t) V(t)
-  static constexpr int P_BUFS = (KT == 128 || (KT == 64 && ROWS <= 32)) ? 2 : 1;
+  static constexpr int P_BUFS = 2;
   static constexpr int P_BYTES = P_BUFS * P_ONE;
-  // 128 rows with 128-key tiles: four slots, so that two P buffers still fit in shared memory
-  static constexpr int SLOTS = (ROWS == 128 && KT == 128) ? 4 : kMaxSlots;
+  // four slots where five would not leave room for the second P buffer (128 rows with 128-key
+  // tiles in one CTA; 64 rows with 64-key tiles in two CTAs per SM)
+  static constexpr int SLOTS = ((ROWS == 128 && KT == 128) || (ROWS == 64 && KT == 64)) ? 4 : kMaxSlots;
   static constexpr int RING_BYTES = SLOTS * TILE_BYTES;
   static constexpr uint32_t TMEM_COLS = KT == 64 ? 256 : 512;   // S: [0,KT) and [KT,2KT); O: [2KT, 2KT+128)
   static constexpr uint32_t O_COL = 2 * KT;
@@ -192,23 +193,6 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
   const int hk = blockIdx.y / p.row_blocks, rb = blockIdx.y % p.row_blocks;
   const int b = blockIdx.z;
 
-  grid_dependency_sync();
-  // ---- per-request metadata; every exit below is uniform over the cluster ----
-  const int n = p.n_nodes[b], L = p.kv_len[b];
-  const int my_parent = tid < p.t_max ? p.parent[(long long)b * p.t_max + tid] : -1;
-  if (n == 0) return;
-  const bool first = split == 0 && blockIdx.y == 0 && tid == 0;
-  if (n < 0 || n > p.t_max) {
-    if (first) flag_status(p.dev_status, b, TWIG_DEV_BAD_TREE);
-    return;
-  }
-  if (L < 0 || L > p.max_len) {
-    if (first) flag_status(p.dev_status, b, TWIG_DEV_OVERFLOW);
-    return;
-  }
-  const int rows_total = n * p.group, row0 = rb * ROWS;
-  if (row0 >= rows_total) return;
-
   const uint32_t q_s = smem_u32(smem);
   const uint32_t p_s = q_s + C::Q_BYTES;
   const uint32_t ring_s = p_s + C::P_BYTES;
@@ -221,6 +205,51 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
   const uint32_t bar_q = bars + 8 * (2 * kMaxSlots + 6);
   constexpr int PB = C::P_BUFS;
 
+  // ---- what needs nothing from global memory comes first, while the preceding kernel of the
+  // stream may still be draining: barriers (all but the one whose count depends on the request)
+  // and tensor memory ----
+  if (tid == 0) {
+    s_bad = 0;
+    s_fail = 0;
+    for (int i = 0; i < kSlots; ++i) {
+      mbar_init(bar_full(i), 32);       // every loader lane arrives once per unit
+      mbar_init(bar_empty(i), 1);       // one tcgen05.commit
+    }
+    mbar_init(bar_s(0), 1);
+    mbar_init(bar_s(1), 1);
+    mbar_init(bar_o(0), 1);
+    mbar_init(bar_o(1), 1);
+    mbar_init(bar_q, 32);
+  }
+  if (warp == 5) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem)), "r"(C::TMEM_COLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  if (warp == 4 && lane == 0) {         // the two tensor maps (kernel parameters) into the descriptor cache
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&kmap)) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&vmap)) : "memory");
+  }
+  // every exit before the key loop hands the tensor memory back
+  auto leave = [&]() {
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (warp == 5) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(s_tmem), "r"(C::TMEM_COLS) : "memory");
+  };
+
+  grid_dependency_sync();
+  // ---- per-request metadata; every exit below is uniform over the cluster ----
+  const int n = p.n_nodes[b], L = p.kv_len[b];
+  const int my_parent = tid < p.t_max ? p.parent[(long long)b * p.t_max + tid] : -1;
+  const bool first = split == 0 && blockIdx.y == 0 && tid == 0;
+  const int rows_total = n * p.group, row0 = rb * ROWS;
+  if (n <= 0 || n > p.t_max || L < 0 || L > p.max_len || row0 >= rows_total) {
+    if (first && (n < 0 || n > p.t_max)) flag_status(p.dev_status, b, TWIG_DEV_BAD_TREE);
+    else if (first && n > 0 && (L < 0 || L > p.max_len)) flag_status(p.dev_status, b, TWIG_DEV_OVERFLOW);
+    leave();
+    return;
+  }
+
   const int NK = L + n;
   const int n_tiles = (NK + KT - 1) / KT;
   const int per = (n_tiles + n_splits - 1) / n_splits;
@@ -231,11 +260,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
   constexpr int RPW = C::ROWS_PER_WARP;
   const int n_soft = min((ROWS + RPW - 1) / RPW, (rows_total - row0 + RPW - 1) / RPW);
 
-  // ---- parents, validation, ancestor masks; barriers; tensor memory ---------------
-  if (tid == 0) {
-    s_bad = 0;
-    s_fail = 0;
-  }
+  // ---- parents, validation, ancestor masks ---------------
   __syncthreads();
   if (tid < n) {
     s_par[tid] = my_parent;
@@ -244,6 +269,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
   __syncthreads();
   if (s_bad) {
     if (first) flag_status(p.dev_status, b, TWIG_DEV_BAD_TREE);
+    leave();
     return;
   }
   if (tid < n) {
@@ -256,22 +282,8 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
     s_mask[tid] = m;
   }
   if (tid == 0) {
-    for (int i = 0; i < kSlots; ++i) {
-      mbar_init(bar_full(i), 32);       // every loader lane arrives once per unit
-      mbar_init(bar_empty(i), 1);       // one tcgen05.commit
-    }
-    mbar_init(bar_s(0), 1);
-    mbar_init(bar_s(1), 1);
-    for (int i = 0; i < 2; ++i) {
-      mbar_init(bar_p(i), n_soft);      // one arrival per softmax warp
-      mbar_init(bar_o(i), 1);
-    }
-    mbar_init(bar_q, 32);
+    for (int i = 0; i < 2; ++i) mbar_init(bar_p(i), n_soft);      // one arrival per softmax warp
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
-  if (warp == 5) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem)), "r"(C::TMEM_COLS) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   tc_fence_before();
   __syncthreads();
@@ -296,19 +308,27 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
     const __nv_bfloat16 *tv = p.tree_v + ((long long)b * p.n_kv_heads + hk) * p.t_max * kD;
     const int c = lane & 15, rbase = lane >> 4;      // chunk c of rows rbase, rbase + 2, ...
     const uint32_t panel = (uint32_t)((c >> 3) * kPanelBytes);
-    // Q tile (zero rows past the request's last row): part of the first commit group
-    for (int r = rbase; r < ROWS && n_my > 0; r += 2) {
-      const int grow = row0 + r;
-      const bool valid = grow < rows_total;
-      const int node = valid ? grow / p.group : 0, g = valid ? grow % p.group : 0;
-      const __nv_bfloat16 *src =
-          p.q + (((long long)b * p.t_max + node) * p.n_q_heads + hk * p.group + g) * kD + c * 8;
-      cp_async_16(q_s + (c >> 3) * ROWS * 128 + r * 128 + (((c & 7) ^ (r & 7)) << 4), src, valid);
-    }
-    cp_async_commit();
-    bool q_published = false;
+    // Q tile (zero rows past the request's last row).  Lane pairs walk the rows two apart; the
+    // (node, query head of the group) pair of a row is stepped, not divided.
+    bool q_issued = false, q_published = false;
+    auto issue_q = [&]() {
+      int node = (row0 + rbase) / p.group, g = (row0 + rbase) % p.group;
+      for (int r = rbase; r < ROWS; r += 2) {
+        const bool valid = row0 + r < rows_total;
+        const __nv_bfloat16 *src =
+            p.q + (((long long)b * p.t_max + (valid ? node : 0)) * p.n_q_heads + hk * p.group + (valid ? g : 0)) * kD + c * 8;
+        cp_async_16(q_s + (c >> 3) * ROWS * 128 + r * 128 + (((c & 7) ^ (r & 7)) << 4), src, valid);
+        g += 2;
+        while (g >= p.group) {
+          g -= p.group;
+          ++node;
+        }
+      }
+      cp_async_commit();
+      q_issued = true;
+    };
     auto publish_q = [&]() {                    // Q has landed: publish it once
-      if (!q_published) {
+      if (q_issued && !q_published) {
         cp_async_wait<0>();
         fence_async_smem();
         mbar_arrive(bar_q);
@@ -317,13 +337,8 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
     };
     const int n_units = 2 * n_my;
     bool ok = true;
-    for (int u = 0; u < n_units && ok; ++u) {
-      const int slot = u % kSlots, round = u / kSlots;
-      if (round > 0) {
-        publish_q();                            // (all ring slots are in flight by now)
-        ok = mbar_wait(bar_empty(slot), (round - 1) & 1, fail);
-      }
-      if (!ok) break;
+    auto issue_unit = [&](int u) {
+      const int slot = u % kSlots;
       const int t = t_begin + (u >> 1);
       const uint32_t dst = ring_s + slot * kTileBytes;
       if (t * KT + KT <= L) {                   // whole tile inside the cached prefix: two TMA boxes
@@ -353,14 +368,24 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
           cp_async_16(dst + panel + r * 128 + (((c & 7) ^ (r & 7)) << 4), src, valid);
         }
         cp_async_commit();
-        cp_async_wait<0>();                     // (this also completes the Q copies)
+        cp_async_wait<0>();                     // (this also completes the Q copies, if they were issued)
         fence_async_smem();
-        if (!q_published) {
+        if (q_issued && !q_published) {
           mbar_arrive(bar_q);
           q_published = true;
         }
         mbar_arrive(bar_full(slot));
       }
+    };
+    // the first ring of tiles is requested before Q: they are the long pole
+    const int n_first = min(n_units, kSlots);
+    for (int u = 0; u < n_first; ++u) issue_unit(u);
+    if (n_my > 0) issue_q();
+    for (int u = n_first; u < n_units && ok; ++u) {
+      publish_q();                              // (all ring slots are in flight by now)
+      ok = mbar_wait(bar_empty(u % kSlots), (u / kSlots - 1) & 1, fail);
+      if (!ok) break;
+      issue_unit(u);
     }
     publish_q();
     if (!ok) s_fail = 1;
