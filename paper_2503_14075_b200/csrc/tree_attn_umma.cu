@@ -120,6 +120,16 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
       : TWIG_R8(v, 0), TWIG_R8(v, 8), TWIG_R8(v, 16), TWIG_R8(v, 24)
       : "r"(taddr));
 }
+// 64 consecutive fp32 columns of 16 lanes (the 16 lanes from the address's lane on), spread over
+// the warp like an mma.sync accumulator: for every 8-column group g, lane t holds columns
+// 8g + 2(t % 4) + {0, 1} of row t / 4 in v[4g], v[4g+1] and of row t / 4 + 8 in v[4g+2], v[4g+3].
+__device__ __forceinline__ void tmem_ld_16rows_64cols(uint32_t taddr, uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.16x256b.x8.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : TWIG_R8(v, 0), TWIG_R8(v, 8), TWIG_R8(v, 16), TWIG_R8(v, 24)
+      : "r"(taddr));
+}
 #undef TWIG_R8
 #define TWIG_S8(a, o) "r"(a[o]), "r"(a[o + 1]), "r"(a[o + 2]), "r"(a[o + 3]), "r"(a[o + 4]), "r"(a[o + 5]), "r"(a[o + 6]), "r"(a[o + 7])
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32]) {
@@ -435,8 +445,154 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
       }
       if (!ok) s_fail = 1;
     }
+  } else if (warp < n_soft && C::MMA_M == 64) {
+    // ================= softmax, 64-row accumulators =================
+    // Such an accumulator keeps only 16 rows in a warp's 32 tensor-memory lanes; read one row per
+    // lane, half of every warp would idle.  The 16-lane load shape spreads the 16 rows over all 32
+    // lanes instead (lane t: rows t/4 and t/4 + 8, two adjacent columns of every 8-column group),
+    // so a quad shares a row: maxima and sums take two shuffles, every lane does half the work.
+    const int gq = lane >> 2, tq = lane & 3;
+    const int r_lo = 16 * warp + gq, r_hi = r_lo + 8;
+    const int g_lo = row0 + r_lo, g_hi = row0 + r_hi;
+    const unsigned long long mask_lo = g_lo < rows_total ? s_mask[g_lo / p.group] : 0ull;
+    const unsigned long long mask_hi = g_hi < rows_total ? s_mask[g_hi / p.group] : 0ull;
+    float m_lo = -INFINITY, m_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;     // l: this lane's columns only
+    const int row_src = 4 * (lane & 7);          // a lane that holds row (lane & 15) of this warp
+    constexpr int NH = KT / 64;
+    bool ok = true;
+    for (int it = 0; it < n_my; ++it) {
+      const int t = t_begin + it;
+      ok = mbar_wait(bar_s(it & 1), (it >> 1) & 1, fail);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t ts = t_lane + (it & 1) * KT;
+      uint32_t sr[NH][32];
+#pragma unroll
+      for (int h = 0; h < NH; ++h) tmem_ld_16rows_64cols(ts + h * 64, sr[h]);
+      tmem_ld_wait();
+      // the keys that hold the prefix end and / or the tree are masked
+#pragma unroll
+      for (int h = 0; h < NH; ++h) {
+        const int key0 = t * KT + h * 64;
+        if (key0 + 64 > L) {
+          // bit j of vis_*: key key0 + j is visible to the row (every prefix key; tree keys by the
+          // ancestor mask, whose bits at and above n are clear)
+          const int rel0 = key0 - L;               // > -64
+          unsigned long long vis_lo, vis_hi;
+          if (rel0 >= 0) {
+            vis_lo = rel0 < 64 ? mask_lo >> rel0 : 0ull;
+            vis_hi = rel0 < 64 ? mask_hi >> rel0 : 0ull;
+          } else {
+            const unsigned long long pre = (1ull << -rel0) - 1ull;
+            vis_lo = (mask_lo << -rel0) | pre;
+            vis_hi = (mask_hi << -rel0) | pre;
+          }
+          vis_lo >>= tq * 2;
+          vis_hi >>= tq * 2;
+#pragma unroll
+          for (int g = 0; g < 8; ++g)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const unsigned long long v = (e & 2) ? vis_hi : vis_lo;
+              if (!((v >> (g * 8 + (e & 1))) & 1ull)) sr[h][4 * g + e] = 0xff800000u;     // -inf
+            }
+        }
+      }
+      float mx_lo = -INFINITY, mx_hi = -INFINITY;
+#pragma unroll
+      for (int h = 0; h < NH; ++h)
+#pragma unroll
+        for (int g = 0; g < 8; ++g) {
+          mx_lo = fmaxf(mx_lo, fmaxf(__uint_as_float(sr[h][4 * g]), __uint_as_float(sr[h][4 * g + 1])));
+          mx_hi = fmaxf(mx_hi, fmaxf(__uint_as_float(sr[h][4 * g + 2]), __uint_as_float(sr[h][4 * g + 3])));
+        }
+      mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 1));
+      mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 2));
+      mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 1));
+      mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 2));
+      mx_lo *= p.scale_log2;                      // scale > 0, so the max commutes with it
+      mx_hi *= p.scale_log2;
+      const bool raise_lo = mx_lo > m_lo + kLazyMax, raise_hi = mx_hi > m_hi + kLazyMax;   // also the first finite maximum
+      const float mn_lo = raise_lo ? mx_lo : m_lo, mn_hi = raise_hi ? mx_hi : m_hi;
+      const float use_lo = mn_lo == -INFINITY ? 0.f : mn_lo, use_hi = mn_hi == -INFINITY ? 0.f : mn_hi;
+      const int pb = it % PB;
+      if (it >= PB) {                             // this P buffer is free once P(it-PB) V(it-PB) is done
+        ok = mbar_wait(bar_o(pb), (it / PB - 1) & 1, fail);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after();
+      }
+      if (it > 0 && __any_sync(0xffffffffu, raise_lo || raise_hi)) {
+        if (PB > 1) {                             // O must be stable: wait for P(it-1) V(it-1) as well
+          ok = mbar_wait(bar_o((it - 1) % PB), ((it - 1) / PB) & 1, fail);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          tc_fence_after();
+        }
+        const float a_lo = fast_exp2(m_lo - use_lo), a_hi = fast_exp2(m_hi - use_hi);   // 1 for rows that keep their maximum
+        l_lo *= a_lo;
+        l_hi *= a_hi;
+        // O is read one row per lane (lanes 0-15 of the warp): fetch that row's factor from its quad
+        const float al = __shfl_sync(0xffffffffu, a_lo, row_src), ah = __shfl_sync(0xffffffffu, a_hi, row_src);
+        const float alpha = lane >= 16 ? 1.f : ((lane & 8) ? ah : al);
+#pragma unroll
+        for (int ch = 0; ch < 4; ++ch) {
+          uint32_t v[32];
+          tmem_ld32(t_lane + C::O_COL + ch * 32, v);
+          tmem_ld_wait();
+#pragma unroll
+          for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) * alpha);
+          tmem_st32(t_lane + C::O_COL + ch * 32, v);
+        }
+        tmem_st_wait();
+      }
+      m_lo = mn_lo;
+      m_hi = mn_hi;
+      // P = exp2(S * scale - m) as bf16 to shared memory (rows of 128 bytes per 64 keys, 16-byte
+      // chunks XORed with the row), row sums
+      float sum_lo = 0.f, sum_hi = 0.f;
+#pragma unroll
+      for (int h = 0; h < NH; ++h) {
+        const uint32_t pl = p_s + pb * C::P_ONE + h * ROWS * 128 + r_lo * 128 + tq * 4;
+        const uint32_t ph = p_s + pb * C::P_ONE + h * ROWS * 128 + r_hi * 128 + tq * 4;
+#pragma unroll
+        for (int g = 0; g < 8; ++g) {
+          const float p0 = fast_exp2(fmaf(__uint_as_float(sr[h][4 * g]), p.scale_log2, -use_lo));
+          const float p1 = poly_exp2(fmaf(__uint_as_float(sr[h][4 * g + 1]), p.scale_log2, -use_lo));
+          const float p2 = fast_exp2(fmaf(__uint_as_float(sr[h][4 * g + 2]), p.scale_log2, -use_hi));
+          const float p3 = poly_exp2(fmaf(__uint_as_float(sr[h][4 * g + 3]), p.scale_log2, -use_hi));
+          sum_lo += p0 + p1;
+          sum_hi += p2 + p3;
+          asm volatile("st.shared.b32 [%0], %1;" ::"r"(pl + ((g ^ (r_lo & 7)) << 4)), "r"(pack_bf16(p0, p1)) : "memory");
+          asm volatile("st.shared.b32 [%0], %1;" ::"r"(ph + ((g ^ (r_hi & 7)) << 4)), "r"(pack_bf16(p2, p3)) : "memory");
+        }
+      }
+      l_lo += sum_lo;
+      l_hi += sum_hi;
+      fence_async_smem();            // P was written with ordinary stores
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_p(pb));
+    }
+    if (ok && n_my > 0) {
+      ok = mbar_wait(bar_o((n_my - 1) % PB), ((n_my - 1) / PB) & 1, fail);   // the last P V product has completed
+      tc_fence_after();
+    }
+    // hand the rows' state to the one-row-per-lane layout of the epilogue (lanes 0-15)
+    l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1);
+    l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
+    l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1);
+    l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
+    {
+      const float ml = __shfl_sync(0xffffffffu, m_lo, row_src), mh = __shfl_sync(0xffffffffu, m_hi, row_src);
+      const float ll = __shfl_sync(0xffffffffu, l_lo, row_src), lh = __shfl_sync(0xffffffffu, l_hi, row_src);
+      m_run = (lane & 8) ? mh : ml;
+      l_run = (lane & 8) ? lh : ll;
+    }
+    if (!ok) s_fail = 1;
   } else if (warp < n_soft) {
-    // ================= softmax: thread r owns row r =================
+    // ================= softmax, 128-row accumulators: thread r owns row r =================
     const unsigned long long my_mask = row_valid ? s_mask[gr / p.group] : 0ull;
     bool ok = true;
     for (int it = 0; it < n_my; ++it) {
