@@ -126,7 +126,7 @@ tree_accept_compact_kernel(const int *__restrict__ parent, const int *__restrict
 
 // ---------------------------------------------------------------------------
 // Greedy target token per tree node: argmax over the vocabulary, lowest index on ties.
-// One CTA per (request, node) row; 16-byte loads, 4 in flight per thread.
+// One CTA per (request, node) row; 16-byte loads, 8 in flight per thread.
 // ---------------------------------------------------------------------------
 constexpr int kArgmaxThreads = 256;
 
@@ -176,12 +176,13 @@ base_argmax_kernel(const void *__restrict__ logits, long long row_stride, int vo
     }
   };
   int c = tid;
-  for (; c + 3 * kArgmaxThreads < chunks; c += 4 * kArgmaxThreads) {
-    uint4 w[4];
+  constexpr int kDeep = 8;                          // 16-byte loads in flight per thread
+  for (; c + (kDeep - 1) * kArgmaxThreads < chunks; c += kDeep * kArgmaxThreads) {
+    uint4 w[kDeep];
 #pragma unroll
-    for (int u = 0; u < 4; ++u) w[u] = ld_nc_16(row + (long long)(c + u * kArgmaxThreads) * 16);
+    for (int u = 0; u < kDeep; ++u) w[u] = ld_nc_16(row + (long long)(c + u * kArgmaxThreads) * 16);
 #pragma unroll
-    for (int u = 0; u < 4; ++u) take_chunk(w[u], c + u * kArgmaxThreads);
+    for (int u = 0; u < kDeep; ++u) take_chunk(w[u], c + u * kArgmaxThreads);
   }
   for (; c < chunks; c += kArgmaxThreads) take_chunk(ld_nc_16(row + (long long)c * 16), c);
   for (int i = chunks * EPC + tid; i < vocab; i += kArgmaxThreads) {     // tail that is no whole chunk
