@@ -546,6 +546,25 @@ def extra_rooflines(torch, tw, peaks, dev):
                                    "frac": round(by / us / 1e3 / peaks["hbm_gbs"], 4),
                                    "l2": f"chain of {n_chain} launches over {n_sets} rotating 394 MB source sets"}
     del sets
+    # P-Head score with its gates applied in the kernel (Eq. 7) on the high-resolution prompts: K and the
+    # key gates are each read once (2 x 98.6 MB, larger than L2 together), logits go through the scratch
+    pre4 = synth.make_prefill(wl, rng, n_layers=1)
+    q4, k4 = bf(pre4["twig_q"]), bf(pre4["twig_k"])
+    qg4, kg4 = bf(synth.gate_bf16(rng, pre4["twig_q"].shape)), bf(synth.gate_bf16(rng, pre4["twig_k"].shape))
+    sc4 = torch.zeros((B, max(wl.n_vis)), dtype=torch.float32, device=dev)
+    ws4 = torch.empty(tw.twig_workspace_bytes(B, Hq, d, k4.shape[2], T), dtype=torch.uint8, device=dev)
+    m4 = (i32(pre4["prefix_len"]), i32(pre4["vis_start"]), i32(pre4["n_vis"]))
+    for _ in range(3):
+        tw.ttp_score_gated(q4, qg4, k4, kg4, *m4, sc4, ws4)
+    e0.record(stream)
+    for _ in range(n_chain):
+        tw.ttp_score_gated(q4, qg4, k4, kg4, *m4, sc4, ws4)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    us = e0.elapsed_time(e1) * 1e3 / n_chain
+    res["ttp_score_gated_c4"] = hbm_entry(us, int(2 * sum(Hkv * n * d * 2 for n in wl.n_vis)))
+    res["ttp_score_gated_c4"]["launches"] = "logits + softmax/mean (2 kernels)"
+    del pre4, q4, k4, qg4, kg4
     # greedy target token per tree node over the heterogeneous batch's trees (32000-entry bf16 rows);
     # six logits buffers in turn, 190 MB together, so that every read is cold
     V = 32000

@@ -103,6 +103,23 @@ twig_status ttp_score(const void *twig_q, const void *twig_k, int64_t k_stride_b
                       int32_t norm_scope, float softmax_scale, float *scores, int32_t m_max,
                       int32_t *dev_status, void *ws, size_t ws_bytes, void *stream);
 
+/* ---- P-Head score with its gates applied in the kernel ----------------------
+ * Eq. 7: s = (1/H) sum_h softmax( (G_q(x_q)^(h) * q^(h)) . (G_k(X_k)^(h) * K^(h))^T / sqrt(d_h) ), the
+ * products element-wise.  ttp_score on q_gate * twig_q and k_gate * twig_k, the products formed in
+ * fp32 inside the kernel (the gated tensors are never written).  The gates themselves (a linear
+ * layer and an activation each) are inputs.
+ *   q_gate  [batch, n_q_heads, head_dim] bf16, like twig_q
+ *   k_gate  bf16, same strides and extent as twig_k (entry (b, h_kv, j, c) gates K's entry there)
+ * Everything else as in ttp_score; Eq. 7 normalises over the visual span: norm_scope = 1.
+ */
+twig_status ttp_score_gated(const void *twig_q, const void *q_gate, const void *twig_k,
+                            const void *k_gate, int64_t k_stride_batch, int64_t k_stride_head,
+                            int64_t k_stride_pos, int32_t k_max_len, const int32_t *prefix_len,
+                            const int32_t *vis_start, const int32_t *n_vis, int32_t batch,
+                            int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim,
+                            int32_t norm_scope, float softmax_scale, float *scores, int32_t m_max,
+                            int32_t *dev_status, void *ws, size_t ws_bytes, void *stream);
+
 /* ---- ttp_score without any caller-provided or allocated scratch --------------
  * (No counterpart in the paper: this is a deployment convenience.)
  * Some hosts of this library may not allocate device memory at the point where

@@ -76,6 +76,34 @@ def ttp_scores(q, k, prefix_len, vis_start, n_vis, norm_scope=0, scale=None):
     return s
 
 
+def ttp_scores_gated(q, q_gate, k, k_gate, prefix_len, vis_start, n_vis, norm_scope=1, scale=None):
+    """Eq. 7, written out: for head h (KV head h // G) and key j of the scope
+      z_j = sum_c (q_gate[b,h,c] * q[b,h,c]) * (k_gate[b,h//G,j,c] * k[b,h//G,j,c]) / sqrt(d),
+    p = softmax_j(z), s[b,m] = mean_h p_h[visual token m].  q, q_gate [B,Hq,d]; k, k_gate
+    [B,Hkv,Lmax,d].  Eq. 7 normalises over the visual tokens (norm_scope 1)."""
+    q, q_gate = np.asarray(q, dtype=np.float64), np.asarray(q_gate, dtype=np.float64)
+    k, k_gate = np.asarray(k, dtype=np.float64), np.asarray(k_gate, dtype=np.float64)
+    B, Hq, d = q.shape
+    G = Hq // k.shape[1]
+    if scale is None:
+        scale = 1.0 / np.sqrt(d)
+    m_max = int(np.max(n_vis)) if B else 0
+    s = np.zeros((B, m_max), dtype=np.float64)
+    for b in range(B):
+        lp, vs, m = int(prefix_len[b]), int(vis_start[b]), int(n_vis[b])
+        if m == 0:
+            continue
+        lo, hi = (0, lp) if norm_scope == 0 else (vs, vs + m)
+        for h in range(Hq):
+            gq = q_gate[b, h] * q[b, h]                               # [d]
+            gk = k_gate[b, h // G, lo:hi] * k[b, h // G, lo:hi]       # [scope, d]
+            z = np.sum(gk * gq[None, :], axis=1) * scale
+            e = np.exp(z - np.max(z))
+            s[b, :m] += (e / np.sum(e))[vs - lo: vs - lo + m]
+        s[b, :m] /= Hq
+    return s
+
+
 # --------------------------------------------------------------------------
 # O2: TopR with the lowest-index tie rule (Eq. 3)
 # --------------------------------------------------------------------------

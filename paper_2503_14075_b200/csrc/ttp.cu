@@ -27,9 +27,12 @@ __device__ __forceinline__ bool layout_ok(int lp, int vs, int nv, int k_max_len,
 // One CTA = 128 keys of one kv head; the G query heads of the group share the
 // key read.  D/8 lanes cover one key row (16 bytes each).
 // ---------------------------------------------------------------------------
-template <int D>
+// GATED (Eq. 7): q is multiplied element-wise by q_gate and every key row by the row of k_gate at the
+// same place (k_gate has K's strides), in fp32, before the dot product.
+template <int D, bool GATED>
 __global__ void __launch_bounds__(kScoreThreads)
 ttp_logits_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restrict__ k,
+                  const __nv_bfloat16 *__restrict__ q_gate, const __nv_bfloat16 *__restrict__ k_gate,
                   long long ksb, long long ksh, long long ksp, int k_max_len,
                   const int *__restrict__ prefix_len, const int *__restrict__ vis_start,
                   const int *__restrict__ n_vis, int n_q_heads, int group, int norm_scope,
@@ -50,17 +53,39 @@ ttp_logits_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__re
   const int j0 = blockIdx.x * kScoreKeysPerCta;
   if (j0 >= hi || j0 + kScoreKeysPerCta <= lo) return;
 
-  for (int i = threadIdx.x; i < group * D; i += kScoreThreads)
-    qs[i] = __bfloat162float(q[((long long)b * n_q_heads + hk * group) * D + i]) * scale;
+  for (int i = threadIdx.x; i < group * D; i += kScoreThreads) {
+    const long long at = ((long long)b * n_q_heads + hk * group) * D + i;
+    float v = __bfloat162float(q[at]) * scale;
+    if (GATED) v *= __bfloat162float(q_gate[at]);
+    qs[i] = v;
+  }
   __syncthreads();
 
   const int sub = threadIdx.x % LPK, slot = threadIdx.x / LPK;
   const __nv_bfloat16 *kb = k + b * ksb + hk * ksh + sub * 8;
-  uint4 kr[PASSES];
+  const __nv_bfloat16 *gb = GATED ? k_gate + b * ksb + hk * ksh + sub * 8 : nullptr;
+  uint4 kr[PASSES], gr[GATED ? PASSES : 1];
 #pragma unroll
   for (int p = 0; p < PASSES; ++p) {
     const int j = j0 + p * KPP + slot;
-    kr[p] = (j >= lo && j < hi) ? ld_nc_16(kb + (long long)j * ksp) : make_uint4(0, 0, 0, 0);
+    const bool in = j >= lo && j < hi;
+    kr[p] = in ? ld_nc_16(kb + (long long)j * ksp) : make_uint4(0, 0, 0, 0);
+    if (GATED) gr[p] = in ? ld_nc_16(gb + (long long)j * ksp) : make_uint4(0, 0, 0, 0);
+  }
+  // the (gated) key row of every pass as eight floats
+  float kf[PASSES][8];
+#pragma unroll
+  for (int p = 0; p < PASSES; ++p) {
+    kf[p][0] = bf16_lo(kr[p].x); kf[p][1] = bf16_hi(kr[p].x);
+    kf[p][2] = bf16_lo(kr[p].y); kf[p][3] = bf16_hi(kr[p].y);
+    kf[p][4] = bf16_lo(kr[p].z); kf[p][5] = bf16_hi(kr[p].z);
+    kf[p][6] = bf16_lo(kr[p].w); kf[p][7] = bf16_hi(kr[p].w);
+    if (GATED) {
+      kf[p][0] *= bf16_lo(gr[p].x); kf[p][1] *= bf16_hi(gr[p].x);
+      kf[p][2] *= bf16_lo(gr[p].y); kf[p][3] *= bf16_hi(gr[p].y);
+      kf[p][4] *= bf16_lo(gr[p].z); kf[p][5] *= bf16_hi(gr[p].z);
+      kf[p][6] *= bf16_lo(gr[p].w); kf[p][7] *= bf16_hi(gr[p].w);
+    }
   }
   for (int g = 0; g < group; ++g) {
     const float4 qa = *reinterpret_cast<const float4 *>(qs + g * D + sub * 8);
@@ -68,14 +93,14 @@ ttp_logits_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__re
     float *lrow = logits + ((long long)b * n_q_heads + hk * group + g) * lstride;
 #pragma unroll
     for (int p = 0; p < PASSES; ++p) {
-      float acc = bf16_lo(kr[p].x) * qa.x;
-      acc = fmaf(bf16_hi(kr[p].x), qa.y, acc);
-      acc = fmaf(bf16_lo(kr[p].y), qa.z, acc);
-      acc = fmaf(bf16_hi(kr[p].y), qa.w, acc);
-      acc = fmaf(bf16_lo(kr[p].z), qb.x, acc);
-      acc = fmaf(bf16_hi(kr[p].z), qb.y, acc);
-      acc = fmaf(bf16_lo(kr[p].w), qb.z, acc);
-      acc = fmaf(bf16_hi(kr[p].w), qb.w, acc);
+      float acc = kf[p][0] * qa.x;
+      acc = fmaf(kf[p][1], qa.y, acc);
+      acc = fmaf(kf[p][2], qa.z, acc);
+      acc = fmaf(kf[p][3], qa.w, acc);
+      acc = fmaf(kf[p][4], qb.x, acc);
+      acc = fmaf(kf[p][5], qb.y, acc);
+      acc = fmaf(kf[p][6], qb.z, acc);
+      acc = fmaf(kf[p][7], qb.w, acc);
 #pragma unroll
       for (int o = LPK / 2; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
       const int j = j0 + p * KPP + slot;
@@ -427,6 +452,7 @@ struct ScoreArgs {
   float softmax_scale;
   float *scores;
   int m_max;
+  const void *q_gate = nullptr, *k_gate = nullptr;     // both or neither (Eq. 7's gates)
 };
 
 static twig_status check_score_args(const ScoreArgs &a, const void *ws, size_t ws_bytes) {
@@ -453,14 +479,18 @@ static twig_status launch_logits(const ScoreArgs &a, int *dev_status, void *ws, 
   const int ls = logits_stride(a.k_max_len);
   auto q = static_cast<const __nv_bfloat16 *>(a.twig_q);
   auto k = static_cast<const __nv_bfloat16 *>(a.twig_k);
-  if (a.head_dim == 128)
-    ttp_logits_kernel<128><<<grid, kScoreThreads, 0, st>>>(q, k, a.ksb, a.ksh, a.ksp, a.k_max_len,
-        a.prefix_len, a.vis_start, a.n_vis, a.n_q_heads, group, a.norm_scope, scale,
-        static_cast<float *>(ws), ls, a.m_max, dev_status);
-  else
-    ttp_logits_kernel<64><<<grid, kScoreThreads, 0, st>>>(q, k, a.ksb, a.ksh, a.ksp, a.k_max_len,
-        a.prefix_len, a.vis_start, a.n_vis, a.n_q_heads, group, a.norm_scope, scale,
-        static_cast<float *>(ws), ls, a.m_max, dev_status);
+  auto qg = static_cast<const __nv_bfloat16 *>(a.q_gate);
+  auto kg = static_cast<const __nv_bfloat16 *>(a.k_gate);
+#define TWIG_LOGITS(D_, G_)                                                                              \
+  ttp_logits_kernel<D_, G_><<<grid, kScoreThreads, 0, st>>>(q, k, qg, kg, a.ksb, a.ksh, a.ksp, a.k_max_len, \
+      a.prefix_len, a.vis_start, a.n_vis, a.n_q_heads, group, a.norm_scope, scale,                       \
+      static_cast<float *>(ws), ls, a.m_max, dev_status)
+  if (a.head_dim == 128) {
+    if (qg) TWIG_LOGITS(128, true); else TWIG_LOGITS(128, false);
+  } else {
+    if (qg) TWIG_LOGITS(64, true); else TWIG_LOGITS(64, false);
+  }
+#undef TWIG_LOGITS
   return launch_status();
 }
 
@@ -530,6 +560,27 @@ extern "C" twig_status ttp_score(const void *twig_q, const void *twig_k, int64_t
   ScoreArgs a{twig_q, twig_k, k_stride_batch, k_stride_head, k_stride_pos, k_max_len, prefix_len,
               vis_start, n_vis, batch, n_q_heads, n_kv_heads, head_dim, norm_scope, softmax_scale,
               scores, m_max};
+  twig_status s = check_score_args(a, ws, ws_bytes);
+  if (s != TWIG_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  s = launch_logits(a, dev_status, ws, st);
+  if (s != TWIG_OK) return s;
+  return launch_finalize(static_cast<const float *>(ws), a, nullptr, nullptr, 0, dev_status, 1, st);
+}
+
+extern "C" twig_status ttp_score_gated(const void *twig_q, const void *q_gate, const void *twig_k,
+                                       const void *k_gate, int64_t k_stride_batch, int64_t k_stride_head,
+                                       int64_t k_stride_pos, int32_t k_max_len, const int32_t *prefix_len,
+                                       const int32_t *vis_start, const int32_t *n_vis, int32_t batch,
+                                       int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim,
+                                       int32_t norm_scope, float softmax_scale, float *scores,
+                                       int32_t m_max, int32_t *dev_status, void *ws, size_t ws_bytes,
+                                       void *stream) {
+  if (!q_gate || !k_gate) return TWIG_ERR_NULL;
+  if (!aligned16(q_gate) || !aligned16(k_gate)) return TWIG_ERR_ALIGN;
+  ScoreArgs a{twig_q, twig_k, k_stride_batch, k_stride_head, k_stride_pos, k_max_len, prefix_len,
+              vis_start, n_vis, batch, n_q_heads, n_kv_heads, head_dim, norm_scope, softmax_scale,
+              scores, m_max, q_gate, k_gate};
   twig_status s = check_score_args(a, ws, ws_bytes);
   if (s != TWIG_OK) return s;
   cudaStream_t st = static_cast<cudaStream_t>(stream);

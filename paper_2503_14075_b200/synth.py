@@ -64,6 +64,12 @@ def normal_bf16(rng: np.random.Generator, shape, head_dim: int, gain: float = 1.
 # --------------------------------------------------------------------------
 # draft trees (parent arrays; node 0 is the root, parent[0] = -1)
 # --------------------------------------------------------------------------
+def gate_bf16(rng: np.random.Generator, shape) -> np.ndarray:
+    """Gate values as a bounded activation would give them: 2 * sigmoid(N(0, 1)), in (0, 2), as bf16 bits."""
+    x = rng.standard_normal(shape, dtype=np.float32)
+    return f32_to_bf16((2.0 / (1.0 + np.exp(-x))).astype(np.float32))
+
+
 def node_depths(parent: Sequence[int]) -> np.ndarray:
     dep = np.zeros(len(parent), dtype=np.int32)
     for i in range(1, len(parent)):

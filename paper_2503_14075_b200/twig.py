@@ -26,7 +26,7 @@ STATUS_NAMES = {0: "TWIG_OK", 1: "TWIG_ERR_NULL", 2: "TWIG_ERR_SHAPE", 3: "TWIG_
 DEV_OK, DEV_BAD_LAYOUT, DEV_BAD_KEEP, DEV_BAD_INDEX, DEV_BAD_TREE, DEV_OVERFLOW, DEV_INTERNAL = range(7)
 MAX_NODES, MAX_VISUAL, MAX_BATCH = 64, 16384, 4096
 
-EXPORTS = ["twig_status_str", "twig_set_launch_overlap", "twig_set_early_prefix", "twig_set_attention_path", "twig_set_attention_splits", "twig_workspace_bytes", "ttp_score", "ttp_score_noalloc", "ttp_topk", "ttp_compact", "ttp_compact_rows",
+EXPORTS = ["twig_status_str", "twig_set_launch_overlap", "twig_set_early_prefix", "twig_set_attention_path", "twig_set_attention_splits", "twig_workspace_bytes", "ttp_score", "ttp_score_gated", "ttp_score_noalloc", "ttp_topk", "ttp_compact", "ttp_compact_rows",
            "ttp_score_topk_compact", "tree_verify_attention", "tree_base_argmax", "tree_accept_compact"]
 
 
@@ -71,6 +71,9 @@ _lib.twig_workspace_bytes.argtypes = [_i32] * 5
 _lib.ttp_score.restype = C.c_int
 _lib.ttp_score.argtypes = [_vp, _vp, _i64, _i64, _i64, _i32, _vp, _vp, _vp, _i32, _i32, _i32, _i32, _i32,
                            _f32, _vp, _i32, _vp, _vp, _sz, _vp]
+_lib.ttp_score_gated.restype = C.c_int
+_lib.ttp_score_gated.argtypes = [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _vp, _vp, _vp, _i32, _i32, _i32, _i32,
+                                 _i32, _f32, _vp, _i32, _vp, _vp, _sz, _vp]
 _lib.ttp_score_noalloc.restype = C.c_int
 _lib.ttp_score_noalloc.argtypes = [_vp, _vp, _i64, _i64, _i64, _i32, _vp, _vp, _vp, _i32, _i32, _i32, _i32, _i32,
                                    _f32, _vp, _i32, _vp, _vp]
@@ -146,6 +149,19 @@ def ttp_score(twig_q, twig_k, prefix_len, vis_start, n_vis, scores, ws, norm_sco
                           twig_k.shape[2], _p(prefix_len), _p(vis_start), _p(n_vis), B, Hq,
                           twig_k.shape[1], d, norm_scope, softmax_scale, _p(scores), scores.shape[1],
                           _p(dev_status), _p(ws), ws.numel() * ws.element_size(), _stream(stream)))
+
+
+def ttp_score_gated(twig_q, q_gate, twig_k, k_gate, prefix_len, vis_start, n_vis, scores, ws, norm_scope=1,
+                    softmax_scale=0.0, dev_status=None, stream=None):
+    """ttp_score of (q_gate * twig_q, k_gate * twig_k), element-wise products formed in the kernel;
+    q_gate like twig_q, k_gate with twig_k's shape and strides."""
+    B, Hq, d = twig_q.shape
+    assert q_gate.shape == twig_q.shape and q_gate.is_contiguous()
+    assert k_gate.shape == twig_k.shape and k_gate.stride() == twig_k.stride()
+    _check(_lib.ttp_score_gated(_p(twig_q), _p(q_gate), _p(twig_k), _p(k_gate), twig_k.stride(0), twig_k.stride(1),
+                                twig_k.stride(2), twig_k.shape[2], _p(prefix_len), _p(vis_start), _p(n_vis), B, Hq,
+                                twig_k.shape[1], d, norm_scope, softmax_scale, _p(scores), scores.shape[1],
+                                _p(dev_status), _p(ws), ws.numel() * ws.element_size(), _stream(stream)))
 
 
 def ttp_score_noalloc(twig_q, twig_k, prefix_len, vis_start, n_vis, scores, norm_scope=0,

@@ -64,6 +64,37 @@ def test_scores_match_oracle(tw, name, scope, gain_mult):
             assert abs(float(got[b, :m].astype(np.float64).sum()) - 1.0) < 1e-4
 
 
+@pytest.mark.parametrize("name", ["c1", "hetero", "gqa64", "gqa7"])
+@pytest.mark.parametrize("scope", [1, 0])
+def test_gated_scores_match_oracle(tw, name, scope):
+    """Eq. 7 with the gates applied inside the kernel."""
+    wl = WORKLOADS[name]()
+    rng = synth.rng_for(wl.index, 11)
+    pre = synth.make_prefill(wl, rng, n_layers=1, gain=wl.head_dim ** 0.5)
+    qg, kg = synth.gate_bf16(rng, pre["twig_q"].shape), synth.gate_bf16(rng, pre["twig_k"].shape)
+    B = wl.batch
+    m_max = max(1, int(pre["n_vis"].max()))
+    q, k = dev_bf16(pre["twig_q"]), dev_bf16(pre["twig_k"])
+    scores = torch.full((B, m_max), -1.0, dtype=torch.float32, device=DEV)
+    ws = torch.empty(tw.twig_workspace_bytes(B, wl.n_q_heads, wl.head_dim, k.shape[2], 64), dtype=torch.uint8, device=DEV)
+    status = torch.zeros(B, dtype=torch.int32, device=DEV)
+    tw.ttp_score_gated(q, dev_bf16(qg), k, dev_bf16(kg), dev_i32(pre["prefix_len"]), dev_i32(pre["vis_start"]),
+                       dev_i32(pre["n_vis"]), scores, ws, norm_scope=scope, dev_status=status)
+    torch.cuda.synchronize()
+    assert status.cpu().tolist() == [0] * B
+    got = scores.cpu().numpy()
+    want = O.ttp_scores_gated(f64(pre["twig_q"]), f64(qg), f64(pre["twig_k"]), f64(kg), pre["prefix_len"], pre["vis_start"],
+                              pre["n_vis"], scope)
+    ungated = O.ttp_scores(f64(pre["twig_q"]), f64(pre["twig_k"]), pre["prefix_len"], pre["vis_start"], pre["n_vis"], scope)
+    for b in range(B):
+        m = pre["n_vis"][b]
+        assert max_abs(got[b, :m], want[b, :m]) <= MAX_ABS_TOL
+        assert rel_l2_rows(got[b, :m].astype(np.float64), want[b, :m]) <= REL_L2_TOL
+        assert np.all(got[b, m:] == 0)
+        if m > 1:      # the gates matter on these inputs: the ungated score is far outside the tolerance
+            assert rel_l2_rows(ungated[b, :m], want[b, :m]) > 10 * REL_L2_TOL
+
+
 def _run_topk(tw, s, n_vis, keep, r_max=None):
     B, m_max = s.shape
     r_max = r_max or max(1, int(max(keep)))

@@ -17,6 +17,9 @@ MUTATIONS = [
     ("scores: wrong kv head for a query head", "z = np.matmul(k[b, h // G, lo:hi, :]", "z = np.matmul(k[b, h % Hkv, lo:hi, :]"),
     ("scores: visual slice off by one", "p[vs - lo: vs - lo + m]", "p[vs - lo + 1: vs - lo + m + 1]"),
     ("scores: eq. 7 scope ignored", "lo, hi = (0, lp) if norm_scope == 0 else (vs, vs + m)", "lo, hi = (0, lp)"),
+    ("gated scores: key gate dropped", "gk = k_gate[b, h // G, lo:hi] * k[b, h // G, lo:hi]", "gk = k[b, h // G, lo:hi]"),
+    ("gated scores: query gate of another head", "gq = q_gate[b, h] * q[b, h]", "gq = q_gate[b, 0] * q[b, h]"),
+    ("gated scores: gate of the wrong kv head", "gk = k_gate[b, h // G, lo:hi] *", "gk = k_gate[b, h % k.shape[1], lo:hi] *"),
     ("top-k: ties to the higher index", "key=lambda m: (-s[m], m)", "key=lambda m: (-s[m], -m)"),
     ("top-k: smallest instead of largest", "key=lambda m: (-s[m], m)", "key=lambda m: (s[m], m)"),
     ("prune: text after the image dropped", "+ list(range(vis_start + n_vis, prefix_len))", ""),

@@ -471,6 +471,42 @@ def test_speculative_decoding_is_lossless_with_toy_target():
     assert seq[:len(greedy)] == greedy
 
 
+def test_gated_scores_brute_force_and_reductions():
+    """Eq. 7: against a loop-by-loop evaluation on a tiny case; gates of one give the ungated
+    score; a gate can be moved between q and K; a key whose gate is zero gets the uniform share
+    of a zero logit."""
+    import math
+    rng = np.random.default_rng(17)
+    B, Hq, Hkv, L, d = 2, 4, 2, 9, 8
+    q, gq = rng.standard_normal((B, Hq, d)), rng.uniform(0.2, 1.5, (B, Hq, d))
+    k, gk = rng.standard_normal((B, Hkv, L, d)), rng.uniform(0.2, 1.5, (B, Hkv, L, d))
+    lp, vs, nv = [9, 7], [2, 1], [5, 4]
+    got = O.ttp_scores_gated(q, gq, k, gk, lp, vs, nv)
+    for b in range(B):
+        want = [0.0] * nv[b]
+        for h in range(Hq):
+            z = []
+            for m in range(nv[b]):
+                j = vs[b] + m
+                z.append(sum(gq[b, h, c] * q[b, h, c] * gk[b, h // 2, j, c] * k[b, h // 2, j, c] for c in range(d)) / math.sqrt(d))
+            den = sum(math.exp(x) for x in z)
+            for m in range(nv[b]):
+                want[m] += math.exp(z[m]) / den / Hq
+        assert np.allclose(got[b, :nv[b]], want, rtol=1e-12, atol=1e-15)
+        assert abs(got[b, :nv[b]].sum() - 1.0) < 1e-12
+    one_q, one_k = np.ones_like(q), np.ones_like(k)
+    assert np.allclose(O.ttp_scores_gated(q, one_q, k, one_k, lp, vs, nv, norm_scope=0), O.ttp_scores(q, k, lp, vs, nv, 0), rtol=1e-12)
+    assert np.allclose(O.ttp_scores_gated(q, one_q, k, one_k, lp, vs, nv, norm_scope=1), O.ttp_scores(q, k, lp, vs, nv, 1), rtol=1e-12)
+    # the same product whichever side carries the factor
+    assert np.allclose(got, O.ttp_scores(q * gq, k * gk, lp, vs, nv, 1), rtol=1e-12)
+    g0 = gk.copy()
+    g0[:, :, 3, :] = 0.0                      # key 3: logit 0 in every head
+    z0 = O.ttp_scores_gated(q, gq, k, g0, [9, 9], [0, 0], [9, 9])
+    k0 = k.copy()
+    k0[:, :, 3, :] = 0.0
+    assert np.allclose(z0, O.ttp_scores_gated(q, gq, k0, gk, [9, 9], [0, 0], [9, 9]), rtol=1e-12)
+
+
 def test_base_argmax_library_and_ties():
     rng = np.random.default_rng(31)
     x = rng.integers(-3, 4, size=(2, 5, 40)).astype(np.float64)          # many exact ties
