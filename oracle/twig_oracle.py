@@ -104,6 +104,32 @@ def ttp_scores_gated(q, q_gate, k, k_gate, prefix_len, vis_start, n_vis, norm_sc
     return s
 
 
+def text_to_visual_scores(q_text, k, prefix_len, vis_start, n_vis, scale=None):
+    """Eq. 3's guide "sum_{i=M+1}^{M+N} A[i, 1:M]": attention that the textual tokens after the
+    image pay to every visual token, with A the causal attention map averaged over heads.
+    q_text [B,Hq,Nmax,d]: row i is the query at prompt position vis_start + n_vis + i
+    (N_b = prefix_len - vis_start - n_vis of them); k [B,Hkv,Lmax,d].  For head h and query i at
+    position t: p = softmax_{j <= t}(q . k_j * scale);  s[b,m] = (1/Hq) sum_h sum_i p[vis_start + m]."""
+    q_text = np.asarray(q_text, dtype=np.float64)
+    k = np.asarray(k, dtype=np.float64)
+    B, Hq, _, d = q_text.shape
+    G = Hq // k.shape[1]
+    if scale is None:
+        scale = 1.0 / np.sqrt(d)
+    m_max = int(np.max(n_vis)) if B else 0
+    s = np.zeros((B, m_max), dtype=np.float64)
+    for b in range(B):
+        lp, vs, m = int(prefix_len[b]), int(vis_start[b]), int(n_vis[b])
+        for h in range(Hq):
+            for i in range(lp - vs - m):
+                t = vs + m + i
+                z = np.matmul(k[b, h // G, :t + 1, :], q_text[b, h, i, :]) * scale
+                e = np.exp(z - np.max(z))
+                s[b, :m] += (e / np.sum(e))[vs:vs + m]
+        s[b, :m] /= Hq
+    return s
+
+
 # --------------------------------------------------------------------------
 # O2: TopR with the lowest-index tie rule (Eq. 3)
 # --------------------------------------------------------------------------

@@ -20,6 +20,9 @@ MUTATIONS = [
     ("gated scores: key gate dropped", "gk = k_gate[b, h // G, lo:hi] * k[b, h // G, lo:hi]", "gk = k[b, h // G, lo:hi]"),
     ("gated scores: query gate of another head", "gq = q_gate[b, h] * q[b, h]", "gq = q_gate[b, 0] * q[b, h]"),
     ("gated scores: gate of the wrong kv head", "gk = k_gate[b, h // G, lo:hi] *", "gk = k_gate[b, h % k.shape[1], lo:hi] *"),
+    ("eq. 3 guide: not causal", "z = np.matmul(k[b, h // G, :t + 1, :], q_text[b, h, i, :]) * scale", "z = np.matmul(k[b, h // G, :lp, :], q_text[b, h, i, :]) * scale"),
+    ("eq. 3 guide: query position off by one", "                t = vs + m + i\n", "                t = vs + m + i - 1\n"),
+    ("eq. 3 guide: only the last text token", "for i in range(lp - vs - m):", "for i in range(lp - vs - m - 1, lp - vs - m):"),
     ("top-k: ties to the higher index", "key=lambda m: (-s[m], m)", "key=lambda m: (-s[m], -m)"),
     ("top-k: smallest instead of largest", "key=lambda m: (-s[m], m)", "key=lambda m: (s[m], m)"),
     ("prune: text after the image dropped", "+ list(range(vis_start + n_vis, prefix_len))", ""),

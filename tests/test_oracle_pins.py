@@ -507,6 +507,43 @@ def test_gated_scores_brute_force_and_reductions():
     assert np.allclose(z0, O.ttp_scores_gated(q, gq, k0, gk, [9, 9], [0, 0], [9, 9]), rtol=1e-12)
 
 
+def test_text_to_visual_scores_pins():
+    """Eq. 3's multi-query guide: brute force on a tiny case; one query at the last prompt position
+    is the single-query score over the full causal row; causality (a key after a query's position
+    does not reach that query's share); each query spreads at most 1 over the visual tokens."""
+    import math
+    rng = np.random.default_rng(23)
+    B, Hq, Hkv, L, d, N = 2, 4, 2, 12, 8, 4
+    k = rng.standard_normal((B, Hkv, L, d))
+    qt = rng.standard_normal((B, Hq, N, d))
+    lp, vs, nv = [12, 9], [3, 2], [5, 6]          # 4 and 1 text tokens after the image
+    got = O.text_to_visual_scores(qt, k, lp, vs, nv)
+    for b in range(B):
+        want = [0.0] * nv[b]
+        for h in range(Hq):
+            for i in range(lp[b] - vs[b] - nv[b]):
+                t = vs[b] + nv[b] + i
+                z = [sum(qt[b, h, i, c] * k[b, h // 2, j, c] for c in range(d)) / math.sqrt(d) for j in range(t + 1)]
+                den = sum(math.exp(x) for x in z)
+                for m in range(nv[b]):
+                    want[m] += math.exp(z[vs[b] + m]) / den / Hq
+        assert np.allclose(got[b, :nv[b]], want, rtol=1e-12, atol=1e-15)
+        assert got[b, :nv[b]].sum() <= (lp[b] - vs[b] - nv[b]) + 1e-12
+        assert np.all(got[b, nv[b]:] == 0)
+    # request 1 has exactly one text token after the image, at the last prompt position
+    single = O.ttp_scores(qt[1:2, :, 0, :], k[1:2], [9], [2], [6], norm_scope=0)
+    assert np.allclose(got[1, :6], single[0, :6], rtol=1e-12)
+    # causality: the last key (position 11) is seen by request 0's last query only
+    k2 = k.copy()
+    k2[0, :, 11, :] += 3.0
+    got2 = O.text_to_visual_scores(qt, k2, lp, vs, nv)
+    first3 = O.text_to_visual_scores(qt[:, :, :3], k, [11, 9], vs, nv)      # prompt cut before its last token
+    first3_2 = O.text_to_visual_scores(qt[:, :, :3], k2, [11, 9], vs, nv)
+    assert np.allclose(first3, first3_2, rtol=0, atol=0)
+    assert np.allclose(got2[0] - first3_2[0], O.text_to_visual_scores(qt, k2, lp, vs, nv)[0] - first3[0], rtol=1e-12)
+    assert not np.allclose(got2[0], got[0])
+
+
 def test_base_argmax_library_and_ties():
     rng = np.random.default_rng(31)
     x = rng.integers(-3, 4, size=(2, 5, 40)).astype(np.float64)          # many exact ties
