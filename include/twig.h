@@ -120,6 +120,27 @@ twig_status ttp_score_gated(const void *twig_q, const void *q_gate, const void *
                             int32_t norm_scope, float softmax_scale, float *scores, int32_t m_max,
                             int32_t *dev_status, void *ws, size_t ws_bytes, void *stream);
 
+/* ---- Multi-query pruning guide (FastV's form of the TopR argument) ----------
+ * Eq. 3: "sum_{i=M+1}^{M+N} A[i, 1:M]", the attention the textual tokens after the image pay to
+ * every visual token, A the causal attention map averaged over heads:
+ *   scores[b, m] = (1/n_q_heads) sum_h sum_i softmax_{j <= t_i}(q_text[b,h,i] . twig_k[b,h/G,j] * scale)[vis_start[b] + m],
+ * i < N_b = prefix_len[b] - vis_start[b] - n_vis[b], t_i = vis_start[b] + n_vis[b] + i (text token i's
+ * prompt position).  With one text token this is ttp_score with norm_scope 0.
+ *   q_text  [batch, n_q_heads, n_text_max, head_dim] bf16 contiguous; rows i >= N_b are ignored.
+ *           N_b > n_text_max is reported as TWIG_DEV_BAD_LAYOUT (scores of that request: 0)
+ *   twig_k, strides, k_max_len, prefix_len, vis_start, n_vis, scores, m_max: as in ttp_score
+ * Scratch: ttp_multiquery_workspace_bytes(batch, n_q_heads, n_text_max, m_max).  The result is
+ * reproducible from run to run (partial sums are added in a fixed order).
+ */
+size_t ttp_multiquery_workspace_bytes(int32_t batch, int32_t n_q_heads, int32_t n_text_max, int32_t m_max);
+twig_status ttp_score_multiquery(const void *q_text, int32_t n_text_max, const void *twig_k,
+                                 int64_t k_stride_batch, int64_t k_stride_head, int64_t k_stride_pos,
+                                 int32_t k_max_len, const int32_t *prefix_len, const int32_t *vis_start,
+                                 const int32_t *n_vis, int32_t batch, int32_t n_q_heads,
+                                 int32_t n_kv_heads, int32_t head_dim, float softmax_scale,
+                                 float *scores, int32_t m_max, int32_t *dev_status, void *ws,
+                                 size_t ws_bytes, void *stream);
+
 /* ---- ttp_score without any caller-provided or allocated scratch --------------
  * (No counterpart in the paper: this is a deployment convenience.)
  * Some hosts of this library may not allocate device memory at the point where

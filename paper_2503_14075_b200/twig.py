@@ -26,7 +26,7 @@ STATUS_NAMES = {0: "TWIG_OK", 1: "TWIG_ERR_NULL", 2: "TWIG_ERR_SHAPE", 3: "TWIG_
 DEV_OK, DEV_BAD_LAYOUT, DEV_BAD_KEEP, DEV_BAD_INDEX, DEV_BAD_TREE, DEV_OVERFLOW, DEV_INTERNAL = range(7)
 MAX_NODES, MAX_VISUAL, MAX_BATCH = 64, 16384, 4096
 
-EXPORTS = ["twig_status_str", "twig_set_launch_overlap", "twig_set_early_prefix", "twig_set_attention_path", "twig_set_attention_splits", "twig_workspace_bytes", "ttp_score", "ttp_score_gated", "ttp_score_noalloc", "ttp_topk", "ttp_compact", "ttp_compact_rows",
+EXPORTS = ["twig_status_str", "twig_set_launch_overlap", "twig_set_early_prefix", "twig_set_attention_path", "twig_set_attention_splits", "twig_workspace_bytes", "ttp_score", "ttp_score_gated", "ttp_multiquery_workspace_bytes", "ttp_score_multiquery", "ttp_score_noalloc", "ttp_topk", "ttp_compact", "ttp_compact_rows",
            "ttp_score_topk_compact", "tree_verify_attention", "tree_base_argmax", "tree_accept_compact"]
 
 
@@ -74,6 +74,11 @@ _lib.ttp_score.argtypes = [_vp, _vp, _i64, _i64, _i64, _i32, _vp, _vp, _vp, _i32
 _lib.ttp_score_gated.restype = C.c_int
 _lib.ttp_score_gated.argtypes = [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _vp, _vp, _vp, _i32, _i32, _i32, _i32,
                                  _i32, _f32, _vp, _i32, _vp, _vp, _sz, _vp]
+_lib.ttp_multiquery_workspace_bytes.restype = _sz
+_lib.ttp_multiquery_workspace_bytes.argtypes = [_i32] * 4
+_lib.ttp_score_multiquery.restype = C.c_int
+_lib.ttp_score_multiquery.argtypes = [_vp, _i32, _vp, _i64, _i64, _i64, _i32, _vp, _vp, _vp, _i32, _i32, _i32, _i32,
+                                      _f32, _vp, _i32, _vp, _vp, _sz, _vp]
 _lib.ttp_score_noalloc.restype = C.c_int
 _lib.ttp_score_noalloc.argtypes = [_vp, _vp, _i64, _i64, _i64, _i32, _vp, _vp, _vp, _i32, _i32, _i32, _i32, _i32,
                                    _f32, _vp, _i32, _vp, _vp]
@@ -162,6 +167,23 @@ def ttp_score_gated(twig_q, q_gate, twig_k, k_gate, prefix_len, vis_start, n_vis
                                 twig_k.stride(2), twig_k.shape[2], _p(prefix_len), _p(vis_start), _p(n_vis), B, Hq,
                                 twig_k.shape[1], d, norm_scope, softmax_scale, _p(scores), scores.shape[1],
                                 _p(dev_status), _p(ws), ws.numel() * ws.element_size(), _stream(stream)))
+
+
+def ttp_multiquery_workspace_bytes(batch, n_q_heads, n_text_max, m_max):
+    return int(_lib.ttp_multiquery_workspace_bytes(batch, n_q_heads, n_text_max, m_max))
+
+
+def ttp_score_multiquery(q_text, twig_k, prefix_len, vis_start, n_vis, scores, ws, softmax_scale=0.0,
+                         dev_status=None, stream=None):
+    """q_text [B,Hq,Nmax,d] (the text tokens after the image, in order), twig_k [B,Hkv,Lmax,d] bf16;
+    scores [B,m_max] fp32 (out): attention from those tokens to every visual token, summed over
+    tokens, averaged over heads."""
+    B, Hq, N, d = q_text.shape
+    assert q_text.is_contiguous()
+    _check(_lib.ttp_score_multiquery(_p(q_text), N, _p(twig_k), twig_k.stride(0), twig_k.stride(1), twig_k.stride(2),
+                                     twig_k.shape[2], _p(prefix_len), _p(vis_start), _p(n_vis), B, Hq, twig_k.shape[1],
+                                     d, softmax_scale, _p(scores), scores.shape[1], _p(dev_status), _p(ws),
+                                     ws.numel() * ws.element_size(), _stream(stream)))
 
 
 def ttp_score_noalloc(twig_q, twig_k, prefix_len, vis_start, n_vis, scores, norm_scope=0,

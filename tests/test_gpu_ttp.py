@@ -95,6 +95,49 @@ def test_gated_scores_match_oracle(tw, name, scope):
             assert rel_l2_rows(ungated[b, :m], want[b, :m]) > 10 * REL_L2_TOL
 
 
+@pytest.mark.parametrize("name", ["c1", "c2", "hetero", "gqa64", "gqa7"])
+@pytest.mark.parametrize("gain_mult", [1.0, "sharp"])
+def test_multiquery_scores_match_oracle(tw, name, gain_mult):
+    """Eq. 3's guide: attention from the text tokens after the image to the visual tokens."""
+    wl = WORKLOADS[name]()
+    gain = {1.0: 1.0, "sharp": wl.head_dim ** 0.5}[gain_mult]
+    rng = synth.rng_for(wl.index, 12)
+    pre = synth.make_prefill(wl, rng, n_layers=1, gain=gain)
+    B, Hq, d = wl.batch, wl.n_q_heads, wl.head_dim
+    n_text = [int(pre["prefix_len"][b] - pre["vis_start"][b] - pre["n_vis"][b]) for b in range(B)]
+    n_max = max(1, max(n_text)) + 3                     # a few rows nobody may read
+    qt = synth.normal_bf16(rng, (B, Hq, n_max, d), d, gain)
+    for b in range(B):
+        qt[b, :, n_text[b]:, :] = 0x7FC1                # NaN past the last text token
+    m_max = max(1, int(pre["n_vis"].max()))
+    scores = torch.full((B, m_max), -1.0, dtype=torch.float32, device=DEV)
+    ws = torch.full((tw.ttp_multiquery_workspace_bytes(B, Hq, n_max, m_max) // 4,), float("nan"), dtype=torch.float32,
+                    device=DEV)
+    status = torch.zeros(B, dtype=torch.int32, device=DEV)
+    args = (dev_bf16(qt), dev_bf16(pre["twig_k"]), dev_i32(pre["prefix_len"]), dev_i32(pre["vis_start"]),
+            dev_i32(pre["n_vis"]), scores, ws)
+    tw.ttp_score_multiquery(*args, dev_status=status)
+    torch.cuda.synchronize()
+    assert status.cpu().tolist() == [0] * B
+    got = scores.cpu().numpy()
+    qt_clean = qt.copy()
+    for b in range(B):
+        qt_clean[b, :, n_text[b]:, :] = 0
+    want = O.text_to_visual_scores(f64(qt_clean), f64(pre["twig_k"]), pre["prefix_len"], pre["vis_start"], pre["n_vis"])
+    for b in range(B):
+        m = pre["n_vis"][b]
+        scale = max(1, n_text[b])                       # up to n_text probabilities add up in an entry
+        assert max_abs(got[b, :m], want[b, :m]) <= MAX_ABS_TOL * scale
+        if m > 0 and n_text[b] > 0:
+            assert rel_l2_rows(got[b, :m].astype(np.float64), want[b, :m]) <= REL_L2_TOL
+        assert np.all(got[b, m:] == 0)
+    # same bits on a second run (fixed summation order)
+    scores2 = torch.full_like(scores, -2.0)
+    tw.ttp_score_multiquery(*args[:5], scores2, ws, dev_status=status)
+    torch.cuda.synchronize()
+    assert torch.equal(scores, scores2)
+
+
 def _run_topk(tw, s, n_vis, keep, r_max=None):
     B, m_max = s.shape
     r_max = r_max or max(1, int(max(keep)))
