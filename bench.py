@@ -564,7 +564,25 @@ def extra_rooflines(torch, tw, peaks, dev):
     us = e0.elapsed_time(e1) * 1e3 / n_chain
     res["ttp_score_gated_c4"] = hbm_entry(us, int(2 * sum(Hkv * n * d * 2 for n in wl.n_vis)))
     res["ttp_score_gated_c4"]["launches"] = "logits + softmax/mean (2 kernels)"
-    del pre4, q4, k4, qg4, kg4
+    # multi-query guide of Eq. 3 on the same prompts: every text token after the image against the whole
+    # prompt (K once per kv head is the algorithmic traffic; the two passes of the query blocks re-read it from L2)
+    n_txt = max(wl.text_after)
+    qt4 = bf(synth.normal_bf16(rng, (B, Hq, n_txt, d), d))
+    wsm = torch.empty(tw.ttp_multiquery_workspace_bytes(B, Hq, n_txt, max(wl.n_vis)), dtype=torch.uint8, device=dev)
+    for _ in range(3):
+        tw.ttp_score_multiquery(qt4, k4, *m4, sc4, wsm)
+    e0.record(stream)
+    for _ in range(n_chain):
+        tw.ttp_score_multiquery(qt4, k4, *m4, sc4, wsm)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    us = e0.elapsed_time(e1) * 1e3 / n_chain
+    # per head and text token i: a + n + i + 1 keys for the statistics, n more for the probabilities
+    fl = sum(2 * Hq * d * c * (a + 2 * n + (c + 1) / 2) for a, n, c in zip(wl.text_before, wl.n_vis, wl.text_after))
+    res["ttp_score_multiquery_c4"] = hbm_entry(us, int(sum(Hkv * p * d * 2 for p in wl.prefix_len)))
+    res["ttp_score_multiquery_c4"].update({"text_tokens": n_txt, "flops_per_launch": int(fl),
+                                           "tflops": round(fl / us / 1e6, 1), "launches": "partial sums + reduce (2 kernels)"})
+    del pre4, q4, k4, qg4, kg4, qt4
     # greedy target token per tree node over the heterogeneous batch's trees (32000-entry bf16 rows);
     # six logits buffers in turn, 190 MB together, so that every read is cold
     V = 32000

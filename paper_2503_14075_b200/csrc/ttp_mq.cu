@@ -3,11 +3,16 @@
 //   a[m] = (1/H) sum_h sum_i softmax_{j <= t_i}(q_i . k_j / sqrt(d))[vis_start + m],
 // t_i = vis_start + n_vis + i the prompt position of text token i.  Unlike the single-query score
 // this is an N x L attention-map reduction: S = Q_text K^T runs on tensor cores (bf16
-// mma.sync.m16n8k16, fp32 accumulation).  A CTA owns 64 query rows of one head and walks the keys
-// twice: once for the rows' softmax statistics (max, sum), once more over the visual span for the
-// normalised probabilities, whose column sums it writes to its own slice of the scratch; a second
-// kernel adds the slices in a fixed order, so the result does not depend on scheduling.
+// mma.sync.m16n8k16, fp32 accumulation).  A thread-block cluster owns 64 query rows of one head and
+// walks the keys twice, its CTAs sharing the key tiles: once for the rows' softmax statistics
+// (max, sum; exchanged through distributed shared memory), once more over the visual span for
+// the normalised probabilities, whose column sums go to the block's own slice of the scratch;
+// a second kernel adds the slices in a fixed order, so the result does not depend on scheduling.
+#include <cooperative_groups.h>
+
 #include "tree_attn.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace twig {
 
@@ -33,8 +38,11 @@ ttp_mq_partial_kernel(const __nv_bfloat16 *__restrict__ q_text, int n_text_max,
   constexpr int TILE_BYTES = 64 * D * 2;
   extern __shared__ __align__(1024) unsigned char smem[];
   __shared__ float s_col[4][kMqKeys];
+  __shared__ float2 s_ml[8][kMqRows];            // (max, sum) of every row from every CTA of the cluster
 
-  const int qb = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+  cg::cluster_group cluster = cg::this_cluster();
+  const int n_splits = cluster.num_blocks(), split = cluster.block_rank();
+  const int qb = blockIdx.x / n_splits, h = blockIdx.y, b = blockIdx.z;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int lp = prefix_len[b], vs = vis_start[b], nv = n_vis[b];
   const int n_text = lp - vs - nv;
@@ -101,16 +109,19 @@ ttp_mq_partial_kernel(const __nv_bfloat16 *__restrict__ q_text, int n_text_max,
 
   // ---- pass 1: running maximum and sum of every row over its causal span ----
   float m_lo = -INFINITY, m_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;
-  const int t_end1 = (t_first + rows - 1) / kMqKeys + 1;      // tiles up to the last query's own position
-  load_keys(0, 0);
+  const int n_t1 = (t_first + rows - 1) / kMqKeys + 1;        // tiles up to the last query's own position
+  const int per1 = (n_t1 + n_splits - 1) / n_splits;
+  const int t_begin1 = split * per1, t_end1 = min(n_t1, t_begin1 + per1);     // this CTA's share
+  if (t_begin1 < t_end1) load_keys(t_begin1, 0);
   cp_async_commit();                                          // (this group also carries Q)
-  for (int t = 0; t < t_end1; ++t) {
-    if (t + 1 < t_end1) load_keys(t + 1, (t + 1) & 1);
+  for (int t = t_begin1; t < t_end1; ++t) {
+    const int it = t - t_begin1;
+    if (t + 1 < t_end1) load_keys(t + 1, (it + 1) & 1);
     cp_async_commit();
     cp_async_wait<1>();
     __syncthreads();
     float s[NT][4];
-    scores_of(t, t & 1, s);
+    scores_of(t, it & 1, s);
     float mx_lo = -INFINITY, mx_hi = -INFINITY;
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
@@ -139,13 +150,41 @@ ttp_mq_partial_kernel(const __nv_bfloat16 *__restrict__ q_text, int n_text_max,
   l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
   l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1);
   l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
+  // every CTA of the cluster tells every other its rows' (max, sum); then all hold the same totals
+  if (n_splits > 1) {
+    if (tq == 0) {
+      for (int c = 0; c < n_splits; ++c) {
+        float2 *dst = cluster.map_shared_rank(&s_ml[split][0], c);
+        dst[r_lo] = make_float2(m_lo, l_lo);
+        dst[r_hi] = make_float2(m_hi, l_hi);
+      }
+    }
+    cluster.sync();
+    float M_lo = -INFINITY, M_hi = -INFINITY;
+    for (int c = 0; c < n_splits; ++c) {
+      M_lo = fmaxf(M_lo, s_ml[c][r_lo].x);
+      M_hi = fmaxf(M_hi, s_ml[c][r_hi].x);
+    }
+    const float U_lo = M_lo == -INFINITY ? 0.f : M_lo, U_hi = M_hi == -INFINITY ? 0.f : M_hi;
+    float L_lo = 0.f, L_hi = 0.f;
+    for (int c = 0; c < n_splits; ++c) {          // index order: the same sum in every CTA
+      L_lo += s_ml[c][r_lo].y * fast_exp2(s_ml[c][r_lo].x - U_lo);
+      L_hi += s_ml[c][r_hi].y * fast_exp2(s_ml[c][r_hi].x - U_hi);
+    }
+    m_lo = M_lo;
+    m_hi = M_hi;
+    l_lo = L_lo;
+    l_hi = L_hi;
+  }
   const float inv_lo = l_lo > 0.f ? 1.f / l_lo : 0.f, inv_hi = l_hi > 0.f ? 1.f / l_hi : 0.f;
   const float use_lo = m_lo == -INFINITY ? 0.f : m_lo, use_hi = m_hi == -INFINITY ? 0.f : m_hi;
 
   // ---- pass 2: normalised probabilities over the visual span, summed down the 64 rows ----
-  float *out = partial + (((long long)b * n_q_heads + h) * gridDim.x + qb) * m_max;
-  const int t_begin2 = vs / kMqKeys, t_end2 = (vs + nv - 1) / kMqKeys + 1;
-  load_keys(t_begin2, 0);
+  float *out = partial + (((long long)b * n_q_heads + h) * (gridDim.x / n_splits) + qb) * m_max;
+  const int t_vis0 = vs / kMqKeys, n_t2 = (vs + nv - 1) / kMqKeys + 1 - t_vis0;
+  const int per2 = (n_t2 + n_splits - 1) / n_splits;
+  const int t_begin2 = t_vis0 + split * per2, t_end2 = min(t_vis0 + n_t2, t_begin2 + per2);
+  if (t_begin2 < t_end2) load_keys(t_begin2, 0);
   cp_async_commit();
   for (int t = t_begin2; t < t_end2; ++t) {
     const int it = t - t_begin2;
@@ -234,8 +273,22 @@ extern "C" twig_status ttp_score_multiquery(const void *q_text, int32_t n_text_m
   auto q = static_cast<const __nv_bfloat16 *>(q_text);
   auto k = static_cast<const __nv_bfloat16 *>(twig_k);
   float *partial = static_cast<float *>(ws);
-  dim3 grid(n_blocks, n_q_heads, batch);
   const int group = n_q_heads / n_kv_heads;
+  // key tiles are shared by the CTAs of a cluster: as many as still fit one wave (4 CTAs per SM)
+  int n_splits = 8;
+  while (n_splits > 1 && (long long)n_blocks * n_q_heads * batch * n_splits > 4 * 148) n_splits >>= 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(n_blocks * n_splits, n_q_heads, batch);
+  cfg.blockDim = dim3(kMqThreads);
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = n_splits;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaError_t err;
   if (head_dim == 128) {
     constexpr int smem = 3 * 64 * 128 * 2;
     static bool attr_set = false;
@@ -244,13 +297,17 @@ extern "C" twig_status ttp_score_multiquery(const void *q_text, int32_t n_text_m
         return TWIG_ERR_CUDA;
       attr_set = true;
     }
-    ttp_mq_partial_kernel<128><<<grid, kMqThreads, smem, st>>>(q, n_text_max, k, k_stride_batch, k_stride_head,
-        k_stride_pos, k_max_len, prefix_len, vis_start, n_vis, n_q_heads, group, scale_log2, partial, m_max, dev_status);
+    cfg.dynamicSmemBytes = smem;
+    err = cudaLaunchKernelEx(&cfg, ttp_mq_partial_kernel<128>, q, n_text_max, k, (long long)k_stride_batch,
+                             (long long)k_stride_head, (long long)k_stride_pos, k_max_len, prefix_len, vis_start, n_vis,
+                             n_q_heads, group, scale_log2, partial, m_max, dev_status);
   } else {
-    constexpr int smem = 3 * 64 * 64 * 2;
-    ttp_mq_partial_kernel<64><<<grid, kMqThreads, smem, st>>>(q, n_text_max, k, k_stride_batch, k_stride_head,
-        k_stride_pos, k_max_len, prefix_len, vis_start, n_vis, n_q_heads, group, scale_log2, partial, m_max, dev_status);
+    cfg.dynamicSmemBytes = 3 * 64 * 64 * 2;
+    err = cudaLaunchKernelEx(&cfg, ttp_mq_partial_kernel<64>, q, n_text_max, k, (long long)k_stride_batch,
+                             (long long)k_stride_head, (long long)k_stride_pos, k_max_len, prefix_len, vis_start, n_vis,
+                             n_q_heads, group, scale_log2, partial, m_max, dev_status);
   }
+  if (err != cudaSuccess) return TWIG_ERR_CUDA;
   if (cudaGetLastError() != cudaSuccess) return TWIG_ERR_CUDA;
   ttp_mq_reduce_kernel<<<dim3((m_max + 255) / 256, batch), 256, 0, st>>>(partial, n_blocks, n_q_heads, n_text_max,
       prefix_len, vis_start, n_vis, k_max_len, scores, m_max);
