@@ -5,6 +5,8 @@
   python -m paper_2503_14075_b200.profile_cases score  --workload 4 --iters 3
   python -m paper_2503_14075_b200.profile_cases accept --workload 2 --layers 32 --iters 3
   python -m paper_2503_14075_b200.profile_cases argmax --workload 4 --iters 3
+  python -m paper_2503_14075_b200.profile_cases gscore --workload 4 --iters 3
+  python -m paper_2503_14075_b200.profile_cases mqscore --workload 4 --iters 3
 
 Every case holds well under a few GB on the device and launches a handful of kernels, so
 that a profiler capture ends by itself.  Prints the mean launch time from CUDA events.
@@ -141,9 +143,41 @@ def case_argmax(a):
     print(f"argmax {wl.name} V={V}: {us:.2f} us/launch, {by / us / 1e3:.1f} GB/s algorithmic ({by} B/launch)")
 
 
+def case_gscore(a):
+    wl = synth.workload(a.workload)
+    rng = synth.rng_for(a.workload, 905)
+    pre = synth.make_prefill(wl, rng, n_layers=1)
+    B = wl.batch
+    q, k = _bf(pre["twig_q"]), _bf(pre["twig_k"])
+    qg, kg = _bf(synth.gate_bf16(rng, pre["twig_q"].shape)), _bf(synth.gate_bf16(rng, pre["twig_k"].shape))
+    scores = torch.zeros((B, max(wl.n_vis)), dtype=torch.float32, device=DEV)
+    ws = torch.empty(tw.twig_workspace_bytes(B, wl.n_q_heads, wl.head_dim, k.shape[2], 64), dtype=torch.uint8,
+                     device=DEV)
+    pl, vs, nv = _i32(pre["prefix_len"]), _i32(pre["vis_start"]), _i32(pre["n_vis"])
+    us = _time(lambda: tw.ttp_score_gated(q, qg, k, kg, pl, vs, nv, scores, ws), a.iters)
+    by = 2 * sum(wl.n_kv_heads * n * wl.head_dim * 2 for n in wl.n_vis)
+    print(f"gated score {wl.name}: {us:.2f} us per call (2 kernels), {by / us / 1e3:.1f} GB/s algorithmic ({by} B)")
+
+
+def case_mqscore(a):
+    wl = synth.workload(a.workload)
+    rng = synth.rng_for(a.workload, 906)
+    pre = synth.make_prefill(wl, rng, n_layers=1)
+    B, n_txt = wl.batch, max(1, max(wl.text_after))
+    k = _bf(pre["twig_k"])
+    qt = _bf(synth.normal_bf16(rng, (B, wl.n_q_heads, n_txt, wl.head_dim), wl.head_dim))
+    scores = torch.zeros((B, max(wl.n_vis)), dtype=torch.float32, device=DEV)
+    ws = torch.empty(tw.ttp_multiquery_workspace_bytes(B, wl.n_q_heads, n_txt, max(wl.n_vis)), dtype=torch.uint8, device=DEV)
+    pl, vs, nv = _i32(pre["prefix_len"]), _i32(pre["vis_start"]), _i32(pre["n_vis"])
+    us = _time(lambda: tw.ttp_score_multiquery(qt, k, pl, vs, nv, scores, ws), a.iters)
+    fl = sum(2 * wl.n_q_heads * wl.head_dim * c * (t + 2 * n + (c + 1) / 2)
+             for t, n, c in zip(wl.text_before, wl.n_vis, wl.text_after))
+    print(f"multi-query score {wl.name}: {us:.2f} us per call (2 kernels), {fl / us / 1e6:.1f} TFLOP/s algorithmic")
+
+
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("case", choices=["attn", "gather", "score", "accept", "argmax"])
+    ap.add_argument("case", choices=["attn", "gather", "score", "accept", "argmax", "gscore", "mqscore"])
     ap.add_argument("--workload", type=int, default=4)
     ap.add_argument("--kv-len", type=int, default=0)
     ap.add_argument("--layers", type=int, default=2)
@@ -152,7 +186,8 @@ def main():
     ap.add_argument("--splits", type=int, default=0, help="force key splits (0 auto)")
     ap.add_argument("--path", type=int, default=0, help="attention kernel: 0 auto, 1 mma.sync, 2 tcgen05")
     a = ap.parse_args()
-    {"attn": case_attn, "gather": case_gather, "score": case_score, "accept": case_accept, "argmax": case_argmax}[a.case](a)
+    {"attn": case_attn, "gather": case_gather, "score": case_score, "accept": case_accept, "argmax": case_argmax, "gscore": case_gscore,
+     "mqscore": case_mqscore}[a.case](a)
 
 
 if __name__ == "__main__":
