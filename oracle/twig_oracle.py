@@ -313,6 +313,64 @@ def base_argmax(logits, n_nodes):
 
 
 # --------------------------------------------------------------------------
+# Draft-side token tree (Sec. 4.3 "tree-based SSD", Appendix "Tree-based self-speculative decoding")
+# --------------------------------------------------------------------------
+def topk_tokens(logits_row, E: int):
+    """The E most probable tokens of one draft distribution, most probable first (equal logits:
+    lower token id first), with their log-probabilities log softmax(logits)[token]."""
+    x = np.asarray(logits_row, dtype=np.float64)
+    order = sorted(range(len(x)), key=lambda v: (-x[v], v))[:E]
+    mx = np.max(x)
+    lse = mx + np.log(np.sum(np.exp(x - mx)))
+    return np.array(order, dtype=np.int32), np.array([x[v] - lse for v in order], dtype=np.float64)
+
+
+def select_top_nodes(score, lo: int, hi: int, K: int):
+    """Node ids of the K highest scores among nodes lo..hi-1 (all of them if fewer), equal scores to
+    the lower id; returned ascending."""
+    ids = sorted(range(lo, hi), key=lambda i: (-score[i], i))[:K]
+    return sorted(ids)
+
+
+def build_token_tree(level_logits, E: int, K: int, n_max: int):
+    """The token tree of one request, level by level.  level_logits[l] is [rows_l, V]: row r of
+    level 0 is the draft distribution after the root (one row); row r of level l >= 1 is the draft
+    distribution after the r-th node selected for expansion at that level (ascending node id).
+    Level 1: the top-E tokens are the root's children.  Level l > 1: the K nodes of level l-1 with
+    the highest score are expanded into E children each.  A node's score is the log of the joint
+    probability of its root-to-node path (root: 0).  Finally the root and the n_max - 1 other nodes
+    with the highest scores are kept (equal scores: lower id, i.e. the ancestor first, so the kept
+    set is closed under parents) and renumbered in creation order.
+    Returns (parent [n], token [n] (root: -1), score [n], kept_old_ids [n]) of the pruned tree and
+    the full tree's (parent, token, score) for inspection."""
+    tok, par, sc = [-1], [-1], [0.0]
+    level_lo, level_hi = 0, 1
+    expand = [0]
+    for l, logits in enumerate(level_logits):
+        logits = np.asarray(logits)
+        assert logits.shape[0] >= len(expand)
+        new_lo = len(tok)
+        for r, u in enumerate(expand):
+            t, lp = topk_tokens(logits[r], E)
+            for e in range(len(t)):
+                tok.append(int(t[e]))
+                par.append(u)
+                sc.append(sc[u] + float(lp[e]))
+        level_lo, level_hi = new_lo, len(tok)
+        expand = select_top_nodes(sc, level_lo, level_hi, K)
+    keep = [0] + select_top_nodes(sc, 1, len(tok), max(0, n_max - 1))
+    new_id = {old: i for i, old in enumerate(keep)}
+    for old in keep[1:]:
+        if par[old] not in new_id:
+            raise ValueError("kept set is not closed under parents")
+    parent = np.array([-1] + [new_id[par[old]] for old in keep[1:]], dtype=np.int32)
+    token = np.array([tok[old] for old in keep], dtype=np.int32)
+    score = np.array([sc[old] for old in keep], dtype=np.float64)
+    full = (np.array(par, dtype=np.int32), np.array(tok, dtype=np.int32), np.array(sc, dtype=np.float64))
+    return parent, token, score, np.array(keep, dtype=np.int32), full
+
+
+# --------------------------------------------------------------------------
 # O6: append the accepted nodes' K/V rows to the cache
 # --------------------------------------------------------------------------
 def accept_compact(tree_k, tree_v, cache_k, cache_v, kv_len, paths):

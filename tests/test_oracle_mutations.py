@@ -23,6 +23,10 @@ MUTATIONS = [
     ("eq. 3 guide: not causal", "z = np.matmul(k[b, h // G, :t + 1, :], q_text[b, h, i, :]) * scale", "z = np.matmul(k[b, h // G, :lp, :], q_text[b, h, i, :]) * scale"),
     ("eq. 3 guide: query position off by one", "                t = vs + m + i\n", "                t = vs + m + i - 1\n"),
     ("eq. 3 guide: only the last text token", "for i in range(lp - vs - m):", "for i in range(lp - vs - m - 1, lp - vs - m):"),
+    ("tree: conditional instead of joint probability", "sc.append(sc[u] + float(lp[e]))", "sc.append(float(lp[e]))"),
+    ("tree: expansion picks the lowest scores", "ids = sorted(range(lo, hi), key=lambda i: (-score[i], i))[:K]", "ids = sorted(range(lo, hi), key=lambda i: (score[i], i))[:K]"),
+    ("tree: children attached to the root", "                par.append(u)\n", "                par.append(0)\n"),
+    ("tree: log-probability without the normaliser", "[x[v] - lse for v in order]", "[x[v] for v in order]"),
     ("top-k: ties to the higher index", "key=lambda m: (-s[m], m)", "key=lambda m: (-s[m], -m)"),
     ("top-k: smallest instead of largest", "key=lambda m: (-s[m], m)", "key=lambda m: (s[m], m)"),
     ("prune: text after the image dropped", "+ list(range(vis_start + n_vis, prefix_len))", ""),

@@ -560,6 +560,60 @@ def test_base_argmax_library_and_ties():
     assert np.array_equal(O.base_argmax(z, [4]), O.base_argmax(sp.softmax(z, axis=-1), [4]))
 
 
+def test_token_tree_pins():
+    """Tree builder: enumeration of every path of a tiny vocabulary; chain and full-tree limits;
+    tie rules; closure under parents."""
+    import itertools, math
+    rng = np.random.default_rng(29)
+    V, E, K, D = 5, 2, 2, 3
+    levels = [rng.standard_normal((1, V))] + [rng.standard_normal((K, V)) for _ in range(D - 1)]
+    parent, token, score, keep, (fpar, ftok, fsc) = O.build_token_tree(levels, E, K, n_max=100)
+    # (a) sizes: 1 + E + (D-1) K E, nothing pruned
+    assert len(fpar) == 1 + E + (D - 1) * K * E == len(parent)
+    # (b) every node's score is the log joint probability of its path, recomputed with plain math
+    def softmax(row):
+        m = max(row)
+        z = [math.exp(x - m) for x in row]
+        return [x / sum(z) for x in z]
+    # replay: which row fed which node
+    row_of = {0: (0, 0)}                      # node -> (level, row) of the distribution after it
+    lo, hi = 1, 1 + E
+    for l in range(1, D):
+        sel = sorted(sorted(range(lo, hi), key=lambda i: (-fsc[i], i))[:K])
+        for r, u in enumerate(sel):
+            row_of[u] = (l, r)
+        lo, hi = hi, hi + K * E
+    for i in range(1, len(fpar)):
+        l, r = row_of[int(fpar[i])]
+        p = softmax(list(levels[l][r]))
+        assert math.isclose(fsc[i], fsc[fpar[i]] + math.log(p[ftok[i]]), rel_tol=1e-12, abs_tol=1e-12)
+        # children of a node are its top-E tokens
+        sibs = [int(ftok[j]) for j in range(1, len(fpar)) if fpar[j] == fpar[i]]
+        assert sorted(sibs, key=lambda v: (-levels[l][r][v], v)) == sorted(range(V), key=lambda v: (-levels[l][r][v], v))[:E]
+    # (c) pruning to n_max keeps the root and the n_max - 1 highest joint probabilities, parents included
+    for n_max in (1, 2, 4, 7):
+        p2, t2, s2, keep2, _ = O.build_token_tree(levels, E, K, n_max)
+        best = sorted(range(1, len(fsc)), key=lambda i: (-fsc[i], i))[:n_max - 1]
+        assert sorted(keep2.tolist()) == sorted([0] + best)
+        assert p2[0] == -1 and all(0 <= p2[i] < i for i in range(1, len(p2)))
+        for i in range(1, len(p2)):
+            assert keep2[p2[i]] == fpar[keep2[i]]          # the renumbered parent is the old parent
+    # (d) E = K = 1: the chain of greedy tokens of the rows
+    chain = O.build_token_tree([lv[:1] for lv in levels], 1, 1, 100)
+    assert chain[0].tolist() == [-1, 0, 1, 2] and chain[1].tolist() == [-1] + [int(np.argmax(lv[0])) for lv in levels]
+    # (e) ties: equal logits go to the lower token id, equal scores to the lower node id
+    flat = [np.zeros((1, 4)), np.zeros((2, 4))]
+    p3, t3, s3, keep3, (fp3, ft3, fs3) = O.build_token_tree(flat, 2, 2, 4)
+    assert ft3.tolist() == [-1, 0, 1, 0, 1, 0, 1] and fp3.tolist() == [-1, 0, 0, 1, 1, 2, 2]
+    assert keep3.tolist() == [0, 1, 2, 3]                    # level 1 (higher score) first, then the lowest id
+    # (f) top-E log-probabilities against scipy
+    import scipy.special as sp
+    x = rng.standard_normal(50)
+    t, lp = O.topk_tokens(x, 5)
+    assert t.tolist() == np.argsort(-x, kind="stable")[:5].tolist()
+    assert np.allclose(lp, sp.log_softmax(x)[t], rtol=1e-12)
+
+
 # ---------------------------------------------------------------- O6 accept-compact
 def test_accept_compact_tail_rows_and_canaries():
     nl, B, H, T, L, d = 2, 2, 2, 5, 12, 3
