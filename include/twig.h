@@ -269,6 +269,46 @@ int32_t twig_set_early_prefix(int32_t on);
  * 1, 2, 4 or 8; 0 = automatic (default).  A tuning control.  Returns the previous value. */
 int32_t twig_set_attention_splits(int32_t splits);
 
+/* ---- Draft-side token tree ---------------------------------------------------
+ * Sec. 4.3 and the appendix's "Tree-based self-speculative decoding": the tree is rooted at the last
+ * accepted token and grown level by level with an expansion width E, a selection width K and a
+ * depth D; level 1 holds the root's top-E tokens, at every later level the K best nodes of the level
+ * before are expanded into their top-E tokens; the finished tree is cut to N_max nodes.  The draft
+ * model runs between these calls (its logits are inputs).  A node's score is the log of the joint
+ * probability of its root-to-node path; "best" is by score, equal scores to the lower node id, equal
+ * logits to the lower token id.  Logits must not be NaN.
+ *
+ * Tree state of request b: node_tok / node_parent / node_score [batch, cap], node 0 the root, nodes in
+ * creation order (level 1 at 1..E, each later level after it).  tree_reset writes the roots.
+ *
+ * tree_expand_level: row r of logits ([batch, rows, vocab] at (b*rows + r)*row_stride ELEMENTS, bf16 or
+ *   fp32, rows 16-byte aligned) is the draft distribution after node src_node[b, r] (-1: unused row);
+ *   its n_children (<= 16) most probable tokens become nodes level_base + r*n_children + e, best
+ *   first, with score = score[src] + log softmax(row)[token].  level_base = first node id of the new
+ *   level (1 for level 1); every src must be older than level_base (else TWIG_DEV_BAD_TREE).
+ * tree_select_expansion: expand_node[b, 0..n_select) = ids of the n_select best nodes among
+ *   level_lo..level_hi-1, ascending: the src_node of the next tree_expand_level.  n_select may not
+ *   exceed the level's size (TWIG_ERR_SHAPE), so that every row of the next level has a node.
+ * tree_finalize: keeps the root and the n_max - 1 best of the nodes 1..n_built-1 (a set closed under
+ *   parents, since a child's score never exceeds its parent's), renumbers them in creation order and
+ *   writes parent / draft_tok [batch, t_max] (root: parent -1, token -1; unused entries -1 / 0) and
+ *   n_nodes[b]: the arrays tree_verify_attention and tree_accept_compact take.  kept_node (optional)
+ *   [batch, t_max]: the state id of every kept node.  n_max <= t_max <= TWIG_MAX_NODES; cap <= 6144.
+ */
+twig_status tree_reset(int32_t *node_tok, int32_t *node_parent, float *node_score, int32_t cap,
+                       int32_t batch, void *stream);
+twig_status tree_expand_level(const void *logits, int32_t logits_fp32, int64_t row_stride, int32_t vocab,
+                              int32_t rows, const int32_t *src_node, int32_t n_children, int32_t level_base,
+                              int32_t *node_tok, int32_t *node_parent, float *node_score, int32_t cap,
+                              int32_t batch, int32_t *dev_status, void *stream);
+twig_status tree_select_expansion(const float *node_score, int32_t cap, int32_t level_lo, int32_t level_hi,
+                                  int32_t n_select, int32_t *expand_node, int32_t batch,
+                                  int32_t *dev_status, void *stream);
+twig_status tree_finalize(const int32_t *node_tok, const int32_t *node_parent, const float *node_score,
+                          int32_t cap, int32_t n_built, int32_t n_max, int32_t *parent, int32_t *draft_tok,
+                          int32_t *n_nodes, int32_t *kept_node, int32_t t_max, int32_t batch,
+                          int32_t *dev_status, void *stream);
+
 /* ---- Greedy target token of every tree node (input of tree_accept_compact) -----
  * Algorithm 2 ("argmax(tgt_probs[...])"), Sec. 5.4: base_argmax[b, i] = the index of the largest of
  * logits[b, i, 0..vocab), the LOWEST index among equal values, for i < n_nodes[b]; other entries

@@ -1,0 +1,313 @@
+// Draft-side token tree of tree-based self-speculative decoding (Sec. 4.3; Appendix, "Tree-based
+// self-speculative decoding"): level by level, every node selected for expansion gets its E most
+// probable next tokens as children; the K best nodes of a level are expanded at the next; at the end
+// the tree is cut to N_max nodes.  A node's score is the log of the joint probability of its path.
+// The draft model itself runs between these calls: its logits are inputs.
+//
+// Tree state per request (capacity `cap` nodes, node 0 = root): token, parent, score, all in
+// creation order (a parent always precedes its children).
+#include "twig_common.cuh"
+
+namespace twig {
+
+namespace {
+
+constexpr int kTopThreads = 256;
+constexpr int kMaxE = 16;            // children per expanded node
+constexpr int kSelThreads = 256;
+
+// (value, index) order of the top lists: larger value first, equal values: lower index first
+__device__ __forceinline__ bool comes_first(float v, int i, float w, int j) { return v > w || (v == w && i < j); }
+
+// One CTA per (expansion slot, request): log-sum-exp of the row and its E largest logits.
+template <bool FP32>
+__global__ void __launch_bounds__(kTopThreads)
+tree_expand_kernel(const void *__restrict__ logits, long long row_stride, int vocab, int rows,
+                   const int *__restrict__ src_node, int E, int level_base, int cap,
+                   int *__restrict__ node_tok, int *__restrict__ node_parent, float *__restrict__ node_score,
+                   int *dev_status) {
+  constexpr int EPC = FP32 ? 4 : 8;
+  __shared__ float s_v[kTopThreads / 32];
+  __shared__ int s_i[kTopThreads / 32];
+  __shared__ float s_m[kTopThreads / 32], s_s[kTopThreads / 32];
+  __shared__ float s_top_v[kMaxE];
+  __shared__ int s_top_i[kMaxE];
+  __shared__ int s_winner;
+  const int r = blockIdx.x, b = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int u = src_node[(long long)b * rows + r];
+  if (u < 0) return;                                       // unused slot
+  const int first = level_base + r * E;
+  if (u >= level_base || first + E > cap) {
+    if (tid == 0) flag_status(dev_status, b, TWIG_DEV_BAD_TREE);
+    return;
+  }
+  const unsigned char *row = static_cast<const unsigned char *>(logits) +
+                             ((long long)b * rows + r) * row_stride * (FP32 ? 4 : 2);
+  // per-thread: running (max, sum of exp) and the thread's own top list, best first
+  float tv[kMaxE];
+  int ti[kMaxE];
+#pragma unroll
+  for (int e = 0; e < kMaxE; ++e) {
+    tv[e] = -INFINITY;
+    ti[e] = 0x7fffffff;
+  }
+  float m = -INFINITY, s = 0.f;
+  auto take = [&](float v, int i) {
+    if (v > m) {
+      s = s * __expf(m - v) + 1.f;          // (m = -inf: s is 0)
+      m = v;
+    } else {
+      s += __expf(v - m);
+    }
+    if (comes_first(v, i, tv[kMaxE - 1], ti[kMaxE - 1])) {
+      // insert: bubble the newcomer up from the tail
+      tv[kMaxE - 1] = v;
+      ti[kMaxE - 1] = i;
+#pragma unroll
+      for (int e = kMaxE - 1; e > 0; --e) {
+        if (comes_first(tv[e], ti[e], tv[e - 1], ti[e - 1])) {
+          const float fv = tv[e];
+          tv[e] = tv[e - 1];
+          tv[e - 1] = fv;
+          const int fi = ti[e];
+          ti[e] = ti[e - 1];
+          ti[e - 1] = fi;
+        }
+      }
+    }
+  };
+  const int chunks = vocab / EPC;
+  for (int c = tid; c < chunks; c += kTopThreads) {
+    const uint4 w = ld_nc_16(row + (long long)c * 16);
+    const int base = c * EPC;
+    if (FP32) {
+      take(__uint_as_float(w.x), base);
+      take(__uint_as_float(w.y), base + 1);
+      take(__uint_as_float(w.z), base + 2);
+      take(__uint_as_float(w.w), base + 3);
+    } else {
+      take(bf16_lo(w.x), base);
+      take(bf16_hi(w.x), base + 1);
+      take(bf16_lo(w.y), base + 2);
+      take(bf16_hi(w.y), base + 3);
+      take(bf16_lo(w.z), base + 4);
+      take(bf16_hi(w.z), base + 5);
+      take(bf16_lo(w.w), base + 6);
+      take(bf16_hi(w.w), base + 7);
+    }
+  }
+  for (int i = chunks * EPC + tid; i < vocab; i += kTopThreads)
+    take(FP32 ? reinterpret_cast<const float *>(row)[i]
+              : __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(row)[i]), i);
+
+  // ---- log-sum-exp of the row ----
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float om = __shfl_xor_sync(0xffffffffu, m, o), os = __shfl_xor_sync(0xffffffffu, s, o);
+    const float nm = fmaxf(m, om);
+    s = (m == -INFINITY ? 0.f : s * __expf(m - nm)) + (om == -INFINITY ? 0.f : os * __expf(om - nm));
+    m = nm;
+  }
+  if (lane == 0) {
+    s_m[warp] = m;
+    s_s[warp] = s;
+  }
+  __syncthreads();
+  float M = -INFINITY;
+  for (int w = 0; w < kTopThreads / 32; ++w) M = fmaxf(M, s_m[w]);
+  float S = 0.f;
+  for (int w = 0; w < kTopThreads / 32; ++w) S += s_m[w] == -INFINITY ? 0.f : s_s[w] * __expf(s_m[w] - M);
+  const float lse = M + logf(S);
+
+  // ---- E rounds: the best head among all threads' lists wins and is popped ----
+  for (int e = 0; e < E; ++e) {
+    float bv = tv[0];
+    int bi = ti[0];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+      const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+      if (comes_first(ov, oi, bv, bi)) {
+        bv = ov;
+        bi = oi;
+      }
+    }
+    if (lane == 0) {
+      s_v[warp] = bv;
+      s_i[warp] = bi;
+    }
+    __syncthreads();
+    if (tid == 0) {
+      for (int w = 1; w < kTopThreads / 32; ++w)
+        if (comes_first(s_v[w], s_i[w], bv, bi)) {
+          bv = s_v[w];
+          bi = s_i[w];
+        }
+      s_top_v[e] = bv;
+      s_top_i[e] = bi;
+      s_winner = bi;
+    }
+    __syncthreads();
+    if (ti[0] == s_winner) {              // token ids are unique: exactly one thread pops
+#pragma unroll
+      for (int k = 0; k < kMaxE - 1; ++k) {
+        tv[k] = tv[k + 1];
+        ti[k] = ti[k + 1];
+      }
+      tv[kMaxE - 1] = -INFINITY;
+      ti[kMaxE - 1] = 0x7fffffff;
+    }
+  }
+  if (tid < E) {
+    const long long at = (long long)b * cap + first + tid;
+    node_tok[at] = s_top_i[tid];
+    node_parent[at] = u;
+    node_score[at] = node_score[(long long)b * cap + u] + (s_top_v[tid] - lse);
+  }
+}
+
+// One CTA per request.  Ranks the nodes lo..hi-1 by (score desc, id asc) and takes the first `take`:
+//  * expansion mode (parent_out == nullptr): their ids, ascending, to sel_out[b, 0..take) (-1 padded);
+//  * final mode: the root and the selected nodes are renumbered in creation order and written as
+//    parent_out / tok_out [b, t_max] with n_nodes_out[b]; kept_out[b, i] = the old id of new node i.
+__global__ void __launch_bounds__(kSelThreads)
+tree_select_kernel(const float *__restrict__ node_score, const int *__restrict__ node_tok,
+                   const int *__restrict__ node_parent, int cap, int lo, int hi, int take,
+                   int *__restrict__ sel_out, int sel_stride, int *__restrict__ parent_out,
+                   int *__restrict__ tok_out, int *__restrict__ n_nodes_out, int *__restrict__ kept_out,
+                   int t_max, int *dev_status) {
+  extern __shared__ unsigned char sel_smem[];
+  float *sc = reinterpret_cast<float *>(sel_smem);                 // [hi]
+  int *new_id = reinterpret_cast<int *>(sel_smem) + cap;           // [hi]: position among the kept, or -1
+  const int b = blockIdx.x, tid = threadIdx.x;
+  const float *score = node_score + (long long)b * cap;
+  for (int i = tid; i < hi; i += kSelThreads) {
+    sc[i] = score[i];
+    new_id[i] = -1;
+  }
+  __syncthreads();
+  const bool final_mode = parent_out != nullptr;
+  for (int i = lo + tid; i < hi; i += kSelThreads) {
+    int rank = 0;
+    const float v = sc[i];
+    for (int j = lo; j < hi; ++j) rank += comes_first(sc[j], j, v, i) ? 1 : 0;
+    if (rank < take) new_id[i] = 0;                                // selected (position follows)
+  }
+  if (final_mode && tid == 0) new_id[0] = 0;                       // the root is always kept
+  __syncthreads();
+  const int from = final_mode ? 0 : lo;
+  for (int i = from + tid; i < hi; i += kSelThreads) {
+    if (new_id[i] < 0) continue;
+    int pos = 0;
+    for (int j = from; j < i; ++j) pos += new_id[j] >= 0 ? 1 : 0;
+    // (positions are written after every thread has counted)
+    sc[i] = __int_as_float(pos);
+  }
+  __syncthreads();
+  for (int i = from + tid; i < hi; i += kSelThreads)
+    if (new_id[i] >= 0) new_id[i] = __float_as_int(sc[i]);
+  __syncthreads();
+  if (!final_mode) {
+    for (int k = tid; k < sel_stride; k += kSelThreads) sel_out[(long long)b * sel_stride + k] = -1;
+    __syncthreads();
+    for (int i = lo + tid; i < hi; i += kSelThreads)
+      if (new_id[i] >= 0 && new_id[i] < sel_stride) sel_out[(long long)b * sel_stride + new_id[i]] = i;
+    return;
+  }
+  int total = 0;
+  for (int j = 0; j < hi; ++j) total += new_id[j] >= 0 ? 1 : 0;    // (hi <= a few hundred)
+  if (tid == 0) n_nodes_out[b] = total;
+  for (int k = total + tid; k < t_max; k += kSelThreads) {
+    parent_out[(long long)b * t_max + k] = -1;
+    tok_out[(long long)b * t_max + k] = 0;
+    if (kept_out) kept_out[(long long)b * t_max + k] = -1;
+  }
+  for (int i = tid; i < hi; i += kSelThreads) {
+    const int ni = new_id[i];
+    if (ni < 0) continue;
+    int np = -1;
+    if (i > 0) {
+      np = new_id[node_parent[(long long)b * cap + i]];
+      if (np < 0) flag_status(dev_status, b, TWIG_DEV_BAD_TREE);   // kept set not closed under parents
+    }
+    parent_out[(long long)b * t_max + ni] = np;
+    tok_out[(long long)b * t_max + ni] = i > 0 ? node_tok[(long long)b * cap + i] : -1;
+    if (kept_out) kept_out[(long long)b * t_max + ni] = i;
+  }
+}
+
+}  // namespace
+
+}  // namespace twig
+
+using namespace twig;
+
+extern "C" twig_status tree_reset(int32_t *node_tok, int32_t *node_parent, float *node_score, int32_t cap,
+                                  int32_t batch, void *stream) {
+  if (!node_tok || !node_parent || !node_score) return TWIG_ERR_NULL;
+  if (cap <= 0 || batch <= 0) return TWIG_ERR_SHAPE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // node 0 of every request: token -1, parent -1, score 0 (the other entries are written before they are read)
+  if (cudaMemset2DAsync(node_tok, (size_t)cap * 4, 0xff, 4, batch, st) != cudaSuccess) return TWIG_ERR_CUDA;
+  if (cudaMemset2DAsync(node_parent, (size_t)cap * 4, 0xff, 4, batch, st) != cudaSuccess) return TWIG_ERR_CUDA;
+  if (cudaMemset2DAsync(node_score, (size_t)cap * 4, 0, 4, batch, st) != cudaSuccess) return TWIG_ERR_CUDA;
+  return TWIG_OK;
+}
+
+extern "C" twig_status tree_expand_level(const void *logits, int32_t logits_fp32, int64_t row_stride,
+                                         int32_t vocab, int32_t rows, const int32_t *src_node, int32_t n_children,
+                                         int32_t level_base, int32_t *node_tok, int32_t *node_parent,
+                                         float *node_score, int32_t cap, int32_t batch, int32_t *dev_status,
+                                         void *stream) {
+  if (!logits || !src_node || !node_tok || !node_parent || !node_score) return TWIG_ERR_NULL;
+  if (vocab <= 0 || rows <= 0 || batch <= 0 || cap <= 0 || level_base <= 0 || row_stride < vocab) return TWIG_ERR_SHAPE;
+  if (n_children <= 0 || n_children > kMaxE || n_children > vocab) return TWIG_ERR_UNSUPPORTED;
+  if (batch > TWIG_MAX_BATCH || rows > 65535) return TWIG_ERR_UNSUPPORTED;
+  if (level_base + (long long)rows * n_children > cap) return TWIG_ERR_SHAPE;
+  const int esz = logits_fp32 ? 4 : 2;
+  if (!aligned16(logits) || (row_stride * esz) % 16) return TWIG_ERR_ALIGN;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  dim3 grid(rows, batch);
+  if (logits_fp32)
+    tree_expand_kernel<true><<<grid, kTopThreads, 0, st>>>(logits, row_stride, vocab, rows, src_node, n_children,
+        level_base, cap, node_tok, node_parent, node_score, dev_status);
+  else
+    tree_expand_kernel<false><<<grid, kTopThreads, 0, st>>>(logits, row_stride, vocab, rows, src_node, n_children,
+        level_base, cap, node_tok, node_parent, node_score, dev_status);
+  return launch_status();
+}
+
+static twig_status launch_select(const float *node_score, const int32_t *node_tok, const int32_t *node_parent,
+                                 int cap, int lo, int hi, int take, int *sel_out, int sel_stride, int *parent_out,
+                                 int *tok_out, int *n_nodes_out, int *kept_out, int t_max, int batch,
+                                 int *dev_status, cudaStream_t st) {
+  const size_t smem = (size_t)cap * 8;
+  if (smem > 48 * 1024) return TWIG_ERR_UNSUPPORTED;
+  tree_select_kernel<<<batch, kSelThreads, smem, st>>>(node_score, node_tok, node_parent, cap, lo, hi, take, sel_out,
+                                                       sel_stride, parent_out, tok_out, n_nodes_out, kept_out, t_max,
+                                                       dev_status);
+  return launch_status();
+}
+
+extern "C" twig_status tree_select_expansion(const float *node_score, int32_t cap, int32_t level_lo, int32_t level_hi,
+                                             int32_t n_select, int32_t *expand_node, int32_t batch,
+                                             int32_t *dev_status, void *stream) {
+  if (!node_score || !expand_node) return TWIG_ERR_NULL;
+  if (cap <= 0 || batch <= 0 || n_select <= 0 || level_lo < 0 || level_hi <= level_lo || level_hi > cap)
+    return TWIG_ERR_SHAPE;
+  if (batch > TWIG_MAX_BATCH) return TWIG_ERR_UNSUPPORTED;
+  if (n_select > level_hi - level_lo) return TWIG_ERR_SHAPE;     // every expansion row gets a node
+  return launch_select(node_score, nullptr, nullptr, cap, level_lo, level_hi, n_select, expand_node, n_select, nullptr,
+                       nullptr, nullptr, nullptr, 0, batch, dev_status, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" twig_status tree_finalize(const int32_t *node_tok, const int32_t *node_parent, const float *node_score,
+                                     int32_t cap, int32_t n_built, int32_t n_max, int32_t *parent, int32_t *draft_tok,
+                                     int32_t *n_nodes, int32_t *kept_node, int32_t t_max, int32_t batch,
+                                     int32_t *dev_status, void *stream) {
+  if (!node_tok || !node_parent || !node_score || !parent || !draft_tok || !n_nodes) return TWIG_ERR_NULL;
+  if (cap <= 0 || batch <= 0 || n_built <= 0 || n_built > cap || n_max <= 0 || t_max <= 0) return TWIG_ERR_SHAPE;
+  if (n_max > t_max || t_max > TWIG_MAX_NODES || batch > TWIG_MAX_BATCH) return TWIG_ERR_UNSUPPORTED;
+  return launch_select(node_score, node_tok, node_parent, cap, 1, n_built, n_max - 1, nullptr, 0, parent, draft_tok,
+                       n_nodes, kept_node, t_max, batch, dev_status, static_cast<cudaStream_t>(stream));
+}

@@ -27,7 +27,7 @@ DEV_OK, DEV_BAD_LAYOUT, DEV_BAD_KEEP, DEV_BAD_INDEX, DEV_BAD_TREE, DEV_OVERFLOW,
 MAX_NODES, MAX_VISUAL, MAX_BATCH = 64, 16384, 4096
 
 EXPORTS = ["twig_status_str", "twig_set_launch_overlap", "twig_set_early_prefix", "twig_set_attention_path", "twig_set_attention_splits", "twig_workspace_bytes", "ttp_score", "ttp_score_gated", "ttp_multiquery_workspace_bytes", "ttp_score_multiquery", "ttp_score_noalloc", "ttp_topk", "ttp_compact", "ttp_compact_rows",
-           "ttp_score_topk_compact", "tree_verify_attention", "tree_base_argmax", "tree_accept_compact"]
+           "ttp_score_topk_compact", "tree_verify_attention", "tree_reset", "tree_expand_level", "tree_select_expansion", "tree_finalize", "tree_base_argmax", "tree_accept_compact"]
 
 
 class TwigError(RuntimeError):
@@ -97,6 +97,14 @@ _lib.ttp_score_topk_compact.argtypes = [_vp, _vp, _i64, _i64, _i64, _i32, _vp, _
 _lib.tree_verify_attention.restype = C.c_int
 _lib.tree_verify_attention.argtypes = [_vp, _vp, _vp, _kvp, _i32, _vp, _vp, _vp, _i32, _i32, _f32, _vp, _vp,
                                        _vp, _vp, _sz, _vp]
+_lib.tree_reset.restype = C.c_int
+_lib.tree_reset.argtypes = [_vp, _vp, _vp, _i32, _i32, _vp]
+_lib.tree_expand_level.restype = C.c_int
+_lib.tree_expand_level.argtypes = [_vp, _i32, _i64, _i32, _i32, _vp, _i32, _i32, _vp, _vp, _vp, _i32, _i32, _vp, _vp]
+_lib.tree_select_expansion.restype = C.c_int
+_lib.tree_select_expansion.argtypes = [_vp, _i32, _i32, _i32, _i32, _vp, _i32, _vp, _vp]
+_lib.tree_finalize.restype = C.c_int
+_lib.tree_finalize.argtypes = [_vp, _vp, _vp, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _i32, _i32, _vp, _vp]
 _lib.tree_base_argmax.restype = C.c_int
 _lib.tree_base_argmax.argtypes = [_vp, _i32, _i64, _i32, _vp, _i32, _i32, _vp, _vp, _vp]
 _lib.tree_accept_compact.restype = C.c_int
@@ -245,6 +253,44 @@ def tree_verify_attention(q, tree_k, tree_v, cache: KV, layer, kv_len, n_nodes, 
     _check(_lib.tree_verify_attention(_p(q), _p(tree_k), _p(tree_v), C.byref(cache), layer, _p(kv_len),
                                       _p(n_nodes), _p(parent), T, Hq, softmax_scale, _p(out), _p(lse),
                                       _p(dev_status), _p(ws), ws_bytes, _stream(stream)))
+
+
+class TreeState:
+    """Device arrays of the token trees under construction: node_tok / node_parent (int32) and
+    node_score (fp32), [batch, cap] each."""
+
+    def __init__(self, batch, cap, device):
+        self.batch, self.cap = batch, cap
+        self.tok = torch.empty((batch, cap), dtype=torch.int32, device=device)
+        self.parent = torch.empty((batch, cap), dtype=torch.int32, device=device)
+        self.score = torch.empty((batch, cap), dtype=torch.float32, device=device)
+
+
+def tree_reset(state: TreeState, stream=None):
+    _check(_lib.tree_reset(_p(state.tok), _p(state.parent), _p(state.score), state.cap, state.batch, _stream(stream)))
+
+
+def tree_expand_level(logits, src_node, n_children, level_base, state: TreeState, dev_status=None, stream=None):
+    """logits [B, rows, V] bf16 or fp32 (last dim contiguous); src_node [B, rows] int32 (-1: unused row)."""
+    B, rows, V = logits.shape
+    assert logits.stride(2) == 1 and logits.stride(0) == rows * logits.stride(1)
+    _check(_lib.tree_expand_level(_p(logits), 1 if logits.dtype == torch.float32 else 0, logits.stride(1), V, rows,
+                                  _p(src_node), n_children, level_base, _p(state.tok), _p(state.parent), _p(state.score),
+                                  state.cap, B, _p(dev_status), _stream(stream)))
+
+
+def tree_select_expansion(state: TreeState, level_lo, level_hi, expand_node, dev_status=None, stream=None):
+    """expand_node [B, K] int32 (out): the K best nodes of level_lo..level_hi-1, ascending, -1 padded."""
+    _check(_lib.tree_select_expansion(_p(state.score), state.cap, level_lo, level_hi, expand_node.shape[1],
+                                      _p(expand_node), state.batch, _p(dev_status), _stream(stream)))
+
+
+def tree_finalize(state: TreeState, n_built, n_max, parent, draft_tok, n_nodes, kept_node=None, dev_status=None,
+                  stream=None):
+    """parent, draft_tok [B, t_max], n_nodes [B] int32 (out): the pruned trees in verification layout."""
+    _check(_lib.tree_finalize(_p(state.tok), _p(state.parent), _p(state.score), state.cap, n_built, n_max, _p(parent),
+                              _p(draft_tok), _p(n_nodes), _p(kept_node), parent.shape[1], state.batch, _p(dev_status),
+                              _stream(stream)))
 
 
 def tree_base_argmax(logits, n_nodes, base_argmax, dev_status=None, stream=None):

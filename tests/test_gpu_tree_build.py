@@ -1,0 +1,112 @@
+"""GPU parity: the draft-side token tree (top-E expansion, top-K selection, pruning to N_max)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import twig_oracle as O
+from paper_2503_14075_b200 import synth
+from gpu_common import DEV, dev_bf16, dev_i32
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def tw():
+    from paper_2503_14075_b200 import twig
+    return twig
+
+
+def gpu_tree(tw, level_logits_dev, E, K, n_max, t_max):
+    """Drives the four entry points for a whole batch; returns host arrays."""
+    B = level_logits_dev[0].shape[0]
+    D = len(level_logits_dev)
+    cap = 1 + E + (D - 1) * K * E
+    st = tw.TreeState(B, cap, DEV)
+    st.tok.fill_(-77)
+    st.parent.fill_(-77)
+    st.score.fill_(float("nan"))
+    status = torch.zeros(B, dtype=torch.int32, device=DEV)
+    tw.tree_reset(st)
+    src = torch.zeros((B, 1), dtype=torch.int32, device=DEV)
+    lo, hi = 0, 1
+    for l in range(D):
+        rows = level_logits_dev[l].shape[1]
+        if src.shape[1] < rows:                       # unused rows
+            pad = torch.full((B, rows - src.shape[1]), -1, dtype=torch.int32, device=DEV)
+            src = torch.cat([src, pad], dim=1).contiguous()
+        tw.tree_expand_level(level_logits_dev[l], src, E, hi, st, dev_status=status)
+        lo, hi = hi, hi + (1 if l == 0 else K) * E
+        if l + 1 < D:
+            src = torch.full((B, K), -5, dtype=torch.int32, device=DEV)
+            tw.tree_select_expansion(st, lo, min(hi, cap), src, dev_status=status)
+    parent = torch.full((B, t_max), -9, dtype=torch.int32, device=DEV)
+    tok = torch.full((B, t_max), -9, dtype=torch.int32, device=DEV)
+    n_nodes = torch.full((B,), -9, dtype=torch.int32, device=DEV)
+    kept = torch.full((B, t_max), -9, dtype=torch.int32, device=DEV)
+    tw.tree_finalize(st, cap, n_max, parent, tok, n_nodes, kept_node=kept, dev_status=status)
+    torch.cuda.synchronize()
+    return (parent.cpu().numpy(), tok.cpu().numpy(), n_nodes.cpu().numpy(), kept.cpu().numpy(), status.cpu().numpy(),
+            st.score.cpu().numpy())
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "fp32"])
+@pytest.mark.parametrize("cfg", [(10, 10, 4, 60, 64, 32000), (3, 2, 3, 7, 8, 1003), (16, 4, 2, 64, 64, 4096), (1, 1, 5, 6, 6, 77)],
+                         ids=["paper-default", "small-ragged", "wide", "chain"])
+def test_token_tree_matches_oracle(tw, cfg, dtype):
+    E, K, D, n_max, t_max, V = cfg
+    B = 3
+    rng = synth.rng_for(7, 21)
+    stride = (V + 7) // 8 * 8
+    host, dev = [], []
+    for l in range(D):
+        rows = 1 if l == 0 else K
+        x = (rng.standard_normal((B, rows, V)) * 3.0).astype(np.float32)
+        if dtype == "bf16":
+            bits = synth.f32_to_bf16(x)
+            padded = np.full((B, rows, stride), 0x7F7F, dtype=bits.dtype)          # a huge value nobody may read
+            padded[..., :V] = bits
+            dev.append(dev_bf16(padded)[..., :V])
+            host.append(synth.bf16_to_f64(bits))
+        else:
+            padded = np.full((B, rows, stride), 3e38, dtype=np.float32)
+            padded[..., :V] = x
+            dev.append(torch.from_numpy(padded).to(DEV)[..., :V])
+            host.append(x.astype(np.float64))
+    parent, tok, n_nodes, kept, status, score = gpu_tree(tw, dev, E, K, n_max, t_max)
+    assert not status.any()
+    for b in range(B):
+        p_o, t_o, s_o, keep_o, (fp, ft, fs) = O.build_token_tree([h[b] for h in host], E, K, n_max)
+        # (scores are fp32 on the GPU and fp64 in the oracle; the seeded rows have no near-ties at a selection
+        # boundary, exact ties are covered by test_token_tree_ties)
+        n = len(p_o)
+        assert n_nodes[b] == n
+        assert np.array_equal(kept[b, :n], keep_o)
+        assert np.array_equal(parent[b, :n], p_o) and np.array_equal(tok[b, :n], t_o)
+        assert np.all(parent[b, n:] == -1) and np.all(tok[b, n:] == 0) and np.all(kept[b, n:] == -1)
+        assert np.allclose(score[b, :len(fs)], fs, rtol=0, atol=2e-4 * D)
+
+
+def test_token_tree_ties(tw):
+    """Equal logits go to the lower token id, equal scores to the lower node id (exact ties: rows that are
+    bit-identical give bit-identical scores)."""
+    E, K, D, n_max, t_max, V = 2, 2, 2, 4, 8, 64
+    flat = [torch.zeros((1, 1, V), dtype=torch.float32, device=DEV), torch.zeros((1, K, V), dtype=torch.float32, device=DEV)]
+    parent, tok, n_nodes, kept, status, _ = gpu_tree(tw, flat, E, K, n_max, t_max)
+    p_o, t_o, _, keep_o, _ = O.build_token_tree([np.zeros((1, V)), np.zeros((K, V))], E, K, n_max)
+    assert not status.any() and n_nodes[0] == 4
+    assert kept[0, :4].tolist() == keep_o.tolist() == [0, 1, 2, 3]
+    assert parent[0, :4].tolist() == p_o.tolist() and tok[0, :4].tolist() == t_o.tolist() == [-1, 0, 1, 0]
+
+
+def test_tree_feeds_verification(tw):
+    """The finalised arrays are valid inputs of the verification side: parents precede children."""
+    E, K, D, n_max, t_max, V = 4, 3, 3, 20, 32, 512
+    rng = synth.rng_for(7, 22)
+    dev = [torch.from_numpy(rng.standard_normal((2, 1 if l == 0 else K, V)).astype(np.float32)).to(DEV) for l in range(D)]
+    parent, tok, n_nodes, kept, status, _ = gpu_tree(tw, dev, E, K, n_max, t_max)
+    assert not status.any()
+    for b in range(2):
+        n = int(n_nodes[b])
+        assert n == n_max and parent[b, 0] == -1
+        assert all(0 <= parent[b, i] < i for i in range(1, n))
+        O.tree_mask(parent[b, :n], n, 5)               # the oracle accepts it as a tree
