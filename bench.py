@@ -598,6 +598,41 @@ def extra_rooflines(torch, tw, peaks, dev):
     torch.cuda.synchronize()
     us = e0.elapsed_time(e1) * 1e3 / n_chain
     res["base_argmax_c3_V32000"] = hbm_entry(us, int(sum(wl3.n_nodes)) * V * 2)
+    # draft-side token tree with the paper's settings (E = K = 10, D = 4, N_max = 60) for the heterogeneous
+    # batch: 4 expansions (1 + 3 x 10 draft rows of 32000 bf16 logits per request), 3 selections, 1 pruning;
+    # three sets of logits in turn (95 MB together with the argmax buffers evicted: cold reads)
+    E_, K_, D_, NMAX = 10, 10, 4, 60
+    Bt = wl3.batch
+    cap = 1 + E_ + (D_ - 1) * K_ * E_
+    state = tw.TreeState(Bt, cap, dev)
+    lsets = [[torch.randn((Bt, 1 if l == 0 else K_, V), dtype=torch.bfloat16, device=dev) for l in range(D_)]
+             for _ in range(3)]
+    t_par = torch.zeros((Bt, 64), dtype=torch.int32, device=dev)
+    t_tok, t_n = torch.zeros_like(t_par), torch.zeros(Bt, dtype=torch.int32, device=dev)
+    root = torch.zeros((Bt, 1), dtype=torch.int32, device=dev)
+    nxt = torch.zeros((Bt, K_), dtype=torch.int32, device=dev)
+
+    def build_tree(logit_levels):
+        tw.tree_reset(state)
+        src, lo, hi = root, 0, 1
+        for l in range(D_):
+            tw.tree_expand_level(logit_levels[l], src, E_, hi, state)
+            lo, hi = hi, hi + (1 if l == 0 else K_) * E_
+            if l + 1 < D_:
+                tw.tree_select_expansion(state, lo, hi, nxt)
+                src = nxt
+        tw.tree_finalize(state, cap, NMAX, t_par, t_tok, t_n)
+
+    for ls in lsets:
+        build_tree(ls)
+    e0.record(stream)
+    for i in range(n_chain):
+        build_tree(lsets[i % 3])
+    e1.record(stream)
+    torch.cuda.synchronize()
+    us = e0.elapsed_time(e1) * 1e3 / n_chain
+    res["tree_build_c3_E10_K10_D4"] = hbm_entry(us, int(Bt * (1 + (D_ - 1) * K_) * V * 2))
+    res["tree_build_c3_E10_K10_D4"]["launches"] = "4 expansions + 3 selections + 1 pruning + 3 memsets, launched one by one"
     return res
 
 

@@ -12,7 +12,7 @@ namespace twig {
 
 namespace {
 
-constexpr int kTopThreads = 256;
+constexpr int kTopThreads = 512;
 constexpr int kMaxE = 16;            // children per expanded node
 constexpr int kSelThreads = 256;
 
@@ -20,19 +20,22 @@ constexpr int kSelThreads = 256;
 __device__ __forceinline__ bool comes_first(float v, int i, float w, int j) { return v > w || (v == w && i < j); }
 
 // One CTA per (expansion slot, request): log-sum-exp of the row and its E largest logits.
+// The row is read from global memory once: it is kept in shared memory (when it fits) for the E
+// selection rounds.  Round e finds the best entry that comes strictly after round e-1's winner in
+// the (value, index) order, so nothing has to be marked as taken and no lane takes a long branch.
 template <bool FP32>
 __global__ void __launch_bounds__(kTopThreads)
 tree_expand_kernel(const void *__restrict__ logits, long long row_stride, int vocab, int rows,
-                   const int *__restrict__ src_node, int E, int level_base, int cap,
+                   const int *__restrict__ src_node, int E, int level_base, int cap, int staged,
                    int *__restrict__ node_tok, int *__restrict__ node_parent, float *__restrict__ node_score,
                    int *dev_status) {
   constexpr int EPC = FP32 ? 4 : 8;
+  extern __shared__ __align__(16) unsigned char row_s[];
   __shared__ float s_v[kTopThreads / 32];
   __shared__ int s_i[kTopThreads / 32];
   __shared__ float s_m[kTopThreads / 32], s_s[kTopThreads / 32];
   __shared__ float s_top_v[kMaxE];
   __shared__ int s_top_i[kMaxE];
-  __shared__ int s_winner;
   const int r = blockIdx.x, b = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int u = src_node[(long long)b * rows + r];
   if (u < 0) return;                                       // unused slot
@@ -43,64 +46,50 @@ tree_expand_kernel(const void *__restrict__ logits, long long row_stride, int vo
   }
   const unsigned char *row = static_cast<const unsigned char *>(logits) +
                              ((long long)b * rows + r) * row_stride * (FP32 ? 4 : 2);
-  // per-thread: running (max, sum of exp) and the thread's own top list, best first
-  float tv[kMaxE];
-  int ti[kMaxE];
-#pragma unroll
-  for (int e = 0; e < kMaxE; ++e) {
-    tv[e] = -INFINITY;
-    ti[e] = 0x7fffffff;
-  }
-  float m = -INFINITY, s = 0.f;
-  auto take = [&](float v, int i) {
-    if (v > m) {
-      s = s * __expf(m - v) + 1.f;          // (m = -inf: s is 0)
-      m = v;
+  auto element = [&](const unsigned char *base, int i) {
+    return FP32 ? reinterpret_cast<const float *>(base)[i]
+                : __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(base)[i]);
+  };
+  auto unpack = [&](const uint4 &w, float (&v)[8]) {
+    if (FP32) {
+      v[0] = __uint_as_float(w.x); v[1] = __uint_as_float(w.y); v[2] = __uint_as_float(w.z); v[3] = __uint_as_float(w.w);
     } else {
-      s += __expf(v - m);
-    }
-    if (comes_first(v, i, tv[kMaxE - 1], ti[kMaxE - 1])) {
-      // insert: bubble the newcomer up from the tail
-      tv[kMaxE - 1] = v;
-      ti[kMaxE - 1] = i;
-#pragma unroll
-      for (int e = kMaxE - 1; e > 0; --e) {
-        if (comes_first(tv[e], ti[e], tv[e - 1], ti[e - 1])) {
-          const float fv = tv[e];
-          tv[e] = tv[e - 1];
-          tv[e - 1] = fv;
-          const int fi = ti[e];
-          ti[e] = ti[e - 1];
-          ti[e - 1] = fi;
-        }
-      }
+      v[0] = bf16_lo(w.x); v[1] = bf16_hi(w.x); v[2] = bf16_lo(w.y); v[3] = bf16_hi(w.y);
+      v[4] = bf16_lo(w.z); v[5] = bf16_hi(w.z); v[6] = bf16_lo(w.w); v[7] = bf16_hi(w.w);
     }
   };
   const int chunks = vocab / EPC;
+
+  // ---- pass over global memory: stage the row, running (max, sum of exp) per thread ----
+  float m = -INFINITY, s = 0.f;
+  auto soft = [&](float v) {
+    const float nm = fmaxf(m, v);
+    s = s * __expf(m - nm) + __expf(v - nm);      // (m = -inf: s is 0 and exp(-inf) = 0)
+    m = nm;
+  };
   for (int c = tid; c < chunks; c += kTopThreads) {
     const uint4 w = ld_nc_16(row + (long long)c * 16);
-    const int base = c * EPC;
-    if (FP32) {
-      take(__uint_as_float(w.x), base);
-      take(__uint_as_float(w.y), base + 1);
-      take(__uint_as_float(w.z), base + 2);
-      take(__uint_as_float(w.w), base + 3);
-    } else {
-      take(bf16_lo(w.x), base);
-      take(bf16_hi(w.x), base + 1);
-      take(bf16_lo(w.y), base + 2);
-      take(bf16_hi(w.y), base + 3);
-      take(bf16_lo(w.z), base + 4);
-      take(bf16_hi(w.z), base + 5);
-      take(bf16_lo(w.w), base + 6);
-      take(bf16_hi(w.w), base + 7);
-    }
+    if (staged) *reinterpret_cast<uint4 *>(row_s + (size_t)c * 16) = w;
+    float v[8];
+    unpack(w, v);
+    float cm = v[0];
+#pragma unroll
+    for (int k = 1; k < EPC; ++k) cm = fmaxf(cm, v[k]);
+    const float nm = fmaxf(m, cm);
+    float acc = s * __expf(m - nm);
+#pragma unroll
+    for (int k = 0; k < EPC; ++k) acc += __expf(v[k] - nm);
+    s = acc;
+    m = nm;
   }
-  for (int i = chunks * EPC + tid; i < vocab; i += kTopThreads)
-    take(FP32 ? reinterpret_cast<const float *>(row)[i]
-              : __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(row)[i]), i);
-
-  // ---- log-sum-exp of the row ----
+  for (int i = chunks * EPC + tid; i < vocab; i += kTopThreads) {
+    const float v = element(row, i);
+    if (staged) {
+      if (FP32) reinterpret_cast<float *>(row_s)[i] = v;
+      else reinterpret_cast<__nv_bfloat16 *>(row_s)[i] = reinterpret_cast<const __nv_bfloat16 *>(row)[i];
+    }
+    soft(v);
+  }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
     const float om = __shfl_xor_sync(0xffffffffu, m, o), os = __shfl_xor_sync(0xffffffffu, s, o);
@@ -112,17 +101,54 @@ tree_expand_kernel(const void *__restrict__ logits, long long row_stride, int vo
     s_m[warp] = m;
     s_s[warp] = s;
   }
-  __syncthreads();
+  __syncthreads();                         // (also: the staged row is complete)
   float M = -INFINITY;
   for (int w = 0; w < kTopThreads / 32; ++w) M = fmaxf(M, s_m[w]);
   float S = 0.f;
   for (int w = 0; w < kTopThreads / 32; ++w) S += s_m[w] == -INFINITY ? 0.f : s_s[w] * __expf(s_m[w] - M);
   const float lse = M + logf(S);
 
-  // ---- E rounds: the best head among all threads' lists wins and is popped ----
+  // ---- E rounds over the (staged) row ----
+  const unsigned char *src = staged ? row_s : row;
+  float pv = INFINITY;                     // previous winner; every finite logit comes after (+inf, -1)
+  int pi = -1;
   for (int e = 0; e < E; ++e) {
-    float bv = tv[0];
-    int bi = ti[0];
+    float bv = -INFINITY;
+    int bi = 0x7fffffff;
+    auto offer = [&](float v, int i) {
+      const bool after_prev = pv > v || (pv == v && pi < i);
+      if (after_prev && comes_first(v, i, bv, bi)) {
+        bv = v;
+        bi = i;
+      }
+    };
+    for (int c = tid; c < chunks; c += kTopThreads) {
+      const uint4 w = *reinterpret_cast<const uint4 *>(src + (size_t)c * 16);
+      float v[8];
+      int ix[8];
+      unpack(w, v);
+      // entries at or before the previous winner drop out; then a tournament inside the chunk (equal
+      // values: the left, lower-index entry stays), and one comparison with the running best
+#pragma unroll
+      for (int k = 0; k < EPC; ++k) {
+        ix[k] = c * EPC + k;
+        const bool after_prev = pv > v[k] || (pv == v[k] && pi < ix[k]);
+        v[k] = after_prev ? v[k] : -INFINITY;
+      }
+#pragma unroll
+      for (int span = 1; span < EPC; span <<= 1)
+#pragma unroll
+        for (int k = 0; k + span < EPC; k += 2 * span)
+          if (v[k + span] > v[k]) {
+            v[k] = v[k + span];
+            ix[k] = ix[k + span];
+          }
+      if (v[0] > -INFINITY && comes_first(v[0], ix[0], bv, bi)) {
+        bv = v[0];
+        bi = ix[0];
+      }
+    }
+    for (int i = chunks * EPC + tid; i < vocab; i += kTopThreads) offer(element(src, i), i);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
       const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
@@ -137,26 +163,19 @@ tree_expand_kernel(const void *__restrict__ logits, long long row_stride, int vo
       s_i[warp] = bi;
     }
     __syncthreads();
-    if (tid == 0) {
-      for (int w = 1; w < kTopThreads / 32; ++w)
-        if (comes_first(s_v[w], s_i[w], bv, bi)) {
-          bv = s_v[w];
-          bi = s_i[w];
-        }
-      s_top_v[e] = bv;
-      s_top_i[e] = bi;
-      s_winner = bi;
-    }
-    __syncthreads();
-    if (ti[0] == s_winner) {              // token ids are unique: exactly one thread pops
+    pv = s_v[0];
+    pi = s_i[0];
 #pragma unroll
-      for (int k = 0; k < kMaxE - 1; ++k) {
-        tv[k] = tv[k + 1];
-        ti[k] = ti[k + 1];
+    for (int w = 1; w < kTopThreads / 32; ++w)
+      if (comes_first(s_v[w], s_i[w], pv, pi)) {
+        pv = s_v[w];
+        pi = s_i[w];
       }
-      tv[kMaxE - 1] = -INFINITY;
-      ti[kMaxE - 1] = 0x7fffffff;
+    if (tid == 0) {
+      s_top_v[e] = pv;
+      s_top_i[e] = pi;
     }
+    __syncthreads();                       // s_v / s_i are free for the next round
   }
   if (tid < E) {
     const long long at = (long long)b * cap + first + tid;
@@ -268,12 +287,23 @@ extern "C" twig_status tree_expand_level(const void *logits, int32_t logits_fp32
   if (!aligned16(logits) || (row_stride * esz) % 16) return TWIG_ERR_ALIGN;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   dim3 grid(rows, batch);
+  // the row is staged in shared memory when it fits (else the selection rounds re-read it through L2)
+  const size_t row_bytes = ((size_t)vocab * esz + 15) & ~(size_t)15;
+  const int staged = row_bytes <= 200 * 1024;
+  const size_t smem = staged ? row_bytes : 0;
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(tree_expand_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess ||
+        cudaFuncSetAttribute(tree_expand_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess)
+      return TWIG_ERR_CUDA;
+    attr_set = true;
+  }
   if (logits_fp32)
-    tree_expand_kernel<true><<<grid, kTopThreads, 0, st>>>(logits, row_stride, vocab, rows, src_node, n_children,
-        level_base, cap, node_tok, node_parent, node_score, dev_status);
+    tree_expand_kernel<true><<<grid, kTopThreads, smem, st>>>(logits, row_stride, vocab, rows, src_node, n_children,
+        level_base, cap, staged, node_tok, node_parent, node_score, dev_status);
   else
-    tree_expand_kernel<false><<<grid, kTopThreads, 0, st>>>(logits, row_stride, vocab, rows, src_node, n_children,
-        level_base, cap, node_tok, node_parent, node_score, dev_status);
+    tree_expand_kernel<false><<<grid, kTopThreads, smem, st>>>(logits, row_stride, vocab, rows, src_node, n_children,
+        level_base, cap, staged, node_tok, node_parent, node_score, dev_status);
   return launch_status();
 }
 
