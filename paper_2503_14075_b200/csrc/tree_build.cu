@@ -14,15 +14,19 @@ namespace {
 
 constexpr int kTopThreads = 512;
 constexpr int kMaxE = 16;            // children per expanded node
+constexpr int kMaxCand = 1024;       // entries at or above the threshold that the short list holds
 constexpr int kSelThreads = 256;
 
 // (value, index) order of the top lists: larger value first, equal values: lower index first
 __device__ __forceinline__ bool comes_first(float v, int i, float w, int j) { return v > w || (v == w && i < j); }
 
 // One CTA per (expansion slot, request): log-sum-exp of the row and its E largest logits.
-// The row is read from global memory once: it is kept in shared memory (when it fits) for the E
-// selection rounds.  Round e finds the best entry that comes strictly after round e-1's winner in
-// the (value, index) order, so nothing has to be marked as taken and no lane takes a long branch.
+// The row is read from global memory once and kept in shared memory (when it fits).  The E-th
+// largest of the half-warp groups' maxima is a lower bound of the E-th largest logit, so one more pass
+// over the staged row collects the few entries at or above it into a short list; the E selection
+// rounds run over that list (over the whole row if the list overflows, e.g. a row of equal logits).
+// Round e finds the best entry that comes strictly after round e-1's winner in the (value, index)
+// order, so nothing has to be marked as taken and no lane takes a long branch.
 template <bool FP32>
 __global__ void __launch_bounds__(kTopThreads)
 tree_expand_kernel(const void *__restrict__ logits, long long row_stride, int vocab, int rows,
@@ -36,6 +40,10 @@ tree_expand_kernel(const void *__restrict__ logits, long long row_stride, int vo
   __shared__ float s_m[kTopThreads / 32], s_s[kTopThreads / 32];
   __shared__ float s_top_v[kMaxE];
   __shared__ int s_top_i[kMaxE];
+  __shared__ float s_tmax[kTopThreads / 16];       // maxima of the half-warp groups
+  __shared__ float s_cand_v[kMaxCand];
+  __shared__ int s_cand_i[kMaxCand];
+  __shared__ int s_n_cand;
   const int r = blockIdx.x, b = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int u = src_node[(long long)b * rows + r];
   if (u < 0) return;                                       // unused slot
@@ -62,7 +70,9 @@ tree_expand_kernel(const void *__restrict__ logits, long long row_stride, int vo
 
   // ---- pass over global memory: stage the row, running (max, sum of exp) per thread ----
   float m = -INFINITY, s = 0.f;
+  float t_max = -INFINITY;                       // (equals m; kept apart for clarity)
   auto soft = [&](float v) {
+    t_max = fmaxf(t_max, v);
     const float nm = fmaxf(m, v);
     s = s * __expf(m - nm) + __expf(v - nm);      // (m = -inf: s is 0 and exp(-inf) = 0)
     m = nm;
@@ -75,6 +85,7 @@ tree_expand_kernel(const void *__restrict__ logits, long long row_stride, int vo
     float cm = v[0];
 #pragma unroll
     for (int k = 1; k < EPC; ++k) cm = fmaxf(cm, v[k]);
+    t_max = fmaxf(t_max, cm);
     const float nm = fmaxf(m, cm);
     float acc = s * __expf(m - nm);
 #pragma unroll
@@ -108,8 +119,54 @@ tree_expand_kernel(const void *__restrict__ logits, long long row_stride, int vo
   for (int w = 0; w < kTopThreads / 32; ++w) S += s_m[w] == -INFINITY ? 0.f : s_s[w] * __expf(s_m[w] - M);
   const float lse = M + logf(S);
 
-  // ---- E rounds over the (staged) row ----
+  // ---- threshold: the E-th largest of the maxima of the 32 half-warp groups (E <= 16 distinct
+  // entries are at or above it, so it is a lower bound of the E-th largest logit) ----
   const unsigned char *src = staged ? row_s : row;
+  float g_max = t_max;
+#pragma unroll
+  for (int o = 8; o > 0; o >>= 1) g_max = fmaxf(g_max, __shfl_xor_sync(0xffffffffu, g_max, o));
+  constexpr int kGroups = kTopThreads / 16;
+  if ((lane & 15) == 0) s_tmax[tid >> 4] = g_max;
+  if (tid == 0) s_n_cand = 0;
+  __syncthreads();
+  if (tid < kGroups) {
+    const float mine = s_tmax[tid];
+    int above = 0;                                   // group maxima ranked before mine (ties: lower group first)
+    for (int j = 0; j < kGroups; ++j) above += (s_tmax[j] > mine || (s_tmax[j] == mine && j < tid)) ? 1 : 0;
+    if (above == E - 1) s_v[0] = mine;               // exactly one group has this rank
+  }
+  __syncthreads();
+  const float thr = s_v[0];
+  __syncthreads();
+  for (int c = tid; c < chunks; c += kTopThreads) {
+    const uint4 w = *reinterpret_cast<const uint4 *>(src + (size_t)c * 16);
+    float v[8];
+    unpack(w, v);
+#pragma unroll
+    for (int k = 0; k < EPC; ++k)
+      if (v[k] >= thr) {
+        const int at = atomicAdd(&s_n_cand, 1);
+        if (at < kMaxCand) {
+          s_cand_v[at] = v[k];
+          s_cand_i[at] = c * EPC + k;
+        }
+      }
+  }
+  for (int i = chunks * EPC + tid; i < vocab; i += kTopThreads) {
+    const float v = element(src, i);
+    if (v >= thr) {
+      const int at = atomicAdd(&s_n_cand, 1);
+      if (at < kMaxCand) {
+        s_cand_v[at] = v;
+        s_cand_i[at] = i;
+      }
+    }
+  }
+  __syncthreads();
+  const int n_cand = s_n_cand;
+  const bool short_list = n_cand <= kMaxCand;       // (n_cand >= E always: the E maxima are in it)
+
+  // ---- E rounds over the short list (or the whole row) ----
   float pv = INFINITY;                     // previous winner; every finite logit comes after (+inf, -1)
   int pi = -1;
   for (int e = 0; e < E; ++e) {
@@ -122,7 +179,9 @@ tree_expand_kernel(const void *__restrict__ logits, long long row_stride, int vo
         bi = i;
       }
     };
-    for (int c = tid; c < chunks; c += kTopThreads) {
+    if (short_list)
+      for (int j = tid; j < n_cand; j += kTopThreads) offer(s_cand_v[j], s_cand_i[j]);
+    for (int c = tid; c < (short_list ? 0 : chunks); c += kTopThreads) {
       const uint4 w = *reinterpret_cast<const uint4 *>(src + (size_t)c * 16);
       float v[8];
       int ix[8];
@@ -148,7 +207,8 @@ tree_expand_kernel(const void *__restrict__ logits, long long row_stride, int vo
         bi = ix[0];
       }
     }
-    for (int i = chunks * EPC + tid; i < vocab; i += kTopThreads) offer(element(src, i), i);
+    if (!short_list)
+      for (int i = chunks * EPC + tid; i < vocab; i += kTopThreads) offer(element(src, i), i);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
       const float ov = __shfl_xor_sync(0xffffffffu, bv, o);

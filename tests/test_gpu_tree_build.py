@@ -86,10 +86,12 @@ def test_token_tree_matches_oracle(tw, cfg, dtype):
         assert np.allclose(score[b, :len(fs)], fs, rtol=0, atol=2e-4 * D)
 
 
-def test_token_tree_ties(tw):
+@pytest.mark.parametrize("V", [64, 4096])
+def test_token_tree_ties(tw, V):
     """Equal logits go to the lower token id, equal scores to the lower node id (exact ties: rows that are
-    bit-identical give bit-identical scores)."""
-    E, K, D, n_max, t_max, V = 2, 2, 2, 4, 8, 64
+    bit-identical give bit-identical scores).  With 4096 equal logits the kernel's short candidate list
+    overflows and the selection runs over the whole row."""
+    E, K, D, n_max, t_max = 2, 2, 2, 4, 8
     flat = [torch.zeros((1, 1, V), dtype=torch.float32, device=DEV), torch.zeros((1, K, V), dtype=torch.float32, device=DEV)]
     parent, tok, n_nodes, kept, status, _ = gpu_tree(tw, flat, E, K, n_max, t_max)
     p_o, t_o, _, keep_o, _ = O.build_token_tree([np.zeros((1, V)), np.zeros((K, V))], E, K, n_max)
