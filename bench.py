@@ -345,7 +345,7 @@ def run_ours(args):
         wl.n_kv_heads * max(wl.prefix_len) * wl.head_dim * 2
 
     # ---- end to end through the public API with host buffers -----------------------------------
-    e2e = run_e2e(torch, tw, wl, reps, stream, world, dev, dist if world > 1 else None)
+    e2e = run_e2e(torch, tw, wl, reps, stream, world, dev, dist if world > 1 else None, graphs[0] if graphs else None)
 
     out = {
         "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -375,11 +375,13 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
-def run_e2e(torch, tw, wl, reps, stream, world, dev, dist):
+def run_e2e(torch, tw, wl, reps, stream, world, dev, dist, step_graphs):
     """Same loop through the public API, every verify step's inputs (Q, tree K/V of all
     layers, tree and token ids) copied from pinned host memory and its result (accept
     length, path, bonus token) read back before the next step.  The prompt's KV cache is
-    device-resident state, like the model weights."""
+    device-resident state, like the model weights.  The step's kernels are launched as in the
+    device-resident loop: the captured graph of the step (one launch per layer + accept) where
+    graphs are in use, one by one otherwise."""
     rp = reps[0]
     pin = []
     for (q, tk, tv) in rp.pool_host:
@@ -390,7 +392,7 @@ def run_e2e(torch, tw, wl, reps, stream, world, dev, dist):
     tgt_pin = torch.from_numpy(rp.tgt_host).pin_memory()
     res_pin = torch.zeros((wl.batch, 2 + wl.t_max), dtype=torch.int32).pin_memory()
     res_dev = torch.zeros((wl.batch, 2 + wl.t_max), dtype=torch.int32, device=dev)
-    d_q, d_tk, d_tv = (torch.empty_like(rp.q[0]), torch.empty_like(rp.tree_k[0]), torch.empty_like(rp.tree_v[0]))
+    stage = (torch.empty_like(rp.q[0]), torch.empty_like(rp.tree_k[0]), torch.empty_like(rp.tree_v[0]))
     h2d = d2h = 0
 
     def request():
@@ -402,18 +404,23 @@ def run_e2e(torch, tw, wl, reps, stream, world, dev, dist):
         rp.prune(tw)
         for s in range(rp.n_steps):
             slot = s % POOL
+            # (with graphs the copies land in the buffers the step's graph reads)
+            d_q, d_tk, d_tv = (rp.q[slot], rp.tree_k[slot], rp.tree_v[slot]) if step_graphs else stage
             d_q.view(torch.int16).copy_(pin[slot][0], non_blocking=True)
             d_tk.view(torch.int16).copy_(pin[slot][1], non_blocking=True)
             d_tv.view(torch.int16).copy_(pin[slot][2], non_blocking=True)
             rp.parent.copy_(par_pin, non_blocking=True)
             rp.draft[s].copy_(draft_pin[s], non_blocking=True)
             rp.tgt[s].copy_(tgt_pin[s], non_blocking=True)
-            h2d += 2 * (d_q.numel() + d_tk.numel() + d_tv.numel()) + 4 * 3 * par_pin.numel()
-            for layer in range(wl.n_layers):
-                tw.tree_verify_attention(d_q[layer], d_tk[layer], d_tv[layer], rp.cache, layer, rp.kv_len,
-                                         rp.n_nodes, rp.parent, rp.out, dev_status=rp.status)
-            tw.tree_accept_compact(rp.parent, rp.draft[s], rp.tgt[s], rp.n_nodes, d_tk, d_tv, rp.cache, rp.kv_len,
-                                   rp.accept_len, rp.path, rp.bonus, dev_status=rp.status)
+            h2d += 2 * (d_q.numel() + d_tk.numel() + d_tv.numel()) + 4 * (par_pin.numel() + 2 * draft_pin[s].numel())
+            if step_graphs:
+                step_graphs[s].replay()
+            else:
+                for layer in range(wl.n_layers):
+                    tw.tree_verify_attention(d_q[layer], d_tk[layer], d_tv[layer], rp.cache, layer, rp.kv_len,
+                                             rp.n_nodes, rp.parent, rp.out, dev_status=rp.status)
+                tw.tree_accept_compact(rp.parent, rp.draft[s], rp.tgt[s], rp.n_nodes, d_tk, d_tv, rp.cache, rp.kv_len,
+                                       rp.accept_len, rp.path, rp.bonus, dev_status=rp.status)
             res_dev[:, 0] = rp.accept_len
             res_dev[:, 1] = rp.bonus
             res_dev[:, 2:] = rp.path
@@ -440,7 +447,8 @@ def run_e2e(torch, tw, wl, reps, stream, world, dev, dist):
         ms = float(tt.item())
     return {"value": round(rp.n_steps * n_req * world / (ms * 1e-3), 1), "unit": UNIT,
             "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
-            "note": "per bench step = one request; Q and tree K/V of all layers cross PCIe every verify step"}
+            "note": "per bench step = one request; Q and tree K/V of all layers cross PCIe every verify step; "
+                    + ("kernels replayed from the step's graph" if step_graphs else "kernels launched one by one")}
 
 
 def _time_attention(torch, tw, wl, kv_lens, nl, stream_id, dev, reps=10):
