@@ -96,6 +96,10 @@ __device__ __forceinline__ void st_async_b32x2(uint32_t dst, uint32_t a, uint32_
   asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v2.b32 [%0], {%1, %2}, [%3];"
                ::"r"(dst), "r"(a), "r"(b), "r"(bar) : "memory");
 }
+__device__ __forceinline__ void st_async_b32x4(uint32_t dst, uint32_t a, uint32_t b, uint32_t c, uint32_t d, uint32_t bar) {
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.b32 [%0], {%1, %2, %3, %4}, [%5];"
+               ::"r"(dst), "r"(a), "r"(b), "r"(c), "r"(d), "r"(bar) : "memory");
+}
 __device__ __forceinline__ void st_async_f32x2(uint32_t dst, float a, float b, uint32_t bar) {
   asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v2.f32 [%0], {%1, %2}, [%3];"
                ::"r"(dst), "f"(a), "f"(b), "r"(bar) : "memory");

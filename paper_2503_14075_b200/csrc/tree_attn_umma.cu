@@ -79,15 +79,6 @@ __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.a
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
 // One box of the 5-D cache tensor map -> shared memory; completion is counted on `bar`.
 __device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int pos,
                                             int head, int batch, int layer) {
@@ -191,11 +182,13 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
   extern __shared__ __align__(1024) unsigned char smem[];
   __shared__ unsigned long long s_mask[TWIG_MAX_NODES];
   __shared__ int s_par[TWIG_MAX_NODES];
-  __shared__ float r_m[ROWS], r_l[ROWS];
+  __shared__ float2 r_ml[ROWS];                      // received (m, l): [sender][owned row]
+  __shared__ __align__(8) unsigned long long s_recv_bar;      // counts what peers push to this CTA (split merge)
   // barriers: full[5], empty[5] (ring slots), s_ready[2], p_ready[2], o_done[2], q_ready
   __shared__ __align__(8) unsigned long long s_bar[2 * kMaxSlots + 7];
   __shared__ uint32_t s_tmem;
   __shared__ int s_bad, s_fail;
+  __shared__ volatile int s_never;                   // stays 0
 
   cg::cluster_group cluster = cg::this_cluster();
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -221,6 +214,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
   if (tid == 0) {
     s_bad = 0;
     s_fail = 0;
+    s_never = 0;
     for (int i = 0; i < kSlots; ++i) {
       mbar_init(bar_full(i), 32);       // every loader lane arrives once per unit
       mbar_init(bar_empty(i), 1);       // one tcgen05.commit
@@ -230,6 +224,13 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
     mbar_init(bar_o(0), 1);
     mbar_init(bar_o(1), 1);
     mbar_init(bar_q, 32);
+    if (n_splits > 1) {
+      // split merge: one arrival that announces the peers' bytes (every peer sends each of this
+      // CTA's ROWS / n_splits rows as 128 fp16 and an (m, l) pair), one per softmax warp for this
+      // CTA's own share
+      mbar_init(smem_u32(&s_recv_bar), 1 + 4);
+      mbar_arrive_expect_tx(smem_u32(&s_recv_bar), (uint32_t)((n_splits - 1) * (ROWS / n_splits) * (kD * 2 + 8)));
+    }
   }
   if (warp == 5) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem)), "r"(C::TMEM_COLS) : "memory");
@@ -737,15 +738,24 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
     return;
   }
 
-  // ---- merge the key splits of the cluster (push to the row's owner, then reduce) ----
+  // ---- merge the key splits of the cluster ----
+  // Every CTA owns ROWS / n_splits rows.  Once all CTAs have left their key loops (the receive
+  // buffer lies in the stage ring) each thread sends its row's (m, l) and O / l as fp16 (|O / l| is
+  // bounded by the largest |V| entry; fp16 rounds eight times finer than the bf16 output) to the
+  // row's owner: asynchronous stores that the owner's barrier counts, plain stores for the CTA's
+  // own share.  The owner waits for its bytes (bounded), combines and stores.
   const int rows_per = ROWS / n_splits;
-  float *recv = reinterpret_cast<float *>(smem + C::Q_BYTES + C::P_BYTES);
+  unsigned char *recv = smem + C::Q_BYTES + C::P_BYTES;      // [sender * rows_per + owned row][128] fp16
+  const uint32_t recv_bar = smem_u32(&s_recv_bar);
   cluster.sync();                          // every CTA has left its key loop: the rings are free
   if (warp < 4) {
     const int rl_ = row_active ? row_local : 0;
     const int owner = rl_ / rows_per, lr = rl_ % rows_per;
     const int slot = split * rows_per + lr;
-    float *ro = cluster.map_shared_rank(recv + (size_t)slot * kD, owner);
+    const bool remote = owner != split;
+    unsigned char *ro = recv + (size_t)slot * kD * 2;
+    const uint32_t ro_c = map_to_cta(smem_u32(ro), owner), bar_c = map_to_cta(recv_bar, owner);
+    const float inv_l = (have_o && l_run > 0.f) ? 1.f / l_run : 0.f;
 #pragma unroll
     for (int ch = 0; ch < 4; ++ch) {
       uint32_t v[32];
@@ -758,23 +768,40 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
       }
       if (row_active) {
 #pragma unroll
-        for (int i = 0; i < 8; ++i)         // float4 slots are XOR-swizzled by the row to spread banks
-          *reinterpret_cast<float4 *>(ro + (((ch * 8 + i) ^ (lr & 31)) << 2)) =
-              make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]), __uint_as_float(v[4 * i + 2]),
-                          __uint_as_float(v[4 * i + 3]));
+        for (int i = 0; i < 4; ++i) {       // 16-byte chunks (8 columns) are XOR-swizzled by the row to spread banks
+          uint32_t h[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e)
+            h[e] = pack_f16(__uint_as_float(v[8 * i + 2 * e]) * inv_l, __uint_as_float(v[8 * i + 2 * e + 1]) * inv_l);
+          const int off = ((ch * 4 + i) ^ (lr & 15)) << 4;
+          if (remote) st_async_b32x4(ro_c + off, h[0], h[1], h[2], h[3], bar_c);
+          else *reinterpret_cast<uint4 *>(ro + off) = make_uint4(h[0], h[1], h[2], h[3]);
+        }
       }
     }
     if (row_active) {
-      *cluster.map_shared_rank(r_m + slot, owner) = m_run;
-      *cluster.map_shared_rank(r_l + slot, owner) = l_run;
+      const float mm = have_o ? m_run : -INFINITY, ll = have_o ? l_run : 0.f;
+      if (remote) st_async_f32x2(map_to_cta(smem_u32(r_ml + slot), owner), mm, ll, bar_c);
+      else r_ml[slot] = make_float2(mm, ll);
     }
+    __syncwarp();                           // the lanes' own-share stores come before lane 0's arrival
+    if (lane == 0) mbar_arrive(recv_bar);
   }
   tc_fence_before();
-  cluster.sync();
+  __syncthreads();                          // every tensor-memory load of this CTA is done
   if (warp == 5) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(C::TMEM_COLS) : "memory");
+  {
+    // (bounded by the spin limit alone: a CTA whose own key loop failed must still stay until its
+    // peers' stores have landed)
+    const bool landed = mbar_wait(recv_bar, 0, &s_never);
+    if (!landed) {                          // a peer never delivered: reported, not waited for
+      if (tid == 0) flag_status(p.dev_status, b, TWIG_DEV_INTERNAL);
+      return;
+    }
+  }
 
   {
-    constexpr int TPR = kD / 4;                       // 32 threads per row, one float4 each
+    constexpr int TPR = kD / 4;                       // 32 threads per row, 4 columns each
     constexpr int RPP = kThreads / TPR;
     const int i4 = tid % TPR;
     for (int lr = tid / TPR; lr < rows_per; lr += RPP) {
@@ -784,22 +811,23 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
       float mstar = -INFINITY;
 #pragma unroll
       for (int sd = 0; sd < 8; ++sd) {
-        mv[sd] = sd < n_splits ? r_m[sd * rows_per + lr] : -INFINITY;
+        mv[sd] = sd < n_splits ? r_ml[sd * rows_per + lr].x : -INFINITY;
         mstar = fmaxf(mstar, mv[sd]);
       }
       float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
       float lsum = 0.f;
-      const int col = (i4 ^ (lr & 31)) << 2;
+      const int off = (((i4 >> 1) ^ (lr & 15)) << 4) + (i4 & 1) * 8;
 #pragma unroll
       for (int sd = 0; sd < 8; ++sd) {
         if (sd < n_splits) {
-          const float wgt = fast_exp2(mv[sd] - mstar);
-          lsum = fmaf(wgt, r_l[sd * rows_per + lr], lsum);
-          const float4 v = *reinterpret_cast<const float4 *>(recv + (size_t)(sd * rows_per + lr) * kD + col);
-          acc.x = fmaf(wgt, v.x, acc.x);
-          acc.y = fmaf(wgt, v.y, acc.y);
-          acc.z = fmaf(wgt, v.z, acc.z);
-          acc.w = fmaf(wgt, v.w, acc.w);
+          const float wgt = fast_exp2(mv[sd] - mstar) * r_ml[sd * rows_per + lr].y;
+          lsum += wgt;
+          const uint2 raw = *reinterpret_cast<const uint2 *>(recv + (size_t)(sd * rows_per + lr) * kD * 2 + off);
+          const float2 v01 = unpack_f16(raw.x), v23 = unpack_f16(raw.y);
+          acc.x = fmaf(wgt, v01.x, acc.x);
+          acc.y = fmaf(wgt, v01.y, acc.y);
+          acc.z = fmaf(wgt, v23.x, acc.z);
+          acc.w = fmaf(wgt, v23.y, acc.w);
         }
       }
       const float inv = 1.f / lsum;
