@@ -41,7 +41,8 @@ namespace twig {
 namespace {
 
 constexpr int kD = 128;          // head_dim
-constexpr int kThreads = 192;          // warps 0-3 softmax, warp 4 loader, warp 5 MMA issuer
+// warps 0-3 softmax, warp 4 loader, warp 5 MMA issuer; with 128-row accumulators warps 6-9 are a
+// second softmax group (UmmaCfg::THREADS)
 constexpr int kMaxSlots = 5;                      // ring of K / V tiles (K0 V0 K1 V1 K2 ...)
 constexpr float kLazyMax = 8.f;                   // raise the running max only beyond this (log2 units)
 constexpr int kSpinLimit = 1 << 22;
@@ -164,25 +165,33 @@ struct UmmaCfg {
   static constexpr int RING_BYTES = SLOTS * TILE_BYTES;
   static constexpr uint32_t TMEM_COLS = KT == 64 ? 256 : 512;   // S: [0,KT) and [KT,2KT); O: [2KT, 2KT+128)
   static constexpr uint32_t O_COL = 2 * KT;
-  static constexpr int MIN_CTAS = KT == 64 ? 2 : 1;
+  static constexpr int MIN_CTAS = (KT == 64 && ROWS <= 64) ? 2 : 1;     // (128 rows: shared memory allows one CTA per SM)
   static constexpr int RECV_BYTES = ROWS * kD * 4;
   static_assert(RECV_BYTES <= RING_BYTES, "split-merge buffer must fit in the stage ring");
   static_assert(Q_BYTES % 1024 == 0 && P_BYTES % 1024 == 0, "swizzled tiles start on 1024 bytes");
   static constexpr int SMEM_BYTES = Q_BYTES + P_BYTES + RING_BYTES;
   static constexpr int MMA_M = ROWS <= 64 ? 64 : 128;
   static constexpr int ROWS_PER_WARP = MMA_M == 64 ? 16 : 32;    // rows a softmax warp owns
+  // 128-row accumulators: two warps share the rows of a lane quadrant, half of a tile's keys each
+  static constexpr int SOFT_GROUPS = MMA_M == 128 ? 2 : 1;
+  static constexpr int THREADS = 32 * (6 + 4 * (SOFT_GROUPS - 1));
 };
 
 template <int ROWS, int KT>
-__global__ void __launch_bounds__(kThreads, UmmaCfg<ROWS, KT>::MIN_CTAS)
+__global__ void __launch_bounds__(UmmaCfg<ROWS, KT>::THREADS, UmmaCfg<ROWS, KT>::MIN_CTAS)
 tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap,
                       const __grid_constant__ CUtensorMap vmap) {
   using C = UmmaCfg<ROWS, KT>;
   constexpr int kTileBytes = C::TILE_BYTES, kPanelBytes = C::PANEL_BYTES, kSlots = C::SLOTS;
   extern __shared__ __align__(1024) unsigned char smem[];
   __shared__ unsigned long long s_mask[TWIG_MAX_NODES];
-  __shared__ int s_par[TWIG_MAX_NODES];
-  __shared__ float2 r_ml[ROWS];                      // received (m, l): [sender][owned row]
+  // one scratch area, used in turn for: the parent array (set-up), the values the two softmax
+  // groups exchange (key loop; [tile parity][key half][row]), the received (m, l) pairs of the
+  // split merge ([sender][owned row])
+  __shared__ __align__(16) float s_scratch[2 * 2 * 128];
+  int *s_par = reinterpret_cast<int *>(s_scratch);
+  float (*s_pair)[2][128] = reinterpret_cast<float (*)[2][128]>(s_scratch);
+  float2 *r_ml = reinterpret_cast<float2 *>(s_scratch);
   __shared__ __align__(8) unsigned long long s_recv_bar;      // counts what peers push to this CTA (split merge)
   // barriers: full[5], empty[5] (ring slots), s_ready[2], p_ready[2], o_done[2], q_ready
   __shared__ __align__(8) unsigned long long s_bar[2 * kMaxSlots + 7];
@@ -293,7 +302,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
     s_mask[tid] = m;
   }
   if (tid == 0) {
-    for (int i = 0; i < 2; ++i) mbar_init(bar_p(i), n_soft);      // one arrival per softmax warp
+    for (int i = 0; i < 2; ++i) mbar_init(bar_p(i), n_soft * C::SOFT_GROUPS);      // one arrival per softmax warp
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   tc_fence_before();
@@ -592,112 +601,120 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
       l_run = (lane & 8) ? lh : ll;
     }
     if (!ok) s_fail = 1;
-  } else if (warp < n_soft) {
-    // ================= softmax, 128-row accumulators: thread r owns row r =================
-    const unsigned long long my_mask = row_valid ? s_mask[gr / p.group] : 0ull;
+  } else if (C::MMA_M == 128 && (warp & 3) < n_soft) {
+    // ================= softmax, 128-row accumulators =================
+    // Lane quadrant q of tensor memory (rows 32q .. 32q+31, one per lane) is served by two warps:
+    // warp q takes the first half of a tile's keys, the warp of 6..9 with the same index modulo 4
+    // the second half.  They agree on the rows' maxima through shared memory; each keeps the row
+    // sums of its own keys, rescales its half of O's columns and writes its half of P.  No wait
+    // below is followed by a break: a failed wait marks the request and the rest runs through, so
+    // that both warps meet at every pair barrier.
+    const int quad = warp & 3, half = warp >= 6 ? 1 : 0;
+    const int row = 32 * quad + lane;
+    const int grow = row0 + row;
+    const unsigned long long my_mask = grow < rows_total ? s_mask[grow / p.group] : 0ull;
+    constexpr int NV = KT / 2;                  // keys of a tile this thread handles
+    constexpr int NC = NV / 32;
+    auto pair_sync = [&]() { asm volatile("bar.sync %0, 64;" ::"r"(1 + quad) : "memory"); };
+    float m_r = -INFINITY, l_r = 0.f;           // l_r: this thread's keys only
     bool ok = true;
     for (int it = 0; it < n_my; ++it) {
       const int t = t_begin + it;
-      ok = mbar_wait(bar_s(it & 1), (it >> 1) & 1, fail);
+      ok = ok && mbar_wait(bar_s(it & 1), (it >> 1) & 1, fail);
       ok = __all_sync(0xffffffffu, ok);
-      if (!ok) break;
       tc_fence_after();
-      const uint32_t ts = t_lane + (it & 1) * KT;
-      // 64 keys of this row's S; the keys that hold the prefix end and / or the tree are masked
-      auto load_s = [&](int half, uint32_t (&sr)[2][32]) {
-        tmem_ld32(ts + half * 64, sr[0]);
-        tmem_ld32(ts + half * 64 + 32, sr[1]);
-        tmem_ld_wait();
-        const int key0 = t * KT + half * 64;
-        if (key0 + 64 > L) {
+      const uint32_t ts = t_lane + (it & 1) * KT + half * NV;
+      uint32_t sr[NC][32];
 #pragma unroll
-          for (int h = 0; h < 2; ++h)
+      for (int c = 0; c < NC; ++c) tmem_ld32(ts + 32 * c, sr[c]);
+      tmem_ld_wait();
+      const int key0 = t * KT + half * NV;
+      if (key0 + NV > L) {                      // the prefix end and / or the tree: mask
+        const int rel0 = key0 - L;              // > -NV
+        unsigned long long vis;                 // bit j: key key0 + j is visible to this row
+        if (rel0 >= 0) vis = rel0 < 64 ? my_mask >> rel0 : 0ull;
+        else vis = (my_mask << -rel0) | ((1ull << -rel0) - 1ull);
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-              const int vj = key0 + h * 32 + j;
-              const bool vis = vj < L || (vj < NK && ((my_mask >> (vj - L)) & 1ull));
-              if (!vis) sr[h][j] = 0xff800000u;     // -inf
-            }
-        }
-      };
-      // pass 1: the tile's row maximum (with 64-key tiles the row then stays in registers)
+        for (int c = 0; c < NC; ++c)
+#pragma unroll
+          for (int j = 0; j < 32; ++j)
+            if (!((vis >> (32 * c + j)) & 1ull)) sr[c][j] = 0xff800000u;     // -inf
+      }
       float mx = -INFINITY;
-      uint32_t sr[2][32];
-#pragma unroll 1
-      for (int half = 0; half < KT / 64; ++half) {
-        load_s(half, sr);
+#pragma unroll
+      for (int c = 0; c < NC; ++c)
 #pragma unroll
         for (int j = 0; j < 32; j += 2)
-          mx = fmaxf(mx, fmaxf(fmaxf(__uint_as_float(sr[0][j]), __uint_as_float(sr[0][j + 1])),
-                               fmaxf(__uint_as_float(sr[1][j]), __uint_as_float(sr[1][j + 1]))));
-      }
-      mx *= p.scale_log2;                         // scale > 0, so the max commutes with it
-      const bool raise = row_active && mx > m_run + kLazyMax;   // also true for the first finite maximum
-      const float m_new = raise ? mx : m_run;
+          mx = fmaxf(mx, fmaxf(__uint_as_float(sr[c][j]), __uint_as_float(sr[c][j + 1])));
+      mx *= p.scale_log2;                       // scale > 0, so the max commutes with it
+      s_pair[it & 1][half][row] = mx;
+      pair_sync();
+      mx = fmaxf(mx, s_pair[it & 1][half ^ 1][row]);
+      const bool raise = mx > m_r + kLazyMax;   // also true for the first finite maximum
+      const float m_new = raise ? mx : m_r;
       const float m_use = m_new == -INFINITY ? 0.f : m_new;
       const int pb = it % PB;
-      if (it >= PB) {                             // this P buffer is free once P(it-PB) V(it-PB) is done
-        ok = mbar_wait(bar_o(pb), (it / PB - 1) & 1, fail);
+      if (it >= PB) {                           // this P buffer is free once P(it-PB) V(it-PB) is done
+        ok = ok && mbar_wait(bar_o(pb), (it / PB - 1) & 1, fail);
         ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
         tc_fence_after();
       }
-      if (it > 0 && __any_sync(0xffffffffu, raise)) {
-        if (PB > 1) {                             // O must be stable: wait for P(it-1) V(it-1) as well
-          ok = mbar_wait(bar_o((it - 1) % PB), ((it - 1) / PB) & 1, fail);
+      if (it > 0 && __any_sync(0xffffffffu, raise)) {     // (the same decision in both warps of the pair)
+        if (PB > 1) {                           // O must be stable: wait for P(it-1) V(it-1) as well
+          ok = ok && mbar_wait(bar_o((it - 1) % PB), ((it - 1) / PB) & 1, fail);
           ok = __all_sync(0xffffffffu, ok);
-          if (!ok) break;
           tc_fence_after();
         }
-        {
-          const float alpha = fast_exp2(m_run - m_use);   // 1 for rows that keep their maximum
-          l_run *= alpha;
+        const float alpha = fast_exp2(m_r - m_use);       // 1 for rows that keep their maximum
+        l_r *= alpha;
 #pragma unroll
-          for (int ch = 0; ch < 4; ++ch) {
-            uint32_t v[32];
-            tmem_ld32(t_lane + C::O_COL + ch * 32, v);
-            tmem_ld_wait();
+        for (int ch = 0; ch < 2; ++ch) {        // this warp's 64 of O's 128 columns
+          uint32_t v[32];
+          const uint32_t col = t_lane + C::O_COL + half * 64 + ch * 32;
+          tmem_ld32(col, v);
+          tmem_ld_wait();
 #pragma unroll
-            for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) * alpha);
-            tmem_st32(t_lane + C::O_COL + ch * 32, v);
-          }
-          tmem_st_wait();
+          for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) * alpha);
+          tmem_st32(col, v);
         }
+        tmem_st_wait();
       }
-      m_run = m_new;
-      // pass 2: P = exp2(S * scale - m), row sums, P (bf16) to shared memory
+      m_r = m_new;
+      // P = exp2(S * scale - m) as bf16 to shared memory, row sums
       float sum0 = 0.f, sum1 = 0.f;
-#pragma unroll 1
-      for (int half = 0; half < KT / 64; ++half) {
-        if (KT > 64) load_s(half, sr);
-        const uint32_t prow = p_s + pb * C::P_ONE + half * ROWS * 128 + row_local * 128;
+      constexpr int panel = KT == 128 ? 1 : 0;  // with 128-key tiles the second half is the second 64-key panel
+      const uint32_t prow = p_s + pb * C::P_ONE + half * panel * ROWS * 128 + row * 128;
+      const int chunk0 = KT == 128 ? 0 : half * 4;
 #pragma unroll
-        for (int c = 0; c < 8; ++c) {          // chunk c = keys 8c .. 8c+7 of this row
-          uint32_t w[4];
+      for (int cc = 0; cc < NV / 8; ++cc) {     // chunk: 8 keys of this row
+        uint32_t w[4];
 #pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const int j = c * 8 + e * 2;
-            const float p0 = fast_exp2(fmaf(__uint_as_float(sr[j >> 5][j & 31]), p.scale_log2, -m_use));
-            const float p1 = poly_exp2(fmaf(__uint_as_float(sr[(j + 1) >> 5][(j + 1) & 31]), p.scale_log2, -m_use));
-            sum0 += p0;
-            sum1 += p1;
-            w[e] = pack_bf16(p0, p1);
-          }
-          if (row_active)
-            asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(prow + ((c ^ (row_local & 7)) << 4)), "r"(w[0]),
-                         "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
+        for (int e = 0; e < 4; ++e) {
+          const int j = cc * 8 + e * 2;
+          const float p0 = fast_exp2(fmaf(__uint_as_float(sr[j >> 5][j & 31]), p.scale_log2, -m_use));
+          const float p1 = poly_exp2(fmaf(__uint_as_float(sr[(j + 1) >> 5][(j + 1) & 31]), p.scale_log2, -m_use));
+          sum0 += p0;
+          sum1 += p1;
+          w[e] = pack_bf16(p0, p1);
         }
+        asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(prow + (((chunk0 + cc) ^ (row & 7)) << 4)), "r"(w[0]),
+                     "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
       }
-      l_run += sum0 + sum1;
+      l_r += sum0 + sum1;
       fence_async_smem();            // P was written with ordinary stores
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_p(pb));
     }
-    if (ok && n_my > 0) {
-      ok = mbar_wait(bar_o((n_my - 1) % PB), ((n_my - 1) / PB) & 1, fail);   // the last P V product has completed
+    if (n_my > 0) {
+      ok = ok && mbar_wait(bar_o((n_my - 1) % PB), ((n_my - 1) / PB) & 1, fail);   // the last P V product has completed
       tc_fence_after();
     }
+    // row sums: add the other warp's share (the buffer of the parity no tile is using)
+    s_pair[n_my & 1][half][row] = l_r;
+    pair_sync();
+    l_run = l_r + s_pair[n_my & 1][half ^ 1][row];
+    m_run = m_r;
     if (!ok) s_fail = 1;
   }
   __syncthreads();
@@ -802,7 +819,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
 
   {
     constexpr int TPR = kD / 4;                       // 32 threads per row, 4 columns each
-    constexpr int RPP = kThreads / TPR;
+    constexpr int RPP = C::THREADS / TPR;
     const int i4 = tid % TPR;
     for (int lr = tid / TPR; lr < rows_per; lr += RPP) {
       const int grow = row0 + split * rows_per + lr;
@@ -921,7 +938,7 @@ twig_status launch_umma(const AttnParams &p, const MapEntry *maps, int batch, in
   }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(n_splits, p.n_kv_heads * p.row_blocks, batch);
-  cfg.blockDim = dim3(kThreads);
+  cfg.blockDim = dim3(UmmaCfg<ROWS, KT>::THREADS);
   cfg.dynamicSmemBytes = C::SMEM_BYTES;
   cfg.stream = st;
   cudaLaunchAttribute attr[2];
