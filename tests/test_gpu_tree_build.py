@@ -5,7 +5,7 @@ import torch
 
 from oracle import twig_oracle as O
 from paper_2503_14075_b200 import synth
-from gpu_common import DEV, dev_bf16, dev_i32
+from gpu_common import DEV, MAX_ABS_TOL, REL_L2_TOL, dev_bf16, dev_i32, f64, host_bits, max_abs, rel_l2_rows
 
 pytestmark = pytest.mark.gpu
 
@@ -112,3 +112,90 @@ def test_tree_feeds_verification(tw):
         assert n == n_max and parent[b, 0] == -1
         assert all(0 <= parent[b, i] < i for i in range(1, n))
         O.tree_mask(parent[b, :n], n, 5)               # the oracle accepts it as a tree
+
+
+def test_draft_verify_accept_chain(tw):
+    """The device arrays flow from one entry point into the next without touching the host: token tree ->
+    target tokens -> tree attention -> acceptance + KV append, against the same chain of oracle functions."""
+    E, K, D, n_max, t_max, V = 3, 2, 3, 10, 16, 512
+    B, Hq, Hkv, d, nl, L0 = 2, 4, 2, 128, 2, 70
+    rng = synth.rng_for(7, 23)
+    levels = [rng.standard_normal((B, 1 if l == 0 else K, V)).astype(np.float32) * 2 for l in range(D)]
+    parent_d, tok_d, n_d = (torch.zeros((B, t_max), dtype=torch.int32, device=DEV), torch.zeros((B, t_max), dtype=torch.int32, device=DEV),
+                            torch.zeros(B, dtype=torch.int32, device=DEV))
+    cap = 1 + E + (D - 1) * K * E
+    st = tw.TreeState(B, cap, DEV)
+    status = torch.zeros(B, dtype=torch.int32, device=DEV)
+    tw.tree_reset(st)
+    src, lo, hi = torch.zeros((B, 1), dtype=torch.int32, device=DEV), 0, 1
+    for l in range(D):
+        tw.tree_expand_level(torch.from_numpy(levels[l]).to(DEV), src, E, hi, st, dev_status=status)
+        lo, hi = hi, hi + (1 if l == 0 else K) * E
+        if l + 1 < D:
+            src = torch.zeros((B, K), dtype=torch.int32, device=DEV)
+            tw.tree_select_expansion(st, lo, hi, src, dev_status=status)
+    tw.tree_finalize(st, cap, n_max, parent_d, tok_d, n_d, dev_status=status)
+    # oracle trees; target logits that follow one root-to-leaf path of each tree and then diverge
+    trees = [O.build_token_tree([lv[b] for lv in levels], E, K, n_max) for b in range(B)]
+    tgt = rng.standard_normal((B, t_max, V)).astype(np.float32)
+    planted = []
+    for b in range(B):
+        par, tk = trees[b][0], trees[b][1]
+        u, depth = 0, 0
+        for _ in range(2 + b):                                  # follow up to 2 (request 0) or 3 (request 1) levels
+            kids = [i for i in range(len(par)) if par[i] == u]
+            if not kids:
+                break
+            tgt[b, u, tk[kids[-1]]] = 40.0                       # the target agrees with the last child
+            u, depth = kids[-1], depth + 1
+        planted.append(depth)
+    assert min(planted) >= 1
+    tgt_d = torch.from_numpy(tgt).to(DEV)
+    base_d = torch.zeros((B, t_max), dtype=torch.int32, device=DEV)
+    tw.tree_base_argmax(tgt_d, n_d, base_d, dev_status=status)
+    # verification inputs
+    q = synth.normal_bf16(rng, (nl, B, t_max, Hq, d), d, d ** 0.5)
+    tkv = [synth.normal_bf16(rng, (nl, B, Hkv, t_max, d), d, d ** 0.5) for _ in range(2)]
+    cache = [synth.normal_bf16(rng, (nl, B, Hkv, L0 + t_max, d), d, d ** 0.5) for _ in range(2)]
+    kv_len = np.array([L0, L0 - 9], dtype=np.int32)
+    ck, cv = dev_bf16(cache[0]), dev_bf16(cache[1])
+    kvl = dev_i32(kv_len)
+    q_d, tk_d, tv_d = dev_bf16(q), dev_bf16(tkv[0]), dev_bf16(tkv[1])
+    out = torch.zeros((nl, B, t_max, Hq, d), dtype=torch.bfloat16, device=DEV)
+    kvc = tw.KV.of(ck, cv)
+    for layer in range(nl):
+        tw.tree_verify_attention(q_d[layer], tk_d[layer], tv_d[layer], kvc, layer, kvl, n_d, parent_d, out[layer], dev_status=status)
+    alen = torch.zeros(B, dtype=torch.int32, device=DEV)
+    path = torch.full((B, t_max), -7, dtype=torch.int32, device=DEV)
+    bonus = torch.zeros(B, dtype=torch.int32, device=DEV)
+    tw.tree_accept_compact(parent_d, tok_d, base_d, n_d, tk_d, tv_d, kvc, kvl, alen, path, bonus, dev_status=status)
+    torch.cuda.synchronize()
+    assert not status.cpu().numpy().any()
+    # the same chain on the CPU
+    base_o = O.base_argmax(tgt.astype(np.float64), [len(t[0]) for t in trees])
+    ok_, ov_ = cache[0].copy(), cache[1].copy()
+    paths = []
+    for b in range(B):
+        par, tk = trees[b][0], trees[b][1]
+        n = len(par)
+        assert n_d.cpu().numpy()[b] == n and np.array_equal(parent_d.cpu().numpy()[b, :n], par)
+        a, pth, bt = O.tree_accept(par, tk, base_o[b], n)
+        assert a == planted[b]                                   # the planted path is what gets accepted
+        assert alen.cpu().numpy()[b] == a and bonus.cpu().numpy()[b] == bt
+        assert path.cpu().numpy()[b, :a + 1].tolist() == pth.tolist()
+        paths.append(pth.tolist())
+    par_pad = np.full((B, t_max), -1, dtype=np.int32)
+    for b in range(B):
+        par_pad[b, :len(trees[b][0])] = trees[b][0]
+    n_list = [len(t[0]) for t in trees]
+    for layer in range(nl):
+        want, _ = O.tree_attention(f64(q[layer]), f64(tkv[0][layer]), f64(tkv[1][layer]), f64(cache[0][layer]),
+                                   f64(cache[1][layer]), kv_len, n_list, par_pad)
+        got = f64(host_bits(out[layer]))
+        for b in range(B):
+            n = n_list[b]
+            assert max_abs(got[b, :n], want[b, :n]) <= MAX_ABS_TOL
+            assert rel_l2_rows(got[b, :n].reshape(-1, d), want[b, :n].reshape(-1, d)) <= REL_L2_TOL
+    new_len = O.accept_compact(tkv[0], tkv[1], ok_, ov_, kv_len, paths)
+    assert np.array_equal(kvl.cpu().numpy(), new_len)
+    assert np.array_equal(host_bits(ck), ok_) and np.array_equal(host_bits(cv), ov_)
