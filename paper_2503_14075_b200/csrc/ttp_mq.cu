@@ -77,6 +77,7 @@ ttp_mq_partial_kernel(const __nv_bfloat16 *__restrict__ q_text, int n_text_max,
   const int see_lo = r_lo < rows ? t_first + r_lo : -1, see_hi = r_hi < rows ? t_first + r_hi : -1;
   const uint32_t q_frag = q_s + (warp * 16 + (lane & 7) + ((lane >> 3) & 1) * 8) * 128;
   const int sw = lane & 7;
+  uint32_t qf[KS][4];                  // this warp's Q fragments: the same for every key tile
 
   // S = Q K^T of this warp's 16 rows against the 64 keys of a stage, scaled into the exp2 domain
   // and masked (causal; keys past the prompt)
@@ -86,16 +87,13 @@ ttp_mq_partial_kernel(const __nv_bfloat16 *__restrict__ q_text, int n_text_max,
     for (int i = 0; i < NT; ++i) s[i][0] = s[i][1] = s[i][2] = s[i][3] = 0.f;
 #pragma unroll
     for (int ks = 0; ks < KS; ++ks) {
-      uint32_t qf[4];
-      const int c = ks * 2 + (lane >> 4);
-      ldsm_x4(q_frag + (c >> 3) * 64 * 128 + (((c & 7) ^ sw) << 4), qf);
 #pragma unroll
       for (int np = 0; np < NT / 2; ++np) {
         uint32_t kb[4];
         const int key = np * 16 + (lane & 7) + (lane >> 4) * 8;
         ldsm_x4(kst + mq_off(key, ks * 2 + ((lane >> 3) & 1)), kb);
-        mma_bf16(s[2 * np], qf, kb[0], kb[1]);
-        mma_bf16(s[2 * np + 1], qf, kb[2], kb[3]);
+        mma_bf16(s[2 * np], qf[ks], kb[0], kb[1]);
+        mma_bf16(s[2 * np + 1], qf[ks], kb[2], kb[3]);
       }
     }
 #pragma unroll
@@ -114,6 +112,13 @@ ttp_mq_partial_kernel(const __nv_bfloat16 *__restrict__ q_text, int n_text_max,
   const int t_begin1 = split * per1, t_end1 = min(n_t1, t_begin1 + per1);     // this CTA's share
   if (t_begin1 < t_end1) load_keys(t_begin1, 0);
   cp_async_commit();                                          // (this group also carries Q)
+  cp_async_wait<0>();
+  __syncthreads();
+#pragma unroll
+  for (int ks = 0; ks < KS; ++ks) {
+    const int c = ks * 2 + (lane >> 4);
+    ldsm_x4(q_frag + (c >> 3) * 64 * 128 + (((c & 7) ^ sw) << 4), qf[ks]);
+  }
   for (int t = t_begin1; t < t_end1; ++t) {
     const int it = t - t_begin1;
     if (t + 1 < t_end1) load_keys(t + 1, (it + 1) & 1);
