@@ -199,3 +199,50 @@ def test_draft_verify_accept_chain(tw):
     new_len = O.accept_compact(tkv[0], tkv[1], ok_, ov_, kv_len, paths)
     assert np.array_equal(kvl.cpu().numpy(), new_len)
     assert np.array_equal(host_bits(ck), ok_) and np.array_equal(host_bits(cv), ov_)
+
+
+def test_next_row_entry_points_report_bad_arguments(tw):
+    """Host-side argument checks return an error and launch nothing; device-side checks set dev_status and
+    leave the outputs of that request untouched.  (None of these cases can read or write out of bounds.)"""
+    from paper_2503_14075_b200.twig import TwigError
+    B, V, E, K = 2, 256, 4, 2
+    st = tw.TreeState(B, 1 + E + K * E, DEV)
+    tw.tree_reset(st)
+    logits = torch.zeros((B, 1, V), dtype=torch.float32, device=DEV)
+    root = torch.zeros((B, 1), dtype=torch.int32, device=DEV)
+    status = torch.zeros(B, dtype=torch.int32, device=DEV)
+    # more children than the state can hold
+    with pytest.raises(TwigError) as e:
+        tw.tree_expand_level(logits, root, 16, 1, st)
+    assert e.value.code == 2          # TWIG_ERR_SHAPE
+    # more children per node than the kernel supports
+    with pytest.raises(TwigError) as e:
+        tw.tree_expand_level(logits, root, 17, 1, tw.TreeState(B, 64, DEV))
+    assert e.value.code == 3          # TWIG_ERR_UNSUPPORTED
+    # selection wider than the level
+    tw.tree_expand_level(logits, root, E, 1, st, dev_status=status)
+    with pytest.raises(TwigError) as e:
+        tw.tree_select_expansion(st, 1, 1 + E, torch.zeros((B, E + 1), dtype=torch.int32, device=DEV))
+    assert e.value.code == 2
+    # a source node that is not older than the level (request 1): flagged on the device, request 0 is built
+    src = torch.tensor([[1, 2], [1, 7]], dtype=torch.int32, device=DEV)
+    lv2 = torch.zeros((B, K, V), dtype=torch.float32, device=DEV)
+    tw.tree_expand_level(lv2, src, E, 1 + E, st, dev_status=status)
+    torch.cuda.synchronize()
+    assert status.cpu().tolist() == [0, 4]                      # TWIG_DEV_BAD_TREE
+    assert st.parent.cpu().numpy()[0, 1 + E:1 + E + K * E].tolist() == [1] * E + [2] * E
+    # target tokens: a node count beyond t_max is flagged, nothing is written for that request
+    out = torch.full((B, 3), -5, dtype=torch.int32, device=DEV)
+    status.zero_()
+    tw.tree_base_argmax(torch.zeros((B, 3, V), dtype=torch.float32, device=DEV), dev_i32([3, 4]), out, dev_status=status)
+    torch.cuda.synchronize()
+    assert status.cpu().tolist() == [0, 4] and out.cpu().numpy()[1].tolist() == [-5, -5, -5]
+    # multi-query guide: more text tokens after the image than q_text holds
+    qt = torch.zeros((1, 4, 2, 128), dtype=torch.bfloat16, device=DEV)
+    k = torch.zeros((1, 4, 32, 128), dtype=torch.bfloat16, device=DEV)
+    sc = torch.full((1, 8), -1.0, dtype=torch.float32, device=DEV)
+    ws = torch.zeros(tw.ttp_multiquery_workspace_bytes(1, 4, 2, 8), dtype=torch.uint8, device=DEV)
+    st1 = torch.zeros(1, dtype=torch.int32, device=DEV)
+    tw.ttp_score_multiquery(qt, k, dev_i32([20]), dev_i32([4]), dev_i32([8]), sc, ws, dev_status=st1)   # 8 text tokens > 2
+    torch.cuda.synchronize()
+    assert st1.cpu().tolist() == [1] and np.all(sc.cpu().numpy() == 0)        # TWIG_DEV_BAD_LAYOUT, scores zeroed
