@@ -269,21 +269,6 @@ int32_t twig_set_early_prefix(int32_t on);
  * 1, 2, 4 or 8; 0 = automatic (default).  A tuning control.  Returns the previous value. */
 int32_t twig_set_attention_splits(int32_t splits);
 
-/* ---- Longest requests first (scheduling aid for batches of unequal length; not in the paper) ----
- * The requests of a tree_verify_attention call are independent and their key axes differ in length.
- * CTAs are handed out in request order; with the long requests last, the GPU ends the launch on
- * a few long CTAs.  tree_order_requests writes order[0..batch) = the requests by decreasing
- * kv_len[b] + n_nodes[b] (equal lengths in index order).  twig_set_request_order(order) makes the
- * following tree_verify_attention calls map their CTAs through it (results are the same, bit for
- * bit; NULL restores request order).  order is a device array that must stay valid, and hold a
- * permutation of 0..batch-1, for as long as it is set; entries outside that range are skipped.
- * With twig_set_early_prefix(1) the array falls under the same promise as kv_len: the kernel
- * that precedes the attention call must not write it.
- */
-twig_status tree_order_requests(const int32_t *kv_len, const int32_t *n_nodes, int32_t batch,
-                                int32_t *order, void *stream);
-void twig_set_request_order(const int32_t *order);
-
 /* ---- Draft-side token tree ---------------------------------------------------
  * Sec. 4.3 and the appendix's "Tree-based self-speculative decoding": the tree is rooted at the last
  * accepted token and grown level by level with an expansion width E, a selection width K and a

@@ -312,13 +312,6 @@ def base_argmax(logits, n_nodes):
     return out
 
 
-def order_requests(kv_len, n_nodes):
-    """Requests by decreasing key-axis length kv_len + n_nodes, equal lengths in index order (a
-    scheduling aid of the GPU library; no counterpart in the paper)."""
-    total = [int(a) + int(b) for a, b in zip(kv_len, n_nodes)]
-    return np.array(sorted(range(len(total)), key=lambda i: (-total[i], i)), dtype=np.int32)
-
-
 # --------------------------------------------------------------------------
 # Draft-side token tree (Sec. 4.3 "tree-based SSD", Appendix "Tree-based self-speculative decoding")
 # --------------------------------------------------------------------------

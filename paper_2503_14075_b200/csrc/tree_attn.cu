@@ -84,6 +84,7 @@ tree_attn_kernel(const AttnParams p) {
   const int wm = warp / WN, wn = warp % WN;
   const int split = blockIdx.x, n_splits = gridDim.x;
   const int hk = blockIdx.y / p.row_blocks, rb = blockIdx.y % p.row_blocks;
+  const int b = blockIdx.z;
   // barrier of the WN warps that share a row group (ids 1..WM; 0 is __syncthreads)
   auto group_sync = [&]() {
     if (WN > 1) asm volatile("bar.sync %0, %1;" ::"r"(1 + wm), "n"(32 * WN) : "memory");
@@ -94,9 +95,6 @@ tree_attn_kernel(const AttnParams p) {
   // the parent array nor cache rows below kv_len: those are then read (and the prefix tiles
   // prefetched) while that kernel is still draining, and only Q and the tree's rows wait.
   if (!p.early_prefix) grid_dependency_sync();
-  // which request this CTA works on (all CTAs of a cluster share blockIdx.z, so the exits below stay uniform)
-  const int b = p.order ? p.order[blockIdx.z] : (int)blockIdx.z;
-  if (b < 0 || b >= p.batch) return;            // not a request: nothing to do (the caller's order array is wrong)
   // ---- per-request metadata; every exit below is uniform over the cluster ----
   const int n = p.n_nodes[b], L = p.kv_len[b];
   const int my_parent = tid < p.t_max ? p.parent[(long long)b * p.t_max + tid] : -1;   // (in flight with n, L)
@@ -617,40 +615,12 @@ static twig_status dispatch_attn(AttnParams &p, int batch, int rows, cudaStream_
   }
 }
 
-// order[i] = the request with the i-th longest key axis (kv_len + n_nodes), equal lengths in index order.
-// One CTA; rank by counting.
-__global__ void __launch_bounds__(256)
-order_requests_kernel(const int *__restrict__ kv_len, const int *__restrict__ n_nodes, int batch, int *__restrict__ order) {
-  extern __shared__ int s_len[];
-  grid_dependency_sync();
-  for (int i = threadIdx.x; i < batch; i += blockDim.x) s_len[i] = kv_len[i] + n_nodes[i];
-  __syncthreads();
-  for (int i = threadIdx.x; i < batch; i += blockDim.x) {
-    const int mine = s_len[i];
-    int rank = 0;
-    for (int j = 0; j < batch; ++j) rank += (s_len[j] > mine || (s_len[j] == mine && j < i)) ? 1 : 0;
-    order[rank] = i;
-  }
-}
-
 }  // namespace twig
 
 using namespace twig;
 
-extern "C" twig_status tree_order_requests(const int32_t *kv_len, const int32_t *n_nodes, int32_t batch,
-                                           int32_t *order, void *stream) {
-  if (!kv_len || !n_nodes || !order) return TWIG_ERR_NULL;
-  if (batch <= 0) return TWIG_ERR_SHAPE;
-  if (batch > TWIG_MAX_BATCH) return TWIG_ERR_UNSUPPORTED;
-  order_requests_kernel<<<1, 256, (size_t)batch * sizeof(int), static_cast<cudaStream_t>(stream)>>>(kv_len, n_nodes, batch, order);
-  return launch_status();
-}
-
 static int g_attention_path = 0;
 static int g_early_prefix = 0;
-static const int32_t *g_request_order = nullptr;
-
-extern "C" void twig_set_request_order(const int32_t *order) { g_request_order = order; }
 
 extern "C" int32_t twig_set_early_prefix(int32_t on) {
   const int prev = g_early_prefix;
@@ -716,7 +686,6 @@ extern "C" twig_status tree_verify_attention(const void *q, const void *tree_k, 
   p.max_len = cache->max_len;
   p.row_blocks = 1;
   p.early_prefix = (g_early_prefix && launch_overlap_enabled()) ? 1 : 0;
-  p.order = g_request_order;
   const float scale = softmax_scale != 0.f ? softmax_scale : 1.f / sqrtf((float)cache->head_dim);
   p.scale_log2 = scale * 1.4426950408889634f;
   const int rows = t_max * p.group;

@@ -21,7 +21,6 @@ struct AttnParams {
   long long c_sl;
   int layer, n_layers, batch;
   int early_prefix;   // see twig_set_early_prefix
-  const int *order;   // see twig_set_request_order: blockIdx.z -> request, or nullptr for the identity
   float scale_log2;   // softmax_scale * log2(e)
 };
 

@@ -203,6 +203,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int split = blockIdx.x, n_splits = gridDim.x;
   const int hk = blockIdx.y / p.row_blocks, rb = blockIdx.y % p.row_blocks;
+  const int b = blockIdx.z;
 
   const uint32_t q_s = smem_u32(smem);
   const uint32_t p_s = q_s + C::Q_BYTES;
@@ -257,12 +258,6 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
   };
 
   grid_dependency_sync();
-  // which request this CTA works on (all CTAs of a cluster share blockIdx.z)
-  const int b = p.order ? p.order[blockIdx.z] : (int)blockIdx.z;
-  if (b < 0 || b >= p.batch) {                  // not a request: the caller's order array is wrong
-    leave();
-    return;
-  }
   // ---- per-request metadata; every exit below is uniform over the cluster ----
   const int n = p.n_nodes[b], L = p.kv_len[b];
   const int my_parent = tid < p.t_max ? p.parent[(long long)b * p.t_max + tid] : -1;

@@ -27,7 +27,7 @@ DEV_OK, DEV_BAD_LAYOUT, DEV_BAD_KEEP, DEV_BAD_INDEX, DEV_BAD_TREE, DEV_OVERFLOW,
 MAX_NODES, MAX_VISUAL, MAX_BATCH = 64, 16384, 4096
 
 EXPORTS = ["twig_status_str", "twig_set_launch_overlap", "twig_set_early_prefix", "twig_set_attention_path", "twig_set_attention_splits", "twig_workspace_bytes", "ttp_score", "ttp_score_gated", "ttp_multiquery_workspace_bytes", "ttp_score_multiquery", "ttp_score_noalloc", "ttp_topk", "ttp_compact", "ttp_compact_rows",
-           "ttp_score_topk_compact", "tree_verify_attention", "tree_order_requests", "twig_set_request_order", "tree_reset", "tree_expand_level", "tree_select_expansion", "tree_finalize", "tree_base_argmax", "tree_accept_compact"]
+           "ttp_score_topk_compact", "tree_verify_attention", "tree_reset", "tree_expand_level", "tree_select_expansion", "tree_finalize", "tree_base_argmax", "tree_accept_compact"]
 
 
 class TwigError(RuntimeError):
@@ -97,10 +97,6 @@ _lib.ttp_score_topk_compact.argtypes = [_vp, _vp, _i64, _i64, _i64, _i32, _vp, _
 _lib.tree_verify_attention.restype = C.c_int
 _lib.tree_verify_attention.argtypes = [_vp, _vp, _vp, _kvp, _i32, _vp, _vp, _vp, _i32, _i32, _f32, _vp, _vp,
                                        _vp, _vp, _sz, _vp]
-_lib.tree_order_requests.restype = C.c_int
-_lib.tree_order_requests.argtypes = [_vp, _vp, _i32, _vp, _vp]
-_lib.twig_set_request_order.restype = None
-_lib.twig_set_request_order.argtypes = [_vp]
 _lib.tree_reset.restype = C.c_int
 _lib.tree_reset.argtypes = [_vp, _vp, _vp, _i32, _i32, _vp]
 _lib.tree_expand_level.restype = C.c_int
@@ -257,17 +253,6 @@ def tree_verify_attention(q, tree_k, tree_v, cache: KV, layer, kv_len, n_nodes, 
     _check(_lib.tree_verify_attention(_p(q), _p(tree_k), _p(tree_v), C.byref(cache), layer, _p(kv_len),
                                       _p(n_nodes), _p(parent), T, Hq, softmax_scale, _p(out), _p(lse),
                                       _p(dev_status), _p(ws), ws_bytes, _stream(stream)))
-
-
-def tree_order_requests(kv_len, n_nodes, order, stream=None):
-    """order [B] int32 (out): the requests by decreasing kv_len + n_nodes, equal lengths in index order."""
-    _check(_lib.tree_order_requests(_p(kv_len), _p(n_nodes), kv_len.shape[0], _p(order), _stream(stream)))
-
-
-def twig_set_request_order(order):
-    """Maps the CTAs of the following tree_verify_attention calls through `order` (a device int32
-    permutation that the caller keeps alive); None restores request order."""
-    _lib.twig_set_request_order(_p(order))
 
 
 class TreeState:

@@ -222,41 +222,3 @@ def test_early_prefix_gives_the_same_bits(tw, shape):
         n = n_nodes[b]
         for o in outs:
             assert np.array_equal(host_bits(o)[b, :n], ref[b, :n])
-
-
-@pytest.mark.parametrize("path", [1, 2], ids=["mma", "tcgen05"])
-def test_request_order_gives_the_same_bits(tw, path):
-    """Longest-first scheduling: the order array matches the oracle's sort, and mapping the CTAs through it
-    (or through any permutation) changes nothing in the output; entries that are no request are skipped."""
-    name, B, Hq, Hkv, d, n_nodes, depth, kv_len = [s for s in SHAPES if s[0] == "idle-request"][0]
-    wl = _wl(B, Hq, Hkv, d, n_nodes, depth)
-    rng = synth.rng_for(9, 654)
-    ver = synth.make_verify_inputs(wl, rng, n_layers=1, gain=d ** 0.5)
-    ck, cv = synth.make_cache(wl, rng, max(kv_len) + 70, n_layers=1, gain=d ** 0.5)
-    ref, ref_lse, st0 = run_attention(tw, wl, ver, ck, cv, kv_len, path=path)
-    order = torch.full((B,), -3, dtype=torch.int32, device=DEV)
-    tw.tree_order_requests(dev_i32(kv_len), dev_i32(ver["n_nodes"]), order)
-    torch.cuda.synchronize()
-    assert order.cpu().numpy().tolist() == O.order_requests(kv_len, ver["n_nodes"]).tolist()
-    try:
-        tw.twig_set_request_order(order)
-        got, got_lse, st1 = run_attention(tw, wl, ver, ck, cv, kv_len, path=path)
-        rev = torch.flip(order, dims=[0]).contiguous()
-        tw.twig_set_request_order(rev)
-        got2, got2_lse, st2 = run_attention(tw, wl, ver, ck, cv, kv_len, path=path)
-        # an entry that is no request: that CTA group does nothing, its request keeps the canary
-        bad = order.clone()
-        skipped = int(bad[0].item())
-        bad[0] = B + 5
-        tw.twig_set_request_order(bad)
-        got3, _, st3 = run_attention(tw, wl, ver, ck, cv, kv_len, path=path)
-    finally:
-        tw.twig_set_request_order(None)
-    assert not st0.any() and not st1.any() and not st2.any() and not st3.any()
-    assert np.array_equal(got, ref) and np.array_equal(got_lse, ref_lse)
-    assert np.array_equal(got2, ref) and np.array_equal(got2_lse, ref_lse)
-    for b in range(B):
-        if b == skipped:
-            assert np.all(got3[b] == CANARY)
-        else:
-            assert np.array_equal(got3[b], ref[b])

@@ -560,15 +560,6 @@ def test_base_argmax_library_and_ties():
     assert np.array_equal(O.base_argmax(z, [4]), O.base_argmax(sp.softmax(z, axis=-1), [4]))
 
 
-def test_order_requests_is_a_stable_descending_sort():
-    rng = np.random.default_rng(37)
-    kv, nn = rng.integers(0, 50, 40), rng.integers(0, 5, 40)
-    got = O.order_requests(kv, nn)
-    assert sorted(got.tolist()) == list(range(40))
-    assert got.tolist() == np.argsort(-(kv + nn), kind="stable").tolist()
-    assert O.order_requests([5, 5, 7], [1, 1, 0]).tolist() == [2, 0, 1]
-
-
 def test_token_tree_pins():
     """Tree builder: enumeration of every path of a tiny vocabulary; chain and full-tree limits;
     tie rules; closure under parents."""
