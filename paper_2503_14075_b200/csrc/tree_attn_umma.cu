@@ -397,10 +397,11 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
         mbar_arrive(bar_full(slot));
       }
     };
-    // the first ring of tiles is requested before Q: they are the long pole
+    // K of the first tile, then Q (what S(0) needs), then the rest of the first ring
     const int n_first = min(n_units, kSlots);
-    for (int u = 0; u < n_first; ++u) issue_unit(u);
+    if (n_first > 0) issue_unit(0);
     if (n_my > 0) issue_q();
+    for (int u = 1; u < n_first; ++u) issue_unit(u);
     for (int u = n_first; u < n_units && ok; ++u) {
       publish_q();                              // (all ring slots are in flight by now)
       ok = mbar_wait(bar_empty(u % kSlots), (u / kSlots - 1) & 1, fail);
