@@ -157,11 +157,11 @@ struct UmmaCfg {
   static constexpr int Q_BYTES = ROWS * kD * 2;          // two 64-column panels of ROWS x 128 B
   static constexpr int P_ONE = ROWS * KT * 2;            // ROWS x KT keys bf16, KT/64 panels of ROWS x 128 B
   // two P buffers where shared memory allows: the softmax of tile t+1 then never waits for P(t) V(t)
-  static constexpr int P_BUFS = 2;
+  // (64 rows with 64-key tiles, two CTAs per SM: a fifth ring slot measured better than the second P buffer)
+  static constexpr int P_BUFS = (ROWS == 64 && KT == 64) ? 1 : 2;
   static constexpr int P_BYTES = P_BUFS * P_ONE;
-  // four slots where five would not leave room for the second P buffer (128 rows with 128-key
-  // tiles in one CTA; 64 rows with 64-key tiles in two CTAs per SM)
-  static constexpr int SLOTS = ((ROWS == 128 && KT == 128) || (ROWS == 64 && KT == 64)) ? 4 : kMaxSlots;
+  // 128 rows with 128-key tiles: four slots, so that two P buffers still fit in shared memory
+  static constexpr int SLOTS = (ROWS == 128 && KT == 128) ? 4 : kMaxSlots;
   static constexpr int RING_BYTES = SLOTS * TILE_BYTES;
   static constexpr uint32_t TMEM_COLS = KT == 64 ? 256 : 512;   // S: [0,KT) and [KT,2KT); O: [2KT, 2KT+128)
   static constexpr uint32_t O_COL = 2 * KT;
