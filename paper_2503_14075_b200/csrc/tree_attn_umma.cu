@@ -43,7 +43,7 @@ namespace {
 constexpr int kD = 128;          // head_dim
 // warps 0-3 softmax, warp 4 loader, warp 5 MMA issuer; with 128-row accumulators warps 6-9 are a
 // second softmax group (UmmaCfg::THREADS)
-constexpr int kMaxSlots = 5;                      // ring of K / V tiles (K0 V0 K1 V1 K2 ...)
+constexpr int kMaxSlots = 6;                      // ring of K / V tiles (K0 V0 K1 V1 K2 ...)
 constexpr float kLazyMax = 8.f;                   // raise the running max only beyond this (log2 units)
 constexpr int kSpinLimit = 1 << 22;
 
@@ -157,11 +157,11 @@ struct UmmaCfg {
   static constexpr int Q_BYTES = ROWS * kD * 2;          // two 64-column panels of ROWS x 128 B
   static constexpr int P_ONE = ROWS * KT * 2;            // ROWS x KT keys bf16, KT/64 panels of ROWS x 128 B
   // two P buffers where shared memory allows: the softmax of tile t+1 then never waits for P(t) V(t)
-  // (64 rows with 64-key tiles, two CTAs per SM: a fifth ring slot measured better than the second P buffer)
-  static constexpr int P_BUFS = (ROWS == 64 && KT == 64) ? 1 : 2;
+  // (64-key tiles with two CTAs per SM: one more ring slot measured better than the second P buffer)
+  static constexpr int P_BUFS = (ROWS <= 64 && KT == 64) ? 1 : 2;
   static constexpr int P_BYTES = P_BUFS * P_ONE;
   // 128 rows with 128-key tiles: four slots, so that two P buffers still fit in shared memory
-  static constexpr int SLOTS = (ROWS == 128 && KT == 128) ? 4 : kMaxSlots;
+  static constexpr int SLOTS = (ROWS == 128 && KT == 128) ? 4 : (ROWS == 32 && KT == 64) ? 6 : 5;
   static constexpr int RING_BYTES = SLOTS * TILE_BYTES;
   static constexpr uint32_t TMEM_COLS = KT == 64 ? 256 : 512;   // S: [0,KT) and [KT,2KT); O: [2KT, 2KT+128)
   static constexpr uint32_t O_COL = 2 * KT;
