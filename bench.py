@@ -160,6 +160,9 @@ class Replica:
         self.bonus = torch.zeros(B, dtype=torch.int32, device=dev)
         self.n_steps = MAX_STEPS
         self.early_prefix = True
+        self.attn_kernel, self.attn_splits, self.plain_launch = 0, 0, False
+        # scratch of the persistent attention kernel: zero-filled once, used by the attention calls only
+        self.attn_ws = torch.zeros(tw.tree_attention_workspace_bytes(B, Hq, T), dtype=torch.uint8, device=dev)
 
     def prune(self, tw):
         tw.ttp_score_topk_compact(self.twig_q, self.twig_k, self.prefix_len, self.vis_start, self.n_vis, self.keep,
@@ -172,10 +175,10 @@ class Replica:
         for layer in range(self.wl.n_layers):
             # layer 0 follows the accept (or prune) kernel, which writes kv_len; the other layers follow
             # the previous layer's attention, which leaves lengths and cache alone
-            tw.twig_set_early_prefix(1 if (layer > 0 and self.early_prefix) else 0)
+            flags = tw.attn_flags(kernel=self.attn_kernel, splits=self.attn_splits, plain_launch=self.plain_launch,
+                                  early_prefix=layer > 0 and self.early_prefix)
             tw.tree_verify_attention(q[layer], tk[layer], tv[layer], self.cache, layer, self.kv_len, self.n_nodes,
-                                     self.parent, self.out, dev_status=self.status)
-        tw.twig_set_early_prefix(0)
+                                     self.parent, self.out, dev_status=self.status, ws=self.attn_ws, flags=flags)
 
     def accept(self, tw, s):
         slot = s % POOL
@@ -210,14 +213,13 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device(dev))
     wl = synth.workload(args.workload)
     peaks = load_peaks()
-    tw.twig_set_attention_path(args.attn_path)
     tw.twig_set_launch_overlap(0 if args.no_overlap else 1)
-    tw.twig_set_attention_splits(args.attn_splits)
     max_len = ((max(wl.pruned_len) + max(wl.gen_target) + wl.t_max + 8 + 31) // 32) * 32
 
     reps = [Replica(wl, sid, torch, tw, dev, max_len) for sid in replicas.replica_streams(rank, N_ROT)]
     for rp in reps:
         rp.early_prefix = not args.no_early_prefix
+        rp.attn_kernel, rp.attn_splits = args.attn_path, args.attn_splits
     stream = torch.cuda.current_stream()
 
     # ---- dry run: how many verify steps each request needs to emit its target ------------
@@ -418,7 +420,8 @@ def run_e2e(torch, tw, wl, reps, stream, world, dev, dist, step_graphs):
             else:
                 for layer in range(wl.n_layers):
                     tw.tree_verify_attention(d_q[layer], d_tk[layer], d_tv[layer], rp.cache, layer, rp.kv_len,
-                                             rp.n_nodes, rp.parent, rp.out, dev_status=rp.status)
+                                             rp.n_nodes, rp.parent, rp.out, dev_status=rp.status, ws=rp.attn_ws,
+                                             flags=tw.attn_flags(kernel=rp.attn_kernel, splits=rp.attn_splits))
                 tw.tree_accept_compact(rp.parent, rp.draft[s], rp.tgt[s], rp.n_nodes, d_tk, d_tv, rp.cache, rp.kv_len,
                                        rp.accept_len, rp.path, rp.bonus, dev_status=rp.status)
             res_dev[:, 0] = rp.accept_len
@@ -451,11 +454,19 @@ def run_e2e(torch, tw, wl, reps, stream, world, dev, dist, step_graphs):
                     + ("kernels replayed from the step's graph" if step_graphs else "kernels launched one by one")}
 
 
-def _time_attention(torch, tw, wl, kv_lens, nl, stream_id, dev, reps=10):
-    """Mean launch time (us) of tree_verify_attention over `nl` resident layers (their KV does
-    not fit L2 together), plus the algorithmic bytes and flops of one launch."""
+L2_BYTES = 126 * 1024 * 1024
+
+
+def _time_attention(torch, tw, wl, kv_lens, nl, stream_id, dev, reps=20, kernel=0, early_prefix=False, splits=0):
+    """Launch time (us: median and best over `reps` timed passes) of tree_verify_attention over `nl`
+    resident layers visited in turn (nl = 0: as many as it takes for their KV to exceed twice the L2,
+    so that no launch finds its cache in L2), plus the algorithmic bytes and flops of one launch.
+    kernel: 0 automatic, 1 mma.sync, 2 tcgen05 with cluster splits, 3 persistent tcgen05."""
     rng = synth.rng_for(wl.index, stream_id)
     B, Hq, Hkv, d, T = wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.t_max
+    by = attn_bytes_per_launch(wl, kv_lens)
+    if nl <= 0:
+        nl = int(min(40, max(2, -(-2 * L2_BYTES // by))))
 
     def bf(x):
         return torch.from_numpy(np.ascontiguousarray(x).view(np.int16)).to(dev).view(torch.bfloat16)
@@ -468,24 +479,29 @@ def _time_attention(torch, tw, wl, kv_lens, nl, stream_id, dev, reps=10):
     nn = torch.from_numpy(ver["n_nodes"]).to(dev)
     kvl = torch.from_numpy(np.asarray(kv_lens, dtype=np.int32)).to(dev)
     out = torch.zeros((B, T, Hq, d), dtype=torch.bfloat16, device=dev)
+    ws = torch.zeros(tw.tree_attention_workspace_bytes(B, Hq, T), dtype=torch.uint8, device=dev)
+    status = torch.zeros(B, dtype=torch.int32, device=dev)
     cache = tw.KV.of(ck, cv)
     stream = torch.cuda.current_stream()
+    # nothing but these launches runs in the stream, so the early-prefix promise holds for every launch
+    flags = tw.attn_flags(kernel=kernel, early_prefix=early_prefix, splits=splits)
 
     def loop():
         for layer in range(nl):
-            tw.tree_verify_attention(q[layer], tk[layer], tv[layer], cache, layer, kvl, nn, par, out)
+            tw.tree_verify_attention(q[layer], tk[layer], tv[layer], cache, layer, kvl, nn, par, out,
+                                     dev_status=status, ws=ws, flags=flags)
     for _ in range(3):
         loop()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
-    for _ in range(reps):
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(reps + 1)]
+    evs[0].record(stream)
+    for r in range(reps):
         loop()
-    e1.record(stream)
+        evs[r + 1].record(stream)
     torch.cuda.synchronize()
-    us = e0.elapsed_time(e1) * 1e3 / (reps * nl)
-    by = attn_bytes_per_launch(wl, kv_lens)
+    assert not status.cpu().numpy().any(), "device status set"
+    per = sorted(evs[r].elapsed_time(evs[r + 1]) * 1e3 / nl for r in range(reps))
     flops = sum(4 * Hq * n * d * (int(l) + n) for n, l in zip(wl.n_nodes, kv_lens))
-    return us, by, flops
+    return {"us": statistics.median(per), "us_best": per[0], "bytes": by, "flops": flops, "layers": nl, "reps": reps}
 
 
 def extra_rooflines(torch, tw, peaks, dev):
@@ -502,24 +518,38 @@ def extra_rooflines(torch, tw, peaks, dev):
                 "achieved": round(by / us / 1e3, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": round(by / us / 1e3 / peaks["hbm_gbs"], 4)}
 
+    def attn_entry(t, bound="hbm"):
+        """Median of the timed passes is the figure; the best pass and, where the call was also timed
+        with the early-prefix promise (the launches of a verification step other than its first may make
+        it), that figure are reported beside it."""
+        us, by, fl = t["us"], t["bytes"], t["flops"]
+        e = hbm_entry(us, by)
+        if bound == "tensor":
+            e = {"bound": "tensor", "flops_per_launch": fl, "bytes_per_launch": by, "us_per_launch": round(us, 2),
+                 "achieved": round(fl / us / 1e6, 1), "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                 "frac": round(fl / us / 1e6 / peaks["bf16_tflops"], 4), "hbm_gbs": round(by / us / 1e3, 1)}
+        e.update({"us_best": round(t["us_best"], 2), "reps": t["reps"], "layers_in_rotation": t["layers"]})
+        return e
+
+    def attn_both(wl_, lens_, sid, bound="hbm"):
+        e = attn_entry(_time_attention(torch, tw, wl_, lens_, 0, sid, dev), bound)
+        t2 = _time_attention(torch, tw, wl_, lens_, 0, sid, dev, early_prefix=True)
+        e["us_per_launch_early_prefix"] = round(t2["us"], 2)
+        num = t2["flops"] / 1e6 if bound == "tensor" else t2["bytes"] / 1e3
+        e["frac_early_prefix"] = round(num / t2["us"] / (peaks["bf16_tflops"] if bound == "tensor" else peaks["hbm_gbs"]), 4)
+        return e
+
     wl3 = synth.workload(3)
     lens3 = [p + g // 2 for p, g in zip(wl3.pruned_len, wl3.gen_target)]      # half-way through generation
-    us, by, _ = _time_attention(torch, tw, wl3, lens3, 2, 501, dev)
-    res["tree_attn_c3_midway"] = hbm_entry(us, by)
+    res["tree_attn_c3_midway"] = attn_both(wl3, lens3, 501)
     wl = synth.workload(4)
     B, Hq, Hkv, d, T = wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.t_max
-    us, by, _ = _time_attention(torch, tw, wl, [wl.final_kv_len] * B, 8, 500, dev)
-    res["tree_attn_c4_L1472"] = hbm_entry(us, by)
+    res["tree_attn_c4_L1472"] = attn_both(wl, [wl.final_kv_len] * B, 500)
     # the same shape with a long cache (beyond the configuration's 1.5k): the kernel's steady state
-    us, by, _ = _time_attention(torch, tw, wl, [8128] * B, 2, 504, dev, reps=5)
-    res["tree_attn_c4shape_L8128"] = hbm_entry(us, by)
+    res["tree_attn_c4shape_L8128"] = attn_entry(_time_attention(torch, tw, wl, [8128] * B, 0, 504, dev))
     wl5 = synth.workload(5)
-    us, by, fl = _time_attention(torch, tw, wl5, [wl5.final_kv_len] * wl5.batch, 2, 502, dev, reps=5)
-    res["tree_attn_c5_L8128"] = {"bound": "tensor", "flops_per_launch": fl, "bytes_per_launch": by,
-                                 "us_per_launch": round(us, 2), "achieved": round(fl / us / 1e6, 1),
-                                 "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                                 "frac": round(fl / us / 1e6 / peaks["bf16_tflops"], 4),
-                                 "hbm_gbs": round(by / us / 1e3, 1)}
+    for L5 in (384, 2048, wl5.final_kv_len):
+        res[f"tree_attn_c5_L{L5}"] = attn_entry(_time_attention(torch, tw, wl5, [L5] * wl5.batch, 0, 502, dev), "tensor")
     rng = synth.rng_for(4, 503)
     stream = torch.cuda.current_stream()
     # pruning gather, 2 layers at a time of the B=4 x 3008-token prompt cache.  A chain of launches over
@@ -645,6 +675,134 @@ def extra_rooflines(torch, tw, peaks, dev):
 
 
 # ----------------------------------------------------------------------------------
+# single-kernel cases: small, self-contained launch sets for a profiler capture or a quick timing
+#   python bench.py --case attn --workload 4 --kv-len 1472 --layers 2 --iters 3 [--attn-path 3] [--early-prefix]
+#   python bench.py --case gather|score|accept|argmax|gscore|mqscore --workload N [--layers n] [--iters k]
+# Each holds well under a few GB on the device and launches a handful of kernels, so that a
+# capture ends by itself.  Prints one JSON line.
+# ----------------------------------------------------------------------------------
+def run_case(a):
+    import torch
+    from paper_2503_14075_b200 import build as _build
+    _build.build()
+    from paper_2503_14075_b200 import twig as tw
+    dev = "cuda:0"
+    torch.cuda.set_device(0)
+    wl = synth.workload(a.workload)
+    rng = synth.rng_for(a.workload, 900)
+    B, Hq, Hkv, d, T = wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.t_max
+
+    def bf(x):
+        return torch.from_numpy(np.ascontiguousarray(x).view(np.int16)).to(dev).view(torch.bfloat16)
+
+    def i32(x):
+        return torch.from_numpy(np.ascontiguousarray(x, dtype=np.int32)).to(dev)
+
+    def timed(fn):
+        stream = torch.cuda.current_stream()
+        fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(a.iters):
+            fn()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) * 1e3 / a.iters
+
+    out = {"case": a.case, "workload": wl.name}
+    if a.case == "attn":
+        if a.kv_len:
+            lens = [a.kv_len] * B
+        elif wl.index == 3:
+            lens = [p + g // 2 for p, g in zip(wl.pruned_len, wl.gen_target)]
+        else:
+            lens = [wl.final_kv_len or max(wl.pruned_len)] * B
+        t = _time_attention(torch, tw, wl, lens, a.layers, 900, dev, reps=a.iters, kernel=a.attn_path,
+                            early_prefix=a.early_prefix, splits=a.attn_splits)
+        out.update({"kernel": a.attn_path, "early_prefix": a.early_prefix, "kv_len": lens[0] if a.kv_len else "workload",
+                    "us_per_launch": round(t["us"], 2), "us_best": round(t["us_best"], 2), "bytes_per_launch": t["bytes"],
+                    "gbs": round(t["bytes"] / t["us"] / 1e3, 1), "tflops": round(t["flops"] / t["us"] / 1e6, 1),
+                    "layers": t["layers"]})
+    elif a.case == "gather":
+        nl = a.layers or 2
+        pre = synth.make_prefill(wl, rng, n_layers=nl)
+        sk, sv = bf(pre["cache_k"]), bf(pre["cache_v"])
+        kept = np.full((B, max(1, max(wl.keep))), -1, dtype=np.int32)
+        for b in range(B):
+            kept[b, :wl.keep[b]] = np.sort(rng.choice(wl.n_vis[b], wl.keep[b], replace=False))
+        meta = (i32(kept), i32(pre["keep"]), i32(pre["prefix_len"]), i32(pre["vis_start"]), i32(pre["n_vis"]))
+        if a.in_place:
+            src = tw.KV.of(sk, sv)
+            us = timed(lambda: tw.ttp_compact(src, src, *meta))
+        else:
+            dk = torch.zeros((nl, B, Hkv, max(wl.pruned_len) + 8, d), dtype=torch.bfloat16, device=dev)
+            src, dst = tw.KV.of(sk, sv), tw.KV.of(dk, torch.zeros_like(dk))
+            us = timed(lambda: tw.ttp_compact(src, dst, *meta))
+        by = 2 * sum(wl.pruned_len) * wl.kv_row_bytes() * nl
+        out.update({"layers": nl, "in_place": a.in_place, "us_per_launch": round(us, 2), "bytes_per_launch": by,
+                    "gbs": round(by / us / 1e3, 1)})
+    elif a.case in ("score", "gscore", "mqscore", "prune"):
+        nl = (a.layers or wl.n_layers) if a.case == "prune" else 1
+        pre = synth.make_prefill(wl, rng, n_layers=nl)
+        q, k = bf(pre["twig_q"]), bf(pre["twig_k"])
+        scores = torch.zeros((B, max(wl.n_vis)), dtype=torch.float32, device=dev)
+        kept = torch.zeros((B, max(wl.keep)), dtype=torch.int32, device=dev)
+        ws = torch.empty(tw.twig_workspace_bytes(B, Hq, d, k.shape[2], 64), dtype=torch.uint8, device=dev)
+        pl, vs, nv, kp = i32(pre["prefix_len"]), i32(pre["vis_start"]), i32(pre["n_vis"]), i32(pre["keep"])
+        if a.case == "score":
+            def run():
+                tw.ttp_score(q, k, pl, vs, nv, scores, ws)
+                tw.ttp_topk(scores, nv, kp, kept)
+            us = timed(run)
+            out.update({"us_per_score_topk_pair": round(us, 2),
+                        "k_bytes": int(sum(Hkv * lp * d * 2 for lp in wl.prefix_len))})
+        elif a.case == "prune":
+            sk, sv = bf(pre["cache_k"]), bf(pre["cache_v"])
+            dk = torch.zeros((nl, B, Hkv, max(wl.pruned_len) + 8, d), dtype=torch.bfloat16, device=dev)
+            src, dst = tw.KV.of(sk, sv), tw.KV.of(dk, torch.zeros_like(dk))
+            us = timed(lambda: tw.ttp_score_topk_compact(q, k, pl, vs, nv, kp, scores, kept, src, dst, ws))
+            out.update({"layers": nl, "us_per_call": round(us, 2)})
+        elif a.case == "gscore":
+            qg, kg = bf(synth.gate_bf16(rng, pre["twig_q"].shape)), bf(synth.gate_bf16(rng, pre["twig_k"].shape))
+            us = timed(lambda: tw.ttp_score_gated(q, qg, k, kg, pl, vs, nv, scores, ws))
+            by = 2 * sum(Hkv * n * d * 2 for n in wl.n_vis)
+            out.update({"us_per_call": round(us, 2), "bytes": int(by), "gbs": round(by / us / 1e3, 1)})
+        else:
+            n_txt = max(1, max(wl.text_after))
+            qt = bf(synth.normal_bf16(rng, (B, Hq, n_txt, d), d))
+            wsm = torch.empty(tw.ttp_multiquery_workspace_bytes(B, Hq, n_txt, max(wl.n_vis)), dtype=torch.uint8, device=dev)
+            us = timed(lambda: tw.ttp_score_multiquery(qt, k, pl, vs, nv, scores, wsm))
+            fl = sum(2 * Hq * d * c * (t + 2 * n + (c + 1) / 2) for t, n, c in zip(wl.text_before, wl.n_vis, wl.text_after))
+            out.update({"us_per_call": round(us, 2), "tflops": round(fl / us / 1e6, 1)})
+    elif a.case == "accept":
+        nl = a.layers or wl.n_layers
+        ver = synth.make_verify_inputs(wl, rng, n_layers=nl)
+        ck = torch.zeros((nl, B, Hkv, 256 + T, d), dtype=torch.bfloat16, device=dev)
+        cache = tw.KV.of(ck, torch.zeros_like(ck))
+        tk, tv = bf(ver["tree_k"]), bf(ver["tree_v"])
+        par, nn = i32(ver["parent"]), i32(ver["n_nodes"])
+        dt, ba = i32(ver["draft_tok"]), i32(ver["base_argmax"])
+        kvl = torch.zeros(B, dtype=torch.int32, device=dev)
+        alen, bonus = torch.zeros(B, dtype=torch.int32, device=dev), torch.zeros(B, dtype=torch.int32, device=dev)
+        path = torch.zeros((B, T), dtype=torch.int32, device=dev)
+
+        def run():
+            kvl.fill_(100)
+            tw.tree_accept_compact(par, dt, ba, nn, tk, tv, cache, kvl, alen, path, bonus)
+        out.update({"layers": nl, "us_per_fill_accept_pair": round(timed(run), 2)})
+    elif a.case == "argmax":
+        V = 32000
+        logits = torch.from_numpy(rng.standard_normal((B, T, V), dtype=np.float32)).to(dev).to(torch.bfloat16)
+        nn = i32(wl.n_nodes)
+        res = torch.zeros((B, T), dtype=torch.int32, device=dev)
+        us = timed(lambda: tw.tree_base_argmax(logits, nn, res))
+        by = sum(wl.n_nodes) * V * 2
+        out.update({"us_per_launch": round(us, 2), "bytes": int(by), "gbs": round(by / us / 1e3, 1)})
+    print(json.dumps(out))
+
+
+# ----------------------------------------------------------------------------------
 # CPU oracle arm
 # ----------------------------------------------------------------------------------
 def oracle_verify_steps(wl, host, n_steps, n_layers):
@@ -751,8 +909,20 @@ def main():
     ap.add_argument("--no-early-prefix", action="store_true", help="do not prefetch the KV prefix under the previous layer")
     ap.add_argument("--no-overlap", action="store_true", help="plain launches (no programmatic stream serialization)")
     ap.add_argument("--attn-splits", type=int, default=0, help="force key splits per cluster (0 auto)")
-    ap.add_argument("--attn-path", type=int, default=0, help="tree-attention kernel: 0 auto, 1 mma.sync, 2 tcgen05")
+    ap.add_argument("--attn-path", type=int, default=0,
+                    help="tree-attention kernel: 0 auto, 1 mma.sync, 2 tcgen05 (cluster splits), 3 tcgen05 persistent")
+    ap.add_argument("--case", default=None,
+                    choices=["attn", "gather", "score", "prune", "accept", "argmax", "gscore", "mqscore"],
+                    help="run one small single-kernel case (for a profiler capture) instead of the benchmark")
+    ap.add_argument("--kv-len", type=int, default=0, help="--case attn: cache length of every request")
+    ap.add_argument("--layers", type=int, default=0, help="--case: layers resident / per call (0: the case's default)")
+    ap.add_argument("--iters", type=int, default=3, help="--case: timed repetitions")
+    ap.add_argument("--early-prefix", action="store_true", help="--case attn: launch with the early-prefix promise")
+    ap.add_argument("--in-place", action="store_true", help="--case gather: compact the cache in place")
     args = ap.parse_args()
+    if args.case:
+        run_case(args)
+        return
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
         run_reference(args)

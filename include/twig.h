@@ -236,8 +236,10 @@ twig_status ttp_score_topk_compact(
  *   parent   [batch, t_max] int32; parent[b,0] = -1, parent[b,i] in [0, i)
  *   lse      [batch, n_q_heads, t_max] fp32 or NULL
  * t_max <= TWIG_MAX_NODES.  Rows of nodes >= n_nodes[b] are not written.
- * softmax_scale 0 means 1/sqrt(head_dim).  ws may be NULL when ws_bytes is 0
- * (the current kernels combine key splits on chip and use no scratch).
+ * softmax_scale 0 means 1/sqrt(head_dim).  ws may be NULL when ws_bytes is 0: the kernels that
+ * combine key splits on chip need no scratch; a scratch buffer (see tree_verify_attention_ex for
+ * its contract: zero-filled at first use, used by these calls only) lets large calls run on the
+ * persistent kernel.
  */
 twig_status tree_verify_attention(const void *q, const void *tree_k, const void *tree_v,
                                   const twig_kv *cache, int32_t layer, const int32_t *kv_len,
@@ -245,29 +247,56 @@ twig_status tree_verify_attention(const void *q, const void *tree_k, const void 
                                   int32_t n_q_heads, float softmax_scale, void *out, float *lse,
                                   int32_t *dev_status, void *ws, size_t ws_bytes, void *stream);
 
-/* Selects the tree-attention kernel: 0 = automatic (default), 1 = mma.sync kernel,
- * 2 = tcgen05 kernel (head_dim 128 only; other shapes fall back to 1).  Both compute
- * the same function; this is a tuning and testing control.  Returns the previous value. */
-int32_t twig_set_attention_path(int32_t path);
+/* tree_verify_attention with per-call flags (the call above is this one with flags = 0).
+ *
+ * TWIG_ATTN_EARLY_PREFIX: the caller promises that the kernel which precedes this call in its stream
+ *   writes neither kv_len, n_nodes, parent nor cache rows below kv_len (true when that kernel is
+ *   another layer's attention or a projection of the same verification step; false right after
+ *   tree_accept_compact or ttp_compact, which write kv_len).  The kernel then reads the lengths and
+ *   starts fetching the cached prefix while the preceding kernel is still draining; q, tree_k and
+ *   tree_v are still read only after it has completed.  Results do not change when the promise holds.
+ * TWIG_ATTN_PLAIN_LAUNCH: launch without programmatic stream serialization (see twig_set_launch_overlap).
+ * TWIG_ATTN_KERNEL(k): run exactly kernel k, a testing and tuning control (all kernels compute the
+ *   same function).  TWIG_ATTN_KERNEL_AUTO picks by shape; _MMA is the mma.sync kernel (any shape);
+ *   _TCGEN05 the tcgen05 kernel whose key splits are the CTAs of a cluster; _STREAM the persistent
+ *   tcgen05 kernel (needs ws, below).  The tcgen05 kernels need head_dim 128 and a cache layout that a
+ *   tensor map can describe; a named kernel that cannot run the call returns TWIG_ERR_UNSUPPORTED (or
+ *   TWIG_ERR_WORKSPACE); only the automatic choice moves on to another kernel.
+ * TWIG_ATTN_SPLITS(n): force n = 1, 2, 4 or 8 key splits per cluster in the _MMA and _TCGEN05 kernels.
+ *
+ * Scratch of the persistent kernel.  One CTA per SM slot walks an equal share of all (request, kv head,
+ * row block, key tile) work; a work item that straddles two CTAs is finished by whichever of them
+ * arrives last, through ws: per-item arrival counters followed by per-CTA partial results.
+ *   size      tree_attention_workspace_bytes(batch, n_q_heads, max_nodes) (twig_workspace_bytes is
+ *             at least that large)
+ *   contents  the first call that uses a buffer must find it ZERO-FILLED (cudaMemset once after
+ *             allocation); every call leaves its counters at zero again.  Nothing else may write
+ *             the buffer between calls: do not pass the buffer that ttp_score uses.
+ *   sharing   calls whose kernels may overlap on the GPU need a buffer each.
+ * With ws = NULL / ws_bytes = 0 the automatic choice never takes the persistent kernel.
+ */
+#define TWIG_ATTN_EARLY_PREFIX 1u
+#define TWIG_ATTN_KERNEL_AUTO 0u
+#define TWIG_ATTN_KERNEL_MMA 1u
+#define TWIG_ATTN_KERNEL_TCGEN05 2u
+#define TWIG_ATTN_KERNEL_STREAM 3u
+#define TWIG_ATTN_KERNEL(k) ((uint32_t)(k) << 1)
+#define TWIG_ATTN_PLAIN_LAUNCH (1u << 4)
+#define TWIG_ATTN_SPLITS(n) ((uint32_t)(n) << 8)
+twig_status tree_verify_attention_ex(const void *q, const void *tree_k, const void *tree_v,
+                                     const twig_kv *cache, int32_t layer, const int32_t *kv_len,
+                                     const int32_t *n_nodes, const int32_t *parent, int32_t t_max,
+                                     int32_t n_q_heads, float softmax_scale, void *out, float *lse,
+                                     int32_t *dev_status, void *ws, size_t ws_bytes, void *stream,
+                                     uint32_t flags);
+size_t tree_attention_workspace_bytes(int32_t batch, int32_t n_q_heads, int32_t max_nodes);
 
 /* Launch overlap (default on): tree_verify_attention and tree_accept_compact launch their kernels
  * with programmatic stream serialization, so the next kernel of the stream is scheduled while the
  * current one drains; each kernel waits on the device for its predecessor before it reads anything,
- * so results do not change.  0 switches it off.  Returns the previous value. */
+ * so results do not change.  0 switches it off for the whole process (an atomic flag; a testing
+ * control, not meant to be toggled while other threads are launching).  Returns the previous value. */
 int32_t twig_set_launch_overlap(int32_t on);
-
-/* Early prefix (default off; needs launch overlap).  While it is on, the caller promises for every
- * following tree_verify_attention call that the kernel preceding it in its stream writes neither
- * kv_len, n_nodes, parent nor cache rows below kv_len (true between the layers of one verification
- * step, where the preceding kernels are the previous layer's; false right after tree_accept_compact or
- * ttp_compact, which write kv_len).  The small-call kernel then reads the lengths and prefetches the
- * cached prefix while the preceding kernel is still draining; Q, tree_k and tree_v are still read only
- * after it has completed.  Results do not change when the promise holds.  Returns the previous value. */
-int32_t twig_set_early_prefix(int32_t on);
-
-/* Forces the number of key splits (CTAs per cluster) of the tree-attention kernels:
- * 1, 2, 4 or 8; 0 = automatic (default).  A tuning control.  Returns the previous value. */
-int32_t twig_set_attention_splits(int32_t splits);
 
 /* ---- Draft-side token tree ---------------------------------------------------
  * Sec. 4.3 and the appendix's "Tree-based self-speculative decoding": the tree is rooted at the last

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.environ.get("TWIG_LIB") or os.path.join(HERE, "libtwig.so")   # TWIG_LIB: load another build
-SOURCES = ["api.cu", "ttp.cu", "ttp_mq.cu", "tree_attn.cu", "tree_attn_umma.cu", "tree_accept.cu", "tree_build.cu"]
+SOURCES = ["api.cu", "ttp.cu", "ttp_mq.cu", "tree_attn.cu", "tree_attn_umma.cu", "tree_attn_stream.cu", "tree_accept.cu", "tree_build.cu"]
 
 
 def _newest_source_mtime() -> float:
@@ -27,7 +27,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
-           "--use_fast_math" if False else "-DTWIG_BUILD", "-Xcompiler", "-fPIC,-O2", "-shared",
+           "-DTWIG_BUILD", "-Xcompiler", "-fPIC,-O2", "-shared",
            "-I", os.path.join(ROOT, "include"), "-I", CSRC, "-o", LIB]
     if verbose:
         cmd += ["-Xptxas", "-v"]

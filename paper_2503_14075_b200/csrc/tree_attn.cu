@@ -75,7 +75,8 @@ tree_attn_kernel(const AttnParams p) {
   __shared__ unsigned long long s_mask[TWIG_MAX_NODES];
   __shared__ int s_par[TWIG_MAX_NODES];
   __shared__ float s_stat[WN][ROWS];                            // row maxima of a tile, later row sums
-  __shared__ float2 r_ml[ROWS];                                 // received (m, l): [sender][owned row]
+  __shared__ float s_amax[WN][ROWS];                            // largest |O| of a row over a warp's columns
+  __shared__ float4 r_ml[ROWS];                                 // received (m, l, row scale): [sender][owned row]
   __shared__ int s_bad;
   __shared__ __align__(8) unsigned long long s_recv_bar;       // counts the bytes peers have pushed to this CTA
 
@@ -98,18 +99,16 @@ tree_attn_kernel(const AttnParams p) {
   // ---- per-request metadata; every exit below is uniform over the cluster ----
   const int n = p.n_nodes[b], L = p.kv_len[b];
   const int my_parent = tid < p.t_max ? p.parent[(long long)b * p.t_max + tid] : -1;   // (in flight with n, L)
-  if (n == 0) return;
+  // A CTA that leaves early still waits for the preceding kernel first: the kernel after this one
+  // only waits for this one, so every CTA has to carry the dependency on.
   const bool first = split == 0 && blockIdx.y == 0 && tid == 0;
-  if (n < 0 || n > p.t_max) {
-    if (first) flag_status(p.dev_status, b, TWIG_DEV_BAD_TREE);
-    return;
-  }
-  if (L < 0 || L > p.max_len) {
-    if (first) flag_status(p.dev_status, b, TWIG_DEV_OVERFLOW);
-    return;
-  }
   const int rows_total = n * p.group, row0 = rb * ROWS;
-  if (row0 >= rows_total) return;
+  if (n <= 0 || n > p.t_max || L < 0 || L > p.max_len || row0 >= rows_total) {
+    if (p.early_prefix) grid_dependency_sync();
+    if (first && (n < 0 || n > p.t_max)) flag_status(p.dev_status, b, TWIG_DEV_BAD_TREE);
+    else if (first && n > 0 && (L < 0 || L > p.max_len)) flag_status(p.dev_status, b, TWIG_DEV_OVERFLOW);
+    return;
+  }
   // Split merge: every CTA owns ROWS / n_splits rows and receives n_splits partials (m, l, O row)
   // for each of them; its barrier completes when all of those bytes have landed.
   const int rows_per = ROWS / n_splits;
@@ -118,7 +117,7 @@ tree_attn_kernel(const AttnParams p) {
     if (tid == 0) {
       // one arrival that announces the peers' bytes, one per warp for this CTA's own share
       mbar_init(recv_bar, 1 + C::THREADS / 32);
-      mbar_arrive_expect_tx(recv_bar, (uint32_t)((n_splits - 1) * rows_per * (D * 2 + 8)));
+      mbar_arrive_expect_tx(recv_bar, (uint32_t)((n_splits - 1) * rows_per * (D * 2 + 16)));
       mbar_init_fence_cluster();
     }
     __syncthreads();
@@ -214,6 +213,7 @@ tree_attn_kernel(const AttnParams p) {
   }
   __syncthreads();
   if (s_bad) {
+    if (p.early_prefix) grid_dependency_sync();
     if (first) flag_status(p.dev_status, b, TWIG_DEV_BAD_TREE);
     cp_async_wait<0>();       // nothing may still be writing this CTA's shared memory
     return;
@@ -424,16 +424,30 @@ tree_attn_kernel(const AttnParams p) {
   }
   cp_async_wait<0>();
 
-  // ---- row sums: add up the WN warps' shares ---------------------------------------------
+  // ---- row sums: add up the WN warps' shares; the rows' largest |O| -----
   l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1);
   l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
   l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1);
   l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
+  float amax_lo = 0.f, amax_hi = 0.f;
+  {     // (rows pass through the fp16 buffer of the merge even when there is a single split)
+#pragma unroll
+    for (int i = 0; i < OT; ++i) {
+      amax_lo = fmaxf(amax_lo, fmaxf(fabsf(o[i][0]), fabsf(o[i][1])));
+      amax_hi = fmaxf(amax_hi, fmaxf(fabsf(o[i][2]), fabsf(o[i][3])));
+    }
+    amax_lo = fmaxf(amax_lo, __shfl_xor_sync(0xffffffffu, amax_lo, 1));
+    amax_lo = fmaxf(amax_lo, __shfl_xor_sync(0xffffffffu, amax_lo, 2));
+    amax_hi = fmaxf(amax_hi, __shfl_xor_sync(0xffffffffu, amax_hi, 1));
+    amax_hi = fmaxf(amax_hi, __shfl_xor_sync(0xffffffffu, amax_hi, 2));
+  }
   if (WN > 1) {
     // (every warp of the group has read the last tile's maxima: that was before the tile's second barrier)
     if (tq == 0) {
       s_stat[wn][r_lo] = l_lo;
       s_stat[wn][r_hi] = l_hi;
+      s_amax[wn][r_lo] = amax_lo;
+      s_amax[wn][r_hi] = amax_hi;
     }
     group_sync();
     l_lo = l_hi = 0.f;
@@ -441,12 +455,14 @@ tree_attn_kernel(const AttnParams p) {
     for (int w = 0; w < WN; ++w) {
       l_lo += s_stat[w][r_lo];
       l_hi += s_stat[w][r_hi];
+      amax_lo = fmaxf(amax_lo, s_amax[w][r_lo]);
+      amax_hi = fmaxf(amax_hi, s_amax[w][r_hi]);
     }
   }
 
   // ---- merge the key splits of the cluster ------------------------------------------
-  // Each CTA writes its per-row partial (m, l, O / l as fp16: |O / l| is bounded by the largest
-  // |V| entry, and fp16 rounds eight times finer than the bf16 output) into the owner's shared memory (once the owner's
+  // Each CTA writes its per-row partial (m, l, O / l as scaled fp16, see row_scale: finer than the
+  // bf16 output whatever the magnitude of V) into the owner's shared memory (once the owner's
   // buffer is free: at once if it is a buffer of its own, else after every CTA of the cluster has
   // left its key loop) with asynchronous stores that report to the owner's barrier; the owner
   // waits for its bytes, combines its n_splits partials and stores.
@@ -466,7 +482,11 @@ tree_attn_kernel(const AttnParams p) {
     const int slot = split * rows_per + lr;
     unsigned char *ro = recv + (size_t)slot * D * 2;
     const float my_l = odd ? l_hi : l_lo;
-    const float inv_l = my_l > 0.f ? 1.f / my_l : 0.f;
+    // (a row that saw no key in this split carries m = -inf and counts for nothing)
+    const bool seen = (odd ? m_hi : m_lo) > -INFINITY && my_l > 0.f;
+    const float inv_l = seen ? 1.f / my_l : 0.f;
+    float down, up;
+    row_scale((odd ? amax_hi : amax_lo) * inv_l, down, up);
     const bool remote = owner != split;           // (n_splits == 1: never)
     const uint32_t ro_c = remote ? map_to_cta(smem_u32(ro), owner) : 0u;
     const uint32_t bar_c = remote ? map_to_cta(recv_bar, owner) : 0u;
@@ -475,16 +495,16 @@ tree_attn_kernel(const AttnParams p) {
       const float s0 = odd ? o[i][0] : o[i][2], s1 = odd ? o[i][1] : o[i][3];
       const float g0 = __shfl_xor_sync(0xffffffffu, s0, 1), g1 = __shfl_xor_sync(0xffffffffu, s1, 1);
       const float4 v = odd ? make_float4(g0, g1, o[i][2], o[i][3]) : make_float4(o[i][0], o[i][1], g0, g1);
-      const uint32_t h0 = pack_f16(v.x * inv_l, v.y * inv_l), h1 = pack_f16(v.z * inv_l, v.w * inv_l);
+      const uint32_t h0 = pack_f16(v.x * inv_l * down, v.y * inv_l * down), h1 = pack_f16(v.z * inv_l * down, v.w * inv_l * down);
       // 8-column groups of a row are XOR-swizzled by the row to spread banks
       const int off = ((((wn * OT + i) ^ (lr & 7)) << 3) + (tq >> 1) * 4) * 2;
       if (remote) st_async_b32x2(ro_c + off, h0, h1, bar_c);
       else *reinterpret_cast<uint2 *>(ro + off) = make_uint2(h0, h1);
     }
     if (wn == 0 && tq < 2) {
-      const float mm = odd ? m_hi : m_lo, ll = odd ? l_hi : l_lo;
-      if (remote) st_async_f32x2(map_to_cta(smem_u32(r_ml + slot), owner), mm, ll, bar_c);
-      else r_ml[slot] = make_float2(mm, ll);
+      const float mm = seen ? (odd ? m_hi : m_lo) : -INFINITY, ll = seen ? my_l : 0.f;
+      if (remote) st_async_f32x4(map_to_cta(smem_u32(r_ml + slot), owner), mm, ll, up, 0.f, bar_c);
+      else r_ml[slot] = make_float4(mm, ll, up, 0.f);
     }
   }
   if (n_splits > 1) {
@@ -528,8 +548,10 @@ tree_attn_kernel(const AttnParams p) {
 #pragma unroll
       for (int sd = 0; sd < 8; ++sd) {
         if (sd < n_splits) {
-          const float wgt = fast_exp2(mv[sd] - mstar) * r_ml[sd * rows_per + lr].y;
-          lsum += wgt;
+          const float4 ml = r_ml[sd * rows_per + lr];
+          const float wl = fast_exp2(mv[sd] - mstar) * ml.y;
+          lsum += wl;
+          const float wgt = wl * ml.z;
           const uint2 raw = *reinterpret_cast<const uint2 *>(recv + ((size_t)(sd * rows_per + lr) * D + col) * 2);
           const float2 v01 = unpack_f16(raw.x), v23 = unpack_f16(raw.y);
           acc.x = fmaf(wgt, v01.x, acc.x);
@@ -576,15 +598,13 @@ static twig_status launch_attn(const AttnParams &p, int batch, int n_splits, cud
   attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = launch_overlap_enabled() ? 2 : 1;
+  cfg.numAttrs = p.overlap ? 2 : 1;
   if (cudaLaunchKernelEx(&cfg, tree_attn_kernel<C>, p) != cudaSuccess) return TWIG_ERR_CUDA;
   return TWIG_OK;
 }
 
-static int g_forced_splits = 0;
-
-int pick_splits(int items, int max_tiles, int ctas_per_sm) {
-  if (g_forced_splits > 0) return g_forced_splits;
+int pick_splits(int items, int max_tiles, int ctas_per_sm, int forced) {
+  if (forced > 0) return forced;
   int s = 1;
   // double the key splits while all CTAs still fit in one wave
   while (s < 8 && items * s * 2 <= ctas_per_sm * 148 && s * 2 <= max_tiles) s *= 2;
@@ -606,7 +626,7 @@ static twig_status dispatch_attn(AttnParams &p, int batch, int rows, cudaStream_
   p.row_blocks = (rows + rows_per_cta - 1) / rows_per_cta;
   if ((long long)p.n_kv_heads * p.row_blocks > 65535) return TWIG_ERR_UNSUPPORTED;
   const int max_tiles = (p.max_len + p.t_max + 63) / 64;
-  const int n_splits = pick_splits(batch * p.n_kv_heads * p.row_blocks, max_tiles, 2);
+  const int n_splits = pick_splits(batch * p.n_kv_heads * p.row_blocks, max_tiles, 2, p.forced_splits);
   switch (rows_per_cta) {
     case 16: return launch_attn<C16>(p, batch, n_splits, st);
     case 32: return launch_attn<C32>(p, batch, n_splits, st);
@@ -619,37 +639,13 @@ static twig_status dispatch_attn(AttnParams &p, int batch, int rows, cudaStream_
 
 using namespace twig;
 
-static int g_attention_path = 0;
-static int g_early_prefix = 0;
-
-extern "C" int32_t twig_set_early_prefix(int32_t on) {
-  const int prev = g_early_prefix;
-  g_early_prefix = on != 0;
-  return prev;
-}
-
-
-extern "C" int32_t twig_set_attention_path(int32_t path) {
-  const int prev = g_attention_path;
-  if (path >= 0 && path <= 2) g_attention_path = path;
-  return prev;
-}
-
-extern "C" int32_t twig_set_attention_splits(int32_t splits) {
-  const int prev = g_forced_splits;
-  if (splits == 0 || splits == 1 || splits == 2 || splits == 4 || splits == 8) g_forced_splits = splits;
-  return prev;
-}
-
-extern "C" twig_status tree_verify_attention(const void *q, const void *tree_k, const void *tree_v,
-                                             const twig_kv *cache, int32_t layer,
-                                             const int32_t *kv_len, const int32_t *n_nodes,
-                                             const int32_t *parent, int32_t t_max,
-                                             int32_t n_q_heads, float softmax_scale, void *out,
-                                             float *lse, int32_t *dev_status, void *ws,
-                                             size_t ws_bytes, void *stream) {
-  (void)ws;
-  (void)ws_bytes;
+extern "C" twig_status tree_verify_attention_ex(const void *q, const void *tree_k, const void *tree_v,
+                                                const twig_kv *cache, int32_t layer,
+                                                const int32_t *kv_len, const int32_t *n_nodes,
+                                                const int32_t *parent, int32_t t_max,
+                                                int32_t n_q_heads, float softmax_scale, void *out,
+                                                float *lse, int32_t *dev_status, void *ws,
+                                                size_t ws_bytes, void *stream, uint32_t flags) {
   if (!q || !tree_k || !tree_v || !kv_len || !n_nodes || !parent || !out) return TWIG_ERR_NULL;
   twig_status s = check_kv(cache);
   if (s != TWIG_OK) return s;
@@ -657,6 +653,10 @@ extern "C" twig_status tree_verify_attention(const void *q, const void *tree_k, 
   if (n_q_heads % cache->n_kv_heads) return TWIG_ERR_SHAPE;
   if (t_max > TWIG_MAX_NODES) return TWIG_ERR_UNSUPPORTED;
   if (!aligned16(q) || !aligned16(tree_k) || !aligned16(tree_v) || !aligned16(out)) return TWIG_ERR_ALIGN;
+  const int kernel = (int)((flags >> 1) & 3u);
+  const int splits = (int)((flags >> 8) & 15u);
+  if (splits != 0 && splits != 1 && splits != 2 && splits != 4 && splits != 8) return TWIG_ERR_UNSUPPORTED;
+  if (ws_bytes > 0 && (!ws || !aligned16(ws))) return ws ? TWIG_ERR_ALIGN : TWIG_ERR_NULL;
 
   AttnParams p;
   p.q = static_cast<const __nv_bfloat16 *>(q);
@@ -685,19 +685,46 @@ extern "C" twig_status tree_verify_attention(const void *q, const void *tree_k, 
   p.group = n_q_heads / cache->n_kv_heads;
   p.max_len = cache->max_len;
   p.row_blocks = 1;
-  p.early_prefix = (g_early_prefix && launch_overlap_enabled()) ? 1 : 0;
+  p.overlap = (launch_overlap_enabled() && !(flags & TWIG_ATTN_PLAIN_LAUNCH)) ? 1 : 0;
+  p.early_prefix = ((flags & TWIG_ATTN_EARLY_PREFIX) && p.overlap) ? 1 : 0;
+  p.forced_splits = splits;
+  p.ws = static_cast<unsigned char *>(ws);
+  p.ws_bytes = ws_bytes;
   const float scale = softmax_scale != 0.f ? softmax_scale : 1.f / sqrtf((float)cache->head_dim);
   p.scale_log2 = scale * 1.4426950408889634f;
   const int rows = t_max * p.group;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  // automatic choice: the tcgen05 kernel once there are more than 32 query rows per kv head or
-  // enough (request, kv head) pairs to fill the GPU; the mma.sync kernel for small, latency-bound calls
-  const bool big = rows > 32 || (long long)cache->batch * cache->n_kv_heads >= 148;
-  if (cache->head_dim == 128 && softmax_scale >= 0.f &&
-      (g_attention_path == 2 || (g_attention_path == 0 && big))) {
-    const twig_status us = launch_tree_attn_umma(p, cache->batch, rows, st);
-    if (us != TWIG_ERR_UNSUPPORTED) return us;     // no tensor map for this layout: use the mma.sync kernel
+  const bool umma_ok = cache->head_dim == 128 && softmax_scale >= 0.f;
+  // A kernel named in the flags is the kernel that runs: what it cannot do is an error, never a
+  // quiet change of kernel.
+  if (kernel == TWIG_ATTN_KERNEL_TCGEN05 || kernel == TWIG_ATTN_KERNEL_STREAM) {
+    if (!umma_ok) return TWIG_ERR_UNSUPPORTED;
+    return kernel == TWIG_ATTN_KERNEL_STREAM ? launch_tree_attn_stream(p, cache->batch, rows, st)
+                                             : launch_tree_attn_umma(p, cache->batch, rows, st);
+  }
+  if (kernel == TWIG_ATTN_KERNEL_AUTO && umma_ok) {
+    // automatic choice: a tcgen05 kernel once there are more than 32 query rows per kv head or enough
+    // (request, kv head) pairs to fill the GPU (the persistent one when the caller has given it its
+    // scratch), the mma.sync kernel for small, latency-bound calls
+    const bool big = rows > 32 || (long long)cache->batch * cache->n_kv_heads >= 148;
+    if (big) {
+      twig_status us = TWIG_ERR_UNSUPPORTED;
+      if (ws_bytes > 0) us = launch_tree_attn_stream(p, cache->batch, rows, st);
+      if (us == TWIG_ERR_UNSUPPORTED || us == TWIG_ERR_WORKSPACE) us = launch_tree_attn_umma(p, cache->batch, rows, st);
+      if (us != TWIG_ERR_UNSUPPORTED) return us;     // no tensor map for this layout: the mma.sync kernel
+    }
   }
   return cache->head_dim == 128 ? dispatch_attn<128>(p, cache->batch, rows, st)
                                 : dispatch_attn<64>(p, cache->batch, rows, st);
+}
+
+extern "C" twig_status tree_verify_attention(const void *q, const void *tree_k, const void *tree_v,
+                                             const twig_kv *cache, int32_t layer,
+                                             const int32_t *kv_len, const int32_t *n_nodes,
+                                             const int32_t *parent, int32_t t_max,
+                                             int32_t n_q_heads, float softmax_scale, void *out,
+                                             float *lse, int32_t *dev_status, void *ws,
+                                             size_t ws_bytes, void *stream) {
+  return tree_verify_attention_ex(q, tree_k, tree_v, cache, layer, kv_len, n_nodes, parent, t_max, n_q_heads,
+                                  softmax_scale, out, lse, dev_status, ws, ws_bytes, stream, 0u);
 }

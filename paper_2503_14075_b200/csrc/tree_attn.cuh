@@ -2,6 +2,7 @@
 // the tcgen05 path): launch parameters and small PTX wrappers.
 #pragma once
 
+#include <cuda.h>
 #include <cuda_fp16.h>
 
 #include "twig_common.cuh"
@@ -20,8 +21,13 @@ struct AttnParams {
   const __nv_bfloat16 *cache_k0, *cache_v0;
   long long c_sl;
   int layer, n_layers, batch;
-  int early_prefix;   // see twig_set_early_prefix
+  int early_prefix;   // TWIG_ATTN_EARLY_PREFIX of the call
   float scale_log2;   // softmax_scale * log2(e)
+  // host side only: launch with programmatic stream serialization, forced key splits (0: automatic),
+  // the caller's scratch (persistent kernel)
+  int overlap, forced_splits;
+  unsigned char *ws;
+  size_t ws_bytes;
 };
 
 // ---- small PTX wrappers ----------------------------------------------------
@@ -105,6 +111,23 @@ __device__ __forceinline__ void st_async_f32x2(uint32_t dst, float a, float b, u
                ::"r"(dst), "f"(a), "f"(b), "r"(bar) : "memory");
 }
 
+__device__ __forceinline__ void st_async_f32x4(uint32_t dst, float a, float b, float c, float d, uint32_t bar) {
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.f32 [%0], {%1, %2, %3, %4}, [%5];"
+               ::"r"(dst), "f"(a), "f"(b), "f"(c), "f"(d), "r"(bar) : "memory");
+}
+
+// Partial rows cross between CTAs as fp16 of O / l (bounded by the largest |V| among the row's keys)
+// times a power of two that brings the row's largest entry into [1, 2): fp16 then keeps 11 bits of
+// every entry down to 2^-15 of that maximum, whatever the magnitude of V.  `amax` is that largest
+// |O / l|; `down` scales the row before the conversion, `up` = 1 / down travels with the row's (m, l).
+// Zero, infinite and NaN maxima are left unscaled.
+__device__ __forceinline__ void row_scale(float amax, float &down, float &up) {
+  const int ebits = (int)((__float_as_uint(amax) >> 23) & 0xffu);
+  const bool scalable = ebits > 0 && ebits < 255;
+  down = scalable ? __uint_as_float((uint32_t)(254 - ebits) << 23) : 1.f;
+  up = scalable ? __uint_as_float((uint32_t)ebits << 23) : 1.f;
+}
+
 // exp2 on the special-function unit; fast_exp2(-inf) = +0
 __device__ __forceinline__ float fast_exp2(float x) {
   float y;
@@ -112,8 +135,19 @@ __device__ __forceinline__ float fast_exp2(float x) {
   return y;
 }
 
+// Tensor maps (TMA) over the whole K and the whole V cache, dims (d, pos, head, batch, layer), boxes of
+// 64 columns x box_rows rows with the 128-byte swizzle; kept in a small host table per cache layout.
+struct CacheMaps {
+  alignas(64) CUtensorMap kmap;
+  alignas(64) CUtensorMap vmap;
+};
+bool cache_maps(const AttnParams &p, int box_rows, CacheMaps *out);
+
 // tcgen05 path (tree_attn_umma.cu): head_dim 128, rows = t_max * group.
 twig_status launch_tree_attn_umma(AttnParams &p, int batch, int rows, cudaStream_t st);
-int pick_splits(int items, int max_tiles, int ctas_per_sm);
+// persistent tcgen05 path (tree_attn_stream.cu): the same shapes, needs the caller's scratch
+twig_status launch_tree_attn_stream(AttnParams &p, int batch, int rows, cudaStream_t st);
+size_t tree_attn_stream_workspace_bytes(int batch, int n_q_heads, int max_nodes);
+int pick_splits(int items, int max_tiles, int ctas_per_sm, int forced);
 
 }  // namespace twig

@@ -32,7 +32,7 @@
 
 #include <mutex>
 
-#include "tree_attn.cuh"
+#include "tcgen05_common.cuh"
 
 namespace cg = cooperative_groups;
 
@@ -45,111 +45,9 @@ constexpr int kD = 128;          // head_dim
 // second softmax group (UmmaCfg::THREADS)
 constexpr int kMaxSlots = 6;                      // ring of K / V tiles (K0 V0 K1 V1 K2 ...)
 constexpr float kLazyMax = 8.f;                   // raise the running max only beyond this (log2 units)
-constexpr int kSpinLimit = 1 << 22;
-
-// ---- descriptors -------------------------------------------------------------
-// Shared-memory matrix descriptor, 128-byte swizzle, 8-row groups 1024 bytes apart.
-// lbo_bytes is the distance between 64-element groups along the leading (MN) dimension
-// and is only meaningful for MN-major operands.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes) {
-  uint64_t d = 0;
-  d |= (uint64_t)((addr & 0x3ffff) >> 4);
-  d |= (uint64_t)((lbo_bytes >> 4) & 0x3fff) << 16;
-  d |= (uint64_t)((1024u >> 4) & 0x3fff) << 32;
-  d |= (uint64_t)1 << 46;      // descriptor version of this architecture
-  d |= (uint64_t)2 << 61;      // 128-byte swizzle
-  return d;
-}
-// Instruction descriptor: bf16 x bf16 -> fp32, M = m (64 or 128), A K-major.
-__host__ __device__ constexpr uint32_t instr_desc(int m, int n, bool b_mn_major) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((uint32_t)(n >> 3) << 17) |
-         ((uint32_t)(m >> 4) << 24);
-}
-
-__device__ __forceinline__ void umma(uint32_t tmem_d, uint64_t a, uint64_t b, uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(tmem_d), "l"(a), "l"(b), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-// One box of the 5-D cache tensor map -> shared memory; completion is counted on `bar`.
-__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int pos,
-                                            int head, int batch, int layer) {
-  asm volatile(
-      "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
-      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(x), "r"(pos), "r"(head), "r"(batch), "r"(layer)
-      : "memory");
-}
-// Bounded wait on an mbarrier phase; false when the limit ran out or another role has failed.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *fail) {
-  for (int i = 0; i < kSpinLimit; ++i) {
-    if ((i & 1023) == 1023 && *fail) return false;
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    if (ok) return true;
-  }
-  return false;
-}
-
-#define TWIG_R8(a, o) "=r"(a[o]), "=r"(a[o + 1]), "=r"(a[o + 2]), "=r"(a[o + 3]), "=r"(a[o + 4]), "=r"(a[o + 5]), "=r"(a[o + 6]), "=r"(a[o + 7])
-// 32 consecutive fp32 columns of this thread's lane
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
-      : TWIG_R8(v, 0), TWIG_R8(v, 8), TWIG_R8(v, 16), TWIG_R8(v, 24)
-      : "r"(taddr));
-}
-// 64 consecutive fp32 columns of 16 lanes (the 16 lanes from the address's lane on), spread over
-// the warp like an mma.sync accumulator: for every 8-column group g, lane t holds columns
-// 8g + 2(t % 4) + {0, 1} of row t / 4 in v[4g], v[4g+1] and of row t / 4 + 8 in v[4g+2], v[4g+3].
-__device__ __forceinline__ void tmem_ld_16rows_64cols(uint32_t taddr, uint32_t (&v)[32]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.16x256b.x8.b32 "
-      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
-      : TWIG_R8(v, 0), TWIG_R8(v, 8), TWIG_R8(v, 16), TWIG_R8(v, 24)
-      : "r"(taddr));
-}
-#undef TWIG_R8
-#define TWIG_S8(a, o) "r"(a[o]), "r"(a[o + 1]), "r"(a[o + 2]), "r"(a[o + 3]), "r"(a[o + 4]), "r"(a[o + 5]), "r"(a[o + 6]), "r"(a[o + 7])
-__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32]) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
-      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
-      ::"r"(taddr), TWIG_S8(v, 0), TWIG_S8(v, 8), TWIG_S8(v, 16), TWIG_S8(v, 24)
-      : "memory");
-}
-#undef TWIG_S8
-__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // KT = keys per tile: 64 (two CTAs per SM, 256 tensor-memory columns each) or 128 (one CTA per SM
 // with all 512 columns: half as many, twice as large MMA instructions per key).
-// 2^x by range reduction and a cubic on the FMA pipe (relative error < 1e-3, far below the
-// bf16 rounding of P); used for half of the elements so that the special-function unit and
-// the FMA pipe share the exponentials.  Arguments below -126 give 2^-126 (in effect 0).
-__device__ __forceinline__ float poly_exp2(float x) {
-  x = fmaxf(x, -126.f);
-  const float t = x + 12582912.f;                 // 1.5 * 2^23: rounds x to the nearest integer
-  const float f = x - (t - 12582912.f);           // in [-0.5, 0.5]
-  float r = fmaf(f, 0.0555041f, 0.2402265f);
-  r = fmaf(r, f, 0.6931472f);
-  r = fmaf(r, f, 1.f);
-  return __int_as_float(__float_as_int(r) + (__float_as_int(t) << 23));   // * 2^n (the magic's bits shift out)
-}
-
 template <int ROWS, int KT>
 struct UmmaCfg {
   static constexpr int TILE_BYTES = KT * kD * 2;         // one K (or V) tile: 16 or 32 KB
@@ -191,7 +89,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
   __shared__ __align__(16) float s_scratch[2 * 2 * 128];
   int *s_par = reinterpret_cast<int *>(s_scratch);
   float (*s_pair)[2][128] = reinterpret_cast<float (*)[2][128]>(s_scratch);
-  float2 *r_ml = reinterpret_cast<float2 *>(s_scratch);
+  float4 *r_ml = reinterpret_cast<float4 *>(s_scratch);
   __shared__ __align__(8) unsigned long long s_recv_bar;      // counts what peers push to this CTA (split merge)
   // barriers: full[5], empty[5] (ring slots), s_ready[2], p_ready[2], o_done[2], q_ready
   __shared__ __align__(8) unsigned long long s_bar[2 * kMaxSlots + 7];
@@ -235,10 +133,10 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
     mbar_init(bar_q, 32);
     if (n_splits > 1) {
       // split merge: one arrival that announces the peers' bytes (every peer sends each of this
-      // CTA's ROWS / n_splits rows as 128 fp16 and an (m, l) pair), one per softmax warp for this
+      // CTA's ROWS / n_splits rows as 128 fp16 and (m, l, row scale, -)), one per softmax warp for this
       // CTA's own share
       mbar_init(smem_u32(&s_recv_bar), 1 + 4);
-      mbar_arrive_expect_tx(smem_u32(&s_recv_bar), (uint32_t)((n_splits - 1) * (ROWS / n_splits) * (kD * 2 + 8)));
+      mbar_arrive_expect_tx(smem_u32(&s_recv_bar), (uint32_t)((n_splits - 1) * (ROWS / n_splits) * (kD * 2 + 16)));
     }
   }
   if (warp == 5) {
@@ -758,9 +656,8 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
 
   // ---- merge the key splits of the cluster ----
   // Every CTA owns ROWS / n_splits rows.  Once all CTAs have left their key loops (the receive
-  // buffer lies in the stage ring) each thread sends its row's (m, l) and O / l as fp16 (|O / l| is
-  // bounded by the largest |V| entry; fp16 rounds eight times finer than the bf16 output) to the
-  // row's owner: asynchronous stores that the owner's barrier counts, plain stores for the CTA's
+  // buffer lies in the stage ring) each thread sends its row's (m, l) and O / l as scaled fp16 (see
+  // row_scale: finer than the bf16 output whatever the magnitude of V) to the row's owner: asynchronous stores that the owner's barrier counts, plain stores for the CTA's
   // own share.  The owner waits for its bytes (bounded), combines and stores.
   const int rows_per = ROWS / n_splits;
   unsigned char *recv = smem + C::Q_BYTES + C::P_BYTES;      // [sender * rows_per + owned row][128] fp16
@@ -773,7 +670,22 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
     const bool remote = owner != split;
     unsigned char *ro = recv + (size_t)slot * kD * 2;
     const uint32_t ro_c = map_to_cta(smem_u32(ro), owner), bar_c = map_to_cta(recv_bar, owner);
-    const float inv_l = (have_o && l_run > 0.f) ? 1.f / l_run : 0.f;
+    // (a row that saw no key in this split carries m = -inf and counts for nothing)
+    const bool seen = have_o && m_run > -INFINITY && l_run > 0.f;
+    const float inv_l = seen ? 1.f / l_run : 0.f;
+    float amax = 0.f;
+    if (have_o) {                           // warp-uniform: the row's largest |O|
+#pragma unroll
+      for (int ch = 0; ch < 4; ++ch) {
+        uint32_t v[32];
+        tmem_ld32(t_lane + C::O_COL + ch * 32, v);
+        tmem_ld_wait();
+#pragma unroll
+        for (int j = 0; j < 32; ++j) amax = fmaxf(amax, fabsf(__uint_as_float(v[j])));
+      }
+    }
+    float down, up;
+    row_scale(amax * inv_l, down, up);
 #pragma unroll
     for (int ch = 0; ch < 4; ++ch) {
       uint32_t v[32];
@@ -790,7 +702,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
           uint32_t h[4];
 #pragma unroll
           for (int e = 0; e < 4; ++e)
-            h[e] = pack_f16(__uint_as_float(v[8 * i + 2 * e]) * inv_l, __uint_as_float(v[8 * i + 2 * e + 1]) * inv_l);
+            h[e] = pack_f16(__uint_as_float(v[8 * i + 2 * e]) * inv_l * down, __uint_as_float(v[8 * i + 2 * e + 1]) * inv_l * down);
           const int off = ((ch * 4 + i) ^ (lr & 15)) << 4;
           if (remote) st_async_b32x4(ro_c + off, h[0], h[1], h[2], h[3], bar_c);
           else *reinterpret_cast<uint4 *>(ro + off) = make_uint4(h[0], h[1], h[2], h[3]);
@@ -798,9 +710,9 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
       }
     }
     if (row_active) {
-      const float mm = have_o ? m_run : -INFINITY, ll = have_o ? l_run : 0.f;
-      if (remote) st_async_f32x2(map_to_cta(smem_u32(r_ml + slot), owner), mm, ll, bar_c);
-      else r_ml[slot] = make_float2(mm, ll);
+      const float mm = seen ? m_run : -INFINITY, ll = seen ? l_run : 0.f;
+      if (remote) st_async_f32x4(map_to_cta(smem_u32(r_ml + slot), owner), mm, ll, up, 0.f, bar_c);
+      else r_ml[slot] = make_float4(mm, ll, up, 0.f);
     }
     __syncwarp();                           // the lanes' own-share stores come before lane 0's arrival
     if (lane == 0) mbar_arrive(recv_bar);
@@ -838,8 +750,10 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
 #pragma unroll
       for (int sd = 0; sd < 8; ++sd) {
         if (sd < n_splits) {
-          const float wgt = fast_exp2(mv[sd] - mstar) * r_ml[sd * rows_per + lr].y;
-          lsum += wgt;
+          const float4 ml = r_ml[sd * rows_per + lr];
+          const float wl = fast_exp2(mv[sd] - mstar) * ml.y;
+          lsum += wl;
+          const float wgt = wl * ml.z;
           const uint2 raw = *reinterpret_cast<const uint2 *>(recv + (size_t)(sd * rows_per + lr) * kD * 2 + off);
           const float2 v01 = unpack_f16(raw.x), v23 = unpack_f16(raw.y);
           acc.x = fmaf(wgt, v01.x, acc.x);
@@ -861,7 +775,10 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
   }
 }
 
+}  // namespace
+
 // ---- tensor maps over the whole K and V cache: dims (d, pos, head, batch, layer) ----
+namespace {
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -894,8 +811,12 @@ static bool encode_cache_map(EncodeTiledFn fn, CUtensorMap *out, const void *bas
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// Returns the (cached) pair of maps for this cache layout, or nullptr when none can be made.
-static const MapEntry *cache_maps(const AttnParams &p, int box_rows) {
+}  // namespace
+
+// Copies the (cached) pair of maps for this cache layout into `out`; false when none can be made.
+// (The table is a small ring that other threads may overwrite as soon as the lock is gone, so
+// the caller gets a copy, not a pointer into it.)
+bool cache_maps(const AttnParams &p, int box_rows, CacheMaps *out) {
   static std::mutex mu;
   static EncodeTiledFn fn = nullptr;
   static bool fn_tried = false;
@@ -910,25 +831,33 @@ static const MapEntry *cache_maps(const AttnParams &p, int box_rows) {
         qres == cudaDriverEntryPointSuccess)
       fn = reinterpret_cast<EncodeTiledFn>(ptr);
   }
-  if (!fn) return nullptr;
+  if (!fn) return false;
   // strides must be multiples of 16 bytes, and every dimension but the last needs stride * extent in range
-  if (p.c_sp <= 0 || p.c_sh <= 0 || p.c_sb < 0 || p.c_sl < 0) return nullptr;
+  if (p.c_sp <= 0 || p.c_sh <= 0 || p.c_sb < 0 || p.c_sl < 0) return false;
   MapKey key{p.cache_k0, p.cache_v0, p.n_layers > 1 ? p.c_sl : p.c_sp, p.batch > 1 ? p.c_sb : p.c_sp, p.c_sh, p.c_sp,
              p.n_layers, p.batch, p.n_kv_heads, p.max_len, box_rows};
   if (p.n_kv_heads == 1) key.sh = key.sp;      // a stride of an extent-1 dimension is never used
   for (auto &e : table)
-    if (e.valid && e.key == key) return &e;
+    if (e.valid && e.key == key) {
+      out->kmap = e.kmap;
+      out->vmap = e.vmap;
+      return true;
+    }
   MapEntry &e = table[next];
   next = (next + 1) % 16;
   e.valid = false;
-  if (!encode_cache_map(fn, &e.kmap, p.cache_k0, key) || !encode_cache_map(fn, &e.vmap, p.cache_v0, key)) return nullptr;
+  if (!encode_cache_map(fn, &e.kmap, p.cache_k0, key) || !encode_cache_map(fn, &e.vmap, p.cache_v0, key)) return false;
   e.key = key;
   e.valid = true;
-  return &e;
+  out->kmap = e.kmap;
+  out->vmap = e.vmap;
+  return true;
 }
 
+namespace {
+
 template <int ROWS, int KT>
-twig_status launch_umma(const AttnParams &p, const MapEntry *maps, int batch, int n_splits, cudaStream_t st) {
+twig_status launch_umma(const AttnParams &p, const CacheMaps *maps, int batch, int n_splits, cudaStream_t st) {
   using C = UmmaCfg<ROWS, KT>;
   static bool attr_set = false;
   if (!attr_set) {
@@ -950,7 +879,7 @@ twig_status launch_umma(const AttnParams &p, const MapEntry *maps, int batch, in
   attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = launch_overlap_enabled() ? 2 : 1;
+  cfg.numAttrs = p.overlap ? 2 : 1;
   if (cudaLaunchKernelEx(&cfg, tree_attn_umma_kernel<ROWS, KT>, p, maps->kmap, maps->vmap) != cudaSuccess)
     return TWIG_ERR_CUDA;
   return TWIG_OK;
@@ -967,10 +896,11 @@ twig_status launch_tree_attn_umma(AttnParams &p, int batch, int rows, cudaStream
   // memory).  Many items, or short caches: 64-key tiles, two CTAs per SM.
   const bool wide = items <= 148 && ((rows_per_cta == 128 && p.max_len >= 1024) || (rows_per_cta == 64 && p.max_len >= 4096));
   const int kt = wide ? 128 : 64;
-  const MapEntry *maps = cache_maps(p, kt);
-  if (!maps) return TWIG_ERR_UNSUPPORTED;
+  CacheMaps cm;
+  if (!cache_maps(p, kt, &cm)) return TWIG_ERR_UNSUPPORTED;
+  const CacheMaps *maps = &cm;
   const int max_tiles = (p.max_len + p.t_max + kt - 1) / kt;
-  const int n_splits = pick_splits(items, max_tiles, wide ? 1 : 2);
+  const int n_splits = pick_splits(items, max_tiles, wide ? 1 : 2, p.forced_splits);
   if (wide) {
     if (rows_per_cta == 64) return launch_umma<64, 128>(p, maps, batch, n_splits, st);
     return launch_umma<128, 128>(p, maps, batch, n_splits, st);

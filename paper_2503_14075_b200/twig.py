@@ -26,7 +26,7 @@ STATUS_NAMES = {0: "TWIG_OK", 1: "TWIG_ERR_NULL", 2: "TWIG_ERR_SHAPE", 3: "TWIG_
 DEV_OK, DEV_BAD_LAYOUT, DEV_BAD_KEEP, DEV_BAD_INDEX, DEV_BAD_TREE, DEV_OVERFLOW, DEV_INTERNAL = range(7)
 MAX_NODES, MAX_VISUAL, MAX_BATCH = 64, 16384, 4096
 
-EXPORTS = ["twig_status_str", "twig_set_launch_overlap", "twig_set_early_prefix", "twig_set_attention_path", "twig_set_attention_splits", "twig_workspace_bytes", "ttp_score", "ttp_score_gated", "ttp_multiquery_workspace_bytes", "ttp_score_multiquery", "ttp_score_noalloc", "ttp_topk", "ttp_compact", "ttp_compact_rows",
+EXPORTS = ["twig_status_str", "twig_set_launch_overlap", "twig_workspace_bytes", "tree_attention_workspace_bytes", "tree_verify_attention_ex", "ttp_score", "ttp_score_gated", "ttp_multiquery_workspace_bytes", "ttp_score_multiquery", "ttp_score_noalloc", "ttp_topk", "ttp_compact", "ttp_compact_rows",
            "ttp_score_topk_compact", "tree_verify_attention", "tree_reset", "tree_expand_level", "tree_select_expansion", "tree_finalize", "tree_base_argmax", "tree_accept_compact"]
 
 
@@ -58,14 +58,10 @@ _vp, _i32, _i64, _f32, _sz = C.c_void_p, C.c_int32, C.c_int64, C.c_float, C.c_si
 _kvp = C.POINTER(KV)
 _lib.twig_status_str.restype = C.c_char_p
 _lib.twig_status_str.argtypes = [C.c_int]
-_lib.twig_set_attention_path.restype = C.c_int32
-_lib.twig_set_attention_path.argtypes = [C.c_int32]
 _lib.twig_set_launch_overlap.restype = C.c_int32
 _lib.twig_set_launch_overlap.argtypes = [C.c_int32]
-_lib.twig_set_early_prefix.restype = C.c_int32
-_lib.twig_set_early_prefix.argtypes = [C.c_int32]
-_lib.twig_set_attention_splits.restype = C.c_int32
-_lib.twig_set_attention_splits.argtypes = [C.c_int32]
+_lib.tree_attention_workspace_bytes.restype = _sz
+_lib.tree_attention_workspace_bytes.argtypes = [_i32] * 3
 _lib.twig_workspace_bytes.restype = _sz
 _lib.twig_workspace_bytes.argtypes = [_i32] * 5
 _lib.ttp_score.restype = C.c_int
@@ -97,6 +93,19 @@ _lib.ttp_score_topk_compact.argtypes = [_vp, _vp, _i64, _i64, _i64, _i32, _vp, _
 _lib.tree_verify_attention.restype = C.c_int
 _lib.tree_verify_attention.argtypes = [_vp, _vp, _vp, _kvp, _i32, _vp, _vp, _vp, _i32, _i32, _f32, _vp, _vp,
                                        _vp, _vp, _sz, _vp]
+_lib.tree_verify_attention_ex.restype = C.c_int
+_lib.tree_verify_attention_ex.argtypes = _lib.tree_verify_attention.argtypes + [C.c_uint32]
+# per-call flags of tree_verify_attention_ex
+ATTN_EARLY_PREFIX, ATTN_PLAIN_LAUNCH = 1, 1 << 4
+ATTN_KERNEL_AUTO, ATTN_KERNEL_MMA, ATTN_KERNEL_TCGEN05, ATTN_KERNEL_STREAM = 0, 1, 2, 3
+
+
+def attn_flags(kernel=ATTN_KERNEL_AUTO, early_prefix=False, splits=0, plain_launch=False) -> int:
+    """Packs the flags word of tree_verify_attention_ex."""
+    return (int(kernel) << 1) | (ATTN_EARLY_PREFIX if early_prefix else 0) | (int(splits) << 8) | \
+        (ATTN_PLAIN_LAUNCH if plain_launch else 0)
+
+
 _lib.tree_reset.restype = C.c_int
 _lib.tree_reset.argtypes = [_vp, _vp, _vp, _i32, _i32, _vp]
 _lib.tree_expand_level.restype = C.c_int
@@ -129,29 +138,18 @@ def lib_path() -> str:
     return _LIB_PATH
 
 
-def twig_set_attention_path(path: int) -> int:
-    """0 automatic, 1 mma.sync kernel, 2 tcgen05 kernel; returns the previous setting."""
-    return int(_lib.twig_set_attention_path(int(path)))
-
-
 def twig_set_launch_overlap(on: int) -> int:
     """Programmatic stream serialization for the attention and accept kernels (default on)."""
     return int(_lib.twig_set_launch_overlap(int(on)))
 
 
-def twig_set_early_prefix(on: int) -> int:
-    """Promise that the kernel before each following tree_verify_attention call leaves kv_len, n_nodes,
-    parent and the cache rows below kv_len alone (e.g. between the layers of one verify step)."""
-    return int(_lib.twig_set_early_prefix(int(on)))
-
-
-def twig_set_attention_splits(splits: int) -> int:
-    """Force 1, 2, 4 or 8 key splits per (request, kv head, row block); 0 = automatic."""
-    return int(_lib.twig_set_attention_splits(int(splits)))
-
-
 def twig_workspace_bytes(batch, n_q_heads, head_dim, max_len, max_nodes) -> int:
     return int(_lib.twig_workspace_bytes(batch, n_q_heads, head_dim, max_len, max_nodes))
+
+
+def tree_attention_workspace_bytes(batch, n_q_heads, max_nodes) -> int:
+    """Scratch of the persistent attention kernel: zero-filled at first use, passed to no other call."""
+    return int(_lib.tree_attention_workspace_bytes(batch, n_q_heads, max_nodes))
 
 
 def ttp_score(twig_q, twig_k, prefix_len, vis_start, n_vis, scores, ws, norm_scope=0,
@@ -246,13 +244,25 @@ def ttp_score_topk_compact(twig_q, twig_k, prefix_len, vis_start, n_vis, keep, s
 
 
 def tree_verify_attention(q, tree_k, tree_v, cache: KV, layer, kv_len, n_nodes, parent, out, lse=None,
-                          softmax_scale=0.0, dev_status=None, ws=None, stream=None):
-    """q/out [B,T,Hq,d]; tree_k/v [B,Hkv,T,d]; parent [B,T] int32; lse [B,Hq,T] fp32 or None."""
+                          softmax_scale=0.0, dev_status=None, ws=None, stream=None, flags=None):
+    """q/out [B,T,Hq,d]; tree_k/v [B,Hkv,T,d]; parent [B,T] int32; lse [B,Hq,T] fp32 or None.
+    ws: scratch of the persistent kernel (zero-filled at first use, this call's only) or None.
+    flags: None calls tree_verify_attention, an int (see attn_flags) tree_verify_attention_ex."""
     B, T, Hq, d = q.shape
     ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
-    _check(_lib.tree_verify_attention(_p(q), _p(tree_k), _p(tree_v), C.byref(cache), layer, _p(kv_len),
-                                      _p(n_nodes), _p(parent), T, Hq, softmax_scale, _p(out), _p(lse),
-                                      _p(dev_status), _p(ws), ws_bytes, _stream(stream)))
+    args = (_p(q), _p(tree_k), _p(tree_v), C.byref(cache), layer, _p(kv_len), _p(n_nodes), _p(parent), T, Hq,
+            softmax_scale, _p(out), _p(lse), _p(dev_status), _p(ws), ws_bytes, _stream(stream))
+    if flags is None:
+        _check(_lib.tree_verify_attention(*args))
+    else:
+        _check(_lib.tree_verify_attention_ex(*args, int(flags)))
+
+
+def tree_verify_attention_ex(q, tree_k, tree_v, cache: KV, layer, kv_len, n_nodes, parent, out, flags, lse=None,
+                             softmax_scale=0.0, dev_status=None, ws=None, stream=None):
+    """tree_verify_attention with the per-call flags word (see attn_flags)."""
+    tree_verify_attention(q, tree_k, tree_v, cache, layer, kv_len, n_nodes, parent, out, lse=lse,
+                          softmax_scale=softmax_scale, dev_status=dev_status, ws=ws, stream=stream, flags=int(flags))
 
 
 class TreeState:

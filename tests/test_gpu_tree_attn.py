@@ -20,11 +20,25 @@ def tw():
     return twig
 
 
-def run_attention(tw, wl, ver, cache_k, cache_v, kv_len, layer=0, max_len=None, lse=True, path=0):
+_WS = {}
+
+
+def stream_ws(tw, B, Hq, T):
+    """Scratch of the persistent kernel: zero-filled once, then only ever passed to attention calls
+    (which leave it zeroed), so one buffer per size serves the whole test session."""
+    need = tw.tree_attention_workspace_bytes(B, Hq, T)
+    if need not in _WS:
+        _WS[need] = torch.zeros(need, dtype=torch.uint8, device=DEV)
+    return _WS[need]
+
+
+def run_attention(tw, wl, ver, cache_k, cache_v, kv_len, layer=0, max_len=None, lse=True, path=0, splits=0,
+                  early=False):
     """cache_k/v: uint16 [Nl,B,Hkv,Lmax,d].  Returns (out bits [B,T,Hq,d], lse [B,Hq,T], status).
-    path: 0 automatic, 1 mma.sync kernel, 2 tcgen05 kernel."""
+    path: 0 automatic, 1 mma.sync kernel, 2 tcgen05 kernel (cluster splits), 3 persistent tcgen05 kernel.
+    A named kernel is the kernel that runs (the library refuses, it never substitutes)."""
     B, T, Hq, d = ver["q"].shape[1:]
-    tw.twig_set_attention_path(path)
+    ws = stream_ws(tw, B, Hq, T) if path == 3 else None
     ck, cv = dev_bf16(cache_k), dev_bf16(cache_v)
     out = torch.zeros((B, T, Hq, d), dtype=torch.int16, device=DEV)
     out.fill_(CANARY)
@@ -33,9 +47,12 @@ def run_attention(tw, wl, ver, cache_k, cache_v, kv_len, layer=0, max_len=None, 
     status = torch.zeros(B, dtype=torch.int32, device=DEV)
     tw.tree_verify_attention(dev_bf16(ver["q"][layer]), dev_bf16(ver["tree_k"][layer]), dev_bf16(ver["tree_v"][layer]),
                              tw.KV.of(ck, cv), layer, dev_i32(kv_len), dev_i32(ver["n_nodes"]), dev_i32(ver["parent"]),
-                             out, lse=lse_t, dev_status=status)
+                             out, lse=lse_t, dev_status=status, ws=ws,
+                             flags=tw.attn_flags(kernel=path, splits=splits, early_prefix=early))
     torch.cuda.synchronize()
-    tw.twig_set_attention_path(0)
+    if ws is not None:      # the call leaves its arrival counters (the tail of the buffer) at zero
+        n_tail = tw.tree_attention_workspace_bytes(B, Hq, T) - tw.tree_attention_workspace_bytes(1, 1, T) + 8
+        assert not ws[-n_tail:].any()
     return host_bits(out), (lse_t.cpu().numpy() if lse else None), status.cpu().numpy()
 
 
@@ -83,11 +100,11 @@ SHAPES = [
 
 @pytest.mark.parametrize("shape", SHAPES, ids=[s[0] for s in SHAPES])
 @pytest.mark.parametrize("gain_name", ["timing", "sharp", "sharp4"])
-@pytest.mark.parametrize("path", [1, 2], ids=["mma", "tcgen05"])
+@pytest.mark.parametrize("path", [1, 2, 3], ids=["mma", "tcgen05", "stream"])
 def test_tree_attention_matches_oracle(tw, shape, gain_name, path):
     name, B, Hq, Hkv, d, n_nodes, depth, kv_len = shape
-    if path == 2 and d != 128:
-        pytest.skip("the tcgen05 kernel covers head_dim 128")
+    if path >= 2 and d != 128:
+        pytest.skip("the tcgen05 kernels cover head_dim 128")
     gain = {"timing": 1.0, "sharp": d ** 0.5, "sharp4": 2.0 * d ** 0.5}[gain_name]   # logit std 1/d, 1, 4
     wl = _wl(B, Hq, Hkv, d, n_nodes, depth)
     rng = synth.rng_for(9, zlib.crc32(name.encode()) % 1000)
@@ -103,7 +120,7 @@ def test_tree_attention_matches_oracle(tw, shape, gain_name, path):
     check(got, lse, want, want_lse, ver["n_nodes"], name)
 
 
-@pytest.mark.parametrize("path", [1, 2], ids=["mma", "tcgen05"])
+@pytest.mark.parametrize("path", [1, 2, 3], ids=["mma", "tcgen05", "stream"])
 @pytest.mark.parametrize("kind", ["chain", "star"])
 def test_special_trees(tw, kind, path):
     T = 20
@@ -118,7 +135,7 @@ def test_special_trees(tw, kind, path):
     check(got, lse, want, want_lse, ver["n_nodes"], kind)
 
 
-@pytest.mark.parametrize("path", [1, 2], ids=["mma", "tcgen05"])
+@pytest.mark.parametrize("path", [1, 2, 3], ids=["mma", "tcgen05", "stream"])
 def test_bad_tree_and_overflow_set_status(tw, path):
     wl = _wl(4, 4, 4, 128, [6, 6, 6, 6], [3, 3, 3, 3])
     rng = synth.rng_for(9, 78)
@@ -143,7 +160,7 @@ FULL = [
 ]
 
 
-@pytest.mark.parametrize("path", [1, 2], ids=["mma", "tcgen05"])
+@pytest.mark.parametrize("path", [1, 2, 3], ids=["mma", "tcgen05", "stream"])
 @pytest.mark.parametrize("index,lens", FULL, ids=["c2", "c3", "c4", "c5"])
 def test_full_size_configs(tw, index, lens, path):
     """Full-size shapes of the benchmark configurations, one layer, every output row
@@ -189,36 +206,92 @@ class _F64View:
         return synth.bf16_to_f64(self.bits[idx])
 
 
-@pytest.mark.parametrize("shape", [SHAPES[0], SHAPES[2], SHAPES[6]], ids=["c1", "rows32", "d64-rows64"])
-def test_early_prefix_gives_the_same_bits(tw, shape):
-    """With the early-prefix promise kept (nothing before the call writes lengths or cache), the
-    small-call kernel prefetches the prefix under its predecessor and must return identical bits."""
+EARLY = [(SHAPES[0], 1), (SHAPES[2], 1), (SHAPES[6], 1), (SHAPES[2], 3), (SHAPES[3], 3), (SHAPES[5], 3)]
+
+
+@pytest.mark.parametrize("shape,path", EARLY, ids=[f"{s[0]}-{'mma' if k == 1 else 'stream'}" for s, k in EARLY])
+def test_early_prefix_gives_the_same_bits(tw, shape, path):
+    """With the early-prefix promise kept (nothing before the call writes lengths or cache), the kernel
+    fetches the prefix under its predecessor and must return identical bits."""
     name, B, Hq, Hkv, d, n_nodes, depth, kv_len = shape
     wl = _wl(B, Hq, Hkv, d, n_nodes, depth)
     rng = synth.rng_for(9, 321)
     ver = synth.make_verify_inputs(wl, rng, n_layers=1, gain=d ** 0.5)
     ck, cv = synth.make_cache(wl, rng, max(kv_len) + 70, n_layers=1, gain=d ** 0.5)
-    ref, ref_lse, st0 = run_attention(tw, wl, ver, ck, cv, kv_len, path=1)
-    tw.twig_set_early_prefix(1)
-    try:
-        got, got_lse, st1 = run_attention(tw, wl, ver, ck, cv, kv_len, path=1)
-        # twice back to back on one stream: the second call prefetches under the first
-        B_, T, Hq_, d_ = ver["q"].shape[1:]
-        dck, dcv = dev_bf16(ck), dev_bf16(cv)
-        cache = tw.KV.of(dck, dcv)
-        q, tk, tv = dev_bf16(ver["q"][0]), dev_bf16(ver["tree_k"][0]), dev_bf16(ver["tree_v"][0])
-        kvl, nn, par = dev_i32(kv_len), dev_i32(ver["n_nodes"]), dev_i32(ver["parent"])
-        outs = [torch.zeros((B_, T, Hq_, d_), dtype=torch.bfloat16, device=DEV) for _ in range(3)]
-        tw.twig_set_attention_path(1)
-        for o in outs:
-            tw.tree_verify_attention(q, tk, tv, cache, 0, kvl, nn, par, o)
-        torch.cuda.synchronize()
-    finally:
-        tw.twig_set_early_prefix(0)
-        tw.twig_set_attention_path(0)
+    ref, ref_lse, st0 = run_attention(tw, wl, ver, ck, cv, kv_len, path=path)
+    got, got_lse, st1 = run_attention(tw, wl, ver, ck, cv, kv_len, path=path, early=True)
+    # several calls back to back on one stream: each fetches its prefix under the one before
+    B_, T, Hq_, d_ = ver["q"].shape[1:]
+    dck, dcv = dev_bf16(ck), dev_bf16(cv)
+    cache = tw.KV.of(dck, dcv)
+    q, tk, tv = dev_bf16(ver["q"][0]), dev_bf16(ver["tree_k"][0]), dev_bf16(ver["tree_v"][0])
+    kvl, nn, par = dev_i32(kv_len), dev_i32(ver["n_nodes"]), dev_i32(ver["parent"])
+    outs = [torch.zeros((B_, T, Hq_, d_), dtype=torch.bfloat16, device=DEV) for _ in range(4)]
+    ws = stream_ws(tw, B_, Hq_, T) if path == 3 else None
+    for o in outs:
+        tw.tree_verify_attention(q, tk, tv, cache, 0, kvl, nn, par, o, ws=ws,
+                                 flags=tw.attn_flags(kernel=path, early_prefix=True))
+    torch.cuda.synchronize()
     assert not st0.any() and not st1.any()
     assert np.array_equal(got, ref) and np.array_equal(got_lse, ref_lse)
     for b in range(B):
         n = n_nodes[b]
         for o in outs:
             assert np.array_equal(host_bits(o)[b, :n], ref[b, :n])
+
+
+def test_named_kernel_is_never_substituted(tw):
+    """A kernel named in the flags either runs or the call fails on the host: the tcgen05 kernels do not
+    take head_dim 64, the persistent one does not run without its scratch."""
+    wl = _wl(1, 4, 4, 64, [8], [3])
+    rng = synth.rng_for(9, 5)
+    ver = synth.make_verify_inputs(wl, rng, n_layers=1)
+    ck, cv = synth.make_cache(wl, rng, 80, n_layers=1)
+    for path in (2, 3):
+        with pytest.raises(tw.TwigError) as e:
+            run_attention(tw, wl, ver, ck, cv, [10], path=path)
+        assert e.value.code == 3                   # TWIG_ERR_UNSUPPORTED
+    wl = _wl(1, 4, 4, 128, [8], [3])
+    ver = synth.make_verify_inputs(wl, rng, n_layers=1)
+    ck, cv = synth.make_cache(wl, rng, 80, n_layers=1)
+    B, T, Hq, d = ver["q"].shape[1:]
+    out = torch.zeros((B, T, Hq, d), dtype=torch.bfloat16, device=DEV)
+    args = (dev_bf16(ver["q"][0]), dev_bf16(ver["tree_k"][0]), dev_bf16(ver["tree_v"][0]),
+            tw.KV.of(dev_bf16(ck), dev_bf16(cv)), 0, dev_i32([10]), dev_i32(ver["n_nodes"]), dev_i32(ver["parent"]), out)
+    with pytest.raises(tw.TwigError) as e:
+        tw.tree_verify_attention(*args, flags=tw.attn_flags(kernel=3))              # no scratch
+    assert e.value.code == 4                       # TWIG_ERR_WORKSPACE
+    small = torch.zeros(1024, dtype=torch.uint8, device=DEV)
+    with pytest.raises(tw.TwigError) as e:
+        tw.tree_verify_attention(*args, ws=small, flags=tw.attn_flags(kernel=3))
+    assert e.value.code == 4
+    with pytest.raises(tw.TwigError) as e:
+        tw.tree_verify_attention(*args, flags=tw.attn_flags(kernel=1, splits=3))    # not a split count
+    assert e.value.code == 3
+    torch.cuda.synchronize()
+    assert not out.any()                           # nothing was launched
+
+
+@pytest.mark.parametrize("v_scale", [2.0 ** -17, 1.0, 2.0 ** 17], ids=["tinyV", "unitV", "largeV"])
+@pytest.mark.parametrize("path,splits", [(1, 1), (1, 2), (1, 4), (1, 8), (2, 1), (2, 2), (2, 4), (2, 8), (3, 0)],
+                         ids=lambda v: str(v))
+def test_key_splits_and_value_range(tw, path, splits, v_scale):
+    """The result must not depend on how the keys are split between CTAs, nor on the magnitude of V:
+    partial results cross between CTAs in a narrower format than they are accumulated in."""
+    wl = _wl(2, 4, 4, 128, [30, 17], [6, 4])
+    rng = synth.rng_for(9, 4242)
+    ver = synth.make_verify_inputs(wl, rng, n_layers=1, gain=128 ** 0.5)
+    kv_len = [700, 333]
+    ck, cv = synth.make_cache(wl, rng, 800, n_layers=1, gain=128 ** 0.5)
+    # (powers of two: exact in bf16; 2^17 is beyond what fp16 holds, 2^-17 far below its normal range)
+    cv = synth.f32_to_bf16(synth.bf16_to_f32(cv) * np.float32(v_scale))
+    ver["tree_v"] = synth.f32_to_bf16(synth.bf16_to_f32(ver["tree_v"]) * np.float32(v_scale))
+    got, lse, status = run_attention(tw, wl, ver, ck, cv, kv_len, path=path, splits=splits)
+    assert not status.any()
+    want, want_lse = oracle_attention(ver, ck, cv, np.array(kv_len))
+    g = f64(got)
+    for b in range(2):
+        n = int(ver["n_nodes"][b])
+        assert rel_l2_rows(g[b, :n], want[b, :n]) <= REL_L2_TOL
+        assert max_abs(g[b, :n], want[b, :n]) <= MAX_ABS_TOL * max(1.0, np.abs(want[b, :n]).max())
+        assert max_abs(lse[b, :, :n], want_lse[b, :, :n]) <= 1e-3 * max(1.0, np.abs(want_lse[b]).max())
