@@ -236,10 +236,9 @@ twig_status ttp_score_topk_compact(
  *   parent   [batch, t_max] int32; parent[b,0] = -1, parent[b,i] in [0, i)
  *   lse      [batch, n_q_heads, t_max] fp32 or NULL
  * t_max <= TWIG_MAX_NODES.  Rows of nodes >= n_nodes[b] are not written.
- * softmax_scale 0 means 1/sqrt(head_dim).  ws may be NULL when ws_bytes is 0: the kernels that
- * combine key splits on chip need no scratch; a scratch buffer (see tree_verify_attention_ex for
- * its contract: zero-filled at first use, used by these calls only) lets large calls run on the
- * persistent kernel.
+ * softmax_scale 0 means 1/sqrt(head_dim).  ws may be NULL when ws_bytes is 0: the kernels this call
+ * chooses from combine key splits on chip and need no scratch (the persistent kernel of
+ * tree_verify_attention_ex does).
  */
 twig_status tree_verify_attention(const void *q, const void *tree_k, const void *tree_v,
                                   const twig_kv *cache, int32_t layer, const int32_t *kv_len,
@@ -263,6 +262,9 @@ twig_status tree_verify_attention(const void *q, const void *tree_k, const void 
  *   tensor map can describe; a named kernel that cannot run the call returns TWIG_ERR_UNSUPPORTED (or
  *   TWIG_ERR_WORKSPACE); only the automatic choice moves on to another kernel.
  * TWIG_ATTN_SPLITS(n): force n = 1, 2, 4 or 8 key splits per cluster in the _MMA and _TCGEN05 kernels.
+ * TWIG_ATTN_STREAM_SHARES / _WHOLE: how the persistent kernel shares the work between its CTAs: equal
+ *   shares of all key tiles (items may straddle CTAs) or whole items dealt out longest first; by
+ *   default the kernel picks from the lengths it finds on the device.  A testing control.
  *
  * Scratch of the persistent kernel.  One CTA per SM slot walks an equal share of all (request, kv head,
  * row block, key tile) work; a work item that straddles two CTAs is finished by whichever of them
@@ -273,7 +275,8 @@ twig_status tree_verify_attention(const void *q, const void *tree_k, const void 
  *             allocation); every call leaves its counters at zero again.  Nothing else may write
  *             the buffer between calls: do not pass the buffer that ttp_score uses.
  *   sharing   calls whose kernels may overlap on the GPU need a buffer each.
- * With ws = NULL / ws_bytes = 0 the automatic choice never takes the persistent kernel.
+ * The automatic choice does not take the persistent kernel (on the shapes measured so far the
+ * cluster kernel is faster); ws is only read when TWIG_ATTN_KERNEL_STREAM is named.
  */
 #define TWIG_ATTN_EARLY_PREFIX 1u
 #define TWIG_ATTN_KERNEL_AUTO 0u
@@ -283,6 +286,8 @@ twig_status tree_verify_attention(const void *q, const void *tree_k, const void 
 #define TWIG_ATTN_KERNEL(k) ((uint32_t)(k) << 1)
 #define TWIG_ATTN_PLAIN_LAUNCH (1u << 4)
 #define TWIG_ATTN_SPLITS(n) ((uint32_t)(n) << 8)
+#define TWIG_ATTN_STREAM_SHARES (1u << 12)
+#define TWIG_ATTN_STREAM_WHOLE (2u << 12)
 twig_status tree_verify_attention_ex(const void *q, const void *tree_k, const void *tree_v,
                                      const twig_kv *cache, int32_t layer, const int32_t *kv_len,
                                      const int32_t *n_nodes, const int32_t *parent, int32_t t_max,

@@ -688,6 +688,8 @@ extern "C" twig_status tree_verify_attention_ex(const void *q, const void *tree_
   p.overlap = (launch_overlap_enabled() && !(flags & TWIG_ATTN_PLAIN_LAUNCH)) ? 1 : 0;
   p.early_prefix = ((flags & TWIG_ATTN_EARLY_PREFIX) && p.overlap) ? 1 : 0;
   p.forced_splits = splits;
+  p.stream_policy = (int)((flags >> 12) & 3u);
+  if (p.stream_policy == 3) return TWIG_ERR_UNSUPPORTED;
   p.ws = static_cast<unsigned char *>(ws);
   p.ws_bytes = ws_bytes;
   const float scale = softmax_scale != 0.f ? softmax_scale : 1.f / sqrtf((float)cache->head_dim);
@@ -703,14 +705,13 @@ extern "C" twig_status tree_verify_attention_ex(const void *q, const void *tree_
                                              : launch_tree_attn_umma(p, cache->batch, rows, st);
   }
   if (kernel == TWIG_ATTN_KERNEL_AUTO && umma_ok) {
-    // automatic choice: a tcgen05 kernel once there are more than 32 query rows per kv head or enough
-    // (request, kv head) pairs to fill the GPU (the persistent one when the caller has given it its
-    // scratch), the mma.sync kernel for small, latency-bound calls
+    // automatic choice: the tcgen05 kernel with cluster splits once there are more than 32 query rows
+    // per kv head or enough (request, kv head) pairs to fill the GPU, the mma.sync kernel for small,
+    // latency-bound calls.  (The persistent kernel measured slower than the cluster kernel on every
+    // shape tried, so it only runs when it is named.)
     const bool big = rows > 32 || (long long)cache->batch * cache->n_kv_heads >= 148;
     if (big) {
-      twig_status us = TWIG_ERR_UNSUPPORTED;
-      if (ws_bytes > 0) us = launch_tree_attn_stream(p, cache->batch, rows, st);
-      if (us == TWIG_ERR_UNSUPPORTED || us == TWIG_ERR_WORKSPACE) us = launch_tree_attn_umma(p, cache->batch, rows, st);
+      const twig_status us = launch_tree_attn_umma(p, cache->batch, rows, st);
       if (us != TWIG_ERR_UNSUPPORTED) return us;     // no tensor map for this layout: the mma.sync kernel
     }
   }

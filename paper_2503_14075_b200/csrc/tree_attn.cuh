@@ -26,6 +26,7 @@ struct AttnParams {
   // host side only: launch with programmatic stream serialization, forced key splits (0: automatic),
   // the caller's scratch (persistent kernel)
   int overlap, forced_splits;
+  int stream_policy;   // persistent kernel: 0 chosen on the device, 1 equal shares, 2 whole items
   unsigned char *ws;
   size_t ws_bytes;
 };

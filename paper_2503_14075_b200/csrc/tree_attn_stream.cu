@@ -2,12 +2,15 @@
 // tree's ancestor mask) as ONE persistent tcgen05 kernel per call.
 //
 // Work: a call is a list of items (request, kv head, block of query rows), each a run of key
-// tiles (cached prefix followed by the tree's own rows).  All tiles of all items, in item order,
-// form one sequence; the grid has one CTA per SM slot and CTA c takes the c-th equal share
-// (+-1 tile) of that sequence, whatever the lengths of the requests are.  A CTA's share is a list
-// of segments: (item, tile range).  Tensor memory, barriers and the K/V ring are set up once per
-// CTA and run through all of its segments; the loaders run ahead across segment borders, so the
-// ring never drains between items.
+// tiles (cached prefix followed by the tree's own rows).  The grid has one CTA per SM slot; a CTA's
+// share of the call is a list of segments (item, tile range), found on the device from the
+// requests' lengths.  Tensor memory, barriers and the K/V ring are set up once per CTA and run
+// through all of its segments; the loaders run ahead across segment borders, so the ring never
+// drains between items.  Two ways of sharing, chosen on the device:
+//   whole items  when no item is large next to a CTA's share: the items, longest first, are dealt
+//                out to the CTAs back and forth (c, 2G-1-c, 2G+c, ...), every segment is a whole item;
+//   equal shares when items are long or few: all tiles of all items, in item order, form one
+//                sequence and CTA c takes the c-th equal share (+-1 tile) of it.
 //
 // A segment that covers its whole item is finished on the spot.  An item that straddles CTAs is
 // finished by whichever of them arrives last: each writes its partial (row maxima, row sums,
@@ -17,19 +20,25 @@
 //
 // Warp roles (they only meet at mbarriers):
 //   softmax warps   tcgen05.ld of S, running max / sum, P (bf16) to shared memory, epilogue;
-//   loader warp     the ring's only producer: K / V tiles that lie wholly in the cached prefix by TMA
-//                   (two 64-column boxes of a 5-D tensor map over the cache, 128-byte swizzle), the
-//                   tile that holds the prefix end and the tree's rows by 16-byte cp.async with zero
-//                   fill, completed lazily so that the TMA requests behind it are not held up;
+//   loader warp     the only producer: K / V tiles that lie wholly in the cached prefix by TMA (two
+//                   64-column boxes of a 5-D tensor map over the cache, 128-byte swizzle); the tile
+//                   that holds the prefix end and the tree's rows, and the Q tile of every segment
+//                   (one or two segments ahead), by 16-byte cp.async with zero fill, completed lazily
+//                   so that the TMA requests behind them are not held up;
 //   issuer          one thread issues S = Q K^T two tiles ahead (double-buffered S in tensor memory)
-//                   and O += P V (accumulator in tensor memory);
-//   Q warp          the Q tile of every segment, one or two segments ahead.
+//                   and O += P V (accumulator in tensor memory).
 // Every wait is bounded; if one runs out the request is flagged TWIG_DEV_INTERNAL.
 #include "tcgen05_common.cuh"
 
 namespace twig {
 
 namespace {
+
+// 64-row blocks: Q tiles in flight and ring slots (what two CTAs per SM leave room for)
+#ifndef TWIG_STREAM64_QB
+#define TWIG_STREAM64_QB 2
+#define TWIG_STREAM64_SLOTS 4
+#endif
 
 constexpr int kD = 128;                 // head_dim
 constexpr float kLazyMax = 8.f;         // raise the running max only beyond this (log2 units)
@@ -47,9 +56,34 @@ struct Seg {
 
 struct SegIter {
   const int *cum, *sL, *sn;   // shared memory: first global tile of every request (cum[B] = total)
+  const int *cum_items;       // whole-item mode: first item rank of every request in sorted order
+  const unsigned char *order; // whole-item mode: requests, longest items first
   int n_kv_heads, group, row_blocks, rows, kt;
-  int pos, end, b;
+  int pos, end, b;            // equal shares: position in the global tile sequence
+  int whole, round, cta, n_cta, n_items, j;     // whole items: dealing round, position in sorted order
+  __device__ __forceinline__ void fill(Seg &s, int idx) {
+    const int rbs = (s.n * group + rows - 1) / rows;
+    s.hk = idx / rbs;
+    s.rb = idx - s.hk * rbs;
+    s.item = (s.b * n_kv_heads + s.hk) * row_blocks + s.rb;
+  }
   __device__ __forceinline__ bool next(Seg &s) {
+    if (whole) {
+      // item ranks of this CTA: c, 2G-1-c, 2G+c, 4G-1-c, ... (increasing)
+      const int r = (round & 1) ? (round + 1) * n_cta - 1 - cta : round * n_cta + cta;
+      if (r >= n_items) return false;
+      ++round;
+      while (cum_items[j + 1] <= r) ++j;
+      s.b = order[j];
+      s.n = sn[s.b];
+      s.L = sL[s.b];
+      s.tiles = (s.L + s.n + kt - 1) / kt;
+      s.t0 = 0;
+      s.t1 = s.tiles;
+      s.gstart = 0;
+      fill(s, r - cum_items[j]);
+      return true;
+    }
     if (pos >= end) return false;
     while (cum[b + 1] <= pos) ++b;
     s.b = b;
@@ -60,11 +94,8 @@ struct SegIter {
     const int idx = off / s.tiles;
     s.t0 = off - idx * s.tiles;
     s.t1 = min(s.tiles, s.t0 + (end - pos));
-    const int rbs = (s.n * group + rows - 1) / rows;
-    s.hk = idx / rbs;
-    s.rb = idx - s.hk * rbs;
-    s.item = (b * n_kv_heads + s.hk) * row_blocks + s.rb;
     s.gstart = pos - s.t0;
+    fill(s, idx);
     pos += s.t1 - s.t0;
     return true;
   }
@@ -99,9 +130,9 @@ struct StreamCfg {
   static constexpr int ROWS_PER_WARP = MMA_M == 64 ? 16 : 32;
   static constexpr int NSOFT = ROWS / ROWS_PER_WARP;             // warps of a softmax group that own rows
   static constexpr int SOFT_GROUPS = MMA_M == 128 ? 2 : 1;       // 128-row accumulators: two warps per lane quadrant
-  // warps 0-3: softmax group 0 (the first NSOFT of them), 4: loader, 5: issuer, 6: Q tiles,
-  // 7-10: softmax group 1 (128-row accumulators only)
-  static constexpr int WARPS = 7 + 4 * (SOFT_GROUPS - 1);
+  // warps 0-3: softmax group 0 (the first NSOFT of them), 4: loader, 5: issuer,
+  // 6-9: softmax group 1 (128-row accumulators only; warp w serves the lane quadrant w % 4)
+  static constexpr int WARPS = 6 + 4 * (SOFT_GROUPS - 1);
   static constexpr int THREADS = 32 * WARPS;
   static constexpr int SOFT_THREADS = 32 * NSOFT * SOFT_GROUPS;
   // scratch slot of one partial result: ROWS rows of 128 fp16 (16 chunks of [ROWS][16 bytes]), then
@@ -124,12 +155,13 @@ tree_attn_stream_kernel(const AttnParams p, const __grid_constant__ CUtensorMap 
   __shared__ unsigned long long s_mask[TWIG_MAX_NODES];
   __shared__ int s_par[TWIG_MAX_NODES];
   __shared__ int s_cum[kStreamMaxBatch + 1], s_L[kStreamMaxBatch], s_n[kStreamMaxBatch];
-  __shared__ unsigned char s_badtree[kStreamMaxBatch];
+  __shared__ unsigned char s_badtree[kStreamMaxBatch], s_order[kStreamMaxBatch];
+  __shared__ int s_cumi[kStreamMaxBatch + 1], s_whole;
   __shared__ float s_pair[C::SOFT_GROUPS == 2 ? 2 : 1][2][C::SOFT_GROUPS == 2 ? 128 : 1];
   // barriers: full[6], empty[6] (ring slots), s_ready[2], p_ready[2], o_done[2], q_ready[2], q_free[2], o_free
   __shared__ __align__(8) unsigned long long s_bar[2 * kMaxSlots + 11];
   __shared__ uint32_t s_tmem;
-  __shared__ int s_fail, s_last;
+  __shared__ int s_fail, s_last[2];
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int B = p.batch;
@@ -151,7 +183,6 @@ tree_attn_stream_kernel(const AttnParams p, const __grid_constant__ CUtensorMap 
   // stream may still be draining: barriers and tensor memory ----
   if (tid == 0) {
     s_fail = 0;
-    s_last = 0;
     for (int i = 0; i < kSlots; ++i) {
       mbar_init(bar_full(i), 1);        // lane 0 of the loader warp: with the TMA's byte count, or after its cp.async copies
       mbar_init(bar_empty(i), 1);       // one tcgen05.commit
@@ -182,6 +213,18 @@ tree_attn_stream_kernel(const AttnParams p, const __grid_constant__ CUtensorMap 
   else asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   // ---- requests: validation, tiles per request, the global tile sequence ----
+  // (lengths and parents are requested together: one round trip to memory)
+  constexpr int kParRegs = 4;
+  const int n_par = B * p.t_max;
+  const bool par_in_regs = n_par <= kParRegs * C::THREADS;
+  int par_reg[kParRegs];
+  if (par_in_regs) {
+#pragma unroll
+    for (int j = 0; j < kParRegs; ++j) {
+      const int idx = tid + j * C::THREADS;
+      par_reg[j] = idx < n_par ? p.parent[idx] : -1;
+    }
+  }
   for (int b = tid; b < B; b += C::THREADS) {
     const int n = p.n_nodes[b], L = p.kv_len[b];
     int use = n;
@@ -197,46 +240,97 @@ tree_attn_stream_kernel(const AttnParams p, const __grid_constant__ CUtensorMap 
     s_badtree[b] = 0;
   }
   __syncthreads();
-  for (int idx = tid; idx < B * p.t_max; idx += C::THREADS) {
-    const int b = idx / p.t_max, i = idx - b * p.t_max;
-    if (i < s_n[b]) {
-      const int pr = p.parent[idx];
-      if ((i == 0) ? (pr != -1) : (pr < 0 || pr >= i)) s_badtree[b] = 1;
+  if (par_in_regs) {
+#pragma unroll
+    for (int j = 0; j < kParRegs; ++j) {
+      const int idx = tid + j * C::THREADS;
+      if (idx < n_par) {
+        const int b = idx / p.t_max, i = idx - b * p.t_max;
+        if (i < s_n[b] && ((i == 0) ? (par_reg[j] != -1) : (par_reg[j] < 0 || par_reg[j] >= i))) s_badtree[b] = 1;
+      }
+    }
+  } else {
+    for (int idx = tid; idx < n_par; idx += C::THREADS) {
+      const int b = idx / p.t_max, i = idx - b * p.t_max;
+      if (i < s_n[b]) {
+        const int pr = p.parent[idx];
+        if ((i == 0) ? (pr != -1) : (pr < 0 || pr >= i)) s_badtree[b] = 1;
+      }
     }
   }
   __syncthreads();
+  for (int b = tid; b < B; b += C::THREADS)
+    if (s_badtree[b]) {
+      if (blockIdx.x == 0) flag_status(p.dev_status, b, TWIG_DEV_BAD_TREE);
+      s_n[b] = 0;
+    }
+  __syncthreads();
+  // requests by the length of their items, longest first (equal lengths: lower index first)
+  for (int b = tid; b < B; b += C::THREADS) {
+    const int mine = s_n[b] > 0 ? (s_L[b] + s_n[b] + KT - 1) / KT : 0;
+    int rank = 0;
+    for (int o = 0; o < B; ++o) {
+      const int other = s_n[o] > 0 ? (s_L[o] + s_n[o] + KT - 1) / KT : 0;
+      rank += (other > mine || (other == mine && o < b)) ? 1 : 0;
+    }
+    s_order[rank] = (unsigned char)b;
+  }
+  __syncthreads();
   if (warp == 0) {
-    // tiles of request b: (kv heads x row blocks) items of ceil((L + n) / KT) tiles; eight requests per lane
-    int loc[kStreamMaxBatch / 32];
-    int sum = 0;
+    // eight requests per lane: tiles of request b = (kv heads x row blocks) items of ceil((L + n) / KT)
+    // tiles, in request order; items per request in sorted order
+    constexpr int PER = kStreamMaxBatch / 32;
+    int loc[PER], loci[PER];
+    int sum = 0, sumi = 0, mx = 0;
 #pragma unroll
-    for (int j = 0; j < kStreamMaxBatch / 32; ++j) {
-      const int b = lane * (kStreamMaxBatch / 32) + j;
-      int t = 0;
+    for (int j = 0; j < PER; ++j) {
+      const int b = lane * PER + j;
+      int t = 0, it = 0;
       if (b < B) {
-        if (s_badtree[b]) {
-          if (blockIdx.x == 0) flag_status(p.dev_status, b, TWIG_DEV_BAD_TREE);
-          s_n[b] = 0;
-        }
         const int n = s_n[b];
         if (n > 0) t = ((s_L[b] + n + KT - 1) / KT) * p.n_kv_heads * ((n * p.group + ROWS - 1) / ROWS);
+        const int bs = s_order[b], ns = s_n[bs];
+        if (ns > 0) {
+          it = p.n_kv_heads * ((ns * p.group + ROWS - 1) / ROWS);
+          mx = max(mx, (s_L[bs] + ns + KT - 1) / KT);
+        }
       }
       loc[j] = sum;
+      loci[j] = sumi;
       sum += t;
+      sumi += it;
     }
-    int inc = sum;
+    int inc = sum, inci = sumi;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
-      const int y = __shfl_up_sync(0xffffffffu, inc, o);
-      if (lane >= o) inc += y;
+      const int y = __shfl_up_sync(0xffffffffu, inc, o), yi = __shfl_up_sync(0xffffffffu, inci, o);
+      if (lane >= o) {
+        inc += y;
+        inci += yi;
+      }
+      mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, o));
     }
-    const int base = inc - sum;
+    const int base = inc - sum, basei = inci - sumi;
 #pragma unroll
-    for (int j = 0; j < kStreamMaxBatch / 32; ++j) {
-      const int b = lane * (kStreamMaxBatch / 32) + j;
-      if (b < B) s_cum[b] = base + loc[j];
+    for (int j = 0; j < PER; ++j) {
+      const int b = lane * PER + j;
+      if (b < B) {
+        s_cum[b] = base + loc[j];
+        s_cumi[b] = basei + loci[j];
+      }
     }
-    if (lane == 31) s_cum[B] = inc;      // (requests past B count zero tiles)
+    if (lane == 31) {      // (requests past B count nothing)
+      s_cum[B] = inc;
+      s_cumi[B] = inci;
+      // Whole items when every CTA gets one and none of them is long next to a CTA's share of the
+      // tiles (an item that is not split costs its CTA up to its own length in imbalance; a split
+      // costs a trip through scratch memory, a few tiles' worth).
+      const int n_cta = (int)gridDim.x;
+      int whole = inci >= n_cta && mx <= max(12, inc / (2 * n_cta));
+      if (p.stream_policy == 1) whole = 0;
+      if (p.stream_policy == 2) whole = 1;
+      s_whole = whole;
+    }
   }
   tc_fence_before();
   __syncthreads();
@@ -252,6 +346,14 @@ tree_attn_stream_kernel(const AttnParams p, const __grid_constant__ CUtensorMap 
     it.cum = s_cum;
     it.sL = s_L;
     it.sn = s_n;
+    it.cum_items = s_cumi;
+    it.order = s_order;
+    it.whole = s_whole;
+    it.round = 0;
+    it.cta = (int)blockIdx.x;
+    it.n_cta = (int)gridDim.x;
+    it.n_items = s_cumi[B];
+    it.j = 0;
     it.n_kv_heads = p.n_kv_heads;
     it.group = p.group;
     it.row_blocks = p.row_blocks;
@@ -264,54 +366,118 @@ tree_attn_stream_kernel(const AttnParams p, const __grid_constant__ CUtensorMap 
   };
 
   if (warp == 4) {
-    // ================= loader warp: the ring's only producer =================
+    // ================= loader warp: the only producer of the ring and of the Q tiles =================
     // Tiles that lie wholly inside the cached prefix come by TMA (lane 0: two 64-column boxes per
-    // tile); the tile that holds the prefix end and / or the tree's rows by 16-byte cp.async with zero
-    // fill from all lanes.  Those copies are not waited for on the spot: the warp goes on to the next
-    // tile and completes them (wait, proxy fence, arrival on the slots' barriers) just before it
-    // would block on a ring slot anyway.  One producer per ring: every parity wait below is for the
-    // phase that directly precedes the slot's next use.
-    SegIter it = make_iter();
-    Seg s;
+    // tile); the tile that holds the prefix end and / or the tree's rows, and the Q tile of every
+    // segment, by 16-byte cp.async with zero fill from all lanes.  Those copies are not waited for on
+    // the spot: up to two groups of them stay in flight while the warp goes on requesting tiles, and
+    // they are completed (wait, proxy fence, arrival on their barriers) when a third group comes or
+    // when the warp would block on a barrier anyway.  One producer per barrier: every parity wait
+    // below is for the phase that directly precedes the next use.
+    SegIter it = make_iter(), ahead = make_iter();
+    Seg s, sa;
     int u = 0;
     bool ok = true;
-    bool waited_dep = !p.early_prefix;               // the tree's rows may still be in the making
-    int pend0 = -1, pend1 = -1;                      // ring slots whose cp.async copies are in flight
-    auto complete_pending = [&]() {
-      if (pend0 >= 0) {
-        cp_async_wait<0>();
-        fence_async_smem();
-        __syncwarp();
-        if (lane == 0) {
-          mbar_arrive(bar_full(pend0));
-          mbar_arrive(bar_full(pend1));
-        }
-        pend0 = pend1 = -1;
+    bool waited_dep = !p.early_prefix;               // Q and the tree's rows may still be in the making
+    // groups in flight, oldest first: ring slots (or -1) and a Q buffer (or -1) whose barriers they complete
+    int g_slot0[2] = {-1, -1}, g_slot1[2] = {-1, -1}, g_q[2] = {-1, -1};
+    int n_groups = 0;
+    auto arrive_group = [&](int g) {
+      if (lane == 0) {
+        if (g_slot0[g] >= 0) mbar_arrive(bar_full(g_slot0[g]));
+        if (g_slot1[g] >= 0) mbar_arrive(bar_full(g_slot1[g]));
+        if (g_q[g] >= 0) mbar_arrive(bar_q(g_q[g]));
       }
+    };
+    auto complete_oldest = [&]() {              // (with two groups in flight: the older one)
+      if (n_groups == 2) cp_async_wait<1>();
+      else cp_async_wait<0>();
+      fence_async_smem();
+      __syncwarp();
+      arrive_group(0);
+      g_slot0[0] = g_slot0[1];
+      g_slot1[0] = g_slot1[1];
+      g_q[0] = g_q[1];
+      --n_groups;
+    };
+    auto complete_all = [&]() {
+      while (n_groups > 0) complete_oldest();
+    };
+    auto open_group = [&](int slot0, int slot1, int qbuf) {     // after the copies were issued
+      cp_async_commit();
+      g_slot0[n_groups] = slot0;
+      g_slot1[n_groups] = slot1;
+      g_q[n_groups] = qbuf;
+      ++n_groups;
+    };
+    // a wait that would block first completes what is in flight (nothing is lost by waiting there)
+    auto wait_bar = [&](uint32_t bar, uint32_t parity) {
+      bool ready = mbar_try_wait(bar, parity);
+      ready = __all_sync(0xffffffffu, ready);
+      if (ready) return;
+      complete_all();
+      ok = mbar_wait(bar, parity, fail);
+      ok = __all_sync(0xffffffffu, ok);
     };
     const int c = lane & 15, rbase = lane >> 4;      // chunk c of rows rbase, rbase + 2, ...
     const uint32_t panel = (uint32_t)((c >> 3) * kPanelBytes);
-    while (ok && it.next(s)) {
+    int q_next = 0;                                   // segments whose Q tile has been requested
+    auto request_q = [&]() {                          // the Q tile of segment q_next, if there is one
+      if (!ahead.next(sa)) {
+        q_next = 1 << 30;
+        return;
+      }
+      const int buf = q_next % QB;
+      // the buffer's previous segment is done with it once all of its S products have completed
+      if (q_next >= QB) wait_bar(bar_qfree(buf), (q_next / QB - 1) & 1);
+      if (!ok) return;
+      if (!waited_dep) {
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        waited_dep = true;
+      }
+      if (n_groups == 2) complete_oldest();
+      // zero rows past the request's last row.  Lane pairs walk the rows two apart; the (node, query
+      // head of the group) pair of a row is stepped, not divided.
+      const uint32_t qb = q_s + buf * C::Q_ONE;
+      const int row0 = sa.rb * ROWS, rows_total = sa.n * p.group;
+      int node = (row0 + rbase) / p.group, g = (row0 + rbase) % p.group;
+      for (int r = rbase; r < ROWS; r += 2) {
+        const bool valid = row0 + r < rows_total;
+        const __nv_bfloat16 *src =
+            p.q + (((long long)sa.b * p.t_max + (valid ? node : 0)) * p.n_q_heads + sa.hk * p.group + (valid ? g : 0)) * kD + c * 8;
+        cp_async_16(qb + (c >> 3) * ROWS * 128 + r * 128 + (((c & 7) ^ (r & 7)) << 4), src, valid);
+        g += 2;
+        while (g >= p.group) {
+          g -= p.group;
+          ++node;
+        }
+      }
+      open_group(-1, -1, buf);
+      ++q_next;
+    };
+    for (int si = 0; ok && it.next(s); ++si) {
+      if (si == 0) request_q();                       // Q of the first segment goes out before its tiles
       const __nv_bfloat16 *ck = p.cache_k + s.b * p.c_sb + s.hk * p.c_sh;
       const __nv_bfloat16 *cv = p.cache_v + s.b * p.c_sb + s.hk * p.c_sh;
       const __nv_bfloat16 *tk = p.tree_k + ((long long)s.b * p.n_kv_heads + s.hk) * p.t_max * kD;
       const __nv_bfloat16 *tv = p.tree_v + ((long long)s.b * p.n_kv_heads + s.hk) * p.t_max * kD;
       const int NK = s.L + s.n;
       for (int t = s.t0; t < s.t1 && ok; ++t, u += 2) {
-        complete_pending();
         const bool pure = t * KT + KT <= s.L;
-        if (!pure && !waited_dep) {
-          asm volatile("griddepcontrol.wait;" ::: "memory");
-          waited_dep = true;
-        }
-#pragma unroll 1
-        for (int kv = 0; kv < 2; ++kv) {
-          const int uu = u + kv, slot = uu % kSlots;
-          if (uu >= kSlots) {
-            ok = mbar_wait(bar_empty(slot), (uu / kSlots - 1) & 1, fail);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
+        if (!pure) {
+          if (!waited_dep) {
+            asm volatile("griddepcontrol.wait;" ::: "memory");
+            waited_dep = true;
           }
+          if (n_groups == 2) complete_oldest();
+        }
+        int slots_kv[2];
+#pragma unroll 1
+        for (int kv = 0; kv < 2 && ok; ++kv) {
+          const int uu = u + kv, slot = uu % kSlots;
+          slots_kv[kv] = slot;
+          if (uu >= kSlots) wait_bar(bar_empty(slot), (uu / kSlots - 1) & 1);
+          if (!ok) break;
           const uint32_t dst = ring_s + slot * kTileBytes;
           if (pure) {
             if (lane == 0) {
@@ -337,18 +503,24 @@ tree_attn_stream_kernel(const AttnParams p, const __grid_constant__ CUtensorMap 
               }
               cp_async_16(dst + panel + r * 128 + (((c & 7) ^ (r & 7)) << 4), src, valid);
             }
-            if (kv == 0) pend0 = slot;
-            else pend1 = slot;
           }
         }
-        if (!pure) cp_async_commit();
+        // (a wait that failed between the two halves leaves copies without a group: they are
+        // committed and waited for below like the rest, their barrier is never completed)
+        if (!pure) {
+          if (ok) open_group(slots_kv[0], slots_kv[1], -1);
+          else cp_async_commit();
+        }
+        // the next segments' Q tiles, as early as their buffers can be free: with two buffers after
+        // this segment's first tile, with one after its last
+        if (ok && (QB > 1 ? (q_next <= si + QB - 1 && t == s.t0) : (q_next <= si + 1 && t == s.t1 - 1))) request_q();
       }
     }
-    // (after a failed wait the copies in flight are still waited for; their arrivals are harmless)
-    complete_pending();
-    if (!ok) {
-      // giving up: the TMA requests already made still write into this CTA's shared memory, so the CTA
-      // stays for longer than any of them can take before it leaves
+    if (ok) complete_all();
+    else {
+      // giving up: the copies and TMA requests already made still write into this CTA's shared memory,
+      // so the CTA stays for longer than any of them can take before it leaves
+      cp_async_wait<0>();
       s_fail = 1;
       unsigned long long t0, t1;
       asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
@@ -358,44 +530,6 @@ tree_attn_stream_kernel(const AttnParams p, const __grid_constant__ CUtensorMap 
     }
     // every CTA carries the dependency on its predecessor on to its successor
     if (!waited_dep) asm volatile("griddepcontrol.wait;" ::: "memory");
-  } else if (warp == 6) {
-    // ================= Q warp: the Q tile of every segment, QB segments ahead =================
-    if (p.early_prefix) asm volatile("griddepcontrol.wait;" ::: "memory");
-    const int c = lane & 15, rbase = lane >> 4;      // chunk c of rows rbase, rbase + 2, ...
-    SegIter ahead = make_iter();
-    Seg sa;
-    bool ok = true;
-    for (int sj = 0; ok && ahead.next(sa); ++sj) {
-      const int buf = sj % QB;
-      if (sj >= QB) {
-        // the buffer's previous segment is done with it once all of its S products have completed
-        ok = mbar_wait(bar_qfree(buf), (sj / QB - 1) & 1, fail);
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
-      }
-      // zero rows past the request's last row.  Lane pairs walk the rows two apart; the (node, query
-      // head of the group) pair of a row is stepped, not divided.
-      const uint32_t qb = q_s + buf * C::Q_ONE;
-      const int row0 = sa.rb * ROWS, rows_total = sa.n * p.group;
-      int node = (row0 + rbase) / p.group, g = (row0 + rbase) % p.group;
-      for (int r = rbase; r < ROWS; r += 2) {
-        const bool valid = row0 + r < rows_total;
-        const __nv_bfloat16 *src =
-            p.q + (((long long)sa.b * p.t_max + (valid ? node : 0)) * p.n_q_heads + sa.hk * p.group + (valid ? g : 0)) * kD + c * 8;
-        cp_async_16(qb + (c >> 3) * ROWS * 128 + r * 128 + (((c & 7) ^ (r & 7)) << 4), src, valid);
-        g += 2;
-        while (g >= p.group) {
-          g -= p.group;
-          ++node;
-        }
-      }
-      cp_async_commit();
-      cp_async_wait<0>();
-      fence_async_smem();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar_q(buf));
-    }
-    if (!ok) s_fail = 1;
   } else if (warp == 5) {
     // ================= MMA issuer (one thread) =================
     if (lane == 0) {
@@ -468,9 +602,9 @@ tree_attn_stream_kernel(const AttnParams p, const __grid_constant__ CUtensorMap 
       }
       if (!ok) s_fail = 1;
     }
-  } else if ((warp & 3) < NSOFT && (warp < 4 || warp >= 7)) {
+  } else if ((warp & 3) < NSOFT && (warp < 4 || warp >= 6)) {
     // ================= softmax warps =================
-    const int quad = warp & 3, half = warp >= 7 ? 1 : 0;
+    const int quad = warp & 3, half = warp >= 6 ? 1 : 0;
     const int stid = (half * NSOFT + quad) * 32 + lane;              // index among the softmax threads
     const uint32_t t_lane = tmem + ((uint32_t)(quad * 32) << 16);    // this warp's 32 tensor-memory lanes
     auto soft_sync = [&]() { asm volatile("bar.sync 5, %0;" ::"n"(C::SOFT_THREADS) : "memory"); };
@@ -492,6 +626,7 @@ tree_attn_stream_kernel(const AttnParams p, const __grid_constant__ CUtensorMap 
     };
     int gt = 0;            // running tile index of this CTA
     int mask_b = -1;       // request whose ancestor masks are in s_mask
+    int n_partial = 0;     // partial segments so far (the ticket's hand-over word alternates)
     while (it.next(s)) {
       const int row0 = s.rb * ROWS, rows_total = s.n * p.group;
       const int n_it = s.t1 - s.t0;
@@ -809,6 +944,10 @@ tree_attn_stream_kernel(const AttnParams p, const __grid_constant__ CUtensorMap 
           amax *= inv_l;
           float down, up;
           row_scale(amax, down, up);
+          // one factor where it is finite (a row sum below 2^-100 or so overflows it: then two steps)
+          const float f1 = inv_l * down;
+          const bool one_step = f1 < INFINITY;
+          const float fa = one_step ? f1 : inv_l, fb = one_step ? 1.f : down;
 #pragma unroll
           for (int ch = 0; ch < 4; ++ch) {
             uint32_t v[32];
@@ -818,10 +957,10 @@ tree_attn_stream_kernel(const AttnParams p, const __grid_constant__ CUtensorMap 
 #pragma unroll
               for (int i = 0; i < 4; ++i) {
                 uint4 w;
-                w.x = pack_f16(__uint_as_float(v[8 * i]) * inv_l * down, __uint_as_float(v[8 * i + 1]) * inv_l * down);
-                w.y = pack_f16(__uint_as_float(v[8 * i + 2]) * inv_l * down, __uint_as_float(v[8 * i + 3]) * inv_l * down);
-                w.z = pack_f16(__uint_as_float(v[8 * i + 4]) * inv_l * down, __uint_as_float(v[8 * i + 5]) * inv_l * down);
-                w.w = pack_f16(__uint_as_float(v[8 * i + 6]) * inv_l * down, __uint_as_float(v[8 * i + 7]) * inv_l * down);
+                w.x = pack_f16(__uint_as_float(v[8 * i]) * fa * fb, __uint_as_float(v[8 * i + 1]) * fa * fb);
+                w.y = pack_f16(__uint_as_float(v[8 * i + 2]) * fa * fb, __uint_as_float(v[8 * i + 3]) * fa * fb);
+                w.z = pack_f16(__uint_as_float(v[8 * i + 4]) * fa * fb, __uint_as_float(v[8 * i + 5]) * fa * fb);
+                w.w = pack_f16(__uint_as_float(v[8 * i + 6]) * fa * fb, __uint_as_float(v[8 * i + 7]) * fa * fb);
                 st_16(slot + ((size_t)(ch * 4 + i) * ROWS + row_local) * 16, w);
               }
             }
@@ -832,70 +971,111 @@ tree_attn_stream_kernel(const AttnParams p, const __grid_constant__ CUtensorMap 
           __syncwarp();
           if (lane == 0) mbar_arrive(bar_ofree);        // the accumulator may be overwritten
           // ---- ticket: the last of the item's CTAs to get here finishes the item ----
-          __threadfence();
+          // (the barrier orders every thread's stores before thread 0's fence, which publishes them
+          // device-wide before the ticket is taken)
+          const int tk_par = n_partial & 1;
+          ++n_partial;
           group0_sync();
-          if (tid == 0 && ok) {
-            const unsigned int old = atomicAdd(tickets + s.item, 1u);
-            const int last = old == (unsigned int)(n_seg - 1);
-            if (last) tickets[s.item] = 0u;             // nobody else touches it before the next call
-            __threadfence();
-            s_last = last;
+          if (tid == 0) {
+            int last = 0;
+            if (ok) {
+              __threadfence();
+              const unsigned int old = atomicAdd(tickets + s.item, 1u);
+              last = old == (unsigned int)(n_seg - 1);
+              if (last) tickets[s.item] = 0u;           // nobody else touches it before the next call
+              __threadfence();
+            }
+            s_last[tk_par] = last;
           }
           group0_sync();
-          const bool last = s_last != 0;
-          group0_sync();                                // (s_last is rewritten by the next partial segment)
-          if (last && row_valid) {
-            // the partials of the item's CTAs c_first..c_last: first the overall maximum and the row
-            // sum, then the weighted rows, 32 columns at a time
+          if (s_last[tk_par] != 0 && ok) {
+            // ---- this CTA adds up the partials of the item's CTAs c_first..c_last ----
+            // Two threads per row (64 columns each, lanes 16-31 of a warp help lanes 0-15 out with
+            // 64-row accumulators); the partials are fetched four at a time so that a pass over them is
+            // one round trip to L2: first their (m, l, scale), then the rows, 32 columns per pass.
+            constexpr int TPR = C::MMA_M == 64 ? 2 : 1;            // threads per row
+            const int mrow = C::MMA_M == 64 ? 16 * quad + (lane & 15) : row_local;
+            const int chalf = C::MMA_M == 64 ? (lane >> 4) : 0;     // which half of the columns
+            const int mg = row0 + mrow;
+            const bool m_valid = mg < rows_total;
+            const int m_node = m_valid ? mg / p.group : 0, m_h = s.hk * p.group + (m_valid ? mg % p.group : 0);
+            __nv_bfloat16 *m_dst = p.out + (((long long)s.b * p.t_max + m_node) * p.n_q_heads + m_h) * kD;
             auto slot_of = [&](int c) {
               const int sl = 2 * c + ((c == c_first && s.gstart != share_begin(c, total, G)) ? 1 : 0);
               return slots + (size_t)sl * C::SLOT_BYTES;
             };
-            auto stats_of = [&](const unsigned char *sp) {
-              return __ldcg(reinterpret_cast<const float4 *>(sp + (size_t)ROWS * kD * 2 + row_local * 16));
+            auto stats_of = [&](int c) {
+              return __ldcg(reinterpret_cast<const float4 *>(slot_of(c) + (size_t)ROWS * kD * 2 + mrow * 16));
             };
             float mstar = -INFINITY;
-            for (int c = c_first; c <= c_last; ++c) mstar = fmaxf(mstar, stats_of(slot_of(c)).x);
+            for (int c0 = c_first; c0 <= c_last; c0 += 4) {
+              float4 st[4];
+#pragma unroll
+              for (int j = 0; j < 4; ++j) st[j] = stats_of(min(c0 + j, c_last));
+#pragma unroll
+              for (int j = 0; j < 4; ++j) mstar = fmaxf(mstar, st[j].x);
+            }
             float lsum = 0.f;
-            for (int c = c_first; c <= c_last; ++c) {
-              const float4 ml = stats_of(slot_of(c));
-              lsum += fast_exp2(ml.x - mstar) * ml.y;
+            for (int c0 = c_first; c0 <= c_last; c0 += 4) {
+              float4 st[4];
+#pragma unroll
+              for (int j = 0; j < 4; ++j) st[j] = stats_of(min(c0 + j, c_last));
+#pragma unroll
+              for (int j = 0; j < 4; ++j)
+                if (c0 + j <= c_last) lsum += fast_exp2(st[j].x - mstar) * st[j].y;
             }
             const float inv = 1.f / lsum;
 #pragma unroll 1
-            for (int cg4 = 0; cg4 < 4; ++cg4) {
+            for (int pass = 0; pass < (kD / 32) / TPR; ++pass) {
+              const int chunk0 = (chalf * ((kD / 32) / TPR) + pass) * 4;       // first of this pass's four 8-column chunks
               float acc[32];
 #pragma unroll
               for (int j = 0; j < 32; ++j) acc[j] = 0.f;
-              for (int c = c_first; c <= c_last; ++c) {
-                const unsigned char *sp = slot_of(c);
-                const float4 ml = stats_of(sp);
-                const float wgt = fast_exp2(ml.x - mstar) * ml.y * ml.z * inv;   // share of the row sum, times the row's scale
+              for (int c0 = c_first; c0 <= c_last; c0 += 4) {
+                float4 st[4];
+                uint4 raw[4][4];
 #pragma unroll
-                for (int ch = 0; ch < 4; ++ch) {
-                  const uint4 raw = __ldcg(reinterpret_cast<const uint4 *>(sp + ((size_t)(cg4 * 4 + ch) * ROWS + row_local) * 16));
-                  const float2 a0 = unpack_f16(raw.x), a1 = unpack_f16(raw.y), a2 = unpack_f16(raw.z), a3 = unpack_f16(raw.w);
-                  acc[8 * ch + 0] = fmaf(wgt, a0.x, acc[8 * ch + 0]);
-                  acc[8 * ch + 1] = fmaf(wgt, a0.y, acc[8 * ch + 1]);
-                  acc[8 * ch + 2] = fmaf(wgt, a1.x, acc[8 * ch + 2]);
-                  acc[8 * ch + 3] = fmaf(wgt, a1.y, acc[8 * ch + 3]);
-                  acc[8 * ch + 4] = fmaf(wgt, a2.x, acc[8 * ch + 4]);
-                  acc[8 * ch + 5] = fmaf(wgt, a2.y, acc[8 * ch + 5]);
-                  acc[8 * ch + 6] = fmaf(wgt, a3.x, acc[8 * ch + 6]);
-                  acc[8 * ch + 7] = fmaf(wgt, a3.y, acc[8 * ch + 7]);
+                for (int j = 0; j < 4; ++j) {
+                  const int c = min(c0 + j, c_last);
+                  const unsigned char *sp = slot_of(c);
+                  st[j] = __ldcg(reinterpret_cast<const float4 *>(sp + (size_t)ROWS * kD * 2 + mrow * 16));
+#pragma unroll
+                  for (int ch = 0; ch < 4; ++ch)
+                    raw[j][ch] = __ldcg(reinterpret_cast<const uint4 *>(sp + ((size_t)(chunk0 + ch) * ROWS + mrow) * 16));
+                }
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                  // share of the row sum, times the row's scale (nothing for a repeated last partial)
+                  const float wgt = (c0 + j <= c_last) ? fast_exp2(st[j].x - mstar) * st[j].y * st[j].z * inv : 0.f;
+#pragma unroll
+                  for (int ch = 0; ch < 4; ++ch) {
+                    const float2 a0 = unpack_f16(raw[j][ch].x), a1 = unpack_f16(raw[j][ch].y);
+                    const float2 a2 = unpack_f16(raw[j][ch].z), a3 = unpack_f16(raw[j][ch].w);
+                    acc[8 * ch + 0] = fmaf(wgt, a0.x, acc[8 * ch + 0]);
+                    acc[8 * ch + 1] = fmaf(wgt, a0.y, acc[8 * ch + 1]);
+                    acc[8 * ch + 2] = fmaf(wgt, a1.x, acc[8 * ch + 2]);
+                    acc[8 * ch + 3] = fmaf(wgt, a1.y, acc[8 * ch + 3]);
+                    acc[8 * ch + 4] = fmaf(wgt, a2.x, acc[8 * ch + 4]);
+                    acc[8 * ch + 5] = fmaf(wgt, a2.y, acc[8 * ch + 5]);
+                    acc[8 * ch + 6] = fmaf(wgt, a3.x, acc[8 * ch + 6]);
+                    acc[8 * ch + 7] = fmaf(wgt, a3.y, acc[8 * ch + 7]);
+                  }
                 }
               }
+              if (m_valid) {
 #pragma unroll
-              for (int ch = 0; ch < 4; ++ch) {
-                uint4 w;
-                w.x = pack_bf16(acc[8 * ch], acc[8 * ch + 1]);
-                w.y = pack_bf16(acc[8 * ch + 2], acc[8 * ch + 3]);
-                w.z = pack_bf16(acc[8 * ch + 4], acc[8 * ch + 5]);
-                w.w = pack_bf16(acc[8 * ch + 6], acc[8 * ch + 7]);
-                st_16(dst + 32 * cg4 + 8 * ch, w);
+                for (int ch = 0; ch < 4; ++ch) {
+                  uint4 w;
+                  w.x = pack_bf16(acc[8 * ch], acc[8 * ch + 1]);
+                  w.y = pack_bf16(acc[8 * ch + 2], acc[8 * ch + 3]);
+                  w.z = pack_bf16(acc[8 * ch + 4], acc[8 * ch + 5]);
+                  w.w = pack_bf16(acc[8 * ch + 6], acc[8 * ch + 7]);
+                  st_16(m_dst + 8 * (chunk0 + ch), w);
+                }
               }
             }
-            if (lse_dst) *lse_dst = (mstar + log2f(lsum)) * 0.6931471805599453f;
+            if (p.lse && m_valid && chalf == 0)
+              p.lse[((long long)s.b * p.n_q_heads + m_h) * p.t_max + m_node] = (mstar + log2f(lsum)) * 0.6931471805599453f;
           }
         }
       }
@@ -982,7 +1162,7 @@ twig_status launch_tree_attn_stream(AttnParams &p, int batch, int rows, cudaStre
   unsigned char *slots = p.ws;
   unsigned int *tickets = reinterpret_cast<unsigned int *>(p.ws + slot_bytes);
   if (rows_per_cta == 32) return launch_stream<32, 64, 2, 5>(p, maps, grid, tickets, slots, st);
-  return launch_stream<64, 64, 2, 4>(p, maps, grid, tickets, slots, st);
+  return launch_stream<64, 64, TWIG_STREAM64_QB, TWIG_STREAM64_SLOTS>(p, maps, grid, tickets, slots, st);
 }
 
 }  // namespace twig

@@ -32,11 +32,21 @@ def stream_ws(tw, B, Hq, T):
     return _WS[need]
 
 
+# kernels under test: (id, kernel, work sharing of the persistent kernel: 0 its own choice, 1 equal shares, 2 whole items)
+KERNELS = [("mma", 1), ("tcgen05", 2), ("stream", 3), ("stream-shares", (3, 1)), ("stream-whole", (3, 2))]
+KERNEL_IDS = [k[0] for k in KERNELS]
+KERNEL_VALS = [k[1] for k in KERNELS]
+
+
 def run_attention(tw, wl, ver, cache_k, cache_v, kv_len, layer=0, max_len=None, lse=True, path=0, splits=0,
                   early=False):
     """cache_k/v: uint16 [Nl,B,Hkv,Lmax,d].  Returns (out bits [B,T,Hq,d], lse [B,Hq,T], status).
-    path: 0 automatic, 1 mma.sync kernel, 2 tcgen05 kernel (cluster splits), 3 persistent tcgen05 kernel.
+    path: 0 automatic, 1 mma.sync kernel, 2 tcgen05 kernel (cluster splits), 3 persistent tcgen05 kernel,
+    (3, policy) the persistent kernel with its work sharing forced.
     A named kernel is the kernel that runs (the library refuses, it never substitutes)."""
+    policy = 0
+    if isinstance(path, tuple):
+        path, policy = path
     B, T, Hq, d = ver["q"].shape[1:]
     ws = stream_ws(tw, B, Hq, T) if path == 3 else None
     ck, cv = dev_bf16(cache_k), dev_bf16(cache_v)
@@ -48,7 +58,7 @@ def run_attention(tw, wl, ver, cache_k, cache_v, kv_len, layer=0, max_len=None, 
     tw.tree_verify_attention(dev_bf16(ver["q"][layer]), dev_bf16(ver["tree_k"][layer]), dev_bf16(ver["tree_v"][layer]),
                              tw.KV.of(ck, cv), layer, dev_i32(kv_len), dev_i32(ver["n_nodes"]), dev_i32(ver["parent"]),
                              out, lse=lse_t, dev_status=status, ws=ws,
-                             flags=tw.attn_flags(kernel=path, splits=splits, early_prefix=early))
+                             flags=tw.attn_flags(kernel=path, splits=splits, early_prefix=early, stream_policy=policy))
     torch.cuda.synchronize()
     if ws is not None:      # the call leaves its arrival counters (the tail of the buffer) at zero
         n_tail = tw.tree_attention_workspace_bytes(B, Hq, T) - tw.tree_attention_workspace_bytes(1, 1, T) + 8
@@ -100,10 +110,10 @@ SHAPES = [
 
 @pytest.mark.parametrize("shape", SHAPES, ids=[s[0] for s in SHAPES])
 @pytest.mark.parametrize("gain_name", ["timing", "sharp", "sharp4"])
-@pytest.mark.parametrize("path", [1, 2, 3], ids=["mma", "tcgen05", "stream"])
+@pytest.mark.parametrize("path", KERNEL_VALS, ids=KERNEL_IDS)
 def test_tree_attention_matches_oracle(tw, shape, gain_name, path):
     name, B, Hq, Hkv, d, n_nodes, depth, kv_len = shape
-    if path >= 2 and d != 128:
+    if path != 1 and d != 128:
         pytest.skip("the tcgen05 kernels cover head_dim 128")
     gain = {"timing": 1.0, "sharp": d ** 0.5, "sharp4": 2.0 * d ** 0.5}[gain_name]   # logit std 1/d, 1, 4
     wl = _wl(B, Hq, Hkv, d, n_nodes, depth)
@@ -120,7 +130,7 @@ def test_tree_attention_matches_oracle(tw, shape, gain_name, path):
     check(got, lse, want, want_lse, ver["n_nodes"], name)
 
 
-@pytest.mark.parametrize("path", [1, 2, 3], ids=["mma", "tcgen05", "stream"])
+@pytest.mark.parametrize("path", KERNEL_VALS, ids=KERNEL_IDS)
 @pytest.mark.parametrize("kind", ["chain", "star"])
 def test_special_trees(tw, kind, path):
     T = 20
@@ -135,7 +145,7 @@ def test_special_trees(tw, kind, path):
     check(got, lse, want, want_lse, ver["n_nodes"], kind)
 
 
-@pytest.mark.parametrize("path", [1, 2, 3], ids=["mma", "tcgen05", "stream"])
+@pytest.mark.parametrize("path", KERNEL_VALS, ids=KERNEL_IDS)
 def test_bad_tree_and_overflow_set_status(tw, path):
     wl = _wl(4, 4, 4, 128, [6, 6, 6, 6], [3, 3, 3, 3])
     rng = synth.rng_for(9, 78)
@@ -160,7 +170,7 @@ FULL = [
 ]
 
 
-@pytest.mark.parametrize("path", [1, 2, 3], ids=["mma", "tcgen05", "stream"])
+@pytest.mark.parametrize("path", KERNEL_VALS, ids=KERNEL_IDS)
 @pytest.mark.parametrize("index,lens", FULL, ids=["c2", "c3", "c4", "c5"])
 def test_full_size_configs(tw, index, lens, path):
     """Full-size shapes of the benchmark configurations, one layer, every output row
@@ -273,8 +283,8 @@ def test_named_kernel_is_never_substituted(tw):
 
 
 @pytest.mark.parametrize("v_scale", [2.0 ** -17, 1.0, 2.0 ** 17], ids=["tinyV", "unitV", "largeV"])
-@pytest.mark.parametrize("path,splits", [(1, 1), (1, 2), (1, 4), (1, 8), (2, 1), (2, 2), (2, 4), (2, 8), (3, 0)],
-                         ids=lambda v: str(v))
+@pytest.mark.parametrize("path,splits", [(1, 1), (1, 2), (1, 4), (1, 8), (2, 1), (2, 2), (2, 4), (2, 8), ((3, 1), 0),
+                                         ((3, 2), 0)], ids=lambda v: str(v))
 def test_key_splits_and_value_range(tw, path, splits, v_scale):
     """The result must not depend on how the keys are split between CTAs, nor on the magnitude of V:
     partial results cross between CTAs in a narrower format than they are accumulated in."""
