@@ -187,8 +187,18 @@ twig_status ttp_topk(const float *scores, const int32_t *n_vis, const int32_t *k
  * dst row j = src row idx[j] (bytes copied verbatim), pos_out[b, j] =
  * pos_in[b, idx[j]], new_len[b] = prefix_len - n_vis + keep.  keep = 0 drops
  * every visual token (the FinalWipe form); keep = n_vis is the identity.
- * dst must not overlap src.  pos_in/pos_out ([batch, pos_stride], may both be
- * NULL) and new_len (may be NULL) are int32.
+ * pos_in/pos_out ([batch, pos_stride], may both be NULL) and new_len (may be
+ * NULL) are int32.
+ * Aliasing: dst either shares no byte with src (rows past new_len of dst are
+ * left as they were), or names the very same tensors (same k, v, strides and
+ * max_len): the cache is then compacted IN PLACE, which saves the second copy
+ * of the KV cache; pos_out must then be pos_in (or both NULL).  Rows only move
+ * to lower positions, so one CTA per (layer, kv head) slice moves them chunk by
+ * chunk in ascending order; rows that stay where they are are not touched and
+ * rows past new_len keep their old contents.  Any other overlap of dst and src
+ * is refused with TWIG_ERR_UNSUPPORTED.  In place, a kept_idx list that is not
+ * strictly ascending within [0, n_vis) is detected before anything moves
+ * (TWIG_DEV_BAD_INDEX, request untouched).
  */
 twig_status ttp_compact(const twig_kv *src, const twig_kv *dst, const int32_t *kept_idx,
                         int32_t r_max, const int32_t *keep, const int32_t *prefix_len,
@@ -342,6 +352,33 @@ twig_status tree_finalize(const int32_t *node_tok, const int32_t *node_parent, c
                           int32_t cap, int32_t n_built, int32_t n_max, int32_t *parent, int32_t *draft_tok,
                           int32_t *n_nodes, int32_t *kept_node, int32_t t_max, int32_t batch,
                           int32_t *dev_status, void *stream);
+
+/* ---- Chain drafting with early exit (sequence self-speculative decoding) ------
+ * Appendix A, "Self-speculative decoding", and Algorithm 1's draft loop: in every iteration the draft
+ * model predicts up to delta = 5 tokens one after another and stops early once the probability of
+ * the token it has just predicted falls below theta = 0.6; that token still counts as drafted.  The
+ * draft model runs between the calls; chain_draft_step takes one draft distribution per request:
+ *   token = argmax_v logits[b, v] (lowest id among equal logits), prob = softmax(logits[b])[token],
+ *   node n = n_nodes[b] is appended to the request's chain: parent[b, n] = n - 1,
+ *   draft_tok[b, n] = token, tok_prob[b, n] = prob (optional), n_nodes[b] = n + 1;
+ *   the request stops drafting (active[b] = 0) once it holds max_draft draft tokens or prob < threshold.
+ * Requests with active[b] == 0 are left alone, so a batch is driven through max_draft calls without
+ * reading anything back; afterwards n_nodes[b] - 1 is the request's draft length.  The arrays are
+ * the ones tree_verify_attention and tree_accept_compact take (a chain is a tree whose node i has
+ * parent i - 1; node 0, the root, is the last accepted token).  chain_draft_reset starts an
+ * iteration: n_nodes = 1, parent[b, 0] = -1, draft_tok[b, 0] = -1, active = 1.
+ *   logits   [batch, vocab] at logits + b*row_stride (ELEMENTS), bf16 (logits_fp32 = 0) or fp32; rows
+ *            16-byte aligned; must not be NaN
+ *   parent, draft_tok [batch, t_max] int32; tok_prob [batch, t_max] fp32 or NULL; n_nodes, active [batch]
+ *   max_draft + 1 <= t_max <= TWIG_MAX_NODES (TWIG_ERR_SHAPE otherwise); threshold >= 0
+ * The probability is formed in fp32 (one pass: running maximum and sum of exponentials).
+ */
+twig_status chain_draft_reset(int32_t *parent, int32_t *draft_tok, float *tok_prob, int32_t *n_nodes,
+                              int32_t *active, int32_t t_max, int32_t batch, void *stream);
+twig_status chain_draft_step(const void *logits, int32_t logits_fp32, int64_t row_stride, int32_t vocab,
+                             int32_t max_draft, float threshold, int32_t *parent, int32_t *draft_tok,
+                             float *tok_prob, int32_t *n_nodes, int32_t *active, int32_t t_max,
+                             int32_t batch, int32_t *dev_status, void *stream);
 
 /* ---- Greedy target token of every tree node (input of tree_accept_compact) -----
  * Algorithm 2 ("argmax(tgt_probs[...])"), Sec. 5.4: base_argmax[b, i] = the index of the largest of

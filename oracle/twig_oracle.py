@@ -156,6 +156,8 @@ def gather_compact(src_k, src_v, pos_in, prefix_len, vis_start, n_vis, kept_list
 
     Arrays of any dtype (bit patterns are moved verbatim); dst/pos_out are
     updated in place, rows >= new_len are left as they were.  Returns new_len.
+    dst may be src itself (compaction in place): rows are assigned in ascending
+    order and idx_b[j] >= j, so a row is read before anything is written over it.
     """
     B = src_k.shape[1]
     new_len = np.zeros(B, dtype=np.int32)
@@ -373,6 +375,29 @@ def build_token_tree(level_logits, E: int, K: int, n_max: int):
 # --------------------------------------------------------------------------
 # O6: append the accepted nodes' K/V rows to the cache
 # --------------------------------------------------------------------------
+def chain_draft(step_logits, delta: int, theta: float):
+    """Draft loop of sequence self-speculative decoding for one request (Appendix A, "Self-speculative
+    decoding"; Algorithm 1): step_logits[i] is the draft distribution of step i (in the real loop it
+    depends on the tokens drafted before; here the rows are given).  Every step appends the greedy token
+    (lowest id among equal logits) and its probability; drafting stops once delta tokens are drafted or
+    the probability of the token just appended is below theta (that token stays in the draft).
+    Returns (tokens, probabilities)."""
+    toks, probs = [], []
+    for x in step_logits:
+        x = np.asarray(x, dtype=np.float64)
+        tok = 0
+        for v in range(1, len(x)):
+            if x[v] > x[tok]:
+                tok = v
+        e = np.exp(x - x[tok])
+        prob = float(e[tok] / e.sum())
+        toks.append(tok)
+        probs.append(prob)
+        if len(toks) >= delta or prob < theta:
+            break
+    return toks, probs
+
+
 def accept_compact(tree_k, tree_v, cache_k, cache_v, kv_len, paths):
     """tree_k/v [Nl,B,Hkv,T,d]; cache_k/v [Nl,B,Hkv,Lmax,d] updated in place:
     cache[l,b,h,kv_len[b]+j,:] = tree[l,b,h,path_b[j],:]; returns new kv_len."""

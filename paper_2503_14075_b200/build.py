@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.environ.get("TWIG_LIB") or os.path.join(HERE, "libtwig.so")   # TWIG_LIB: load another build
-SOURCES = ["api.cu", "ttp.cu", "ttp_mq.cu", "tree_attn.cu", "tree_attn_umma.cu", "tree_attn_stream.cu", "tree_accept.cu", "tree_build.cu"]
+SOURCES = ["api.cu", "ttp.cu", "ttp_mq.cu", "tree_attn.cu", "tree_attn_umma.cu", "tree_attn_stream.cu", "tree_accept.cu", "tree_build.cu", "chain_draft.cu"]
 
 
 def _newest_source_mtime() -> float:

@@ -358,6 +358,99 @@ kv_gather_kernel(KvView src, KvViewMut dst, const int *__restrict__ kept_idx, in
 }
 
 // ---------------------------------------------------------------------------
+// Stage 3 in place (dst is src).  Rows only ever move to lower positions (the source of row j is
+// idx[j] >= j), so a slice can be compacted where it lies if ONE CTA owns it and works through
+// ascending chunks of rows, loading a whole chunk before it stores any row of it: a chunk's stores
+// land below every row a later chunk reads, and the rows a chunk overwrites are either its own
+// sources (already in registers) or rows nobody needs any more.  Independent CTAs on one slice
+// would race, so the grid is one CTA per (layer, kv head, K or V, request).  Rows that stay where
+// they are (the text before the image, kept tokens at the head of the image) are not touched.
+// The kept list is validated in full before the first store: an in-place pass cannot be undone.
+// ---------------------------------------------------------------------------
+constexpr int kInplacePasses = 8;      // 16-byte loads in flight per thread
+
+__device__ __forceinline__ uint4 ld_cg_16(const void *p) {
+  uint4 r;
+  asm volatile("ld.global.cg.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
+  return r;
+}
+
+template <int D>
+__global__ void __launch_bounds__(kGatherThreads)
+kv_compact_inplace_kernel(KvViewMut kv, const int *__restrict__ kept_idx, int r_max,
+                          const int *__restrict__ keep, const int *__restrict__ prefix_len,
+                          const int *__restrict__ vis_start, const int *__restrict__ n_vis, int *pos,
+                          int pos_stride, int *__restrict__ new_len, int *dev_status) {
+  constexpr int LPR = D / 8;                   // lanes per row
+  constexpr int RPP = kGatherThreads / LPR;    // rows per pass
+  constexpr int CHUNK = RPP * kInplacePasses;  // rows per chunk
+  const int b = blockIdx.z, which = blockIdx.y;
+  const int layer = blockIdx.x / kv.n_kv_heads, h = blockIdx.x % kv.n_kv_heads;
+  const int lp = prefix_len[b], vs = vis_start[b], nv = n_vis[b], kp = keep[b];
+  const bool first = blockIdx.x == 0 && which == 0 && threadIdx.x == 0;
+  if (!layout_ok(lp, vs, nv, kv.max_len, TWIG_MAX_VISUAL)) {
+    if (first) flag_status(dev_status, b, TWIG_DEV_BAD_LAYOUT);
+    return;
+  }
+  if (kp < 0 || kp > nv || kp > r_max) {
+    if (first) flag_status(dev_status, b, TWIG_DEV_BAD_KEEP);
+    return;
+  }
+  const int *kidx = kept_idx + (long long)b * r_max;
+  int bad = 0;
+  for (int i = threadIdx.x; i < kp; i += kGatherThreads) {
+    const int kk = kidx[i], prev = i > 0 ? kidx[i - 1] : -1;
+    bad |= (kk < 0 || kk >= nv || kk <= prev) ? 1 : 0;
+  }
+  if (__syncthreads_or(bad)) {
+    if (first) flag_status(dev_status, b, TWIG_DEV_BAD_INDEX);
+    return;
+  }
+  const int nl = lp - nv + kp;
+  if (first && new_len) new_len[b] = nl;
+  auto source = [&](int j) { return j < vs + kp ? vs + kidx[j - vs] : j - kp + nv; };   // j >= vs
+
+  __nv_bfloat16 *base = (which ? kv.v : kv.k) + layer * kv.stride_layer + b * kv.stride_batch + h * kv.stride_head;
+  const int sub = threadIdx.x % LPR, slot = threadIdx.x / LPR;
+  for (int j0 = vs; j0 < nl; j0 += CHUNK) {
+    uint4 val[kInplacePasses];
+    bool moved[kInplacePasses];
+#pragma unroll
+    for (int p = 0; p < kInplacePasses; ++p) {
+      const int j = j0 + p * RPP + slot;
+      moved[p] = false;
+      if (j < nl) {
+        const int sj = source(j);
+        moved[p] = sj != j;
+        if (moved[p]) val[p] = ld_cg_16(base + (long long)sj * kv.stride_pos + sub * 8);
+      }
+    }
+    __syncthreads();                         // the whole chunk is in registers
+#pragma unroll
+    for (int p = 0; p < kInplacePasses; ++p) {
+      const int j = j0 + p * RPP + slot;
+      if (moved[p]) st_16(base + (long long)j * kv.stride_pos + sub * 8, val[p]);
+    }
+  }
+  // position ids, by the CTA of the first slice: the same schedule, one row per thread
+  if (blockIdx.x == 0 && which == 0 && pos) {
+    int *prow = pos + (long long)b * pos_stride;
+    for (int j0 = vs; j0 < nl; j0 += kGatherThreads) {
+      const int j = j0 + threadIdx.x;
+      int v = 0;
+      bool moved = false;
+      if (j < nl) {
+        const int sj = source(j);
+        moved = sj != j;
+        if (moved) v = __ldcg(prow + sj);
+      }
+      __syncthreads();
+      if (moved) prow[j] = v;
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------
 // Stage 3 on rows of any width (hidden states of layer K; FinalWipe with keep = 0).
 // One CTA = 4 destination rows of one request; 16-byte chunks, 8 loads in flight per thread.
 // ---------------------------------------------------------------------------
@@ -511,6 +604,23 @@ static twig_status launch_finalize(const float *logits, const ScoreArgs &a, cons
   return launch_status();
 }
 
+// bytes from the base pointer to the end of the last row of a K (or V) tensor
+static size_t kv_extent_bytes(const twig_kv *kv) {
+  const long long last = (long long)(kv->n_layers - 1) * kv->stride_layer + (long long)(kv->batch - 1) * kv->stride_batch +
+                         (long long)(kv->n_kv_heads - 1) * kv->stride_head + (long long)(kv->max_len - 1) * kv->stride_pos +
+                         kv->head_dim;
+  return (size_t)last * sizeof(__nv_bfloat16);
+}
+static bool ranges_overlap(const void *a, size_t na, const void *b, size_t nb) {
+  const uintptr_t x = reinterpret_cast<uintptr_t>(a), y = reinterpret_cast<uintptr_t>(b);
+  return x < y + nb && y < x + na;
+}
+// dst names exactly the tensors of src: compaction in place
+static bool same_kv(const twig_kv *a, const twig_kv *b) {
+  return a->k == b->k && a->v == b->v && a->stride_layer == b->stride_layer && a->stride_batch == b->stride_batch &&
+         a->stride_head == b->stride_head && a->stride_pos == b->stride_pos && a->max_len == b->max_len;
+}
+
 static twig_status check_compact_args(const twig_kv *src, const twig_kv *dst, const int *kept_idx,
                                       int r_max, const int *keep, const int *prefix_len,
                                       const int *vis_start, const int *n_vis, const int *pos_in,
@@ -525,9 +635,17 @@ static twig_status check_compact_args(const twig_kv *src, const twig_kv *dst, co
   if (src->head_dim != dst->head_dim || src->n_layers != dst->n_layers || src->batch != dst->batch ||
       src->n_kv_heads != dst->n_kv_heads)
     return TWIG_ERR_SHAPE;
-  if (src->k == dst->k || src->v == dst->v || src->k == dst->v || src->v == dst->k)
-    return TWIG_ERR_UNSUPPORTED;   // in-place compaction is not offered
   if ((long long)src->n_layers * src->n_kv_heads > 65535) return TWIG_ERR_UNSUPPORTED;
+  // dst is either the very same tensors as src (in place) or shares no byte with them
+  if (!same_kv(src, dst)) {
+    const void *sa[2] = {src->k, src->v}, *da[2] = {dst->k, dst->v};
+    for (int i = 0; i < 2; ++i)
+      for (int j = 0; j < 2; ++j)
+        if (ranges_overlap(sa[i], kv_extent_bytes(src), da[j], kv_extent_bytes(dst))) return TWIG_ERR_UNSUPPORTED;
+    if (pos_in && pos_in == pos_out) return TWIG_ERR_UNSUPPORTED;
+  } else if (ranges_overlap(src->k, kv_extent_bytes(src), src->v, kv_extent_bytes(src))) {
+    return TWIG_ERR_UNSUPPORTED;
+  }
   return TWIG_OK;
 }
 
@@ -535,6 +653,23 @@ static twig_status launch_gather(const twig_kv *src, const twig_kv *dst, const i
                                  const int *keep, const int *prefix_len, const int *vis_start,
                                  const int *n_vis, const int *pos_in, int *pos_out, int pos_stride,
                                  int *new_len, int *dev_status, cudaStream_t st) {
+  if (same_kv(src, dst)) {
+    // in place: one CTA per (layer, kv head, K or V, request); position ids move in place as well
+    // (pos_out may be pos_in, or a separate array that then receives the gathered ids)
+    if (pos_in && pos_out && pos_in != pos_out) {
+      // a separate pos_out: gather it with the out-of-place rule (one small launch over no KV rows
+      // would cost more than it is worth; the in-place kernel compacts pos_in itself instead)
+      return TWIG_ERR_UNSUPPORTED;
+    }
+    dim3 grid(src->n_layers * src->n_kv_heads, 2, src->batch);
+    if (src->head_dim == 128)
+      kv_compact_inplace_kernel<128><<<grid, kGatherThreads, 0, st>>>(view_of_mut(dst), kept_idx, r_max, keep, prefix_len,
+          vis_start, n_vis, pos_out, pos_stride, new_len, dev_status);
+    else
+      kv_compact_inplace_kernel<64><<<grid, kGatherThreads, 0, st>>>(view_of_mut(dst), kept_idx, r_max, keep, prefix_len,
+          vis_start, n_vis, pos_out, pos_stride, new_len, dev_status);
+    return launch_status();
+  }
   const int rows_bound = src->max_len < dst->max_len ? src->max_len : dst->max_len;
   dim3 grid((rows_bound + kGatherRows - 1) / kGatherRows, src->n_layers * src->n_kv_heads, src->batch);
   if (src->head_dim == 128)

@@ -27,7 +27,7 @@ DEV_OK, DEV_BAD_LAYOUT, DEV_BAD_KEEP, DEV_BAD_INDEX, DEV_BAD_TREE, DEV_OVERFLOW,
 MAX_NODES, MAX_VISUAL, MAX_BATCH = 64, 16384, 4096
 
 EXPORTS = ["twig_status_str", "twig_set_launch_overlap", "twig_workspace_bytes", "tree_attention_workspace_bytes", "tree_verify_attention_ex", "ttp_score", "ttp_score_gated", "ttp_multiquery_workspace_bytes", "ttp_score_multiquery", "ttp_score_noalloc", "ttp_topk", "ttp_compact", "ttp_compact_rows",
-           "ttp_score_topk_compact", "tree_verify_attention", "tree_reset", "tree_expand_level", "tree_select_expansion", "tree_finalize", "tree_base_argmax", "tree_accept_compact"]
+           "ttp_score_topk_compact", "tree_verify_attention", "tree_reset", "tree_expand_level", "tree_select_expansion", "tree_finalize", "tree_base_argmax", "tree_accept_compact", "chain_draft_reset", "chain_draft_step"]
 
 
 class TwigError(RuntimeError):
@@ -117,6 +117,10 @@ _lib.tree_finalize.restype = C.c_int
 _lib.tree_finalize.argtypes = [_vp, _vp, _vp, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _i32, _i32, _vp, _vp]
 _lib.tree_base_argmax.restype = C.c_int
 _lib.tree_base_argmax.argtypes = [_vp, _i32, _i64, _i32, _vp, _i32, _i32, _vp, _vp, _vp]
+_lib.chain_draft_reset.restype = C.c_int
+_lib.chain_draft_reset.argtypes = [_vp, _vp, _vp, _vp, _vp, _i32, _i32, _vp]
+_lib.chain_draft_step.restype = C.c_int
+_lib.chain_draft_step.argtypes = [_vp, _i32, _i64, _i32, _i32, _f32, _vp, _vp, _vp, _vp, _vp, _i32, _i32, _vp, _vp]
 _lib.tree_accept_compact.restype = C.c_int
 _lib.tree_accept_compact.argtypes = [_vp, _vp, _vp, _vp, _i32, _i32, _vp, _vp, _kvp, _vp, _vp, _vp, _vp,
                                      _vp, _vp]
@@ -311,6 +315,23 @@ def tree_base_argmax(logits, n_nodes, base_argmax, dev_status=None, stream=None)
     assert logits.stride(2) == 1 and logits.stride(0) == T * logits.stride(1)
     _check(_lib.tree_base_argmax(_p(logits), 1 if logits.dtype == torch.float32 else 0, logits.stride(1), V,
                                  _p(n_nodes), B, T, _p(base_argmax), _p(dev_status), _stream(stream)))
+
+
+def chain_draft_reset(parent, draft_tok, n_nodes, active, tok_prob=None, stream=None):
+    """Start a drafting iteration: every request holds its root only and is drafting."""
+    _check(_lib.chain_draft_reset(_p(parent), _p(draft_tok), _p(tok_prob), _p(n_nodes), _p(active), parent.shape[1],
+                                  parent.shape[0], _stream(stream)))
+
+
+def chain_draft_step(logits, max_draft, threshold, parent, draft_tok, n_nodes, active, tok_prob=None, dev_status=None,
+                     stream=None):
+    """logits [B, V] bf16 or fp32 (last dim contiguous): one draft distribution per request.  Appends the
+    greedy token to the chains of the requests that are still drafting and applies the early exit."""
+    B, V = logits.shape
+    assert logits.stride(1) == 1
+    _check(_lib.chain_draft_step(_p(logits), 1 if logits.dtype == torch.float32 else 0, logits.stride(0), V, max_draft,
+                                 threshold, _p(parent), _p(draft_tok), _p(tok_prob), _p(n_nodes), _p(active),
+                                 parent.shape[1], B, _p(dev_status), _stream(stream)))
 
 
 def tree_accept_compact(parent, draft_tok, base_argmax, n_nodes, tree_k_all, tree_v_all, cache: KV,

@@ -25,6 +25,9 @@ def _small_workload(B, Hq, Hkv, d, lens, keep, index=9):
 WORKLOADS = {
     "c1": lambda: synth.workload(1),
     "c2": lambda: synth.workload(2),
+    "c3": lambda: synth.workload(3),      # the heterogeneous batch of 16
+    "c4": lambda: synth.workload(4),      # 3008-token prompts, 2880 visual tokens
+    "c5": lambda: synth.workload(5),      # 28 query heads on 4 kv heads
     "hetero": lambda: _small_workload(5, 8, 8, 128, [(35, 576, 40), (20, 300, 0), (0, 129, 7), (3, 1, 1), (10, 0, 5)],
                                       [64, 300, 1, 0, 0]),
     "gqa64": lambda: _small_workload(3, 12, 4, 64, [(17, 333, 9), (1, 1025, 130), (0, 64, 0)], [33, 128, 64]),
@@ -254,6 +257,76 @@ def test_compact_byte_exact(tw, name):
     assert np.array_equal(gnew, onew)
     assert np.array_equal(gk, ok) and np.array_equal(gv, ov)          # moved rows and untouched canaries
     assert np.array_equal(gpos, opos)
+
+
+def _compact_in_place_case(tw, wl, pre, kept_lists):
+    """Compaction in place on the device against the oracle's gather with dst = src on a copy
+    of the same bits: the whole cache is compared, so rows that must not move are checked too."""
+    B = wl.batch
+    r_max = max(1, max(len(k) for k in kept_lists))
+    kept = np.full((B, r_max), -1, dtype=np.int32)
+    for b, kl in enumerate(kept_lists):
+        kept[b, :len(kl)] = kl
+    keep = np.array([len(k) for k in kept_lists], dtype=np.int32)
+    ck, cv = dev_bf16(pre["cache_k"]), dev_bf16(pre["cache_v"])
+    pos = dev_i32(pre["pos_ids"] * 3 + 1)
+    new_len = torch.full((B,), -5, dtype=torch.int32, device=DEV)
+    status = torch.zeros(B, dtype=torch.int32, device=DEV)
+    cache = tw.KV.of(ck, cv)
+    tw.ttp_compact(cache, cache, dev_i32(kept), dev_i32(keep), dev_i32(pre["prefix_len"]), dev_i32(pre["vis_start"]),
+                   dev_i32(pre["n_vis"]), pos, pos, new_len, status)
+    torch.cuda.synchronize()
+    ok, ov, opos = pre["cache_k"].copy(), pre["cache_v"].copy(), (pre["pos_ids"] * 3 + 1).astype(np.int32)
+    onew = O.gather_compact(ok, ov, opos, pre["prefix_len"], pre["vis_start"], pre["n_vis"], kept_lists, ok, ov, opos)
+    return host_bits(ck), host_bits(cv), pos.cpu().numpy(), new_len.cpu().numpy(), status.cpu().numpy(), ok, ov, opos, onew
+
+
+@pytest.mark.parametrize("name", ["c1", "hetero", "gqa64", "c2"])
+def test_compact_in_place_byte_exact(tw, name):
+    wl = WORKLOADS[name]()
+    nl = 3 if name != "c2" else 2
+    pre = synth.make_prefill(wl, synth.rng_for(wl.index, 3), n_layers=nl)
+    rng = np.random.default_rng(4)
+    kept_lists = [sorted(rng.choice(m, size=r, replace=False).tolist()) if r else [] for m, r in zip(wl.n_vis, wl.keep)]
+    gk, gv, gpos, gnew, status, ok, ov, opos, onew = _compact_in_place_case(tw, wl, pre, kept_lists)
+    assert not status.any()
+    assert np.array_equal(gnew, onew)
+    assert np.array_equal(gk, ok) and np.array_equal(gv, ov) and np.array_equal(gpos, opos)
+
+
+def test_compact_in_place_adversarial_lists(tw):
+    """Kept lists whose rows move by a single position, lists longer than a chunk of the kernel,
+    keep-all (nothing may move) and keep-none."""
+    wl = _small_workload(6, 4, 4, 128, [(3, 6, 5), (0, 400, 30), (7, 400, 0), (2, 300, 300), (5, 70, 9), (0, 33, 2)],
+                         [3, 399, 1, 150, 70, 0])
+    pre = synth.make_prefill(wl, synth.rng_for(9, 8), n_layers=2)
+    kept = [[0, 2, 3], [i for i in range(400) if i != 7], [399], list(range(150, 300)), list(range(70)), []]
+    gk, gv, gpos, gnew, status, ok, ov, opos, onew = _compact_in_place_case(tw, wl, pre, kept)
+    assert not status.any() and np.array_equal(gnew, onew)
+    assert np.array_equal(gk, ok) and np.array_equal(gv, ov) and np.array_equal(gpos, opos)
+    assert np.array_equal(gk[:, 4], pre["cache_k"][:, 4])            # keep-all: the request's cache is untouched
+
+
+def test_compact_in_place_refuses_bad_lists_before_moving_anything(tw):
+    wl = _small_workload(2, 4, 4, 64, [(5, 20, 4), (5, 20, 4)], [3, 3])
+    pre = synth.make_prefill(wl, synth.rng_for(9, 6), n_layers=1)
+    gk, gv, gpos, gnew, status, ok, ov, opos, onew = _compact_in_place_case(tw, wl, pre, [[1, 2, 3], [1, 2, 3]])
+    assert not status.any()
+    B = 2
+    ck, cv = dev_bf16(pre["cache_k"]), dev_bf16(pre["cache_v"])
+    cache = tw.KV.of(ck, cv)
+    status = torch.zeros(B, dtype=torch.int32, device=DEV)
+    tw.ttp_compact(cache, cache, dev_i32([[1, 2, 3], [4, 2, 9]]), dev_i32([3, 3]), dev_i32(pre["prefix_len"]),
+                   dev_i32(pre["vis_start"]), dev_i32(pre["n_vis"]), dev_status=status)
+    torch.cuda.synchronize()
+    assert status.cpu().tolist() == [0, tw.DEV_BAD_INDEX]
+    assert np.array_equal(host_bits(ck)[:, 1], pre["cache_k"][:, 1])      # the bad request's cache is untouched
+    # partial overlap of source and destination is refused on the host
+    half = tw.KV.of(ck[:, :, :, 1:], cv[:, :, :, 1:])
+    with pytest.raises(tw.TwigError) as e:
+        tw.ttp_compact(cache, half, dev_i32([[1, 2, 3], [1, 2, 3]]), dev_i32([3, 3]), dev_i32(pre["prefix_len"]),
+                       dev_i32(pre["vis_start"]), dev_i32(pre["n_vis"]))
+    assert e.value.code == 3
 
 
 def test_compact_keep_all_identity_and_keep_none(tw):

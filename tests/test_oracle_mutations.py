@@ -30,6 +30,8 @@ MUTATIONS = [
     ("top-k: ties to the higher index", "key=lambda m: (-s[m], m)", "key=lambda m: (-s[m], -m)"),
     ("top-k: smallest instead of largest", "key=lambda m: (-s[m], m)", "key=lambda m: (s[m], m)"),
     ("prune: text after the image dropped", "+ list(range(vis_start + n_vis, prefix_len))", ""),
+    ("gather: rows assigned from the top down (breaks compaction in place)", "        for j in range(n):\n            dst_k[:, b, :, j, :]",
+     "        for j in reversed(range(n)):\n            dst_k[:, b, :, j, :]"),
     ("prune: kept indices not offset", "[vis_start + m for m in kept]", "[m for m in kept]"),
     ("attention: node does not see itself", "    while x >= 0:\n        out.append(x)", "    while x >= 0:\n        out.append(x) if x != i or x == 0 else None"),
     ("attention: mask shifted by one key", "vis[i, kv_len + a] = True", "vis[i, min(kv_len + a + 1, kv_len + n_nodes - 1)] = True"),
@@ -46,6 +48,12 @@ MUTATIONS = [
     ("append: rows written one position late", "cache_k[:, b, :, base + j, :]", "cache_k[:, b, :, base + j + 1, :]"),
     ("append: length not advanced by the root", "new_len[b] = base + len(paths[b])", "new_len[b] = base + len(paths[b]) - 1"),
     ("argmax: ties to the higher index", "if logits[b, i, v] > best_v:", "if logits[b, i, v] >= best_v:"),
+    ("chain draft: the token below the threshold is dropped", "        toks.append(tok)\n        probs.append(prob)\n        if len(toks) >= delta or prob < theta:\n            break",
+     "        if prob < theta and toks:\n            break\n        toks.append(tok)\n        probs.append(prob)\n        if len(toks) >= delta or prob < theta:\n            break"),
+    ("chain draft: a probability equal to the threshold exits", "if len(toks) >= delta or prob < theta:", "if len(toks) >= delta or prob <= theta:"),
+    ("chain draft: one token too many", "if len(toks) >= delta or prob < theta:", "if len(toks) > delta or prob < theta:"),
+    ("chain draft: ties to the higher token id", "            if x[v] > x[tok]:", "            if x[v] >= x[tok]:"),
+    ("chain draft: probability without the normaliser", "prob = float(e[tok] / e.sum())", "prob = float(e[tok])"),
     ("eq. 6: K_f ignored", "upper = L if K_f is None else K_f", "upper = L"),
 ]
 

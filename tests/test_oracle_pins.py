@@ -191,6 +191,30 @@ def test_gather_keep_all_is_identity_and_keep_none_is_text_only():
     assert n[0] == 4 and list(dk[0, 0, 0, :4, 0] % 1000) == [0, 1, 7, 8]
 
 
+def test_gather_in_place_equals_gather_into_a_copy():
+    """Compaction in place (dst is src) must give what the gather into a separate buffer gives,
+    whatever the kept list: every source row is still intact when its turn comes.  Lists whose
+    rows move by one position (kept = [0, 2, 3]) are the ones an unordered copy would get wrong."""
+    nl, B, H, L, d = 2, 1, 2, 14, 2
+    rng = np.random.default_rng(5)
+    lists = [[0, 2, 3], [1, 2, 3, 4, 5], [], [0, 1, 2], [5], list(range(6)), [0, 1, 4, 5]]
+    lists += [sorted(rng.choice(6, size=int(rng.integers(0, 7)), replace=False).tolist()) for _ in range(40)]
+    for kept in lists:
+        for vs in (0, 3):
+            k = _tagged_cache(nl, B, H, L, d)
+            v = -k
+            pos = (np.arange(L, dtype=np.int32) * 7 + 1)[None]
+            lp = [vs + 6 + 4]
+            dk, dv, po = k.copy(), v.copy(), pos.copy()           # rows past new_len: what was there
+            n_out = O.gather_compact(k, v, pos, lp, [vs], [6], [kept], dk, dv, po)
+            ik, iv, ip = k.copy(), v.copy(), pos.copy()
+            n_in = O.gather_compact(ik, iv, ip, lp, [vs], [6], [kept], ik, iv, ip)
+            assert list(n_in) == list(n_out) == [lp[0] - 6 + len(kept)]
+            assert np.array_equal(ik, dk) and np.array_equal(iv, dv) and np.array_equal(ip, po), kept
+            if len(kept) == 6:                                        # keep-all: nothing moves
+                assert np.array_equal(ik, k) and np.array_equal(ip, pos)
+
+
 def test_gather_rows_hidden_states_and_finalwipe():
     B, L, D = 2, 11, 5
     x = np.arange(B * L * D, dtype=np.int64).reshape(B, L, D)
@@ -633,6 +657,49 @@ def test_accept_compact_tail_rows_and_canaries():
         assert np.array_equal(ck[:, b, :, :base], before_k[:, b, :, :base])
         assert np.array_equal(ck[:, b, :, new_len[b]:], before_k[:, b, :, new_len[b]:])
         assert np.array_equal(cv[:, b, :, new_len[b]:], before_v[:, b, :, new_len[b]:])
+
+
+# ---------------------------------------------------------------- chain drafting with early exit
+def test_chain_draft_hand_case_and_limits():
+    """Appendix A: up to delta = 5 draft tokens, stop once the predicted token's probability is below
+    theta = 0.6; Algorithm 1 appends the token before it tests the probability, so the token that
+    triggers the exit is part of the draft."""
+    lg = lambda p: np.log(np.asarray(p, dtype=np.float64))
+    rows = [lg([0.1, 0.7, 0.2]), lg([0.8, 0.1, 0.1]), lg([0.3, 0.2, 0.5]), lg([0.9, 0.05, 0.05]), lg([0.9, 0.05, 0.05]),
+            lg([0.9, 0.05, 0.05])]
+    toks, probs = O.chain_draft(rows, 5, 0.6)
+    assert toks == [1, 0, 2] and np.allclose(probs, [0.7, 0.8, 0.5], atol=1e-12)      # 0.5 < 0.6: kept, then stop
+    toks, probs = O.chain_draft(rows, 5, 0.0)                                          # no early exit: delta tokens
+    assert toks == [1, 0, 2, 0, 0] and len(probs) == 5
+    toks, _ = O.chain_draft(rows, 2, 0.0)
+    assert toks == [1, 0]
+    toks, probs = O.chain_draft(rows, 5, 1.5)                                          # nothing is confident enough
+    assert toks == [1] and abs(probs[0] - 0.7) < 1e-12
+    # a probability equal to the threshold is not below it
+    toks, _ = O.chain_draft([lg([0.5, 0.5]), lg([0.25, 0.75]), lg([0.4, 0.6])], 5, 0.5)
+    assert toks == [0, 1, 1]                       # (and equal logits go to the lower token id)
+    # shifting a row's logits changes nothing
+    toks2, probs2 = O.chain_draft([r + 3.25 for r in rows], 5, 0.6)
+    assert toks2 == [1, 0, 2] and np.allclose(probs2, [0.7, 0.8, 0.5], atol=1e-12)
+
+
+def test_chain_draft_against_library_softmax():
+    from scipy.special import softmax
+    rng = np.random.default_rng(21)
+    for trial in range(50):
+        V, delta = int(rng.integers(2, 40)), int(rng.integers(1, 7))
+        theta = float(rng.uniform(0.05, 0.9))
+        rows = rng.standard_normal((8, V)) * rng.uniform(0.5, 4.0)
+        toks, probs = O.chain_draft(rows, delta, theta)
+        want_t, want_p = [], []
+        for r in rows:
+            p = softmax(r)
+            want_t.append(int(np.argmax(p)))
+            want_p.append(float(p.max()))
+            if len(want_t) >= delta or want_p[-1] < theta:
+                break
+        assert toks == want_t and np.allclose(probs, want_p, rtol=1e-12)
+        assert 1 <= len(toks) <= delta and all(p >= theta for p in probs[:-1])
 
 
 # ---------------------------------------------------------------- generator sanity
