@@ -169,15 +169,17 @@ class Replica:
                                   self.scores, self.kept, self.src, self.cache, self.ws, pos_in=self.pos_in,
                                   pos_out=self.pos_out, new_len=self.kv_len, dev_status=self.status)
 
-    def attention_layers(self, tw, s):
+    def attention_layers(self, tw, s, kv_len=None):
+        """The step's attention launches; kv_len: the lengths to read (default: the live ones)."""
         slot = s % POOL
         q, tk, tv = self.q[slot], self.tree_k[slot], self.tree_v[slot]
+        kv_len = self.kv_len if kv_len is None else kv_len
         for layer in range(self.wl.n_layers):
             # layer 0 follows the accept (or prune) kernel, which writes kv_len; the other layers follow
             # the previous layer's attention, which leaves lengths and cache alone
             flags = tw.attn_flags(kernel=self.attn_kernel, splits=self.attn_splits, plain_launch=self.plain_launch,
                                   early_prefix=layer > 0 and self.early_prefix)
-            tw.tree_verify_attention(q[layer], tk[layer], tv[layer], self.cache, layer, self.kv_len, self.n_nodes,
+            tw.tree_verify_attention(q[layer], tk[layer], tv[layer], self.cache, layer, kv_len, self.n_nodes,
                                      self.parent, self.out, dev_status=self.status, ws=self.attn_ws, flags=flags)
 
     def accept(self, tw, s):
@@ -300,7 +302,8 @@ def run_ours(args):
     verify_ms = sum(a.elapsed_time(b) for a, b in ev_pairs)          # attention x layers + accept, per verify step
     value = job_steps / (ms * 1e-3)
 
-    # ---- dominant kernel alone: the 32 attention launches of every verify step, timed live ------
+    # ---- dominant kernel alone ---------------------------------------------------------------------
+    # (a) launched one by one: the attention launches of every verify step between two events
     for rp in reps:
         rp.prune(tw)
     att_pairs = []
@@ -317,9 +320,41 @@ def run_ours(args):
     torch.cuda.synchronize()
     att_ms = sum(a.elapsed_time(b) for a, b in att_pairs)
     att_us_per_launch = att_ms * 1e3 / attn_launches
-    # inside the graph the same launches run back to back; per-launch time there:
-    graph_us_per_launch = verify_ms * 1e3 / (args.steps * total_verify * (wl.n_layers + 1))
-    use_us = min(att_us_per_launch, graph_us_per_launch) if graphs is not None else att_us_per_launch
+    # (b) inside graphs, as the timed loop runs them, but the attention launches ALONE: one graph per
+    # (replica, verify step) with the step's layers only, each reading that step's own lengths (a
+    # snapshot taken in the dry run), replayed in the timed loop's order so that no launch finds its
+    # cache in L2.  This is the figure the roofline uses when graphs are on.
+    graph_us_per_launch = None
+    if graphs is not None:
+        for rp in reps:
+            rp.len_at = [torch.from_numpy(np.ascontiguousarray(l, dtype=np.int32)).to(dev) for l in rp.lens]
+        att_graphs = [[None] * rp.n_steps for rp in reps]
+        with torch.cuda.stream(side):
+            for r, rp in enumerate(reps):
+                for s in range(rp.n_steps):
+                    g = torch.cuda.CUDAGraph()
+                    with torch.cuda.graph(g, stream=side):
+                        rp.attention_layers(tw, s, kv_len=rp.len_at[s])
+                    att_graphs[r][s] = g
+        torch.cuda.synchronize()
+
+        def attention_only():
+            for s in range(max_s):
+                for r, rp in enumerate(reps):
+                    if s < rp.n_steps:
+                        att_graphs[r][s].replay()
+        attention_only()
+        torch.cuda.synchronize()
+        n_att_rep = 3
+        a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a0.record(stream)
+        for _ in range(n_att_rep):
+            attention_only()
+        a1.record(stream)
+        torch.cuda.synchronize()
+        graph_us_per_launch = a0.elapsed_time(a1) * 1e3 / (n_att_rep * attn_launches)
+        del att_graphs
+    use_us = graph_us_per_launch if graph_us_per_launch is not None else att_us_per_launch
     bytes_per_launch = attn_bytes / attn_launches
     achieved = bytes_per_launch / (use_us * 1e-6) / 1e9
     roofline = {"kernel": "tree_attn_kernel", "bound": "hbm", "achieved": round(achieved, 1),
@@ -328,21 +363,50 @@ def run_ours(args):
                 "traffic_note": "dram read+write bytes of one launch at kv_len 227 (algorithmic 4571344 B there), "
                                 "from the ncu capture summarised in profiles/kernels_ncu_full.md",
                 "bytes_per_launch": int(bytes_per_launch), "us_per_launch": round(use_us, 3),
+                "us_per_launch_source": ("graphs of the attention launches alone, replayed in the timed loop's order"
+                                         if graph_us_per_launch is not None else "launched one by one between events"),
                 "us_per_launch_direct": round(att_us_per_launch, 3),
-                "us_per_launch_in_graph": round(graph_us_per_launch, 3),
+                "us_per_launch_in_graph": None if graph_us_per_launch is None else round(graph_us_per_launch, 3),
                 "note": "one launch = one layer of one verify step (3.5-5.6 MB): launch-latency sized"}
 
     # ---- prune latency (the third quantity of the metric) --------------------------------------
-    pr = []
-    for _ in range(3):
-        for rp in reps:
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record(stream)
-            rp.prune(tw)
-            e1.record(stream)
-            pr.append((e0, e1))
-    torch.cuda.synchronize()
-    prune_us = statistics.median(a.elapsed_time(b) for a, b in pr) * 1e3
+    # One ttp_score_topk_compact over all layers.  Launched directly the host's launch time shows in the
+    # figure (three launches of a few microseconds each), so the call is also captured in a graph per
+    # replica and replayed; both are reported, the replayed one is the device-side latency.
+    def time_prune(fn):
+        pr = []
+        for _ in range(5):
+            for i in range(len(reps)):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                fn(i)
+                e1.record(stream)
+                pr.append((e0, e1))
+        torch.cuda.synchronize()
+        return statistics.median(a.elapsed_time(b) for a, b in pr) * 1e3
+    prune_us_direct = time_prune(lambda i: reps[i].prune(tw))
+    prune_us = prune_us_direct
+    prune_us_plain = None
+    if graphs is not None:
+        def prune_graphs():
+            gs = []
+            with torch.cuda.stream(side):
+                for rp in reps:
+                    g = torch.cuda.CUDAGraph()
+                    with torch.cuda.graph(g, stream=side):
+                        rp.prune(tw)
+                    gs.append(g)
+            torch.cuda.synchronize()
+            return gs
+        pg = prune_graphs()
+        prune_us = time_prune(lambda i: pg[i].replay())
+        # the same with plain launches (no programmatic stream serialization): what the overlap of the
+        # gather's text rows with scoring and selection is worth
+        prev = tw.twig_set_launch_overlap(0)
+        pg = prune_graphs()
+        prune_us_plain = time_prune(lambda i: pg[i].replay())
+        tw.twig_set_launch_overlap(prev)
+        del pg
     prune_bytes = 2 * max(wl.pruned_len) * wl.kv_row_bytes() * wl.n_layers + \
         wl.n_kv_heads * max(wl.prefix_len) * wl.head_dim * 2
 
@@ -353,22 +417,23 @@ def run_ours(args):
         "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": round(ms / args.steps, 4), "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": wl.name, "requests_per_step": N_ROT, "layers": wl.n_layers, "heads": wl.n_q_heads,
-                   "head_dim": wl.head_dim, "tree_nodes": wl.t_max, "prefix": wl.prefix_len[0], "keep": wl.keep[0],
-                   "tokens_per_request": wl.gen_target[0], "verify_steps_per_bench_step": total_verify,
-                   "tokens_emitted_per_bench_step": sum(rp.emitted for rp in reps),
-                   "launch_mode": "direct" if graphs is None else "cuda-graph per verify step, one launch per layer",
-                   "l2": f"inputs larger than L2: {N_ROT} request replicas round-robin, >= {3 * 113} MB touched "
-                         "between two uses of a buffer"},
+        "config": bench_config(wl, {
+            "verify_steps_per_bench_step": total_verify,
+            "tokens_emitted_per_bench_step": sum(rp.emitted for rp in reps),
+            "launch_mode": "direct" if graphs is None else "cuda-graph per verify step, one launch per layer",
+            "l2": f"inputs larger than L2: {N_ROT} request replicas round-robin, >= {3 * 113} MB touched "
+                  "between two uses of a buffer"}),
         "clocks": clocks, "gpu_launches": args.steps * (3 * N_ROT + total_verify * (wl.n_layers + 1)),
         "e2e": e2e, "roofline": roofline,
         "verify_us_per_step": round(verify_ms * 1e3 / (args.steps * total_verify), 2),
         "ttp_prune_latency_us": round(prune_us, 2),
+        "ttp_prune_latency_us_direct_launches": round(prune_us_direct, 2),
+        "ttp_prune_latency_us_without_launch_overlap": None if prune_us_plain is None else round(prune_us_plain, 2),
         "ttp_prune_gbs": round(prune_bytes / (prune_us * 1e-6) / 1e9, 1),
         "tokens_per_s": round(sum(rp.emitted for rp in reps) * args.steps * world / (ms * 1e-3), 1),
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        out["cpu_baseline"] = cpu_baseline(wl, reps[0], budget_s=args.cpu_budget)
+        out["cpu_baseline"] = cpu_baseline(wl)
     if rank == 0 and world == 1 and args.extra:
         out["other_kernels"] = extra_rooflines(torch, tw, peaks, dev)
     if rank == 0:
@@ -437,19 +502,17 @@ def run_e2e(torch, tw, wl, reps, stream, world, dev, dist, step_graphs):
         dist.barrier()
     n_req = 3
     t0 = time.perf_counter()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
     for _ in range(n_req):
         request()
-    e1.record(stream)
     torch.cuda.synchronize()
-    ms = max(e0.elapsed_time(e1), (time.perf_counter() - t0) * 1e3 * 0.0)
+    ms = (time.perf_counter() - t0) * 1e3            # wall clock: the host waits for every step's result
     if dist is not None:
         tt = torch.tensor([ms], device=dev)
         dist.all_reduce(tt, op=dist.ReduceOp.MAX)
         ms = float(tt.item())
     return {"value": round(rp.n_steps * n_req * world / (ms * 1e-3), 1), "unit": UNIT,
             "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+            "timer": "host wall clock (time.perf_counter) around the requests",
             "note": "per bench step = one request; Q and tree K/V of all layers cross PCIe every verify step; "
                     + ("kernels replayed from the step's graph" if step_graphs else "kernels launched one by one")}
 
@@ -539,6 +602,19 @@ def extra_rooflines(torch, tw, peaks, dev):
         e["frac_early_prefix"] = round(num / t2["us"] / (peaks["bf16_tflops"] if bound == "tensor" else peaks["hbm_gbs"]), 4)
         return e
 
+    # c2's third launch mode: ONE launch for all 32 layers of a verify step, the layers standing in as
+    # 32 requests of a batch (same shapes, same bytes: 32 x 4.6 MB).  Benchmark only: in a model layer l+1
+    # needs layer l's output, so the layers cannot share a launch.
+    wl2 = synth.workload(2)
+    nl2 = wl2.n_layers
+    wl2x = synth.Workload(2, "c2-all-layers-as-batch", 1, nl2, wl2.n_q_heads, wl2.n_kv_heads, wl2.head_dim,
+                          wl2.text_before * nl2, wl2.n_vis * nl2, wl2.text_after * nl2, wl2.keep * nl2,
+                          wl2.n_nodes * nl2, wl2.depth_levels * nl2, wl2.match_p, branching=wl2.branching)
+    e = attn_entry(_time_attention(torch, tw, wl2x, [227] * nl2, 0, 505, dev))
+    e["note"] = "benchmark-only: the 32 layers of one verify step as one launch (real layers depend on each other)"
+    e["us_per_layer"] = round(e["us_per_launch"] / nl2, 3)
+    res["tree_attn_c2_all_layers_one_launch"] = e
+
     wl3 = synth.workload(3)
     lens3 = [p + g // 2 for p, g in zip(wl3.pruned_len, wl3.gen_target)]      # half-way through generation
     res["tree_attn_c3_midway"] = attn_both(wl3, lens3, 501)
@@ -579,6 +655,28 @@ def extra_rooflines(torch, tw, peaks, dev):
     torch.cuda.synchronize()
     us = e0.elapsed_time(e1) * 1e3 / n_chain
     by = 2 * sum(wl.pruned_len) * wl.kv_row_bytes() * nl
+    # the same compaction in place (dst = src): only rows after the first dropped token move; the
+    # prompt caches are restored by a copy before each timed launch (outside the events)
+    us_ip = []
+    for i in range(6):
+        srcs = sets[i % n_sets][0]
+        backup_k, backup_v = srcs._keep[0].clone(), srcs._keep[1].clone()
+        a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a0.record(stream)
+        tw.ttp_compact(srcs, srcs, *meta)
+        a1.record(stream)
+        torch.cuda.synchronize()
+        us_ip.append(a0.elapsed_time(a1) * 1e3)
+        srcs._keep[0].copy_(backup_k)
+        srcs._keep[1].copy_(backup_v)
+        del backup_k, backup_v
+    moved = 2 * sum(int((np.arange(wl.pruned_len[b]) != np.concatenate([np.arange(wl.text_before[b]), wl.text_before[b] + kept[b],
+                    np.arange(wl.text_before[b] + wl.n_vis[b], wl.prefix_len[b])])).sum()) for b in range(B)) * wl.kv_row_bytes() * nl
+    us_med = statistics.median(us_ip[1:])
+    res["kv_gather_in_place_c4_2layers"] = {"bound": "hbm", "bytes_per_launch": int(moved), "us_per_launch": round(us_med, 2),
+                                            "achieved": round(moved / us_med / 1e3, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                            "frac": round(moved / us_med / 1e3 / peaks["hbm_gbs"], 4),
+                                            "note": "single launches on a cold cache; bytes = rows that move (read + write)"}
     res["kv_gather_c4_2layers"] = {"bound": "hbm", "bytes_per_launch": by, "us_per_launch": round(us, 2),
                                    "achieved": round(by / us / 1e3, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
                                    "frac": round(by / us / 1e3 / peaks["hbm_gbs"], 4),
@@ -825,9 +923,10 @@ def oracle_verify_steps(wl, host, n_steps, n_layers):
     t0 = time.perf_counter()
     for st in range(n_steps):
         ver = vers[st % len(vers)]
+        rows = int(max(kv_len))                      # only the rows in use are widened to fp64
         for layer in range(n_layers):
             O.tree_attention(f64(ver["q"][layer]), f64(ver["tree_k"][layer]), f64(ver["tree_v"][layer]),
-                             f64(ck[layer]), f64(cv[layer]), kv_len, ver["n_nodes"], ver["parent"])
+                             f64(ck[layer][:, :, :rows]), f64(cv[layer][:, :, :rows]), kv_len, ver["n_nodes"], ver["parent"])
         paths = []
         for b in range(B):
             _, p, _ = O.tree_accept(ver["parent"][b], draft[st][b], tgt[st][b], wl.n_nodes[b])
@@ -852,18 +951,29 @@ def oracle_host_inputs(wl, n_pool=2, n_tok=16, stream_id=100):
     return {"pre": pre, "vers": vers, "draft": draft, "tgt": tgt}
 
 
-def cpu_baseline(wl, rep0, budget_s=20.0):
-    """The oracle as it stands, single-threaded, on a bounded sample: the first verify steps of
-    one request (every layer each)."""
+ORACLE_SAMPLE_STEPS = 8      # verify steps of one request per timed oracle sample (both CPU legs)
+
+
+def oracle_sample(wl, host):
+    """One timed sample of the oracle, single-threaded: the first ORACLE_SAMPLE_STEPS verify steps of one
+    request, every layer each.  Returns (verify steps per second, seconds, seconds of the oracle prune)."""
     from threadpoolctl import threadpool_limits
-    host = oracle_host_inputs(wl)
     with threadpool_limits(limits=1):
-        t1, _ = oracle_verify_steps(wl, host, 1, wl.n_layers)
-        n = int(max(1, min(16, budget_s / max(t1, 1e-3))))
-        tn, t_prune = oracle_verify_steps(wl, host, n, wl.n_layers)
-    return {"value": round(n / tn, 3), "unit": UNIT, "cores": 1, "kind": "oracle",
-            "sample": f"first {n} verify steps of one request, all {wl.n_layers} layers each (numpy fp64, 1 thread); "
-                      f"oracle prune of the same request took {t_prune:.2f} s",
+        t, t_prune = oracle_verify_steps(wl, host, ORACLE_SAMPLE_STEPS, wl.n_layers)
+    return ORACLE_SAMPLE_STEPS / t, t, t_prune
+
+
+def oracle_sample_text(wl):
+    return (f"first {ORACLE_SAMPLE_STEPS} verify steps of one request, all {wl.n_layers} layers each "
+            "(numpy fp64, 1 thread)")
+
+
+def cpu_baseline(wl):
+    """The oracle as it stands on one host core, one bounded sample (the same sample the reference arm times)."""
+    host = oracle_host_inputs(wl)
+    value, t, t_prune = oracle_sample(wl, host)
+    return {"value": round(value, 3), "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": oracle_sample_text(wl) + f", {t:.1f} s; oracle prune of the same request took {t_prune:.2f} s",
             "host_cores_available": os.cpu_count()}
 
 
@@ -871,27 +981,34 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    from threadpoolctl import threadpool_limits
     wl = synth.workload(args.workload)
     host = oracle_host_inputs(wl)
-    per = 2          # verify steps per timed step (bounded sample)
-    with threadpool_limits(limits=1):
-        for _ in range(min(args.warmup, 1)):
-            oracle_verify_steps(wl, host, 1, wl.n_layers)
-        tot = 0.0
-        k = max(1, min(args.steps, 5))
-        for _ in range(k):
-            t, _ = oracle_verify_steps(wl, host, per, wl.n_layers)
-            tot += t
-    value = per * k / tot
-    sample = f"{per} verify steps (all {wl.n_layers} layers) per step, {k} steps, numpy fp64, 1 thread"
+    for _ in range(min(args.warmup, 1)):
+        oracle_verify_steps(wl, host, 1, wl.n_layers)
+    k = max(1, min(args.steps, 5))          # each step is one bounded sample; the whole run stays within minutes
+    tot = 0.0
+    for _ in range(k):
+        _, t, _ = oracle_sample(wl, host)
+        tot += t
+    value = ORACLE_SAMPLE_STEPS * k / tot
+    sample = oracle_sample_text(wl) + f" per step, {k} steps"
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": round(value, 3), "unit": UNIT,
         "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": k, "warmup": min(args.warmup, 1),
         "ms_per_step": round(tot / k * 1e3, 2), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f64", "data": "synthetic", "config": {"workload": wl.name},
+        "dtype": "f64", "data": "synthetic", "config": bench_config(wl, None),
         "cpu_baseline": {"value": round(value, 3), "unit": UNIT, "kind": "oracle", "cores": 1, "sample": sample},
         "e2e": {"value": round(value, 3), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+
+
+def bench_config(wl, extra):
+    """The `config` object both arms print: the workload and its shape."""
+    cfg = {"workload": wl.name, "requests_per_step": N_ROT, "layers": wl.n_layers, "heads": wl.n_q_heads,
+           "head_dim": wl.head_dim, "tree_nodes": wl.t_max, "prefix": wl.prefix_len[0], "keep": wl.keep[0],
+           "tokens_per_request": wl.gen_target[0]}
+    if extra:
+        cfg.update(extra)
+    return cfg
 
 
 def main():
@@ -905,7 +1022,6 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extra", dest="extra", action="store_false",
                     help="skip the HBM-sized launches of the attention and gather kernels")
-    ap.add_argument("--cpu-budget", type=float, default=15.0)
     ap.add_argument("--no-early-prefix", action="store_true", help="do not prefetch the KV prefix under the previous layer")
     ap.add_argument("--no-overlap", action="store_true", help="plain launches (no programmatic stream serialization)")
     ap.add_argument("--attn-splits", type=int, default=0, help="force key splits per cluster (0 auto)")
@@ -923,6 +1039,18 @@ def main():
     if args.case:
         run_case(args)
         return
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # not under a launcher: start one rank per GPU ourselves (replicas only, no data-path collective)
+        import socket
+        with socket.socket() as sk:
+            sk.bind(("127.0.0.1", 0))
+            port = sk.getsockname()[1]
+        cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+               "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+        sys.exit(subprocess.call(cmd))
+    world_env = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.gpus != world_env and "WORLD_SIZE" in os.environ:
+        sys.stderr.write(f"bench.py: --gpus {args.gpus} but the launcher started {world_env} ranks; reporting {world_env}\n")
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
         run_reference(args)

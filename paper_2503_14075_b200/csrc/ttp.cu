@@ -43,6 +43,7 @@ ttp_logits_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__re
   constexpr int PASSES = kScoreKeysPerCta / KPP;
   __shared__ float qs[kMaxGroup * D];
 
+  grid_dependency_sync();
   const int b = blockIdx.z, hk = blockIdx.y;
   const int lp = prefix_len[b], vs = vis_start[b], nv = n_vis[b];
   if (!layout_ok(lp, vs, nv, k_max_len, m_max)) {
@@ -159,6 +160,10 @@ ttp_finalize_topk_kernel(const float *__restrict__ logits, int lstride, int n_q_
   __shared__ uint32_t warp_sums[33];
   __shared__ uint32_t sel_digit, sel_remaining;
 
+  // the kernel after this one (the gather of the fused call) may start on what does not depend on the
+  // selection; this kernel itself reads its predecessor's output from here on
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int nv = n_vis[b];
   float *sc = scores + (long long)b * m_max;
@@ -214,6 +219,27 @@ ttp_finalize_topk_kernel(const float *__restrict__ logits, int lstride, int n_q_
   for (int i = R + tid; i < r_max; i += kTopkThreads) out[i] = -1;
   if (R == 0) return;
   __syncthreads();
+
+  if (nv <= kTopkThreads) {
+    // Few visual tokens (one per thread): exact selection by counting.  A token is kept iff fewer
+    // than R tokens come before it in the order (larger score first, lower index first among
+    // equals); an ordered scan of the kept flags gives the ascending output positions.
+    const int m = tid;
+    uint32_t sel = 0;
+    if (m < nv) {
+      const uint32_t mine = keys[m];
+      int before = 0;
+      for (int o = 0; o < nv; ++o) {
+        const uint32_t other = keys[o];                       // (all threads read the same word: a broadcast)
+        before += (other > mine || (other == mine && o < m)) ? 1 : 0;
+      }
+      sel = before < R ? 1u : 0u;
+    }
+    uint32_t total;
+    const uint32_t at = block_exclusive_scan(sel, warp_sums, total);
+    if (sel) out[at] = m;
+    return;
+  }
 
   // radix select, 8 bits per pass from the top: the R-th largest key
   uint32_t prefix = 0, mask = 0;
@@ -288,30 +314,35 @@ kv_gather_kernel(KvView src, KvViewMut dst, const int *__restrict__ kept_idx, in
                  const int *__restrict__ keep, const int *__restrict__ prefix_len,
                  const int *__restrict__ vis_start, const int *__restrict__ n_vis,
                  const int *__restrict__ pos_in, int *__restrict__ pos_out, int pos_stride,
-                 int *__restrict__ new_len, int *dev_status) {
+                 int *__restrict__ new_len, int *dev_status, int early_text) {
   constexpr int LPR = D / 8;                   // lanes per row
   constexpr int RPP = kGatherThreads / LPR;    // rows per pass
   constexpr int PASSES = kGatherRows / RPP;
+  // early_text (the fused call): the kernels before this one in the stream are the call's own scoring
+  // and selection, which write nothing this kernel reads except kept_idx.  The text rows (they do not
+  // depend on the selection) are copied while those kernels are still running; the kept visual rows
+  // follow once the selection has completed.
+  if (!early_text) grid_dependency_sync();
   const int b = blockIdx.z;
   const int layer = blockIdx.y / src.n_kv_heads, h = blockIdx.y % src.n_kv_heads;
   const int lp = prefix_len[b], vs = vis_start[b], nv = n_vis[b], kp = keep[b];
   const bool first = blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0;
-  if (!layout_ok(lp, vs, nv, src.max_len, TWIG_MAX_VISUAL)) {
-    if (first) flag_status(dev_status, b, TWIG_DEV_BAD_LAYOUT);
-    return;
-  }
-  if (kp < 0 || kp > nv || kp > r_max) {
-    if (first) flag_status(dev_status, b, TWIG_DEV_BAD_KEEP);
-    return;
-  }
   const int nl = lp - nv + kp;
-  if (nl > dst.max_len) {
-    if (first) flag_status(dev_status, b, TWIG_DEV_OVERFLOW);
-    return;
-  }
-  if (first && new_len) new_len[b] = nl;
   const int j0 = blockIdx.x * kGatherRows;
-  if (j0 >= nl) return;
+  {
+    int code = 0;
+    if (!layout_ok(lp, vs, nv, src.max_len, TWIG_MAX_VISUAL)) code = TWIG_DEV_BAD_LAYOUT;
+    else if (kp < 0 || kp > nv || kp > r_max) code = TWIG_DEV_BAD_KEEP;
+    else if (nl > dst.max_len) code = TWIG_DEV_OVERFLOW;
+    if (code == 0 && first && new_len) new_len[b] = nl;
+    if (code != 0 || j0 >= nl) {
+      // (a CTA with nothing to do still waits for the preceding kernel before it leaves, so that this
+      // kernel's completion implies that one's)
+      if (early_text) grid_dependency_sync();
+      if (code != 0 && first) flag_status(dev_status, b, code);
+      return;
+    }
+  }
 
   const int sub = threadIdx.x % LPR, slot = threadIdx.x / LPR;
   const long long sbase = layer * src.stride_layer + b * src.stride_batch + h * src.stride_head + sub * 8;
@@ -320,39 +351,42 @@ kv_gather_kernel(KvView src, KvViewMut dst, const int *__restrict__ kept_idx, in
 
   int srow[PASSES];
   uint4 kr[PASSES], vr[PASSES];
+  // phase 0: rows that need no kept_idx (text before and after the image); phase 1: kept visual rows
+  for (int phase = 0; phase < 2; ++phase) {
+    if (phase == 1 && early_text) grid_dependency_sync();
 #pragma unroll
-  for (int p = 0; p < PASSES; ++p) {
-    const int j = j0 + p * RPP + slot;
-    int s = -1;
-    if (j < nl) {
-      if (j < vs) {
-        s = j;
-      } else if (j < vs + kp) {
-        const int kk = kidx[j - vs];
-        const int prev = (j > vs) ? kidx[j - vs - 1] : -1;
-        if (kk < 0 || kk >= nv || kk <= prev) {
-          if (sub == 0 && blockIdx.y == 0) flag_status(dev_status, b, TWIG_DEV_BAD_INDEX);
-        } else {
-          s = vs + kk;
+    for (int p = 0; p < PASSES; ++p) {
+      const int j = j0 + p * RPP + slot;
+      int s = -1;
+      if (j < nl) {
+        const bool visual = j >= vs && j < vs + kp;
+        if (phase == 0 && !visual) {
+          s = j < vs ? j : j - kp + nv;
+        } else if (phase == 1 && visual) {
+          const int kk = kidx[j - vs];
+          const int prev = (j > vs) ? kidx[j - vs - 1] : -1;
+          if (kk < 0 || kk >= nv || kk <= prev) {
+            if (sub == 0 && blockIdx.y == 0) flag_status(dev_status, b, TWIG_DEV_BAD_INDEX);
+          } else {
+            s = vs + kk;
+          }
         }
-      } else {
-        s = j - kp + nv;
+      }
+      srow[p] = s;
+      if (s >= 0) {
+        kr[p] = ld_nc_16(src.k + sbase + (long long)s * src.stride_pos);
+        vr[p] = ld_nc_16(src.v + sbase + (long long)s * src.stride_pos);
       }
     }
-    srow[p] = s;
-    if (s >= 0) {
-      kr[p] = ld_nc_16(src.k + sbase + (long long)s * src.stride_pos);
-      vr[p] = ld_nc_16(src.v + sbase + (long long)s * src.stride_pos);
-    }
-  }
 #pragma unroll
-  for (int p = 0; p < PASSES; ++p) {
-    const int j = j0 + p * RPP + slot;
-    if (srow[p] >= 0) {
-      st_16(dst.k + dbase + (long long)j * dst.stride_pos, kr[p]);
-      st_16(dst.v + dbase + (long long)j * dst.stride_pos, vr[p]);
-      if (blockIdx.y == 0 && sub == 0 && pos_in && pos_out)
-        pos_out[(long long)b * pos_stride + j] = pos_in[(long long)b * pos_stride + srow[p]];
+    for (int p = 0; p < PASSES; ++p) {
+      const int j = j0 + p * RPP + slot;
+      if (srow[p] >= 0) {
+        st_16(dst.k + dbase + (long long)j * dst.stride_pos, kr[p]);
+        st_16(dst.v + dbase + (long long)j * dst.stride_pos, vr[p]);
+        if (blockIdx.y == 0 && sub == 0 && pos_in && pos_out)
+          pos_out[(long long)b * pos_stride + j] = pos_in[(long long)b * pos_stride + srow[p]];
+      }
     }
   }
 }
@@ -565,6 +599,23 @@ static twig_status check_score_args(const ScoreArgs &a, const void *ws, size_t w
   return TWIG_OK;
 }
 
+// Launch configuration with programmatic stream serialization: the kernel may be scheduled while its
+// predecessor in the stream drains; it waits on the device before it reads that kernel's output.
+struct PdlLaunch {
+  cudaLaunchConfig_t cfg = {};
+  cudaLaunchAttribute attr[1];
+  PdlLaunch(dim3 grid, dim3 block, size_t smem, cudaStream_t st) {
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = launch_overlap_enabled() ? 1 : 0;
+  }
+};
+
 static twig_status launch_logits(const ScoreArgs &a, int *dev_status, void *ws, cudaStream_t st) {
   const float scale = a.softmax_scale != 0.f ? a.softmax_scale : 1.f / sqrtf((float)a.head_dim);
   dim3 grid((a.k_max_len + kScoreKeysPerCta - 1) / kScoreKeysPerCta, a.n_kv_heads, a.batch);
@@ -574,17 +625,20 @@ static twig_status launch_logits(const ScoreArgs &a, int *dev_status, void *ws, 
   auto k = static_cast<const __nv_bfloat16 *>(a.twig_k);
   auto qg = static_cast<const __nv_bfloat16 *>(a.q_gate);
   auto kg = static_cast<const __nv_bfloat16 *>(a.k_gate);
-#define TWIG_LOGITS(D_, G_)                                                                              \
-  ttp_logits_kernel<D_, G_><<<grid, kScoreThreads, 0, st>>>(q, k, qg, kg, a.ksb, a.ksh, a.ksp, a.k_max_len, \
-      a.prefix_len, a.vis_start, a.n_vis, a.n_q_heads, group, a.norm_scope, scale,                       \
-      static_cast<float *>(ws), ls, a.m_max, dev_status)
+  PdlLaunch L(grid, dim3(kScoreThreads), 0, st);
+  const long long ksb = a.ksb, ksh = a.ksh, ksp = a.ksp;
+  float *lg = static_cast<float *>(ws);
+  cudaError_t err;
+#define TWIG_LOGITS(D_, G_)                                                                                          \
+  err = cudaLaunchKernelEx(&L.cfg, ttp_logits_kernel<D_, G_>, q, k, qg, kg, ksb, ksh, ksp, a.k_max_len, a.prefix_len, \
+                           a.vis_start, a.n_vis, a.n_q_heads, group, a.norm_scope, scale, lg, ls, a.m_max, dev_status)
   if (a.head_dim == 128) {
     if (qg) TWIG_LOGITS(128, true); else TWIG_LOGITS(128, false);
   } else {
     if (qg) TWIG_LOGITS(64, true); else TWIG_LOGITS(64, false);
   }
 #undef TWIG_LOGITS
-  return launch_status();
+  return err == cudaSuccess ? TWIG_OK : TWIG_ERR_CUDA;
 }
 
 static twig_status launch_finalize(const float *logits, const ScoreArgs &a, const int *keep,
@@ -598,10 +652,12 @@ static twig_status launch_finalize(const float *logits, const ScoreArgs &a, cons
       return TWIG_ERR_CUDA;
     attr_set = true;
   }
-  ttp_finalize_topk_kernel<<<a.batch, kTopkThreads, smem, st>>>(
-      logits, logits_stride(a.k_max_len), a.n_q_heads, a.k_max_len, a.prefix_len, a.vis_start,
-      a.n_vis, keep, a.norm_scope, a.scores, a.m_max, kept_idx, r_max, dev_status, mode);
-  return launch_status();
+  PdlLaunch L(dim3(a.batch), dim3(kTopkThreads), smem, st);
+  const int ls = logits_stride(a.k_max_len);
+  const cudaError_t err = cudaLaunchKernelEx(&L.cfg, ttp_finalize_topk_kernel, logits, ls, a.n_q_heads, a.k_max_len,
+                                             a.prefix_len, a.vis_start, a.n_vis, keep, a.norm_scope, a.scores, a.m_max,
+                                             kept_idx, r_max, dev_status, mode);
+  return err == cudaSuccess ? TWIG_OK : TWIG_ERR_CUDA;
 }
 
 // bytes from the base pointer to the end of the last row of a K (or V) tensor
@@ -652,7 +708,7 @@ static twig_status check_compact_args(const twig_kv *src, const twig_kv *dst, co
 static twig_status launch_gather(const twig_kv *src, const twig_kv *dst, const int *kept_idx, int r_max,
                                  const int *keep, const int *prefix_len, const int *vis_start,
                                  const int *n_vis, const int *pos_in, int *pos_out, int pos_stride,
-                                 int *new_len, int *dev_status, cudaStream_t st) {
+                                 int *new_len, int *dev_status, cudaStream_t st, int early_text = 0) {
   if (same_kv(src, dst)) {
     // in place: one CTA per (layer, kv head, K or V, request); position ids move in place as well
     // (pos_out may be pos_in, or a separate array that then receives the gathered ids)
@@ -672,13 +728,17 @@ static twig_status launch_gather(const twig_kv *src, const twig_kv *dst, const i
   }
   const int rows_bound = src->max_len < dst->max_len ? src->max_len : dst->max_len;
   dim3 grid((rows_bound + kGatherRows - 1) / kGatherRows, src->n_layers * src->n_kv_heads, src->batch);
-  if (src->head_dim == 128)
-    kv_gather_kernel<128><<<grid, kGatherThreads, 0, st>>>(view_of(src), view_of_mut(dst), kept_idx, r_max,
-        keep, prefix_len, vis_start, n_vis, pos_in, pos_out, pos_stride, new_len, dev_status);
-  else
-    kv_gather_kernel<64><<<grid, kGatherThreads, 0, st>>>(view_of(src), view_of_mut(dst), kept_idx, r_max,
-        keep, prefix_len, vis_start, n_vis, pos_in, pos_out, pos_stride, new_len, dev_status);
-  return launch_status();
+  PdlLaunch L(grid, dim3(kGatherThreads), 0, st);
+  const KvView sv = view_of(src);
+  const KvViewMut dv = view_of_mut(dst);
+  if (!launch_overlap_enabled()) early_text = 0;
+  const cudaError_t err =
+      src->head_dim == 128
+          ? cudaLaunchKernelEx(&L.cfg, kv_gather_kernel<128>, sv, dv, kept_idx, r_max, keep, prefix_len, vis_start, n_vis,
+                               pos_in, pos_out, pos_stride, new_len, dev_status, early_text)
+          : cudaLaunchKernelEx(&L.cfg, kv_gather_kernel<64>, sv, dv, kept_idx, r_max, keep, prefix_len, vis_start, n_vis,
+                               pos_in, pos_out, pos_stride, new_len, dev_status, early_text);
+  return err == cudaSuccess ? TWIG_OK : TWIG_ERR_CUDA;
 }
 
 }  // namespace twig
@@ -822,8 +882,10 @@ extern "C" twig_status ttp_score_topk_compact(
   if (s != TWIG_OK) return s;
   s = launch_finalize(static_cast<const float *>(ws), a, keep, kept_idx, r_max, dev_status, 3, st);
   if (s != TWIG_OK) return s;
+  // The gather's predecessors in the stream are this call's own kernels: it may copy the rows that do
+  // not depend on the selection while they run.  (Not in place: there every row move needs the list.)
   return launch_gather(src, dst, kept_idx, r_max, keep, prefix_len, vis_start, n_vis, pos_in, pos_out,
-                       pos_stride, new_len, dev_status, st);
+                       pos_stride, new_len, dev_status, st, same_kv(src, dst) ? 0 : 1);
 }
 
 extern "C" twig_status ttp_compact_rows(const void *src, void *dst, int64_t row_bytes, int64_t src_stride_row,
