@@ -264,6 +264,12 @@ twig_status tree_verify_attention(const void *q, const void *tree_k, const void 
  *   tree_accept_compact or ttp_compact, which write kv_len).  The kernel then reads the lengths and
  *   starts fetching the cached prefix while the preceding kernel is still draining; q, tree_k and
  *   tree_v are still read only after it has completed.  Results do not change when the promise holds.
+ * TWIG_ATTN_EARLY_QUERY (with TWIG_ATTN_EARLY_PREFIX): the second promise, that the preceding kernel does
+ *   not write q, tree_k or tree_v either.  The small-call kernel then waits for nothing before it
+ *   computes and only orders its stores after the preceding kernel, so consecutive calls overlap
+ *   almost entirely.  In a model the layers of a verification step cannot make this promise (a
+ *   layer's q is computed from the previous layer's output): it exists to measure what the launch
+ *   chain costs, and for callers whose q is staged ahead of time.
  * TWIG_ATTN_PLAIN_LAUNCH: launch without programmatic stream serialization (see twig_set_launch_overlap).
  * TWIG_ATTN_KERNEL(k): run exactly kernel k, a testing and tuning control (all kernels compute the
  *   same function).  TWIG_ATTN_KERNEL_AUTO picks by shape; _MMA is the mma.sync kernel (any shape);
@@ -295,6 +301,7 @@ twig_status tree_verify_attention(const void *q, const void *tree_k, const void 
 #define TWIG_ATTN_KERNEL_STREAM 3u
 #define TWIG_ATTN_KERNEL(k) ((uint32_t)(k) << 1)
 #define TWIG_ATTN_PLAIN_LAUNCH (1u << 4)
+#define TWIG_ATTN_EARLY_QUERY (1u << 5)
 #define TWIG_ATTN_SPLITS(n) ((uint32_t)(n) << 8)
 #define TWIG_ATTN_STREAM_SHARES (1u << 12)
 #define TWIG_ATTN_STREAM_WHOLE (2u << 12)

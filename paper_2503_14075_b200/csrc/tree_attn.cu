@@ -104,7 +104,7 @@ tree_attn_kernel(const AttnParams p) {
   const bool first = split == 0 && blockIdx.y == 0 && tid == 0;
   const int rows_total = n * p.group, row0 = rb * ROWS;
   if (n <= 0 || n > p.t_max || L < 0 || L > p.max_len || row0 >= rows_total) {
-    if (p.early_prefix) grid_dependency_sync();
+    if (p.early_prefix) grid_dependency_sync();       // (also with early_query: nothing was launched early yet)
     if (first && (n < 0 || n > p.t_max)) flag_status(p.dev_status, b, TWIG_DEV_BAD_TREE);
     else if (first && n > 0 && (L < 0 || L > p.max_len)) flag_status(p.dev_status, b, TWIG_DEV_OVERFLOW);
     return;
@@ -241,7 +241,10 @@ tree_attn_kernel(const AttnParams p) {
   }
 
   if (p.early_prefix) {     // now wait for the preceding kernel; then Q and the tiles that hold tree rows
-    grid_dependency_sync();
+    // (with the second promise, that Q and the tree's rows are final as well, nothing is waited for
+    // here: the wait moves down to just before this kernel's first store)
+    if (!p.early_query) grid_dependency_sync();
+    else asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     load_q();
 #pragma unroll
     for (int s = 0; s < PRE; ++s)
@@ -528,6 +531,7 @@ tree_attn_kernel(const AttnParams p) {
     __syncthreads();
   }
 
+  if (p.early_query) asm volatile("griddepcontrol.wait;" ::: "memory");     // stores are ordered after the predecessor
   {
     constexpr int TPR = D / 4;                        // threads per row, 4 floats each
     constexpr int RPP = C::THREADS / TPR;             // rows per pass
@@ -687,6 +691,7 @@ extern "C" twig_status tree_verify_attention_ex(const void *q, const void *tree_
   p.row_blocks = 1;
   p.overlap = (launch_overlap_enabled() && !(flags & TWIG_ATTN_PLAIN_LAUNCH)) ? 1 : 0;
   p.early_prefix = ((flags & TWIG_ATTN_EARLY_PREFIX) && p.overlap) ? 1 : 0;
+  p.early_query = (p.early_prefix && (flags & TWIG_ATTN_EARLY_QUERY)) ? 1 : 0;
   p.forced_splits = splits;
   p.stream_policy = (int)((flags >> 12) & 3u);
   if (p.stream_policy == 3) return TWIG_ERR_UNSUPPORTED;

@@ -22,6 +22,7 @@ struct AttnParams {
   long long c_sl;
   int layer, n_layers, batch;
   int early_prefix;   // TWIG_ATTN_EARLY_PREFIX of the call
+  int early_query;    // TWIG_ATTN_EARLY_QUERY as well (mma.sync kernel)
   float scale_log2;   // softmax_scale * log2(e)
   // host side only: launch with programmatic stream serialization, forced key splits (0: automatic),
   // the caller's scratch (persistent kernel)

@@ -54,14 +54,7 @@ ttp_logits_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__re
   const int j0 = blockIdx.x * kScoreKeysPerCta;
   if (j0 >= hi || j0 + kScoreKeysPerCta <= lo) return;
 
-  for (int i = threadIdx.x; i < group * D; i += kScoreThreads) {
-    const long long at = ((long long)b * n_q_heads + hk * group) * D + i;
-    float v = __bfloat162float(q[at]) * scale;
-    if (GATED) v *= __bfloat162float(q_gate[at]);
-    qs[i] = v;
-  }
-  __syncthreads();
-
+  // the key rows are requested first: they are the long pole, q is staged while they fly
   const int sub = threadIdx.x % LPK, slot = threadIdx.x / LPK;
   const __nv_bfloat16 *kb = k + b * ksb + hk * ksh + sub * 8;
   const __nv_bfloat16 *gb = GATED ? k_gate + b * ksb + hk * ksh + sub * 8 : nullptr;
@@ -73,6 +66,14 @@ ttp_logits_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__re
     kr[p] = in ? ld_nc_16(kb + (long long)j * ksp) : make_uint4(0, 0, 0, 0);
     if (GATED) gr[p] = in ? ld_nc_16(gb + (long long)j * ksp) : make_uint4(0, 0, 0, 0);
   }
+  for (int i = threadIdx.x; i < group * D; i += kScoreThreads) {
+    const long long at = ((long long)b * n_q_heads + hk * group) * D + i;
+    float v = __bfloat162float(q[at]) * scale;
+    if (GATED) v *= __bfloat162float(q_gate[at]);
+    qs[i] = v;
+  }
+  __syncthreads();
+
   // the (gated) key row of every pass as eight floats
   float kf[PASSES][8];
 #pragma unroll
@@ -177,12 +178,25 @@ ttp_finalize_topk_kernel(const float *__restrict__ logits, int lstride, int n_q_
     const int lo = norm_scope ? vs : 0, hi = norm_scope ? vs + nv : lp;
     for (int h = warp; h < n_q_heads; h += kTopkThreads / 32) {
       const float *z = logits + ((long long)b * n_q_heads + h) * lstride;
+      // up to 32 x kStatRegs logits of the row stay in registers (all loads in flight at once, one
+      // pass for the maximum and the sum); longer rows take the two-pass loop for the rest
+      constexpr int kStatRegs = 24;
+      float v[kStatRegs];
       float mx = -INFINITY;
-      for (int j = lo + lane; j < hi; j += 32) mx = fmaxf(mx, z[j]);
+#pragma unroll
+      for (int i = 0; i < kStatRegs; ++i) {
+        const int j = lo + lane + 32 * i;
+        v[i] = j < hi ? z[j] : -INFINITY;
+      }
+#pragma unroll
+      for (int i = 0; i < kStatRegs; ++i) mx = fmaxf(mx, v[i]);
+      for (int j = lo + lane + 32 * kStatRegs; j < hi; j += 32) mx = fmaxf(mx, z[j]);
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
       float sum = 0.f;
-      for (int j = lo + lane; j < hi; j += 32) sum += expf(z[j] - mx);
+#pragma unroll
+      for (int i = 0; i < kStatRegs; ++i) sum += v[i] > -INFINITY ? expf(v[i] - mx) : 0.f;   // (nothing past the row's end)
+      for (int j = lo + lane + 32 * kStatRegs; j < hi; j += 32) sum += expf(z[j] - mx);
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
       if (lane == 0) {
@@ -196,7 +210,22 @@ ttp_finalize_topk_kernel(const float *__restrict__ logits, int lstride, int n_q_
       float acc = 0.f;
       if (m < nv) {
         const float *z = logits + (long long)b * n_q_heads * lstride + vs + m;
-        for (int h = 0; h < n_q_heads; ++h) acc += expf(z[(long long)h * lstride] - h_max[h]) * h_inv[h];
+        int h = 0;
+        for (; h + 32 <= n_q_heads; h += 32) {         // 32 heads' logits in flight: one round trip
+          float zz[32];
+#pragma unroll
+          for (int i = 0; i < 32; ++i) zz[i] = z[(long long)(h + i) * lstride];
+#pragma unroll
+          for (int i = 0; i < 32; ++i) acc += expf(zz[i] - h_max[h + i]) * h_inv[h + i];
+        }
+        for (; h + 8 <= n_q_heads; h += 8) {
+          float zz[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) zz[i] = z[(long long)(h + i) * lstride];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) acc += expf(zz[i] - h_max[h + i]) * h_inv[h + i];
+        }
+        for (; h < n_q_heads; ++h) acc += expf(z[(long long)h * lstride] - h_max[h]) * h_inv[h];
         acc *= inv_h;
       }
       sc[m] = acc;
@@ -220,27 +249,6 @@ ttp_finalize_topk_kernel(const float *__restrict__ logits, int lstride, int n_q_
   if (R == 0) return;
   __syncthreads();
 
-  if (nv <= kTopkThreads) {
-    // Few visual tokens (one per thread): exact selection by counting.  A token is kept iff fewer
-    // than R tokens come before it in the order (larger score first, lower index first among
-    // equals); an ordered scan of the kept flags gives the ascending output positions.
-    const int m = tid;
-    uint32_t sel = 0;
-    if (m < nv) {
-      const uint32_t mine = keys[m];
-      int before = 0;
-      for (int o = 0; o < nv; ++o) {
-        const uint32_t other = keys[o];                       // (all threads read the same word: a broadcast)
-        before += (other > mine || (other == mine && o < m)) ? 1 : 0;
-      }
-      sel = before < R ? 1u : 0u;
-    }
-    uint32_t total;
-    const uint32_t at = block_exclusive_scan(sel, warp_sums, total);
-    if (sel) out[at] = m;
-    return;
-  }
-
   // radix select, 8 bits per pass from the top: the R-th largest key
   uint32_t prefix = 0, mask = 0;
   uint32_t remaining = (uint32_t)R;
@@ -248,9 +256,15 @@ ttp_finalize_topk_kernel(const float *__restrict__ logits, int lstride, int n_q_
   for (int shift = 24; shift >= 0; shift -= 8) {
     if (tid < 256) hist[tid] = 0;
     __syncthreads();
-    for (int m = tid; m < nv; m += kTopkThreads) {
-      const uint32_t key = keys[m];
-      if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+    // (scores of one request are close to each other, so in the top passes nearly all keys share a
+    // digit: the lanes of a warp that hold the same digit add their count with one atomic)
+    for (int base = 0; base < nv; base += kTopkThreads) {
+      const int m = base + tid;
+      const uint32_t key = m < nv ? keys[m] : 0u;
+      const bool cand = m < nv && (key & mask) == prefix;
+      const uint32_t digit = cand ? (key >> shift) & 255u : 256u + (uint32_t)lane;     // non-candidates match nobody
+      const unsigned peers = __match_any_sync(0xffffffffu, digit);
+      if (cand && lane == __ffs(peers) - 1) atomicAdd(&hist[digit], (uint32_t)__popc(peers));
     }
     __syncthreads();
     if (warp == 0) {
@@ -303,7 +317,12 @@ ttp_finalize_topk_kernel(const float *__restrict__ logits, int lstride, int n_q_
 
 // ---------------------------------------------------------------------------
 // Stage 3: gather the rows of the pruned sequence, all layers and kv heads.
-// One CTA = 64 destination rows of one (layer, kv head, request), K and V.
+// One CTA = 64 rows of one (layer, kv head, request), K and V.  The rows of a request come in two
+// kinds: text rows (before and after the image), whose source needs nothing but the request's
+// layout, and kept visual rows, whose source is kept_idx.  blockIdx.y walks the text rows first
+// (text_blocks blocks of 64) and the visual rows last (the remaining blocks), so that in the
+// fused call, where the selection may still be running when this kernel starts, the CTAs that do
+// not need it are scheduled first and leave without waiting; only the visual CTAs wait for it.
 // ---------------------------------------------------------------------------
 constexpr int kGatherThreads = 256;
 constexpr int kGatherRows = 64;
@@ -314,79 +333,76 @@ kv_gather_kernel(KvView src, KvViewMut dst, const int *__restrict__ kept_idx, in
                  const int *__restrict__ keep, const int *__restrict__ prefix_len,
                  const int *__restrict__ vis_start, const int *__restrict__ n_vis,
                  const int *__restrict__ pos_in, int *__restrict__ pos_out, int pos_stride,
-                 int *__restrict__ new_len, int *dev_status, int early_text) {
+                 int *__restrict__ new_len, int *dev_status, int text_blocks, int early_text) {
   constexpr int LPR = D / 8;                   // lanes per row
   constexpr int RPP = kGatherThreads / LPR;    // rows per pass
   constexpr int PASSES = kGatherRows / RPP;
   // early_text (the fused call): the kernels before this one in the stream are the call's own scoring
-  // and selection, which write nothing this kernel reads except kept_idx.  The text rows (they do not
-  // depend on the selection) are copied while those kernels are still running; the kept visual rows
-  // follow once the selection has completed.
-  if (!early_text) grid_dependency_sync();
-  const int b = blockIdx.z;
-  const int layer = blockIdx.y / src.n_kv_heads, h = blockIdx.y % src.n_kv_heads;
+  // and selection, which write nothing this kernel reads except kept_idx; text CTAs then run without
+  // waiting for them.  Otherwise nothing is read before the preceding kernel has completed.
+  const bool visual = (int)blockIdx.y >= text_blocks;
+  if (!early_text || visual) grid_dependency_sync();
+  const int slice = blockIdx.x % (src.n_layers * src.n_kv_heads), b = blockIdx.x / (src.n_layers * src.n_kv_heads);
+  const int layer = slice / src.n_kv_heads, h = slice % src.n_kv_heads;
   const int lp = prefix_len[b], vs = vis_start[b], nv = n_vis[b], kp = keep[b];
-  const bool first = blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0;
+  const bool first = slice == 0 && blockIdx.y == 0 && threadIdx.x == 0;
   const int nl = lp - nv + kp;
-  const int j0 = blockIdx.x * kGatherRows;
   {
     int code = 0;
     if (!layout_ok(lp, vs, nv, src.max_len, TWIG_MAX_VISUAL)) code = TWIG_DEV_BAD_LAYOUT;
     else if (kp < 0 || kp > nv || kp > r_max) code = TWIG_DEV_BAD_KEEP;
     else if (nl > dst.max_len) code = TWIG_DEV_OVERFLOW;
-    if (code == 0 && first && new_len) new_len[b] = nl;
-    if (code != 0 || j0 >= nl) {
-      // (a CTA with nothing to do still waits for the preceding kernel before it leaves, so that this
-      // kernel's completion implies that one's)
-      if (early_text) grid_dependency_sync();
-      if (code != 0 && first) flag_status(dev_status, b, code);
+    if (code != 0) {
+      if (first) flag_status(dev_status, b, code);
       return;
     }
+    if (first && new_len) new_len[b] = nl;
   }
+  // this CTA's rows: index i0.. within its kind (text rows: the lp - nv rows outside the image)
+  const int i0 = (visual ? (int)blockIdx.y - text_blocks : (int)blockIdx.y) * kGatherRows;
+  const int n_kind = visual ? kp : lp - nv;
+  if (i0 >= n_kind) return;
 
   const int sub = threadIdx.x % LPR, slot = threadIdx.x / LPR;
   const long long sbase = layer * src.stride_layer + b * src.stride_batch + h * src.stride_head + sub * 8;
   const long long dbase = layer * dst.stride_layer + b * dst.stride_batch + h * dst.stride_head + sub * 8;
   const int *kidx = kept_idx + (long long)b * r_max;
 
-  int srow[PASSES];
+  int srow[PASSES], drow[PASSES];
   uint4 kr[PASSES], vr[PASSES];
-  // phase 0: rows that need no kept_idx (text before and after the image); phase 1: kept visual rows
-  for (int phase = 0; phase < 2; ++phase) {
-    if (phase == 1 && early_text) grid_dependency_sync();
 #pragma unroll
-    for (int p = 0; p < PASSES; ++p) {
-      const int j = j0 + p * RPP + slot;
-      int s = -1;
-      if (j < nl) {
-        const bool visual = j >= vs && j < vs + kp;
-        if (phase == 0 && !visual) {
-          s = j < vs ? j : j - kp + nv;
-        } else if (phase == 1 && visual) {
-          const int kk = kidx[j - vs];
-          const int prev = (j > vs) ? kidx[j - vs - 1] : -1;
-          if (kk < 0 || kk >= nv || kk <= prev) {
-            if (sub == 0 && blockIdx.y == 0) flag_status(dev_status, b, TWIG_DEV_BAD_INDEX);
-          } else {
-            s = vs + kk;
-          }
+  for (int p = 0; p < PASSES; ++p) {
+    const int i = i0 + p * RPP + slot;
+    int s = -1, j = 0;
+    if (i < n_kind) {
+      if (!visual) {                 // text row i: before the image it stays, after it moves up by the dropped tokens
+        s = i < vs ? i : i + nv;
+        j = i < vs ? i : i + kp;
+      } else {
+        const int kk = kidx[i];
+        const int prev = i > 0 ? kidx[i - 1] : -1;
+        if (kk < 0 || kk >= nv || kk <= prev) {
+          if (sub == 0 && slice == 0) flag_status(dev_status, b, TWIG_DEV_BAD_INDEX);
+        } else {
+          s = vs + kk;
+          j = vs + i;
         }
       }
-      srow[p] = s;
-      if (s >= 0) {
-        kr[p] = ld_nc_16(src.k + sbase + (long long)s * src.stride_pos);
-        vr[p] = ld_nc_16(src.v + sbase + (long long)s * src.stride_pos);
-      }
     }
+    srow[p] = s;
+    drow[p] = j;
+    if (s >= 0) {
+      kr[p] = ld_nc_16(src.k + sbase + (long long)s * src.stride_pos);
+      vr[p] = ld_nc_16(src.v + sbase + (long long)s * src.stride_pos);
+    }
+  }
 #pragma unroll
-    for (int p = 0; p < PASSES; ++p) {
-      const int j = j0 + p * RPP + slot;
-      if (srow[p] >= 0) {
-        st_16(dst.k + dbase + (long long)j * dst.stride_pos, kr[p]);
-        st_16(dst.v + dbase + (long long)j * dst.stride_pos, vr[p]);
-        if (blockIdx.y == 0 && sub == 0 && pos_in && pos_out)
-          pos_out[(long long)b * pos_stride + j] = pos_in[(long long)b * pos_stride + srow[p]];
-      }
+  for (int p = 0; p < PASSES; ++p) {
+    if (srow[p] >= 0) {
+      st_16(dst.k + dbase + (long long)drow[p] * dst.stride_pos, kr[p]);
+      st_16(dst.v + dbase + (long long)drow[p] * dst.stride_pos, vr[p]);
+      if (slice == 0 && sub == 0 && pos_in && pos_out)
+        pos_out[(long long)b * pos_stride + drow[p]] = pos_in[(long long)b * pos_stride + srow[p]];
     }
   }
 }
@@ -726,8 +742,13 @@ static twig_status launch_gather(const twig_kv *src, const twig_kv *dst, const i
           vis_start, n_vis, pos_out, pos_stride, new_len, dev_status);
     return launch_status();
   }
+  // text rows of a request fit both tensors; kept visual rows are at most r_max (and at most dst's rows)
   const int rows_bound = src->max_len < dst->max_len ? src->max_len : dst->max_len;
-  dim3 grid((rows_bound + kGatherRows - 1) / kGatherRows, src->n_layers * src->n_kv_heads, src->batch);
+  const int text_blocks = (rows_bound + kGatherRows - 1) / kGatherRows;
+  const int vis_rows = r_max < dst->max_len ? r_max : dst->max_len;
+  const int vis_blocks = (vis_rows + kGatherRows - 1) / kGatherRows;
+  if (text_blocks + vis_blocks > 65535) return TWIG_ERR_UNSUPPORTED;
+  dim3 grid(src->n_layers * src->n_kv_heads * src->batch, text_blocks + vis_blocks);
   PdlLaunch L(grid, dim3(kGatherThreads), 0, st);
   const KvView sv = view_of(src);
   const KvViewMut dv = view_of_mut(dst);
@@ -735,9 +756,9 @@ static twig_status launch_gather(const twig_kv *src, const twig_kv *dst, const i
   const cudaError_t err =
       src->head_dim == 128
           ? cudaLaunchKernelEx(&L.cfg, kv_gather_kernel<128>, sv, dv, kept_idx, r_max, keep, prefix_len, vis_start, n_vis,
-                               pos_in, pos_out, pos_stride, new_len, dev_status, early_text)
+                               pos_in, pos_out, pos_stride, new_len, dev_status, text_blocks, early_text)
           : cudaLaunchKernelEx(&L.cfg, kv_gather_kernel<64>, sv, dv, kept_idx, r_max, keep, prefix_len, vis_start, n_vis,
-                               pos_in, pos_out, pos_stride, new_len, dev_status, early_text);
+                               pos_in, pos_out, pos_stride, new_len, dev_status, text_blocks, early_text);
   return err == cudaSuccess ? TWIG_OK : TWIG_ERR_CUDA;
 }
 

@@ -96,15 +96,17 @@ _lib.tree_verify_attention.argtypes = [_vp, _vp, _vp, _kvp, _i32, _vp, _vp, _vp,
 _lib.tree_verify_attention_ex.restype = C.c_int
 _lib.tree_verify_attention_ex.argtypes = _lib.tree_verify_attention.argtypes + [C.c_uint32]
 # per-call flags of tree_verify_attention_ex
-ATTN_EARLY_PREFIX, ATTN_PLAIN_LAUNCH = 1, 1 << 4
+ATTN_EARLY_PREFIX, ATTN_PLAIN_LAUNCH, ATTN_EARLY_QUERY = 1, 1 << 4, 1 << 5
 ATTN_KERNEL_AUTO, ATTN_KERNEL_MMA, ATTN_KERNEL_TCGEN05, ATTN_KERNEL_STREAM = 0, 1, 2, 3
 
 
-def attn_flags(kernel=ATTN_KERNEL_AUTO, early_prefix=False, splits=0, plain_launch=False, stream_policy=0) -> int:
+def attn_flags(kernel=ATTN_KERNEL_AUTO, early_prefix=False, splits=0, plain_launch=False, stream_policy=0,
+               early_query=False) -> int:
     """Packs the flags word of tree_verify_attention_ex (stream_policy: 0 the kernel's choice,
     1 equal shares of the key tiles, 2 whole items)."""
     return (int(kernel) << 1) | (ATTN_EARLY_PREFIX if early_prefix else 0) | (int(splits) << 8) | \
-        (ATTN_PLAIN_LAUNCH if plain_launch else 0) | (int(stream_policy) << 12)
+        (ATTN_PLAIN_LAUNCH if plain_launch else 0) | (int(stream_policy) << 12) | \
+        (ATTN_EARLY_QUERY if early_query else 0)
 
 
 _lib.tree_reset.restype = C.c_int

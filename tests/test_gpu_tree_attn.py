@@ -238,9 +238,11 @@ def test_early_prefix_gives_the_same_bits(tw, shape, path):
     kvl, nn, par = dev_i32(kv_len), dev_i32(ver["n_nodes"]), dev_i32(ver["parent"])
     outs = [torch.zeros((B_, T, Hq_, d_), dtype=torch.bfloat16, device=DEV) for _ in range(4)]
     ws = stream_ws(tw, B_, Hq_, T) if path == 3 else None
-    for o in outs:
+    for i, o in enumerate(outs):
+        # (the second promise, that Q and the tree rows are final too, holds here as well: nothing in
+        # the stream writes them; the small-call kernel then does not wait before it computes)
         tw.tree_verify_attention(q, tk, tv, cache, 0, kvl, nn, par, o, ws=ws,
-                                 flags=tw.attn_flags(kernel=path, early_prefix=True))
+                                 flags=tw.attn_flags(kernel=path, early_prefix=True, early_query=(i % 2 == 1)))
     torch.cuda.synchronize()
     assert not st0.any() and not st1.any()
     assert np.array_equal(got, ref) and np.array_equal(got_lse, ref_lse)
