@@ -19,6 +19,8 @@
 //                     M = 64, whose accumulator rows sit in lanes 0-15 of each of the four
 //                     32-lane quadrants of tensor memory (row r in lane 32 (r / 16) + r % 16),
 //                     so every warp works on 16 rows; with 128 rows M = 128 and row r is lane r.
+// Blocks of 128 rows keep both A operands in tensor memory instead (Q, written once by the softmax
+// warps, and P, written over the first half of the S tile it came from): see UmmaCfg.
 // The running maximum is only raised when a tile exceeds it by more than 2^8; then (rarely)
 // the O accumulator is rescaled in tensor memory (ld, multiply, st).  P stays below 2^8,
 // which bf16 and the fp32 sums hold without loss of accuracy.
@@ -43,7 +45,7 @@ namespace {
 constexpr int kD = 128;          // head_dim
 // warps 0-3 softmax, warp 4 loader, warp 5 MMA issuer; with 128-row accumulators warps 6-9 are a
 // second softmax group (UmmaCfg::THREADS)
-constexpr int kMaxSlots = 6;                      // ring of K / V tiles (K0 V0 K1 V1 K2 ...)
+constexpr int kMaxSlots = 8;                      // ring of K / V tiles (K0 V0 K1 V1 K2 ...)
 constexpr float kLazyMax = 8.f;                   // raise the running max only beyond this (log2 units)
 
 // KT = keys per tile: 64 (two CTAs per SM, 256 tensor-memory columns each) or 128 (one CTA per SM
@@ -52,21 +54,29 @@ template <int ROWS, int KT>
 struct UmmaCfg {
   static constexpr int TILE_BYTES = KT * kD * 2;         // one K (or V) tile: 16 or 32 KB
   static constexpr int PANEL_BYTES = KT * 128;           // 64-column panel of a K/V tile
-  static constexpr int Q_BYTES = ROWS * kD * 2;          // two 64-column panels of ROWS x 128 B
-  static constexpr int P_ONE = ROWS * KT * 2;            // ROWS x KT keys bf16, KT/64 panels of ROWS x 128 B
+  // 128-row blocks keep the A operands of both products in tensor memory: Q (loaded once) and P
+  // (written by the softmax warps over the first half of the S tile it came from).  Both products
+  // then read only their B operand (K or V) through shared memory, whose port is what limits a
+  // CTA that streams 8 KB per MMA instruction; and the 96 KB that Q and two P buffers took go to
+  // the ring of K / V tiles.
+  static constexpr bool TMEM_AB = ROWS == 128;
+  static constexpr int Q_BYTES = TMEM_AB ? 0 : ROWS * kD * 2;     // two 64-column panels of ROWS x 128 B
+  static constexpr int P_ONE = TMEM_AB ? 0 : ROWS * KT * 2;       // ROWS x KT keys bf16, KT/64 panels of ROWS x 128 B
   // two P buffers where shared memory allows: the softmax of tile t+1 then never waits for P(t) V(t)
   // (64-key tiles with two CTAs per SM: one more ring slot measured better than the second P buffer)
   static constexpr int P_BUFS = (ROWS <= 64 && KT == 64) ? 1 : 2;
   static constexpr int P_BYTES = P_BUFS * P_ONE;
-  // 128 rows with 128-key tiles: four slots, so that two P buffers still fit in shared memory
-  static constexpr int SLOTS = (ROWS == 128 && KT == 128) ? 4 : (ROWS == 32 && KT == 64) ? 6 : 5;
+  static constexpr int SLOTS = TMEM_AB ? (KT == 128 ? 6 : 8) : (ROWS == 32 && KT == 64) ? 6 : 5;
   static constexpr int RING_BYTES = SLOTS * TILE_BYTES;
-  static constexpr uint32_t TMEM_COLS = KT == 64 ? 256 : 512;   // S: [0,KT) and [KT,2KT); O: [2KT, 2KT+128)
+  // S: [0,KT) and [KT,2KT); O: [2KT, 2KT+128); Q (TMEM_AB): [2KT+128, 2KT+192), 64 columns of bf16 pairs
+  static constexpr uint32_t TMEM_COLS = (KT == 64 && !TMEM_AB) ? 256 : 512;
   static constexpr uint32_t O_COL = 2 * KT;
+  static constexpr uint32_t Q_COL = 2 * KT + 128;
   static constexpr int MIN_CTAS = (KT == 64 && ROWS <= 64) ? 2 : 1;     // (128 rows: shared memory allows one CTA per SM)
   static constexpr int RECV_BYTES = ROWS * kD * 4;
   static_assert(RECV_BYTES <= RING_BYTES, "split-merge buffer must fit in the stage ring");
   static_assert(Q_BYTES % 1024 == 0 && P_BYTES % 1024 == 0, "swizzled tiles start on 1024 bytes");
+  static_assert(SLOTS <= kMaxSlots, "ring barriers");
   static constexpr int SMEM_BYTES = Q_BYTES + P_BYTES + RING_BYTES;
   static constexpr int MMA_M = ROWS <= 64 ? 64 : 128;
   static constexpr int ROWS_PER_WARP = MMA_M == 64 ? 16 : 32;    // rows a softmax warp owns
@@ -130,7 +140,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
     mbar_init(bar_s(1), 1);
     mbar_init(bar_o(0), 1);
     mbar_init(bar_o(1), 1);
-    mbar_init(bar_q, 32);
+    if (!C::TMEM_AB) mbar_init(bar_q, 32);     // (with Q in tensor memory: one arrival per softmax warp, set below)
     if (n_splits > 1) {
       // split merge: one arrival that announces the peers' bytes (every peer sends each of this
       // CTA's ROWS / n_splits rows as 128 fp16 and (m, l, row scale, -)), one per softmax warp for this
@@ -201,6 +211,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
   }
   if (tid == 0) {
     for (int i = 0; i < 2; ++i) mbar_init(bar_p(i), n_soft * C::SOFT_GROUPS);      // one arrival per softmax warp
+    if (C::TMEM_AB) mbar_init(bar_q, n_soft * C::SOFT_GROUPS);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   tc_fence_before();
@@ -298,7 +309,7 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
     // K of the first tile, then Q (what S(0) needs), then the rest of the first ring
     const int n_first = min(n_units, kSlots);
     if (n_first > 0) issue_unit(0);
-    if (n_my > 0) issue_q();
+    if (n_my > 0 && !C::TMEM_AB) issue_q();
     for (int u = 1; u < n_first; ++u) issue_unit(u);
     for (int u = n_first; u < n_units && ok; ++u) {
       publish_q();                              // (all ring slots are in flight by now)
@@ -325,9 +336,13 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
         const uint32_t kb = ring_s + (u % kSlots) * kTileBytes;
 #pragma unroll
         for (int ks = 0; ks < kD / 16; ++ks) {
-          const uint32_t qa = q_s + (ks >> 2) * ROWS * 128 + (ks & 3) * 32;
           const uint32_t ka = kb + (ks >> 2) * kPanelBytes + (ks & 3) * 32;
-          umma(tmem + (it & 1) * KT, smem_desc(qa, 16), smem_desc(ka, 16), kIdescS, ks > 0);
+          if (C::TMEM_AB) {            // Q from tensor memory: 16 head-dim entries = 8 columns per step
+            umma_ts(tmem + (it & 1) * KT, tmem + C::Q_COL + ks * 8, smem_desc(ka, 16), kIdescS, ks > 0);
+          } else {
+            const uint32_t qa = q_s + (ks >> 2) * ROWS * 128 + (ks & 3) * 32;
+            umma(tmem + (it & 1) * KT, smem_desc(qa, 16), smem_desc(ka, 16), kIdescS, ks > 0);
+          }
         }
         umma_commit(bar_s(it & 1));
         umma_commit(bar_empty(u % kSlots));
@@ -345,9 +360,13 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
         if (!ok) break;
         const uint32_t vb = ring_s + (u % kSlots) * kTileBytes;
 #pragma unroll
-        for (int j = 0; j < KT / 16; ++j)          // 16 keys per step: P panel j / 4, V rows 16 j ..
-          umma(tmem_o, smem_desc(p_s + pb * C::P_ONE + (j >> 2) * ROWS * 128 + (j & 3) * 32, 16),
-               smem_desc(vb + j * 2048, kPanelBytes), kIdescO, (it > 0) || (j > 0));
+        for (int j = 0; j < KT / 16; ++j) {        // 16 keys per step: V rows 16 j ..
+          if (C::TMEM_AB)              // P(it) lies over the first half of S(it): 8 columns per step
+            umma_ts(tmem_o, tmem + (it & 1) * KT + j * 8, smem_desc(vb + j * 2048, kPanelBytes), kIdescO, (it > 0) || (j > 0));
+          else                         // P panel j / 4 in shared memory
+            umma(tmem_o, smem_desc(p_s + pb * C::P_ONE + (j >> 2) * ROWS * 128 + (j & 3) * 32, 16),
+                 smem_desc(vb + j * 2048, kPanelBytes), kIdescO, (it > 0) || (j > 0));
+        }
         umma_commit(bar_o(pb));
         umma_commit(bar_empty(u % kSlots));
         if (it + 2 < n_my) issue_s(it + 2);
@@ -517,6 +536,33 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
     auto pair_sync = [&]() { asm volatile("bar.sync %0, 64;" ::"r"(1 + quad) : "memory"); };
     float m_r = -INFINITY, l_r = 0.f;           // l_r: this thread's keys only
     bool ok = true;
+    if (C::TMEM_AB && n_my > 0) {
+      // Q into tensor memory, once: the row's 128 bf16 are 64 columns of pairs (the pair of head-dim
+      // entries 2c, 2c+1 in column c, the lower one in the low half: as they lie in memory); this
+      // warp writes the half `half` of its rows' columns.  Rows past the last one are zero.
+      uint32_t qw[32];
+      if (grow < rows_total) {
+        const int node = grow / p.group, g = grow % p.group;
+        const uint4 *src = reinterpret_cast<const uint4 *>(
+            p.q + (((long long)b * p.t_max + node) * p.n_q_heads + hk * p.group + g) * kD + half * 64);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const uint4 w = ld_nc_16(src + i);
+          qw[4 * i] = w.x;
+          qw[4 * i + 1] = w.y;
+          qw[4 * i + 2] = w.z;
+          qw[4 * i + 3] = w.w;
+        }
+      } else {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) qw[i] = 0u;
+      }
+      tmem_st32(t_lane + C::Q_COL + half * 32, qw);
+      tmem_st_wait();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_q);
+    }
     for (int it = 0; it < n_my; ++it) {
       const int t = t_begin + it;
       ok = ok && mbar_wait(bar_s(it & 1), (it >> 1) & 1, fail);
@@ -553,7 +599,9 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
       const float m_new = raise ? mx : m_r;
       const float m_use = m_new == -INFINITY ? 0.f : m_new;
       const int pb = it % PB;
-      if (it >= PB) {                           // this P buffer is free once P(it-PB) V(it-PB) is done
+      // a P buffer in shared memory is free once P(it-PB) V(it-PB) is done; in tensor memory P(it)
+      // lies over S(it), which was only computed after P(it-2) V(it-2) (the products run in order)
+      if (!C::TMEM_AB && it >= PB) {
         ok = ok && mbar_wait(bar_o(pb), (it / PB - 1) & 1, fail);
         ok = __all_sync(0xffffffffu, ok);
         tc_fence_after();
@@ -579,28 +627,47 @@ tree_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap km
         tmem_st_wait();
       }
       m_r = m_new;
-      // P = exp2(S * scale - m) as bf16 to shared memory, row sums
+      // P = exp2(S * scale - m) as bf16, row sums
       float sum0 = 0.f, sum1 = 0.f;
-      constexpr int panel = KT == 128 ? 1 : 0;  // with 128-key tiles the second half is the second 64-key panel
-      const uint32_t prow = p_s + pb * C::P_ONE + half * panel * ROWS * 128 + row * 128;
-      const int chunk0 = KT == 128 ? 0 : half * 4;
+      if (C::TMEM_AB) {
+        // into tensor memory, over the first half of this S tile's columns (the other warp of the pair
+        // has read its S by now: the pair met above): key pairs (2c, 2c+1) in column c of the tile
+        uint32_t pw[NV / 2];
 #pragma unroll
-      for (int cc = 0; cc < NV / 8; ++cc) {     // chunk: 8 keys of this row
-        uint32_t w[4];
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const int j = cc * 8 + e * 2;
+        for (int c = 0; c < NV / 2; ++c) {
+          const int j = 2 * c;
           const float p0 = fast_exp2(fmaf(__uint_as_float(sr[j >> 5][j & 31]), p.scale_log2, -m_use));
           const float p1 = poly_exp2(fmaf(__uint_as_float(sr[(j + 1) >> 5][(j + 1) & 31]), p.scale_log2, -m_use));
           sum0 += p0;
           sum1 += p1;
-          w[e] = pack_bf16(p0, p1);
+          pw[c] = pack_bf16(p0, p1);
         }
-        asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(prow + (((chunk0 + cc) ^ (row & 7)) << 4)), "r"(w[0]),
-                     "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
+        const uint32_t pcol = t_lane + (it & 1) * KT + half * (NV / 2);
+        if constexpr (NV / 2 == 32) tmem_st32(pcol, reinterpret_cast<const uint32_t (&)[32]>(pw));
+        else tmem_st16(pcol, reinterpret_cast<const uint32_t (&)[16]>(pw));
+        tmem_st_wait();
+      } else {
+        constexpr int panel = KT == 128 ? 1 : 0;  // with 128-key tiles the second half is the second 64-key panel
+        const uint32_t prow = p_s + pb * C::P_ONE + half * panel * ROWS * 128 + row * 128;
+        const int chunk0 = KT == 128 ? 0 : half * 4;
+#pragma unroll
+        for (int cc = 0; cc < NV / 8; ++cc) {     // chunk: 8 keys of this row
+          uint32_t w[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const int j = cc * 8 + e * 2;
+            const float p0 = fast_exp2(fmaf(__uint_as_float(sr[j >> 5][j & 31]), p.scale_log2, -m_use));
+            const float p1 = poly_exp2(fmaf(__uint_as_float(sr[(j + 1) >> 5][(j + 1) & 31]), p.scale_log2, -m_use));
+            sum0 += p0;
+            sum1 += p1;
+            w[e] = pack_bf16(p0, p1);
+          }
+          asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(prow + (((chunk0 + cc) ^ (row & 7)) << 4)), "r"(w[0]),
+                       "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
+        }
+        fence_async_smem();            // P was written with ordinary stores
       }
       l_r += sum0 + sum1;
-      fence_async_smem();            // P was written with ordinary stores
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_p(pb));
