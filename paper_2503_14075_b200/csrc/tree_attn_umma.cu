@@ -2,23 +2,25 @@
 // (Sec. 5.4, Appendix A, Algorithm 2; Eq. 2 with the tree's ancestor mask).
 //
 // One CTA owns up to ROWS query rows (tree node x query head of one kv head) and a
-// share of the 64-key tiles.  Its six warps have three roles that only meet at mbarriers:
-//   warp 4 (loader)   brings K and V tiles (16 KB units: K0 V0 K1 V1 ...) into a ring of five
-//                     slots in the 128-byte-swizzled layout the matrix descriptors name: tiles
-//                     that lie wholly in the cached prefix by TMA (two 64 x 64 boxes of a 5-D
-//                     tensor map over the cache, completion counted on the slot's mbarrier),
+// share of the key tiles (64 or 128 keys each).  Its warps (six, or ten with 128-row accumulators)
+// have three roles that only meet at mbarriers:
+//   warp 4 (loader)   brings K and V tiles (units K0 V0 K1 V1 ...) into a ring of five to eight
+//                     slots (UmmaCfg::SLOTS) in the 128-byte-swizzled layout the matrix descriptors
+//                     name: tiles that lie wholly in the cached prefix by TMA (two 64-column boxes of
+//                     a 5-D tensor map over the cache, completion counted on the slot's mbarrier),
 //                     the tile that holds the prefix end and the tree's own rows by 16-byte
 //                     cp.async with zero fill; a slot is refilled when the MMA that read it
 //                     has completed;
-//   warp 5 (issuer)   one thread issues S(t) = Q K(t)^T (tcgen05.mma, M = 128, N = 64, K = 8 x 16)
-//                     two tiles ahead into a double-buffered S in tensor memory, and
-//                     O += P(t) V(t) (M = 128, N = 128, K = 4 x 16, V read MN-major, accumulating
-//                     in tensor memory) as soon as the softmax warps have published P(t);
-//   warps 0-3 (softmax) one thread per row: tcgen05.ld of its S row, running max / sum,
-//                     P (bf16) back to shared memory.  With up to 64 rows the products use
-//                     M = 64, whose accumulator rows sit in lanes 0-15 of each of the four
-//                     32-lane quadrants of tensor memory (row r in lane 32 (r / 16) + r % 16),
-//                     so every warp works on 16 rows; with 128 rows M = 128 and row r is lane r.
+//   warp 5 (issuer)   one thread issues S(t) = Q K(t)^T (tcgen05.mma, M = 64 or 128, N = keys of a
+//                     tile, K = 8 x 16) two tiles ahead into a double-buffered S in tensor memory, and
+//                     O += P(t) V(t) (N = 128, V read MN-major, accumulating in tensor memory) as
+//                     soon as the softmax warps have published P(t);
+//   warps 0-3 (softmax; with 128-row accumulators also warps 6-9, which take the second half of
+//                     every tile's keys): tcgen05.ld of S, running max / sum, P (bf16).  With up
+//                     to 64 rows the products use M = 64, whose accumulator rows sit in lanes 0-15
+//                     of each of the four 32-lane quadrants of tensor memory (row r in lane
+//                     32 (r / 16) + r % 16), so every warp works on 16 rows and P goes to shared
+//                     memory; with 128 rows M = 128 and row r is lane r.
 // Blocks of 128 rows keep both A operands in tensor memory instead (Q, written once by the softmax
 // warps, and P, written over the first half of the S tile it came from): see UmmaCfg.
 // The running maximum is only raised when a tile exceeds it by more than 2^8; then (rarely)
