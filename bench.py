@@ -37,7 +37,7 @@ POOL = 8           # distinct per-step Q / tree-K/V sets per replica (cycled)
 MAX_STEPS = 110    # bound on verify steps per request
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel (tree_attn_kernel,
 # c2 shape, kv_len 227); set to None whenever that kernel changes after the capture
-ATTN_TRAFFIC_NCU = 4413184
+ATTN_TRAFFIC_NCU = 4414464
 
 
 def load_peaks():
