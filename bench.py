@@ -755,7 +755,7 @@ def extra_rooflines(torch, tw, peaks, dev):
     root = torch.zeros((Bt, 1), dtype=torch.int32, device=dev)
     nxt = torch.zeros((Bt, K_), dtype=torch.int32, device=dev)
 
-    def build_tree(logit_levels):
+    def build_tree_calls(logit_levels):
         tw.tree_reset(state)
         src, lo, hi = root, 0, 1
         for l in range(D_):
@@ -766,23 +766,58 @@ def extra_rooflines(torch, tw, peaks, dev):
                 src = nxt
         tw.tree_finalize(state, cap, NMAX, t_par, t_tok, t_n)
 
-    for ls in lsets:
-        build_tree(ls)
+    def build_tree(logit_levels):
+        # one launch per level: the level's last CTA of each request selects / prunes
+        src, hi = root, 1
+        for l in range(D_):
+            if l + 1 < D_:
+                tw.tree_grow_level(logit_levels[l], src, E_, hi, state, expand_node=nxt)
+                src = nxt
+            else:
+                tw.tree_grow_level(logit_levels[l], src, E_, hi, state, n_max=NMAX, parent=t_par, draft_tok=t_tok,
+                                   n_nodes=t_n)
+            hi += (1 if l == 0 else K_) * E_
+
+    def timed(fn):
+        for ls in lsets:
+            fn(ls)
+        e0.record(stream)
+        for i in range(n_chain):
+            fn(lsets[i % 3])
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) * 1e3 / n_chain
+
+    tree_bytes = int(Bt * (1 + (D_ - 1) * K_) * V * 2)
+    us = timed(build_tree)
+    res["tree_build_c3_E10_K10_D4"] = hbm_entry(us, tree_bytes)
+    res["tree_build_c3_E10_K10_D4"]["launches"] = "4 (one per level: expansion + selection / pruning), launched one by one"
+    # the same trees replayed from a CUDA graph (no host time between the launches)
+    side = torch.cuda.Stream()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(g, stream=side):
+            for ls in lsets:
+                build_tree(ls)
+    torch.cuda.synchronize()
+    g.replay()
     e0.record(stream)
-    for i in range(n_chain):
-        build_tree(lsets[i % 3])
+    for _ in range(max(1, n_chain // 3)):
+        g.replay()
     e1.record(stream)
     torch.cuda.synchronize()
-    us = e0.elapsed_time(e1) * 1e3 / n_chain
-    res["tree_build_c3_E10_K10_D4"] = hbm_entry(us, int(Bt * (1 + (D_ - 1) * K_) * V * 2))
-    res["tree_build_c3_E10_K10_D4"]["launches"] = "4 expansions + 3 selections + 1 pruning + 3 memsets, launched one by one"
+    res["tree_build_c3_E10_K10_D4"]["us_per_tree_batch_in_graph"] = round(
+        e0.elapsed_time(e1) * 1e3 / (3 * max(1, n_chain // 3)), 2)
+    us = timed(build_tree_calls)
+    res["tree_build_c3_E10_K10_D4_separate_calls"] = hbm_entry(us, tree_bytes)
+    res["tree_build_c3_E10_K10_D4_separate_calls"]["launches"] = "1 reset + 4 expansions + 3 selections + 1 pruning, launched one by one"
     return res
 
 
 # ----------------------------------------------------------------------------------
 # single-kernel cases: small, self-contained launch sets for a profiler capture or a quick timing
 #   python bench.py --case attn --workload 4 --kv-len 1472 --layers 2 --iters 3 [--attn-path 3] [--early-prefix]
-#   python bench.py --case gather|score|accept|argmax|gscore|mqscore --workload N [--layers n] [--iters k]
+#   python bench.py --case gather|score|accept|argmax|tree|gscore|mqscore --workload N [--layers n] [--iters k]
 # Each holds well under a few GB on the device and launches a handful of kernels, so that a
 # capture ends by itself.  Prints one JSON line.
 # ----------------------------------------------------------------------------------
@@ -904,6 +939,28 @@ def run_case(a):
         us = timed(lambda: tw.tree_base_argmax(logits, nn, res))
         by = sum(wl.n_nodes) * V * 2
         out.update({"us_per_launch": round(us, 2), "bytes": int(by), "gbs": round(by / us / 1e3, 1)})
+    elif a.case == "tree":
+        # the paper's tree settings (E = K = 10, D = 4, N_max = 60), one launch per level
+        V, E_, K_, D_, NMAX = 32000, 10, 10, 4, 60
+        cap = 1 + E_ + (D_ - 1) * K_ * E_
+        state = tw.TreeState(B, cap, dev)
+        levels = [torch.from_numpy(rng.standard_normal((B, 1 if l == 0 else K_, V), dtype=np.float32)).to(dev).to(torch.bfloat16)
+                  for l in range(D_)]
+        t_par = torch.zeros((B, 64), dtype=torch.int32, device=dev)
+        t_tok, t_n = torch.zeros_like(t_par), torch.zeros(B, dtype=torch.int32, device=dev)
+        root = torch.zeros((B, 1), dtype=torch.int32, device=dev)
+        nxt = torch.zeros((B, K_), dtype=torch.int32, device=dev)
+
+        def run():
+            src, hi = root, 1
+            for l in range(D_):
+                if l + 1 < D_:
+                    tw.tree_grow_level(levels[l], src, E_, hi, state, expand_node=nxt)
+                    src = nxt
+                else:
+                    tw.tree_grow_level(levels[l], src, E_, hi, state, n_max=NMAX, parent=t_par, draft_tok=t_tok, n_nodes=t_n)
+                hi += (1 if l == 0 else K_) * E_
+        out.update({"us_per_tree_batch": round(timed(run), 2), "launches_per_tree_batch": D_})
     print(json.dumps(out))
 
 
@@ -1035,7 +1092,7 @@ def main():
     ap.add_argument("--attn-path", type=int, default=0,
                     help="tree-attention kernel: 0 auto, 1 mma.sync, 2 tcgen05 (cluster splits), 3 tcgen05 persistent")
     ap.add_argument("--case", default=None,
-                    choices=["attn", "gather", "score", "prune", "accept", "argmax", "gscore", "mqscore"],
+                    choices=["attn", "gather", "score", "prune", "accept", "argmax", "tree", "gscore", "mqscore"],
                     help="run one small single-kernel case (for a profiler capture) instead of the benchmark")
     ap.add_argument("--kv-len", type=int, default=0, help="--case attn: cache length of every request")
     ap.add_argument("--layers", type=int, default=0, help="--case: layers resident / per call (0: the case's default)")

@@ -330,7 +330,9 @@ int32_t twig_set_launch_overlap(int32_t on);
  * logits to the lower token id.  Logits must not be NaN.
  *
  * Tree state of request b: node_tok / node_parent / node_score [batch, cap], node 0 the root, nodes in
- * creation order (level 1 at 1..E, each later level after it).  tree_reset writes the roots.
+ * creation order (level 1 at 1..E, each later level after it).  tree_reset writes the roots (node 0:
+ * token -1, parent -1, score 0); so does an expansion with level_base == 1, so a caller that starts
+ * every tree with such a call needs no tree_reset.
  *
  * tree_expand_level: row r of logits ([batch, rows, vocab] at (b*rows + r)*row_stride ELEMENTS, bf16 or
  *   fp32, rows 16-byte aligned) is the draft distribution after node src_node[b, r] (-1: unused row);
@@ -345,6 +347,15 @@ int32_t twig_set_launch_overlap(int32_t on);
  *   writes parent / draft_tok [batch, t_max] (root: parent -1, token -1; unused entries -1 / 0) and
  *   n_nodes[b]: the arrays tree_verify_attention and tree_accept_compact take.  kept_node (optional)
  *   [batch, t_max]: the state id of every kept node.  n_max <= t_max <= TWIG_MAX_NODES; cap <= 6144.
+ * tree_grow_level: one level in one launch: tree_expand_level, then, for every request, in the CTA
+ *   that finishes the request's last row, the step that consumes the new level
+ *   (level_hi = level_base + rows*n_children):
+ *     n_select > 0:  tree_select_expansion over level_base..level_hi-1 into expand_node [batch, n_select]
+ *                    (n_max, parent, draft_tok, n_nodes, kept_node, t_max are not used);
+ *     n_select == 0: tree_finalize with n_built = level_hi (expand_node is not used).
+ *   Same results as the two calls one after the other.  A tree of depth D is D calls.
+ *   ticket [batch] int32 (device): zero-filled by the caller before its first use, left zero by every
+ *   call; written only by these calls; one array per stream that builds trees concurrently.
  */
 twig_status tree_reset(int32_t *node_tok, int32_t *node_parent, float *node_score, int32_t cap,
                        int32_t batch, void *stream);
@@ -359,6 +370,12 @@ twig_status tree_finalize(const int32_t *node_tok, const int32_t *node_parent, c
                           int32_t cap, int32_t n_built, int32_t n_max, int32_t *parent, int32_t *draft_tok,
                           int32_t *n_nodes, int32_t *kept_node, int32_t t_max, int32_t batch,
                           int32_t *dev_status, void *stream);
+twig_status tree_grow_level(const void *logits, int32_t logits_fp32, int64_t row_stride, int32_t vocab,
+                            int32_t rows, const int32_t *src_node, int32_t n_children, int32_t level_base,
+                            int32_t *node_tok, int32_t *node_parent, float *node_score, int32_t cap,
+                            int32_t batch, int32_t n_select, int32_t *expand_node, int32_t n_max,
+                            int32_t *parent, int32_t *draft_tok, int32_t *n_nodes, int32_t *kept_node,
+                            int32_t t_max, int32_t *ticket, int32_t *dev_status, void *stream);
 
 /* ---- Chain drafting with early exit (sequence self-speculative decoding) ------
  * Appendix A, "Self-speculative decoding", and Algorithm 1's draft loop: in every iteration the draft

@@ -615,23 +615,6 @@ static twig_status check_score_args(const ScoreArgs &a, const void *ws, size_t w
   return TWIG_OK;
 }
 
-// Launch configuration with programmatic stream serialization: the kernel may be scheduled while its
-// predecessor in the stream drains; it waits on the device before it reads that kernel's output.
-struct PdlLaunch {
-  cudaLaunchConfig_t cfg = {};
-  cudaLaunchAttribute attr[1];
-  PdlLaunch(dim3 grid, dim3 block, size_t smem, cudaStream_t st) {
-    cfg.gridDim = grid;
-    cfg.blockDim = block;
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = st;
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = launch_overlap_enabled() ? 1 : 0;
-  }
-};
-
 static twig_status launch_logits(const ScoreArgs &a, int *dev_status, void *ws, cudaStream_t st) {
   const float scale = a.softmax_scale != 0.f ? a.softmax_scale : 1.f / sqrtf((float)a.head_dim);
   dim3 grid((a.k_max_len + kScoreKeysPerCta - 1) / kScoreKeysPerCta, a.n_kv_heads, a.batch);

@@ -74,6 +74,23 @@ inline KvViewMut view_of_mut(const twig_kv *kv) {
 // stream may be scheduled while this one drains; it waits on the device before reading anything).
 bool launch_overlap_enabled();
 
+// Launch configuration with programmatic stream serialization: the kernel may be scheduled while its
+// predecessor in the stream drains; it waits on the device before it reads that kernel's output.
+struct PdlLaunch {
+  cudaLaunchConfig_t cfg = {};
+  cudaLaunchAttribute attr[1];
+  PdlLaunch(dim3 grid, dim3 block, size_t smem, cudaStream_t st) {
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = launch_overlap_enabled() ? 1 : 0;
+  }
+};
+
 inline twig_status launch_status() {
   return cudaGetLastError() == cudaSuccess ? TWIG_OK : TWIG_ERR_CUDA;
 }

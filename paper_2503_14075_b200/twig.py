@@ -27,7 +27,7 @@ DEV_OK, DEV_BAD_LAYOUT, DEV_BAD_KEEP, DEV_BAD_INDEX, DEV_BAD_TREE, DEV_OVERFLOW,
 MAX_NODES, MAX_VISUAL, MAX_BATCH = 64, 16384, 4096
 
 EXPORTS = ["twig_status_str", "twig_set_launch_overlap", "twig_workspace_bytes", "tree_attention_workspace_bytes", "tree_verify_attention_ex", "ttp_score", "ttp_score_gated", "ttp_multiquery_workspace_bytes", "ttp_score_multiquery", "ttp_score_noalloc", "ttp_topk", "ttp_compact", "ttp_compact_rows",
-           "ttp_score_topk_compact", "tree_verify_attention", "tree_reset", "tree_expand_level", "tree_select_expansion", "tree_finalize", "tree_base_argmax", "tree_accept_compact", "chain_draft_reset", "chain_draft_step"]
+           "ttp_score_topk_compact", "tree_verify_attention", "tree_reset", "tree_expand_level", "tree_select_expansion", "tree_finalize", "tree_grow_level", "tree_base_argmax", "tree_accept_compact", "chain_draft_reset", "chain_draft_step"]
 
 
 class TwigError(RuntimeError):
@@ -117,6 +117,9 @@ _lib.tree_select_expansion.restype = C.c_int
 _lib.tree_select_expansion.argtypes = [_vp, _i32, _i32, _i32, _i32, _vp, _i32, _vp, _vp]
 _lib.tree_finalize.restype = C.c_int
 _lib.tree_finalize.argtypes = [_vp, _vp, _vp, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _i32, _i32, _vp, _vp]
+_lib.tree_grow_level.restype = C.c_int
+_lib.tree_grow_level.argtypes = [_vp, _i32, _i64, _i32, _i32, _vp, _i32, _i32, _vp, _vp, _vp, _i32, _i32,
+                                 _i32, _vp, _i32, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _vp]
 _lib.tree_base_argmax.restype = C.c_int
 _lib.tree_base_argmax.argtypes = [_vp, _i32, _i64, _i32, _vp, _i32, _i32, _vp, _vp, _vp]
 _lib.chain_draft_reset.restype = C.c_int
@@ -281,6 +284,7 @@ class TreeState:
         self.tok = torch.empty((batch, cap), dtype=torch.int32, device=device)
         self.parent = torch.empty((batch, cap), dtype=torch.int32, device=device)
         self.score = torch.empty((batch, cap), dtype=torch.float32, device=device)
+        self.ticket = torch.zeros((batch,), dtype=torch.int32, device=device)    # tree_grow_level's counters
 
 
 def tree_reset(state: TreeState, stream=None):
@@ -308,6 +312,20 @@ def tree_finalize(state: TreeState, n_built, n_max, parent, draft_tok, n_nodes, 
     _check(_lib.tree_finalize(_p(state.tok), _p(state.parent), _p(state.score), state.cap, n_built, n_max, _p(parent),
                               _p(draft_tok), _p(n_nodes), _p(kept_node), parent.shape[1], state.batch, _p(dev_status),
                               _stream(stream)))
+
+
+def tree_grow_level(logits, src_node, n_children, level_base, state: TreeState, expand_node=None, n_max=0, parent=None,
+                    draft_tok=None, n_nodes=None, kept_node=None, dev_status=None, stream=None):
+    """One level in one launch: the expansion, then either the next level's expansion nodes
+    (expand_node [B, K] given) or the final pruning to n_max nodes (parent, draft_tok, n_nodes given)."""
+    B, rows, V = logits.shape
+    assert logits.stride(2) == 1 and logits.stride(0) == rows * logits.stride(1)
+    n_select = expand_node.shape[1] if expand_node is not None else 0
+    t_max = parent.shape[1] if parent is not None else 0
+    _check(_lib.tree_grow_level(_p(logits), 1 if logits.dtype == torch.float32 else 0, logits.stride(1), V, rows,
+                                _p(src_node), n_children, level_base, _p(state.tok), _p(state.parent), _p(state.score),
+                                state.cap, B, n_select, _p(expand_node), n_max, _p(parent), _p(draft_tok), _p(n_nodes),
+                                _p(kept_node), t_max, _p(state.ticket), _p(dev_status), _stream(stream)))
 
 
 def tree_base_argmax(logits, n_nodes, base_argmax, dev_status=None, stream=None):

@@ -49,10 +49,47 @@ def gpu_tree(tw, level_logits_dev, E, K, n_max, t_max):
             st.score.cpu().numpy())
 
 
+def gpu_tree_grown(tw, level_logits_dev, E, K, n_max, t_max, repeats=2):
+    """The same trees with one launch per level (tree_grow_level), no tree_reset, and the state reused
+    `repeats` times (the per-request tickets must come back to zero)."""
+    B = level_logits_dev[0].shape[0]
+    D = len(level_logits_dev)
+    cap = 1 + E + (D - 1) * K * E
+    st = tw.TreeState(B, cap, DEV)
+    status = torch.zeros(B, dtype=torch.int32, device=DEV)
+    for _ in range(repeats):
+        st.tok.fill_(-77)
+        st.parent.fill_(-77)
+        st.score.fill_(float("nan"))
+        parent = torch.full((B, t_max), -9, dtype=torch.int32, device=DEV)
+        tok = torch.full((B, t_max), -9, dtype=torch.int32, device=DEV)
+        n_nodes = torch.full((B,), -9, dtype=torch.int32, device=DEV)
+        kept = torch.full((B, t_max), -9, dtype=torch.int32, device=DEV)
+        src = torch.zeros((B, 1), dtype=torch.int32, device=DEV)
+        hi = 1
+        for l in range(D):
+            if l + 1 < D:
+                nxt = torch.full((B, K), -5, dtype=torch.int32, device=DEV)
+                tw.tree_grow_level(level_logits_dev[l], src, E, hi, st, expand_node=nxt, dev_status=status)
+                src = nxt
+            else:
+                tw.tree_grow_level(level_logits_dev[l], src, E, hi, st, n_max=n_max, parent=parent, draft_tok=tok,
+                                   n_nodes=n_nodes, kept_node=kept, dev_status=status)
+            hi += (1 if l == 0 else K) * E
+        torch.cuda.synchronize()
+        assert not st.ticket.any()
+    return (parent.cpu().numpy(), tok.cpu().numpy(), n_nodes.cpu().numpy(), kept.cpu().numpy(), status.cpu().numpy(),
+            st.score.cpu().numpy())
+
+
+BUILDERS = {"calls": gpu_tree, "one-launch-per-level": gpu_tree_grown}
+
+
+@pytest.mark.parametrize("builder", list(BUILDERS))
 @pytest.mark.parametrize("dtype", ["bf16", "fp32"])
 @pytest.mark.parametrize("cfg", [(10, 10, 4, 60, 64, 32000), (3, 2, 3, 7, 8, 1003), (16, 4, 2, 64, 64, 4096), (1, 1, 5, 6, 6, 77)],
                          ids=["paper-default", "small-ragged", "wide", "chain"])
-def test_token_tree_matches_oracle(tw, cfg, dtype):
+def test_token_tree_matches_oracle(tw, cfg, dtype, builder):
     E, K, D, n_max, t_max, V = cfg
     B = 3
     rng = synth.rng_for(7, 21)
@@ -72,7 +109,7 @@ def test_token_tree_matches_oracle(tw, cfg, dtype):
             padded[..., :V] = x
             dev.append(torch.from_numpy(padded).to(DEV)[..., :V])
             host.append(x.astype(np.float64))
-    parent, tok, n_nodes, kept, status, score = gpu_tree(tw, dev, E, K, n_max, t_max)
+    parent, tok, n_nodes, kept, status, score = BUILDERS[builder](tw, dev, E, K, n_max, t_max)
     assert not status.any()
     for b in range(B):
         p_o, t_o, s_o, keep_o, (fp, ft, fs) = O.build_token_tree([h[b] for h in host], E, K, n_max)
@@ -86,14 +123,15 @@ def test_token_tree_matches_oracle(tw, cfg, dtype):
         assert np.allclose(score[b, :len(fs)], fs, rtol=0, atol=2e-4 * D)
 
 
+@pytest.mark.parametrize("builder", list(BUILDERS))
 @pytest.mark.parametrize("V", [64, 4096])
-def test_token_tree_ties(tw, V):
+def test_token_tree_ties(tw, V, builder):
     """Equal logits go to the lower token id, equal scores to the lower node id (exact ties: rows that are
     bit-identical give bit-identical scores).  With 4096 equal logits the kernel's short candidate list
     overflows and the selection runs over the whole row."""
     E, K, D, n_max, t_max = 2, 2, 2, 4, 8
     flat = [torch.zeros((1, 1, V), dtype=torch.float32, device=DEV), torch.zeros((1, K, V), dtype=torch.float32, device=DEV)]
-    parent, tok, n_nodes, kept, status, _ = gpu_tree(tw, flat, E, K, n_max, t_max)
+    parent, tok, n_nodes, kept, status, _ = BUILDERS[builder](tw, flat, E, K, n_max, t_max)
     p_o, t_o, _, keep_o, _ = O.build_token_tree([np.zeros((1, V)), np.zeros((K, V))], E, K, n_max)
     assert not status.any() and n_nodes[0] == 4
     assert kept[0, :4].tolist() == keep_o.tolist() == [0, 1, 2, 3]
@@ -199,6 +237,33 @@ def test_draft_verify_accept_chain(tw):
     new_len = O.accept_compact(tkv[0], tkv[1], ok_, ov_, kv_len, paths)
     assert np.array_equal(kvl.cpu().numpy(), new_len)
     assert np.array_equal(host_bits(ck), ok_) and np.array_equal(host_bits(cv), ov_)
+
+
+def test_unused_expansion_rows_are_never_selected(tw):
+    """A row with src_node = -1 leaves children with score -inf, which the selection in the same launch
+    ranks after every real node."""
+    B, V, E, K = 2, 300, 3, 3
+    rng = synth.rng_for(7, 24)
+    st = tw.TreeState(B, 1 + E + K * E, DEV)
+    st.score.fill_(7.0)
+    status = torch.zeros(B, dtype=torch.int32, device=DEV)
+    lv1 = torch.from_numpy(rng.standard_normal((B, 1, V)).astype(np.float32)).to(DEV)
+    lv2 = torch.from_numpy(rng.standard_normal((B, K, V)).astype(np.float32)).to(DEV)
+    src = torch.zeros((B, 1), dtype=torch.int32, device=DEV)
+    nxt = torch.zeros((B, K), dtype=torch.int32, device=DEV)
+    tw.tree_grow_level(lv1, src, E, 1, st, expand_node=nxt, dev_status=status)
+    torch.cuda.synchronize()
+    assert nxt.cpu().tolist() == [[1, 2, 3]] * B
+    nxt[1, 1] = -1                                   # request 1 expands only nodes 1 and 3
+    nxt2 = torch.zeros((B, 2 * E), dtype=torch.int32, device=DEV)
+    tw.tree_grow_level(lv2, nxt, E, 1 + E, st, expand_node=nxt2, dev_status=status)
+    torch.cuda.synchronize()
+    score = st.score.cpu().numpy()
+    lo = 1 + E
+    assert np.all(np.isneginf(score[1, lo + E:lo + 2 * E])) and np.all(np.isfinite(score[0, lo:lo + K * E]))
+    assert np.all(np.isfinite(score[1, lo:lo + E])) and np.all(np.isfinite(score[1, lo + 2 * E:lo + 3 * E]))
+    assert nxt2.cpu().numpy()[1].tolist() == list(range(lo, lo + E)) + list(range(lo + 2 * E, lo + 3 * E))
+    assert not status.cpu().numpy().any() and not st.ticket.any()
 
 
 def test_next_row_entry_points_report_bad_arguments(tw):
