@@ -36,12 +36,13 @@ ttp_logits_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__re
                   long long ksb, long long ksh, long long ksp, int k_max_len,
                   const int *__restrict__ prefix_len, const int *__restrict__ vis_start,
                   const int *__restrict__ n_vis, int n_q_heads, int group, int norm_scope,
-                  float scale, float *__restrict__ logits, int lstride, int m_max,
-                  int *dev_status) {
+                  float scale, float *__restrict__ logits, int lstride, float2 *__restrict__ stats,
+                  int n_chunks, int m_max, int *dev_status) {
   constexpr int LPK = D / 8;               // lanes per key row
   constexpr int KPP = kScoreThreads / LPK; // keys per pass of the CTA
   constexpr int PASSES = kScoreKeysPerCta / KPP;
   __shared__ float qs[kMaxGroup * D];
+  __shared__ float s_log[kMaxGroup][kScoreKeysPerCta];
 
   grid_dependency_sync();
   const int b = blockIdx.z, hk = blockIdx.y;
@@ -106,15 +107,42 @@ ttp_logits_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__re
 #pragma unroll
       for (int o = LPK / 2; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
       const int j = j0 + p * KPP + slot;
-      if (sub == 0 && j >= lo && j < hi) lrow[j] = acc;
+      if (sub == 0) {
+        const bool in = j >= lo && j < hi;
+        if (in) lrow[j] = acc;
+        s_log[g][p * KPP + slot] = in ? acc : -INFINITY;
+      }
     }
+  }
+  __syncthreads();
+  // softmax statistics of this CTA's keys (at least one is in scope), one warp per head: the maximum
+  // and the sum of exponentials relative to it; the next stage merges the chunks of a head
+  const int lane = threadIdx.x & 31;
+  for (int g = threadIdx.x >> 5; g < group; g += kScoreThreads / 32) {
+    float v[kScoreKeysPerCta / 32];
+    float mx = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < kScoreKeysPerCta / 32; ++i) {
+      v[i] = s_log[g][lane + 32 * i];
+      mx = fmaxf(mx, v[i]);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    float sum = 0.f;
+#pragma unroll
+    for (int i = 0; i < kScoreKeysPerCta / 32; ++i) sum += v[i] > -INFINITY ? expf(v[i] - mx) : 0.f;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+    if (lane == 0) stats[((long long)b * n_q_heads + hk * group + g) * n_chunks + blockIdx.x] = make_float2(mx, sum);
   }
 }
 
 // ---------------------------------------------------------------------------
 // Stage 1b + 2: softmax per head, mean over heads -> scores; then exact TopR.
-// One CTA of 1024 threads per request.  mode bit 0: compute scores from the
-// logits; bit 1: select.  Without bit 0 the scores are read from `scores`.
+// mode bit 0: compute scores from the logits; bit 1: select.  Without bit 0 the scores are read from
+// `scores`.  With the selection: one CTA of 1024 threads per request.  Scores alone: grid
+// (slices, batch), any CTA size, every CTA takes a slice of the request's visual tokens (the
+// per-head statistics are merged from the logits stage's per-chunk partials by every CTA: cheap).
 // ---------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t order_key(float x) {
   const uint32_t u = __float_as_uint(x);
@@ -150,7 +178,8 @@ __device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t x, uint32_t *w
 }
 
 __global__ void __launch_bounds__(kTopkThreads)
-ttp_finalize_topk_kernel(const float *__restrict__ logits, int lstride, int n_q_heads, int k_max_len,
+ttp_finalize_topk_kernel(const float *__restrict__ logits, int lstride, const float2 *__restrict__ stats,
+                         int n_chunks, int n_q_heads, int k_max_len,
                          const int *__restrict__ prefix_len, const int *__restrict__ vis_start,
                          const int *__restrict__ n_vis, const int *__restrict__ keep, int norm_scope,
                          float *__restrict__ scores, int m_max, int *__restrict__ kept_idx, int r_max,
@@ -165,48 +194,56 @@ ttp_finalize_topk_kernel(const float *__restrict__ logits, int lstride, int n_q_
   // selection; this kernel itself reads its predecessor's output from here on
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   asm volatile("griddepcontrol.wait;" ::: "memory");
-  const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int b = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int nt = blockDim.x;
   const int nv = n_vis[b];
   float *sc = scores + (long long)b * m_max;
 
   if (mode & 1) {
     const int lp = prefix_len[b], vs = vis_start[b];
     if (!layout_ok(lp, vs, nv, k_max_len, m_max)) {
-      if (tid == 0) flag_status(dev_status, b, TWIG_DEV_BAD_LAYOUT);
+      if (tid == 0 && blockIdx.x == 0) flag_status(dev_status, b, TWIG_DEV_BAD_LAYOUT);
       return;
     }
     const int lo = norm_scope ? vs : 0, hi = norm_scope ? vs + nv : lp;
-    for (int h = warp; h < n_q_heads; h += kTopkThreads / 32) {
-      const float *z = logits + ((long long)b * n_q_heads + h) * lstride;
-      // up to 32 x kStatRegs logits of the row stay in registers (all loads in flight at once, one
-      // pass for the maximum and the sum); longer rows take the two-pass loop for the rest
-      constexpr int kStatRegs = 24;
-      float v[kStatRegs];
-      float mx = -INFINITY;
+    // chunks of the logits stage that hold keys of the scope (none for an empty scope)
+    const int c_lo = lo / kScoreKeysPerCta, c_hi = hi > lo ? (hi - 1) / kScoreKeysPerCta : c_lo - 1;
+    // a lane takes the chunks c_lo + lane, + 32, ... of a head; a warp has four heads' partials in
+    // flight (for scopes of up to 4096 keys that is every load of the merge in one round trip)
+    constexpr int kHeadsInFlight = 4;
+    for (int h0 = warp * kHeadsInFlight; h0 < n_q_heads; h0 += (nt / 32) * kHeadsInFlight) {
+      float2 part[kHeadsInFlight];
 #pragma unroll
-      for (int i = 0; i < kStatRegs; ++i) {
-        const int j = lo + lane + 32 * i;
-        v[i] = j < hi ? z[j] : -INFINITY;
+      for (int i = 0; i < kHeadsInFlight; ++i) {
+        const int h = h0 + i, c = c_lo + lane;
+        part[i] = h < n_q_heads && c <= c_hi ? stats[((long long)b * n_q_heads + h) * n_chunks + c]
+                                             : make_float2(-INFINITY, 0.f);
       }
 #pragma unroll
-      for (int i = 0; i < kStatRegs; ++i) mx = fmaxf(mx, v[i]);
-      for (int j = lo + lane + 32 * kStatRegs; j < hi; j += 32) mx = fmaxf(mx, z[j]);
+      for (int i = 0; i < kHeadsInFlight; ++i) {
+        const int h = h0 + i;
+        if (h >= n_q_heads) break;                   // (uniform in the warp)
+        for (int c = c_lo + lane + 32; c <= c_hi; c += 32) {
+          const float2 more = stats[((long long)b * n_q_heads + h) * n_chunks + c];
+          const float m2 = fmaxf(part[i].x, more.x);   // (finite: a chunk of the scope holds a key)
+          part[i].y = part[i].y * expf(part[i].x - m2) + more.y * expf(more.x - m2);
+          part[i].x = m2;
+        }
+        float mx = part[i].x;
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-      float sum = 0.f;
+        for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        float sum = part[i].x > -INFINITY ? part[i].y * expf(part[i].x - mx) : 0.f;
 #pragma unroll
-      for (int i = 0; i < kStatRegs; ++i) sum += v[i] > -INFINITY ? expf(v[i] - mx) : 0.f;   // (nothing past the row's end)
-      for (int j = lo + lane + 32 * kStatRegs; j < hi; j += 32) sum += expf(z[j] - mx);
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-      if (lane == 0) {
-        h_max[h] = mx;
-        h_inv[h] = 1.f / sum;
+        for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+        if (lane == 0) {
+          h_max[h] = mx;
+          h_inv[h] = 1.f / sum;
+        }
       }
     }
     __syncthreads();
     const float inv_h = 1.f / (float)n_q_heads;
-    for (int m = tid; m < m_max; m += kTopkThreads) {
+    for (int m = blockIdx.x * nt + tid; m < m_max; m += gridDim.x * nt) {
       float acc = 0.f;
       if (m < nv) {
         const float *z = logits + (long long)b * n_q_heads * lstride + vs + m;
@@ -229,7 +266,7 @@ ttp_finalize_topk_kernel(const float *__restrict__ logits, int lstride, int n_q_
         acc *= inv_h;
       }
       sc[m] = acc;
-      keys[m] = order_key(acc);
+      if (mode & 2) keys[m] = order_key(acc);
     }
   } else {
     if (nv < 0 || nv > m_max) {
@@ -582,8 +619,14 @@ row_gather_kernel(const unsigned char *__restrict__ src, unsigned char *__restri
 // ---------------------------------------------------------------------------
 static inline int logits_stride(int k_max_len) { return (k_max_len + 3) & ~3; }
 
-size_t score_workspace_bytes(int batch, int n_q_heads, int max_len) {
+static inline int score_chunks(int k_max_len) { return (k_max_len + kScoreKeysPerCta - 1) / kScoreKeysPerCta; }
+
+// scaled logits [batch, heads, stride], then the per-chunk softmax statistics [batch, heads, chunks]
+static inline size_t logits_bytes(int batch, int n_q_heads, int max_len) {
   return (size_t)batch * n_q_heads * logits_stride(max_len) * sizeof(float);
+}
+size_t score_workspace_bytes(int batch, int n_q_heads, int max_len) {
+  return logits_bytes(batch, n_q_heads, max_len) + (size_t)batch * n_q_heads * score_chunks(max_len) * sizeof(float2);
 }
 
 struct ScoreArgs {
@@ -627,10 +670,13 @@ static twig_status launch_logits(const ScoreArgs &a, int *dev_status, void *ws, 
   PdlLaunch L(grid, dim3(kScoreThreads), 0, st);
   const long long ksb = a.ksb, ksh = a.ksh, ksp = a.ksp;
   float *lg = static_cast<float *>(ws);
+  float2 *stats = reinterpret_cast<float2 *>(static_cast<unsigned char *>(ws) + logits_bytes(a.batch, a.n_q_heads, a.k_max_len));
+  const int n_chunks = score_chunks(a.k_max_len);
   cudaError_t err;
 #define TWIG_LOGITS(D_, G_)                                                                                          \
   err = cudaLaunchKernelEx(&L.cfg, ttp_logits_kernel<D_, G_>, q, k, qg, kg, ksb, ksh, ksp, a.k_max_len, a.prefix_len, \
-                           a.vis_start, a.n_vis, a.n_q_heads, group, a.norm_scope, scale, lg, ls, a.m_max, dev_status)
+                           a.vis_start, a.n_vis, a.n_q_heads, group, a.norm_scope, scale, lg, ls, stats, n_chunks,    \
+                           a.m_max, dev_status)
   if (a.head_dim == 128) {
     if (qg) TWIG_LOGITS(128, true); else TWIG_LOGITS(128, false);
   } else {
@@ -644,18 +690,25 @@ static twig_status launch_finalize(const float *logits, const ScoreArgs &a, cons
                                    int *kept_idx, int r_max, int *dev_status, int mode,
                                    cudaStream_t st) {
   static bool attr_set = false;
-  const size_t smem = (size_t)a.m_max * sizeof(uint32_t);
+  const bool select = mode & 2;
+  const size_t smem = select ? (size_t)a.m_max * sizeof(uint32_t) : 0;
   if (smem > 48 * 1024 && !attr_set) {
     if (cudaFuncSetAttribute(ttp_finalize_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              TWIG_MAX_VISUAL * (int)sizeof(uint32_t)) != cudaSuccess)
       return TWIG_ERR_CUDA;
     attr_set = true;
   }
-  PdlLaunch L(dim3(a.batch), dim3(kTopkThreads), smem, st);
+  // the selection needs a request's scores in one CTA; scores alone are spread over slices of 256 tokens
+  constexpr int kSliceThreads = 256;
+  const dim3 grid = select ? dim3(1, a.batch) : dim3((a.m_max + kSliceThreads - 1) / kSliceThreads, a.batch);
+  PdlLaunch L(grid, dim3(select ? kTopkThreads : kSliceThreads), smem, st);
   const int ls = logits_stride(a.k_max_len);
-  const cudaError_t err = cudaLaunchKernelEx(&L.cfg, ttp_finalize_topk_kernel, logits, ls, a.n_q_heads, a.k_max_len,
-                                             a.prefix_len, a.vis_start, a.n_vis, keep, a.norm_scope, a.scores, a.m_max,
-                                             kept_idx, r_max, dev_status, mode);
+  const float2 *stats = logits ? reinterpret_cast<const float2 *>(reinterpret_cast<const unsigned char *>(logits) +
+                                                                  logits_bytes(a.batch, a.n_q_heads, a.k_max_len))
+                               : nullptr;
+  const cudaError_t err = cudaLaunchKernelEx(&L.cfg, ttp_finalize_topk_kernel, logits, ls, stats, score_chunks(a.k_max_len),
+                                             a.n_q_heads, a.k_max_len, a.prefix_len, a.vis_start, a.n_vis, keep,
+                                             a.norm_scope, a.scores, a.m_max, kept_idx, r_max, dev_status, mode);
   return err == cudaSuccess ? TWIG_OK : TWIG_ERR_CUDA;
 }
 
