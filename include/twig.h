@@ -129,10 +129,14 @@ twig_status ttp_score_gated(const void *twig_q, const void *q_gate, const void *
  *   q_text  [batch, n_q_heads, n_text_max, head_dim] bf16 contiguous; rows i >= N_b are ignored.
  *           N_b > n_text_max is reported as TWIG_DEV_BAD_LAYOUT (scores of that request: 0)
  *   twig_k, strides, k_max_len, prefix_len, vis_start, n_vis, scores, m_max: as in ttp_score
- * Scratch: ttp_multiquery_workspace_bytes(batch, n_q_heads, n_text_max, m_max).  The result is
- * reproducible from run to run (partial sums are added in a fixed order).
+ * Scratch: ttp_multiquery_workspace_bytes(batch, n_q_heads, n_text_max, m_max, k_max_len) bytes (it
+ * holds one fp16 per (head, text row, key) between the kernels of the call: 2 * batch * n_q_heads *
+ * n_text_max' * k_max_len' bytes plus statistics, the primes rounded up to 64 rows and 128 keys);
+ * no initial contents are assumed.  softmax_scale must be positive (0: 1/sqrt(head_dim)).  The
+ * result is reproducible from run to run (partial sums are added in a fixed order).
  */
-size_t ttp_multiquery_workspace_bytes(int32_t batch, int32_t n_q_heads, int32_t n_text_max, int32_t m_max);
+size_t ttp_multiquery_workspace_bytes(int32_t batch, int32_t n_q_heads, int32_t n_text_max, int32_t m_max,
+                                      int32_t k_max_len);
 twig_status ttp_score_multiquery(const void *q_text, int32_t n_text_max, const void *twig_k,
                                  int64_t k_stride_batch, int64_t k_stride_head, int64_t k_stride_pos,
                                  int32_t k_max_len, const int32_t *prefix_len, const int32_t *vis_start,

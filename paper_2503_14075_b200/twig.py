@@ -71,7 +71,7 @@ _lib.ttp_score_gated.restype = C.c_int
 _lib.ttp_score_gated.argtypes = [_vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _vp, _vp, _vp, _i32, _i32, _i32, _i32,
                                  _i32, _f32, _vp, _i32, _vp, _vp, _sz, _vp]
 _lib.ttp_multiquery_workspace_bytes.restype = _sz
-_lib.ttp_multiquery_workspace_bytes.argtypes = [_i32] * 4
+_lib.ttp_multiquery_workspace_bytes.argtypes = [_i32] * 5
 _lib.ttp_score_multiquery.restype = C.c_int
 _lib.ttp_score_multiquery.argtypes = [_vp, _i32, _vp, _i64, _i64, _i64, _i32, _vp, _vp, _vp, _i32, _i32, _i32, _i32,
                                       _f32, _vp, _i32, _vp, _vp, _sz, _vp]
@@ -185,8 +185,8 @@ def ttp_score_gated(twig_q, q_gate, twig_k, k_gate, prefix_len, vis_start, n_vis
                                 _p(dev_status), _p(ws), ws.numel() * ws.element_size(), _stream(stream)))
 
 
-def ttp_multiquery_workspace_bytes(batch, n_q_heads, n_text_max, m_max):
-    return int(_lib.ttp_multiquery_workspace_bytes(batch, n_q_heads, n_text_max, m_max))
+def ttp_multiquery_workspace_bytes(batch, n_q_heads, n_text_max, m_max, k_max_len):
+    return int(_lib.ttp_multiquery_workspace_bytes(batch, n_q_heads, n_text_max, m_max, k_max_len))
 
 
 def ttp_score_multiquery(q_text, twig_k, prefix_len, vis_start, n_vis, scores, ws, softmax_scale=0.0,

@@ -306,7 +306,7 @@ def test_next_row_entry_points_report_bad_arguments(tw):
     qt = torch.zeros((1, 4, 2, 128), dtype=torch.bfloat16, device=DEV)
     k = torch.zeros((1, 4, 32, 128), dtype=torch.bfloat16, device=DEV)
     sc = torch.full((1, 8), -1.0, dtype=torch.float32, device=DEV)
-    ws = torch.zeros(tw.ttp_multiquery_workspace_bytes(1, 4, 2, 8), dtype=torch.uint8, device=DEV)
+    ws = torch.zeros(tw.ttp_multiquery_workspace_bytes(1, 4, 2, 8, 32), dtype=torch.uint8, device=DEV)
     st1 = torch.zeros(1, dtype=torch.int32, device=DEV)
     tw.ttp_score_multiquery(qt, k, dev_i32([20]), dev_i32([4]), dev_i32([8]), sc, ws, dev_status=st1)   # 8 text tokens > 2
     torch.cuda.synchronize()

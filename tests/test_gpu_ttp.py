@@ -114,7 +114,7 @@ def test_multiquery_scores_match_oracle(tw, name, gain_mult):
         qt[b, :, n_text[b]:, :] = 0x7FC1                # NaN past the last text token
     m_max = max(1, int(pre["n_vis"].max()))
     scores = torch.full((B, m_max), -1.0, dtype=torch.float32, device=DEV)
-    ws = torch.full((tw.ttp_multiquery_workspace_bytes(B, Hq, n_max, m_max) // 4,), float("nan"), dtype=torch.float32,
+    ws = torch.full((tw.ttp_multiquery_workspace_bytes(B, Hq, n_max, m_max, pre["twig_k"].shape[2]) // 4,), float("nan"), dtype=torch.float32,
                     device=DEV)
     status = torch.zeros(B, dtype=torch.int32, device=DEV)
     args = (dev_bf16(qt), dev_bf16(pre["twig_k"]), dev_i32(pre["prefix_len"]), dev_i32(pre["vis_start"]),
