@@ -12,6 +12,7 @@ namespace twig {
 
 constexpr int kScoreThreads = 256;
 constexpr int kScoreKeysPerCta = 128;
+constexpr int kScoreWarps = kScoreThreads / 32;   // every warp of the logits stage writes one partial (max, sum) per head
 constexpr int kMaxGroup = 16;   // query heads per kv head
 constexpr int kMaxQHeads = 128;
 constexpr int kTopkThreads = 1024;
@@ -37,12 +38,11 @@ ttp_logits_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__re
                   const int *__restrict__ prefix_len, const int *__restrict__ vis_start,
                   const int *__restrict__ n_vis, int n_q_heads, int group, int norm_scope,
                   float scale, float *__restrict__ logits, int lstride, float2 *__restrict__ stats,
-                  int n_chunks, int m_max, int *dev_status) {
+                  int n_parts, int m_max, int *dev_status) {
   constexpr int LPK = D / 8;               // lanes per key row
   constexpr int KPP = kScoreThreads / LPK; // keys per pass of the CTA
   constexpr int PASSES = kScoreKeysPerCta / KPP;
   __shared__ float qs[kMaxGroup * D];
-  __shared__ float s_log[kMaxGroup][kScoreKeysPerCta];
 
   grid_dependency_sync();
   const int b = blockIdx.z, hk = blockIdx.y;
@@ -94,6 +94,7 @@ ttp_logits_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__re
     const float4 qa = *reinterpret_cast<const float4 *>(qs + g * D + sub * 8);
     const float4 qb = *reinterpret_cast<const float4 *>(qs + g * D + sub * 8 + 4);
     float *lrow = logits + ((long long)b * n_q_heads + hk * group + g) * lstride;
+    float a[PASSES];                       // the warp's logits of this head, -inf outside the scope
 #pragma unroll
     for (int p = 0; p < PASSES; ++p) {
       float acc = kf[p][0] * qa.x;
@@ -107,33 +108,26 @@ ttp_logits_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__re
 #pragma unroll
       for (int o = LPK / 2; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
       const int j = j0 + p * KPP + slot;
-      if (sub == 0) {
-        const bool in = j >= lo && j < hi;
-        if (in) lrow[j] = acc;
-        s_log[g][p * KPP + slot] = in ? acc : -INFINITY;
-      }
+      const bool in = j >= lo && j < hi;
+      if (sub == 0 && in) lrow[j] = acc;
+      a[p] = in ? acc : -INFINITY;
     }
-  }
-  __syncthreads();
-  // softmax statistics of this CTA's keys (at least one is in scope), one warp per head: the maximum
-  // and the sum of exponentials relative to it; the next stage merges the chunks of a head
-  const int lane = threadIdx.x & 31;
-  for (int g = threadIdx.x >> 5; g < group; g += kScoreThreads / 32) {
-    float v[kScoreKeysPerCta / 32];
-    float mx = -INFINITY;
+    // softmax statistics of the warp's keys (32 / LPK key rows per pass): the maximum and the sum of
+    // exponentials relative to it, every lane of a row's group holding the row's logit; the next stage
+    // merges the partials of a head.  No barrier and no tail: the CTA is done when its warps are.
+    float mx = a[0];
 #pragma unroll
-    for (int i = 0; i < kScoreKeysPerCta / 32; ++i) {
-      v[i] = s_log[g][lane + 32 * i];
-      mx = fmaxf(mx, v[i]);
-    }
+    for (int p = 1; p < PASSES; ++p) mx = fmaxf(mx, a[p]);
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    for (int o = 16; o >= LPK; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
     float sum = 0.f;
 #pragma unroll
-    for (int i = 0; i < kScoreKeysPerCta / 32; ++i) sum += v[i] > -INFINITY ? expf(v[i] - mx) : 0.f;
+    for (int p = 0; p < PASSES; ++p) sum += a[p] > -INFINITY ? expf(a[p] - mx) : 0.f;
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-    if (lane == 0) stats[((long long)b * n_q_heads + hk * group + g) * n_chunks + blockIdx.x] = make_float2(mx, sum);
+    for (int o = 16; o >= LPK; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+    if ((threadIdx.x & 31) == 0)
+      stats[((long long)b * n_q_heads + hk * group + g) * n_parts + blockIdx.x * kScoreWarps + (threadIdx.x >> 5)] =
+          make_float2(mx, sum);
   }
 }
 
@@ -142,7 +136,7 @@ ttp_logits_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__re
 // mode bit 0: compute scores from the logits; bit 1: select.  Without bit 0 the scores are read from
 // `scores`.  With the selection: one CTA of 1024 threads per request.  Scores alone: grid
 // (slices, batch), any CTA size, every CTA takes a slice of the request's visual tokens (the
-// per-head statistics are merged from the logits stage's per-chunk partials by every CTA: cheap).
+// per-head statistics are merged from the logits stage's per-warp partials by every CTA: cheap).
 // ---------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t order_key(float x) {
   const uint32_t u = __float_as_uint(x);
@@ -179,7 +173,7 @@ __device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t x, uint32_t *w
 
 __global__ void __launch_bounds__(kTopkThreads)
 ttp_finalize_topk_kernel(const float *__restrict__ logits, int lstride, const float2 *__restrict__ stats,
-                         int n_chunks, int n_q_heads, int k_max_len,
+                         int n_parts, int n_q_heads, int k_max_len,
                          const int *__restrict__ prefix_len, const int *__restrict__ vis_start,
                          const int *__restrict__ n_vis, const int *__restrict__ keep, int norm_scope,
                          float *__restrict__ scores, int m_max, int *__restrict__ kept_idx, int r_max,
@@ -206,33 +200,41 @@ ttp_finalize_topk_kernel(const float *__restrict__ logits, int lstride, const fl
       return;
     }
     const int lo = norm_scope ? vs : 0, hi = norm_scope ? vs + nv : lp;
-    // chunks of the logits stage that hold keys of the scope (none for an empty scope)
+    // partials of the logits stage that may hold keys of the scope: those of its chunks (none for an
+    // empty scope); a partial without a key in scope is (-inf, 0)
     const int c_lo = lo / kScoreKeysPerCta, c_hi = hi > lo ? (hi - 1) / kScoreKeysPerCta : c_lo - 1;
-    // a lane takes the chunks c_lo + lane, + 32, ... of a head; a warp has four heads' partials in
-    // flight (for scopes of up to 4096 keys that is every load of the merge in one round trip)
-    constexpr int kHeadsInFlight = 4;
+    const int p_lo = c_lo * kScoreWarps, p_hi = (c_hi + 1) * kScoreWarps;        // [p_lo, p_hi)
+    // a lane takes the partials p_lo + lane, + 32, ... of a head, eight of them in registers, and a warp
+    // has two heads in flight: for scopes of up to 4096 keys every load of a pair of heads is one round trip
+    constexpr int kHeadsInFlight = 2, kPartRegs = 8;
     for (int h0 = warp * kHeadsInFlight; h0 < n_q_heads; h0 += (nt / 32) * kHeadsInFlight) {
-      float2 part[kHeadsInFlight];
+      float2 part[kHeadsInFlight][kPartRegs];
 #pragma unroll
-      for (int i = 0; i < kHeadsInFlight; ++i) {
-        const int h = h0 + i, c = c_lo + lane;
-        part[i] = h < n_q_heads && c <= c_hi ? stats[((long long)b * n_q_heads + h) * n_chunks + c]
-                                             : make_float2(-INFINITY, 0.f);
-      }
+      for (int i = 0; i < kHeadsInFlight; ++i)
+#pragma unroll
+        for (int r = 0; r < kPartRegs; ++r) {
+          const int h = h0 + i, c = p_lo + lane + 32 * r;
+          part[i][r] = h < n_q_heads && c < p_hi ? stats[((long long)b * n_q_heads + h) * n_parts + c]
+                                                 : make_float2(-INFINITY, 0.f);
+        }
 #pragma unroll
       for (int i = 0; i < kHeadsInFlight; ++i) {
         const int h = h0 + i;
         if (h >= n_q_heads) break;                   // (uniform in the warp)
-        for (int c = c_lo + lane + 32; c <= c_hi; c += 32) {
-          const float2 more = stats[((long long)b * n_q_heads + h) * n_chunks + c];
-          const float m2 = fmaxf(part[i].x, more.x);   // (finite: a chunk of the scope holds a key)
-          part[i].y = part[i].y * expf(part[i].x - m2) + more.y * expf(more.x - m2);
-          part[i].x = m2;
-        }
-        float mx = part[i].x;
+        float mx = part[i][0].x;
+#pragma unroll
+        for (int r = 1; r < kPartRegs; ++r) mx = fmaxf(mx, part[i][r].x);
+        for (int c = p_lo + lane + 32 * kPartRegs; c < p_hi; c += 32)
+          mx = fmaxf(mx, stats[((long long)b * n_q_heads + h) * n_parts + c].x);
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-        float sum = part[i].x > -INFINITY ? part[i].y * expf(part[i].x - mx) : 0.f;
+        float sum = 0.f;                             // (exp(-inf - mx) = 0: partials without keys add nothing)
+#pragma unroll
+        for (int r = 0; r < kPartRegs; ++r) sum += part[i][r].y * expf(part[i][r].x - mx);
+        for (int c = p_lo + lane + 32 * kPartRegs; c < p_hi; c += 32) {
+          const float2 more = stats[((long long)b * n_q_heads + h) * n_parts + c];
+          sum += more.y * expf(more.x - mx);
+        }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
         if (lane == 0) {
@@ -619,14 +621,15 @@ row_gather_kernel(const unsigned char *__restrict__ src, unsigned char *__restri
 // ---------------------------------------------------------------------------
 static inline int logits_stride(int k_max_len) { return (k_max_len + 3) & ~3; }
 
-static inline int score_chunks(int k_max_len) { return (k_max_len + kScoreKeysPerCta - 1) / kScoreKeysPerCta; }
+// partial softmax statistics per head: one per warp of the logits stage
+static inline int score_parts(int k_max_len) { return (k_max_len + kScoreKeysPerCta - 1) / kScoreKeysPerCta * kScoreWarps; }
 
-// scaled logits [batch, heads, stride], then the per-chunk softmax statistics [batch, heads, chunks]
+// scaled logits [batch, heads, stride], then the partial softmax statistics [batch, heads, parts]
 static inline size_t logits_bytes(int batch, int n_q_heads, int max_len) {
   return (size_t)batch * n_q_heads * logits_stride(max_len) * sizeof(float);
 }
 size_t score_workspace_bytes(int batch, int n_q_heads, int max_len) {
-  return logits_bytes(batch, n_q_heads, max_len) + (size_t)batch * n_q_heads * score_chunks(max_len) * sizeof(float2);
+  return logits_bytes(batch, n_q_heads, max_len) + (size_t)batch * n_q_heads * score_parts(max_len) * sizeof(float2);
 }
 
 struct ScoreArgs {
@@ -671,11 +674,11 @@ static twig_status launch_logits(const ScoreArgs &a, int *dev_status, void *ws, 
   const long long ksb = a.ksb, ksh = a.ksh, ksp = a.ksp;
   float *lg = static_cast<float *>(ws);
   float2 *stats = reinterpret_cast<float2 *>(static_cast<unsigned char *>(ws) + logits_bytes(a.batch, a.n_q_heads, a.k_max_len));
-  const int n_chunks = score_chunks(a.k_max_len);
+  const int n_parts = score_parts(a.k_max_len);
   cudaError_t err;
 #define TWIG_LOGITS(D_, G_)                                                                                          \
   err = cudaLaunchKernelEx(&L.cfg, ttp_logits_kernel<D_, G_>, q, k, qg, kg, ksb, ksh, ksp, a.k_max_len, a.prefix_len, \
-                           a.vis_start, a.n_vis, a.n_q_heads, group, a.norm_scope, scale, lg, ls, stats, n_chunks,    \
+                           a.vis_start, a.n_vis, a.n_q_heads, group, a.norm_scope, scale, lg, ls, stats, n_parts,     \
                            a.m_max, dev_status)
   if (a.head_dim == 128) {
     if (qg) TWIG_LOGITS(128, true); else TWIG_LOGITS(128, false);
@@ -706,7 +709,7 @@ static twig_status launch_finalize(const float *logits, const ScoreArgs &a, cons
   const float2 *stats = logits ? reinterpret_cast<const float2 *>(reinterpret_cast<const unsigned char *>(logits) +
                                                                   logits_bytes(a.batch, a.n_q_heads, a.k_max_len))
                                : nullptr;
-  const cudaError_t err = cudaLaunchKernelEx(&L.cfg, ttp_finalize_topk_kernel, logits, ls, stats, score_chunks(a.k_max_len),
+  const cudaError_t err = cudaLaunchKernelEx(&L.cfg, ttp_finalize_topk_kernel, logits, ls, stats, score_parts(a.k_max_len),
                                              a.n_q_heads, a.k_max_len, a.prefix_len, a.vis_start, a.n_vis, keep,
                                              a.norm_scope, a.scores, a.m_max, kept_idx, r_max, dev_status, mode);
   return err == cudaSuccess ? TWIG_OK : TWIG_ERR_CUDA;
