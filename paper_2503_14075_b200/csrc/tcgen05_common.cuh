@@ -58,6 +58,14 @@ __device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap *map
       ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(x), "r"(pos), "r"(head), "r"(batch), "r"(layer)
       : "memory");
 }
+// One box of a 4-D tensor map (x, position, head, batch) -> shared memory; completion is counted on `bar`.
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int pos,
+                                            int head, int batch) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(x), "r"(pos), "r"(head), "r"(batch)
+      : "memory");
+}
 // Bounded wait on an mbarrier phase; false when the limit ran out or another role has failed.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *fail) {
   for (int i = 0; i < kSpinLimit; ++i) {
