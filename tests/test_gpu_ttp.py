@@ -141,6 +141,48 @@ def test_multiquery_scores_match_oracle(tw, name, gain_mult):
     assert torch.equal(scores, scores2)
 
 
+@pytest.mark.parametrize("d", [64, 128])
+def test_multiquery_many_text_rows(tw, d):
+    """More text tokens than one 64-row block, a causal edge that crosses 128-key chunks, requests
+    of different layouts in one call, keys past the prompt poisoned (nobody may see them)."""
+    B, Hq, Hkv = 3, 4, 2
+    vis_start = np.array([5, 0, 130], dtype=np.int32)
+    n_vis = np.array([300, 70, 129], dtype=np.int32)
+    n_text = [150, 64, 1]
+    prefix_len = (vis_start + n_vis + np.array(n_text)).astype(np.int32)
+    L_max = int(prefix_len.max()) + 9
+    rng = synth.rng_for(9, 31)
+    gain = d ** 0.5                                     # logits of order one
+    k = synth.normal_bf16(rng, (B, Hkv, L_max, d), d, gain)
+    for b in range(B):
+        k[b, :, prefix_len[b]:, :] = 0x7FC1             # NaN past the prompt
+    n_max = max(n_text) + 2
+    qt = synth.normal_bf16(rng, (B, Hq, n_max, d), d, gain)
+    for b in range(B):
+        qt[b, :, n_text[b]:, :] = 0x7FC1
+    m_max = int(n_vis.max())
+    scores = torch.full((B, m_max), -1.0, dtype=torch.float32, device=DEV)
+    ws = torch.full((tw.ttp_multiquery_workspace_bytes(B, Hq, n_max, m_max, L_max) // 4,), float("nan"),
+                    dtype=torch.float32, device=DEV)
+    status = torch.zeros(B, dtype=torch.int32, device=DEV)
+    tw.ttp_score_multiquery(dev_bf16(qt), dev_bf16(k), dev_i32(prefix_len), dev_i32(vis_start), dev_i32(n_vis), scores, ws,
+                            dev_status=status)
+    torch.cuda.synchronize()
+    assert status.cpu().tolist() == [0] * B
+    got = scores.cpu().numpy()
+    qt_clean, k_clean = qt.copy(), k.copy()
+    for b in range(B):
+        qt_clean[b, :, n_text[b]:, :] = 0
+        k_clean[b, :, prefix_len[b]:, :] = 0
+    want = O.text_to_visual_scores(f64(qt_clean), f64(k_clean), prefix_len, vis_start, n_vis)
+    for b in range(B):
+        m = n_vis[b]
+        assert np.all(np.isfinite(got[b]))
+        assert max_abs(got[b, :m], want[b, :m]) <= MAX_ABS_TOL * n_text[b]
+        assert rel_l2_rows(got[b, :m].astype(np.float64), want[b, :m]) <= REL_L2_TOL
+        assert np.all(got[b, m:] == 0)
+
+
 def _run_topk(tw, s, n_vis, keep, r_max=None):
     B, m_max = s.shape
     r_max = r_max or max(1, int(max(keep)))
