@@ -175,16 +175,22 @@ base_argmax_kernel(const void *__restrict__ logits, long long row_stride, int vo
       argmax_take(bf16_hi(w.w), base + 7, best, bi);
     }
   };
-  int c = tid;
   constexpr int kDeep = 8;                          // 16-byte loads in flight per thread
-  for (; c + (kDeep - 1) * kArgmaxThreads < chunks; c += kDeep * kArgmaxThreads) {
+  // (every batch is predicated, so that a row that is no multiple of the batch never falls back to one
+  // load per round trip)
+  for (int c0 = tid; c0 < chunks; c0 += kDeep * kArgmaxThreads) {
     uint4 w[kDeep];
 #pragma unroll
-    for (int u = 0; u < kDeep; ++u) w[u] = ld_nc_16(row + (long long)(c + u * kArgmaxThreads) * 16);
+    for (int u = 0; u < kDeep; ++u) {
+      const int c = c0 + u * kArgmaxThreads;
+      if (c < chunks) w[u] = ld_nc_16(row + (long long)c * 16);
+    }
 #pragma unroll
-    for (int u = 0; u < kDeep; ++u) take_chunk(w[u], c + u * kArgmaxThreads);
+    for (int u = 0; u < kDeep; ++u) {
+      const int c = c0 + u * kArgmaxThreads;
+      if (c < chunks) take_chunk(w[u], c);
+    }
   }
-  for (; c < chunks; c += kArgmaxThreads) take_chunk(ld_nc_16(row + (long long)c * 16), c);
   for (int i = chunks * EPC + tid; i < vocab; i += kArgmaxThreads) {     // tail that is no whole chunk
     const float v = FP32 ? reinterpret_cast<const float *>(row)[i]
                          : __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(row)[i]);
