@@ -746,6 +746,24 @@ def extra_rooflines(torch, tw, peaks, dev):
     torch.cuda.synchronize()
     us = e0.elapsed_time(e1) * 1e3 / n_chain
     res["base_argmax_c3_V32000"] = hbm_entry(us, int(sum(wl3.n_nodes)) * V * 2)
+    # the same chain replayed from a CUDA graph: what the device needs when the host is not in the way
+    side = torch.cuda.Stream()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(g, stream=side):
+            for bfr in bufs:
+                tw.tree_base_argmax(bfr, nn3, arg)
+    torch.cuda.synchronize()
+    g.replay()
+    reps = max(1, n_chain // 6)
+    e0.record(stream)
+    for _ in range(reps):
+        g.replay()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    us_g = e0.elapsed_time(e1) * 1e3 / (6 * reps)
+    res["base_argmax_c3_V32000"]["us_per_launch_in_graph"] = round(us_g, 2)
+    res["base_argmax_c3_V32000"]["frac_in_graph"] = round(int(sum(wl3.n_nodes)) * V * 2 / us_g / 1e3 / peaks["hbm_gbs"], 4)
     # draft-side token tree with the paper's settings (E = K = 10, D = 4, N_max = 60) for the heterogeneous
     # batch: 4 expansions (1 + 3 x 10 draft rows of 32000 bf16 logits per request), 3 selections, 1 pruning;
     # three sets of logits in turn (95 MB together with the argmax buffers evicted: cold reads)
